@@ -1,0 +1,216 @@
+/*
+ * gg.h -- C interface of the B200 (sm_100a) generalized-Gaussian (GG) pass.
+ *
+ * The library runs, per tensor or per segment of a tensor, the data-parallel pass that the
+ * GG-prior training framework repeats over weights, activations and gradients:
+ *
+ *   moments  ->  fit (shape beta, scale alpha)  ->  penalty + elementwise gradient
+ *            ->  quantise, symbol histogram, empirical entropy;   and GG sampling for init.
+ *
+ * Letters.  The density is the paper's Eq. 1 with location 0,
+ *     f(x) = beta / (2 alpha Gamma(1/beta)) * exp(-(|x|/alpha)^beta),
+ * where THIS interface writes the shape as beta and the scale as alpha (Eq. 1 prints them as
+ * nu and beta).  sigma^2 = alpha^2 Gamma(3/beta)/Gamma(1/beta) (Eq. 2-3).
+ *
+ * Conventions.
+ *  - Every function returns a gg_status; nothing throws, aborts or prints.
+ *  - "device" pointers are CUDA global memory of the context's device; "host" pointers are
+ *    ordinary process memory.  The caller owns every buffer it passes; the library keeps no
+ *    caller pointer beyond the work it has enqueued.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *    enqueue work; they do not wait for the device.  Exception: the first call that sees a new
+ *    segment layout (addresses, lengths, dtype, histogram ids) allocates and uploads a small
+ *    plan with blocking calls; make that first call outside stream capture.  A context serves
+ *    one stream at a time.
+ *  - A segment is a contiguous run of `len` elements.  Pointers need only element alignment;
+ *    16-byte aligned segments take the vectorised path.
+ *  - Per-segment conditions are reported in `flags` (GG_FLAG_*), never as an error status.
+ */
+#ifndef GG_B200_H
+#define GG_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gg_ctx gg_ctx;
+typedef int gg_status;
+
+enum {
+    GG_OK = 0,
+    GG_ERR_INVALID_ARG = 1,   /* null pointer, negative size, inconsistent arguments          */
+    GG_ERR_DTYPE = 2,         /* dtype is not GG_F32 / GG_BF16                                 */
+    GG_ERR_ALIGNMENT = 3,     /* a pointer is not aligned to its element size                  */
+    GG_ERR_WORKSPACE = 4,     /* a fixed-capacity scratch area is too small for the request    */
+    GG_ERR_ARCH = 5,          /* the device is not compute capability 10.x                     */
+    GG_ERR_CUDA = 6,          /* a CUDA call failed; see gg_last_cuda_error                    */
+    GG_ERR_UNIMPLEMENTED = 7,
+    GG_ERR_NOMEM = 8          /* a host or device allocation failed                            */
+};
+
+typedef enum { GG_F32 = 0, GG_BF16 = 1 } gg_dtype;
+
+/* One contiguous segment.  `ptr` is device memory (host memory for gg_fused_host). */
+typedef struct {
+    void   *ptr;
+    int64_t len;
+} gg_seg;
+
+/* Per-segment flag bits written by gg_fit / gg_fused. */
+#define GG_FLAG_DEGENERATE      1u   /* len == 0 or all entries zero: beta = alpha = 0       */
+#define GG_FLAG_BETA_CLAMPED_LO 2u   /* moment ratio below rho(GG_BETA_LO): beta = GG_BETA_LO */
+#define GG_FLAG_BETA_CLAMPED_HI 4u   /* moment ratio above rho(GG_BETA_HI): beta = GG_BETA_HI */
+#define GG_FLAG_NONFINITE       8u   /* an entry was inf or nan (left out of the moments)     */
+#define GG_FLAG_CLAMPED_SYMBOLS 16u  /* a quantised symbol fell outside [qmin, qmax]          */
+
+#define GG_BETA_LO 0.05
+#define GG_BETA_HI 20.0
+
+#define GG_SUM  0   /* penalty = lambda * sum_i (|x_i|/alpha)^beta        */
+#define GG_MEAN 1   /* the same with lambda replaced by lambda / len      */
+
+#define GG_PARAMS_FITTED 0   /* penalty uses the (beta, alpha) fitted by this call: two reads of x */
+#define GG_PARAMS_GIVEN  1   /* penalty uses caller-supplied (beta, alpha); the fit of this call is
+                                still produced: one read of x                                    */
+#define GG_STEP_GIVEN      0 /* quantiser step[s] supplied by the caller                        */
+#define GG_STEP_FROM_ALPHA 1 /* step[s] = (float)(fitted alpha[s] * step_scale), also written out */
+
+/* ---- context ----------------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (which must be compute capability 10.x).  The
+ * context owns plan tables and per-tile scratch, grown on demand and freed by gg_destroy. */
+gg_status gg_create(gg_ctx **out, int device);
+gg_status gg_destroy(gg_ctx *ctx);
+
+const char *gg_status_str(gg_status s);
+int gg_version(void);
+/* Text of the last CUDA error seen by this context ("" if none).  Valid until the next call. */
+const char *gg_last_cuda_error(const gg_ctx *ctx);
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t gg_launch_count(const gg_ctx *ctx);
+
+/* ---- host helpers (no device work) --------------------------------------------------------- */
+
+/* Scale for a wanted standard deviation, Eq. 2: alpha = sigma sqrt(Gamma(1/beta)/Gamma(3/beta)). */
+double gg_alpha_from_std(double sigma, double beta);
+/* Scale of the GG initialisation rule for a d_in x d_out linear layer, Eq. 4-5:
+ * sqrt(xi/d_in * Gamma(1/beta)/Gamma(3/beta)); xi = 1 (no activation / sigmoid), 2 (ReLU),
+ * 2/(1+k^2) (leaky ReLU with negative slope k).  beta = 2, xi = 2 is He initialisation. */
+double gg_init_alpha(int64_t d_in, double xi, double beta);
+/* Differential entropy of Eq. 1 in bits: (1/beta + ln(2 alpha Gamma(1/beta)/beta)) / ln 2. */
+double gg_diff_entropy_bits(double alpha, double beta);
+
+/* ---- the steps ------------------------------------------------------------------------------ */
+
+/* Moments and fit of each segment (the "fitted with GGD" step behind the paper's Fig. 1; the
+ * method is the moment-ratio inversion
+ *     (E|x|)^2 / E[x^2] = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)),
+ * which has one root because the right side increases with beta; then alpha from Eq. 2 with
+ * sigma^2 = sum_sq / count).
+ *   segs      host array of n_seg segments (device data of type `dtype`)
+ *   beta, alpha, sum_abs, sum_sq   device double[n_seg], outputs (sum_abs, sum_sq may be NULL)
+ *   count     device int64[n_seg] output (= len; may be NULL)
+ *   flags     device uint32[n_seg] output (may be NULL)
+ * beta is clamped to [GG_BETA_LO, GG_BETA_HI]; a degenerate segment gives beta = alpha = 0. */
+gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
+                 double *beta, double *alpha, double *sum_abs, double *sum_sq,
+                 int64_t *count, uint32_t *flags, void *stream);
+
+/* GG distribution penalty and its gradient for given per-segment parameters (the rate term of the
+ * rate-distortion objective J = D + lambda R, with R the GG negative log-likelihood without its
+ * constants):
+ *     penalty[s] = lambda_s * sum_i (|x_i|/alpha_s)^beta_s
+ *     g_i        = lambda_s * beta_s * sign(x_i) * |x_i|^(beta_s - 1) / alpha_s^beta_s,  g = 0 at x = 0
+ * with lambda_s = lambda (GG_SUM) or lambda/len_s (GG_MEAN).  beta, alpha are constants with
+ * respect to x.  beta_s <= 0 or alpha_s <= 0 (a degenerate fit) gives zeros.
+ *   beta, alpha   device double[n_seg], inputs
+ *   grad          host array of n_seg segments (device data of grad_dtype); grad[s].len must equal
+ *                 segs[s].len; NULL = penalty only
+ *   accumulate    0: grad = g;  1: grad += g
+ *   penalty       device double[n_seg] output (may be NULL) */
+gg_status gg_penalty_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype in_dtype,
+                          const double *beta, const double *alpha, double lambda, int reduction,
+                          const gg_seg *grad, gg_dtype grad_dtype, int accumulate,
+                          double *penalty, void *stream);
+
+/* Quantised-symbol histogram and empirical entropy, the rate measure.  The quantiser is the
+ * paper's floor quantiser (the forward value of STE(x) = x - sg(x - floor(x)) applied to x/step),
+ * with the scaling defined in fp32 so that every symbol is unique:
+ *     inv = (float)(1.0/(double)step[s]);  q_i = clamp(floor(fl32(x_i * inv)), qmin, qmax).
+ * NaN entries are skipped.
+ *   step        device float[n_seg]
+ *   hist_id     host int32[n_seg] or NULL; segment s adds to histogram hist_id[s] (NULL: s itself,
+ *               which requires n_hist == n_seg)
+ *   hist        device uint64[n_hist * (qmax-qmin+1)]; zeroed first unless accumulate != 0
+ *   entropy_bits  device double[n_hist]: H = log2 N - (1/N) sum_{c>0} c log2 c (may be NULL)
+ *   clamped_lo_hi device uint64[2*n_hist]: symbols moved up to qmin / down to qmax (may be NULL;
+ *               zeroed first unless accumulate) */
+gg_status gg_rate_hist(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
+                       const float *step, const int32_t *hist_id, int32_t n_hist,
+                       int32_t qmin, int32_t qmax, uint64_t *hist, int accumulate,
+                       double *entropy_bits, uint64_t *clamped_lo_hi, void *stream);
+
+/* GG sampling for initialisation ("initialize weights from GGDs", Eq. 4-5).  Element i of segment
+ * s is alpha_s * sign * G^(1/beta_s) with G ~ Gamma(1/beta_s, 1) by the Marsaglia-Tsang method
+ * (normals by Box-Muller), rounded to nearest-even in `dtype`.  All randomness is Philox4x32-10
+ * with counter (i mod 2^32, i div 2^32, attempt, tensor_id0 + s) and key (seed mod 2^32,
+ * seed div 2^32); the block with attempt = 0xFFFFFFFF gives the sign and the extra uniform
+ * of the shape < 1 case.  Any element can therefore be regenerated alone.
+ *   out          host array of n_seg segments (device data of `dtype`), outputs
+ *   beta, alpha  HOST double[n_seg]
+ *   max_attempts device uint32[n_seg] or NULL: largest number of attempts any element needed
+ *                (65 = an element exhausted the 64 allowed attempts and was set to 0) */
+gg_status gg_sample(gg_ctx *ctx, const gg_seg *out, int32_t n_seg, gg_dtype dtype,
+                    const double *beta, const double *alpha, uint64_t seed, uint32_t tensor_id0,
+                    uint32_t *max_attempts, void *stream);
+
+/* Arguments of the fused pass.  Pointer meanings are those of the single-step calls above. */
+typedef struct {
+    const gg_seg *segs;          /* host array [n_seg]                                        */
+    int32_t       n_seg;
+    int32_t       in_dtype;      /* gg_dtype                                                  */
+    /* fit outputs, device [n_seg]; beta and alpha are required                               */
+    double   *beta, *alpha, *sum_abs, *sum_sq;
+    int64_t  *count;
+    uint32_t *flags;
+    /* penalty and gradient                                                                   */
+    int32_t       param_mode;    /* GG_PARAMS_FITTED or GG_PARAMS_GIVEN                       */
+    const double *beta_in, *alpha_in;   /* device [n_seg], GG_PARAMS_GIVEN only               */
+    double        lambda;
+    int32_t       reduction;     /* GG_SUM or GG_MEAN                                         */
+    const gg_seg *grad;          /* host array [n_seg] or NULL                                */
+    int32_t       grad_dtype;
+    int32_t       accumulate_grad;
+    double       *penalty;       /* device [n_seg] or NULL                                    */
+    /* quantiser, histogram, entropy                                                          */
+    int32_t       step_mode;     /* GG_STEP_GIVEN or GG_STEP_FROM_ALPHA (needs PARAMS_FITTED) */
+    const float  *step;          /* device [n_seg], GG_STEP_GIVEN                             */
+    double        step_scale;    /* GG_STEP_FROM_ALPHA                                        */
+    float        *step_out;      /* device [n_seg], GG_STEP_FROM_ALPHA: the steps used        */
+    const int32_t *hist_id;      /* host [n_seg] or NULL                                      */
+    int32_t       n_hist, qmin, qmax;
+    uint64_t     *hist;          /* device; NULL skips the histogram step                     */
+    int32_t       accumulate_hist;
+    double       *entropy_bits;  /* device [n_hist] or NULL                                   */
+    uint64_t     *clamped_lo_hi; /* device [2*n_hist] or NULL                                 */
+} gg_fused_args;
+
+/* The whole pass over a list of segments in the fewest sweeps of x: moments -> fit ->
+ * penalty + gradient + histogram -> entropy, all enqueued on `stream`.
+ * GG_PARAMS_FITTED reads x twice (the gradient needs the fit of the whole segment);
+ * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep). */
+gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *args, void *stream);
+
+/* The same pass for data that lives in HOST memory: every pointer of `args` that gg_fused documents
+ * as device memory (segment data, fit outputs, gradient segments, step, histogram, entropy, ...) is
+ * here a host pointer.  The library stages segments through device buffers of its own in chunks of
+ * at most `chunk_bytes` of input (0 = default), overlapping copies with kernels, and returns after
+ * all results are in host memory.  Pinned host buffers make the copies asynchronous. */
+gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *args, int64_t chunk_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GG_B200_H */

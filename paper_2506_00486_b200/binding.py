@@ -1,0 +1,348 @@
+"""ctypes binding of libgg_b200.so: argument marshalling only.
+
+Every step of the pass runs in the CUDA library; this module turns torch tensors into the
+pointers and sizes of the C interface (include/gg.h) and allocates output tensors.  There is
+no CPU fallback: if the library is missing or the device is not a B200-class GPU the calls raise.
+"""
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgg_b200.so")
+
+GG_F32, GG_BF16 = 0, 1
+GG_SUM, GG_MEAN = 0, 1
+GG_PARAMS_FITTED, GG_PARAMS_GIVEN = 0, 1
+GG_STEP_GIVEN, GG_STEP_FROM_ALPHA = 0, 1
+FLAG_DEGENERATE, FLAG_BETA_CLAMPED_LO, FLAG_BETA_CLAMPED_HI, FLAG_NONFINITE, FLAG_CLAMPED_SYMBOLS = 1, 2, 4, 8, 16
+BETA_LO, BETA_HI = 0.05, 20.0
+
+_SEG_DTYPE = np.dtype([("ptr", np.uint64), ("len", np.int64)])
+_P = ctypes.c_void_p
+
+
+class FusedArgs(ctypes.Structure):
+    """Mirror of gg_fused_args."""
+    _fields_ = [
+        ("segs", _P), ("n_seg", ctypes.c_int32), ("in_dtype", ctypes.c_int32),
+        ("beta", _P), ("alpha", _P), ("sum_abs", _P), ("sum_sq", _P), ("count", _P), ("flags", _P),
+        ("param_mode", ctypes.c_int32), ("beta_in", _P), ("alpha_in", _P),
+        ("lam", ctypes.c_double), ("reduction", ctypes.c_int32),
+        ("grad", _P), ("grad_dtype", ctypes.c_int32), ("accumulate_grad", ctypes.c_int32),
+        ("penalty", _P),
+        ("step_mode", ctypes.c_int32), ("step", _P), ("step_scale", ctypes.c_double), ("step_out", _P),
+        ("hist_id", _P), ("n_hist", ctypes.c_int32), ("qmin", ctypes.c_int32), ("qmax", ctypes.c_int32),
+        ("hist", _P), ("accumulate_hist", ctypes.c_int32), ("entropy_bits", _P), ("clamped_lo_hi", _P),
+    ]
+
+
+class GGError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__(f"gg status {status}: {text}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run paper_2506_00486_b200/build.py "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        i32, i64, u32, u64, d = (ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_uint64,
+                                 ctypes.c_double)
+        L.gg_create.argtypes = [ctypes.POINTER(_P), ctypes.c_int]
+        L.gg_destroy.argtypes = [_P]
+        L.gg_status_str.argtypes = [ctypes.c_int]
+        L.gg_status_str.restype = ctypes.c_char_p
+        L.gg_version.restype = ctypes.c_int
+        L.gg_last_cuda_error.argtypes = [_P]
+        L.gg_last_cuda_error.restype = ctypes.c_char_p
+        L.gg_launch_count.argtypes = [_P]
+        L.gg_launch_count.restype = i64
+        for name, args in (("gg_alpha_from_std", [d, d]), ("gg_init_alpha", [i64, d, d]),
+                           ("gg_diff_entropy_bits", [d, d])):
+            getattr(L, name).argtypes = args
+            getattr(L, name).restype = d
+        L.gg_fit.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, _P, _P, _P, _P, _P]
+        L.gg_penalty_grad.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, d, ctypes.c_int, _P,
+                                      ctypes.c_int, ctypes.c_int, _P, _P]
+        L.gg_rate_hist.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, i32, i32, i32, _P, ctypes.c_int,
+                                   _P, _P, _P]
+        L.gg_sample.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, u64, u32, _P, _P]
+        L.gg_fused.argtypes = [_P, ctypes.POINTER(FusedArgs), _P]
+        L.gg_fused_host.argtypes = [_P, ctypes.POINTER(FusedArgs), i64]
+        for name in ("gg_create", "gg_destroy", "gg_fit", "gg_penalty_grad", "gg_rate_hist", "gg_sample",
+                     "gg_fused", "gg_fused_host"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def gg_alpha_from_std(std, beta):
+    return lib().gg_alpha_from_std(float(std), float(beta))
+
+
+def gg_init_alpha(d_in, xi, beta):
+    return lib().gg_init_alpha(int(d_in), float(xi), float(beta))
+
+
+def gg_diff_entropy_bits(alpha, beta):
+    return lib().gg_diff_entropy_bits(float(alpha), float(beta))
+
+
+def _dtype_code(dt):
+    if dt == torch.float32:
+        return GG_F32
+    if dt == torch.bfloat16:
+        return GG_BF16
+    raise TypeError(f"unsupported dtype {dt}: the library takes float32 and bfloat16")
+
+
+class Segments:
+    """A host array of gg_seg built once from tensors (kept alive here).
+
+    `Segments(list_of_tensors)`: one segment per tensor (flattened, must be contiguous).
+    `Segments.rows(t)`: one segment per row of a contiguous 2-D tensor."""
+
+    def __init__(self, tensors):
+        tensors = list(tensors)
+        self.tensors = tensors
+        self.dtype = tensors[0].dtype if tensors else torch.float32
+        arr = np.zeros(len(tensors), dtype=_SEG_DTYPE)
+        for i, t in enumerate(tensors):
+            if t.dtype != self.dtype:
+                raise TypeError("all segments of one call share a dtype")
+            if not t.is_contiguous():
+                raise ValueError("segments must be contiguous")
+            arr["ptr"][i] = t.data_ptr() if t.numel() else 0
+            arr["len"][i] = t.numel()
+        self.array = arr
+
+    @classmethod
+    def rows(cls, t):
+        if t.dim() != 2 or not t.is_contiguous():
+            raise ValueError("need a contiguous 2-D tensor")
+        self = cls.__new__(cls)
+        self.tensors = [t]
+        self.dtype = t.dtype
+        arr = np.zeros(t.shape[0], dtype=_SEG_DTYPE)
+        row_bytes = t.shape[1] * t.element_size()
+        arr["ptr"] = t.data_ptr() + np.arange(t.shape[0], dtype=np.uint64) * np.uint64(row_bytes)
+        arr["len"] = t.shape[1]
+        self.array = arr
+        return self
+
+    @classmethod
+    def slices(cls, flat, offsets, lens):
+        """Segments flat[offsets[i] : offsets[i] + lens[i]] of one flat tensor."""
+        self = cls.__new__(cls)
+        self.tensors = [flat]
+        self.dtype = flat.dtype
+        arr = np.zeros(len(lens), dtype=_SEG_DTYPE)
+        arr["ptr"] = flat.data_ptr() + np.asarray(offsets, dtype=np.uint64) * np.uint64(flat.element_size())
+        arr["len"] = np.asarray(lens, dtype=np.int64)
+        self.array = arr
+        return self
+
+    def __len__(self):
+        return len(self.array)
+
+    @property
+    def lens(self):
+        return self.array["len"]
+
+    @property
+    def ptr(self):
+        return self.array.ctypes.data
+
+    @property
+    def code(self):
+        return _dtype_code(self.dtype)
+
+    def device(self):
+        return self.tensors[0].device
+
+
+def _as_segments(x):
+    return x if isinstance(x, Segments) else Segments(x)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(device):
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+class Context:
+    """One gg_ctx on one CUDA device.  Use from one stream at a time."""
+
+    def __init__(self, device=0):
+        self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+        if self.device.type != "cuda":
+            raise RuntimeError("the GG library runs on CUDA devices only")
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the GG library has no CPU fallback")
+        torch.cuda.init()
+        with torch.cuda.device(self.device):
+            torch.empty(1, device=self.device)          # make sure the primary context exists
+        h = _P()
+        self._check(lib().gg_create(ctypes.byref(h), self.device.index or 0), None)
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().gg_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, status, h=True):
+        if status != 0:
+            text = lib().gg_status_str(status).decode()
+            if status == 6 and h and getattr(self, "_h", None):
+                text += ": " + lib().gg_last_cuda_error(self._h).decode()
+            raise GGError(status, text)
+
+    @property
+    def launch_count(self):
+        return lib().gg_launch_count(self._h)
+
+    def _new(self, n, dtype):
+        return torch.empty(n, dtype=dtype, device=self.device)
+
+    # ------------------------------------------------------------------ gg_fit
+    def gg_fit(self, segs):
+        """Moments and fit per segment.  Returns a dict of device tensors."""
+        segs = _as_segments(segs)
+        n = len(segs)
+        out = dict(beta=self._new(n, torch.float64), alpha=self._new(n, torch.float64),
+                   sum_abs=self._new(n, torch.float64), sum_sq=self._new(n, torch.float64),
+                   count=self._new(n, torch.int64), flags=self._new(n, torch.int32))
+        self._check(lib().gg_fit(self._h, segs.ptr, n, segs.code, _ptr(out["beta"]), _ptr(out["alpha"]),
+                                 _ptr(out["sum_abs"]), _ptr(out["sum_sq"]), _ptr(out["count"]),
+                                 _ptr(out["flags"]), _stream_ptr(self.device)))
+        return out
+
+    # -------------------------------------------------------- gg_penalty_grad
+    def gg_penalty_grad(self, segs, beta, alpha, lam, grad=None, reduction=GG_SUM, accumulate=False,
+                        want_penalty=True):
+        """Penalty per segment (device float64) and the gradient written into `grad` segments."""
+        segs = _as_segments(segs)
+        n = len(segs)
+        gsegs = None if grad is None else _as_segments(grad)
+        pen = self._new(n, torch.float64) if want_penalty else None
+        self._check(lib().gg_penalty_grad(
+            self._h, segs.ptr, n, segs.code, _ptr(beta), _ptr(alpha), float(lam), int(reduction),
+            None if gsegs is None else gsegs.ptr, GG_F32 if gsegs is None else gsegs.code,
+            int(bool(accumulate)), _ptr(pen), _stream_ptr(self.device)))
+        return pen
+
+    # ------------------------------------------------------------ gg_rate_hist
+    def gg_rate_hist(self, segs, step, hist_id=None, n_hist=None, qmin=-32768, qmax=32767, hist=None,
+                     accumulate=False):
+        """Histogram(s) of the quantised symbols, entropy in bits/symbol, clamp counters."""
+        segs = _as_segments(segs)
+        n = len(segs)
+        n_hist = n if n_hist is None else int(n_hist)
+        nb = qmax - qmin + 1
+        if hist is None:
+            hist = torch.empty((n_hist, nb), dtype=torch.int64, device=self.device)
+            if accumulate:
+                hist.zero_()
+        ent = self._new(n_hist, torch.float64)
+        clamped = torch.zeros((n_hist, 2), dtype=torch.int64, device=self.device)
+        hid = None if hist_id is None else np.ascontiguousarray(hist_id, dtype=np.int32)
+        self._check(lib().gg_rate_hist(
+            self._h, segs.ptr, n, segs.code, _ptr(step), None if hid is None else hid.ctypes.data,
+            n_hist, int(qmin), int(qmax), _ptr(hist), int(bool(accumulate)), _ptr(ent), _ptr(clamped),
+            _stream_ptr(self.device)))
+        return dict(hist=hist, entropy_bits=ent, clamped=clamped)
+
+    # --------------------------------------------------------------- gg_sample
+    def gg_sample(self, out, beta, alpha, seed, tensor_id0=0, want_attempts=True):
+        """Fills the `out` segments with GG variates; beta, alpha are host sequences."""
+        segs = _as_segments(out)
+        n = len(segs)
+        b = np.ascontiguousarray(beta, dtype=np.float64)
+        a = np.ascontiguousarray(alpha, dtype=np.float64)
+        if b.size != n or a.size != n:
+            raise ValueError("beta and alpha need one entry per segment")
+        att = self._new(n, torch.int32) if want_attempts else None
+        self._check(lib().gg_sample(self._h, segs.ptr, n, segs.code, b.ctypes.data, a.ctypes.data,
+                                    int(seed) & (2 ** 64 - 1), int(tensor_id0) & 0xFFFFFFFF, _ptr(att),
+                                    _stream_ptr(self.device)))
+        return att
+
+    # ---------------------------------------------------------------- gg_fused
+    def make_fused(self, segs, grad=None, lam=1e-4, reduction=GG_SUM, accumulate_grad=False,
+                   param_mode=GG_PARAMS_FITTED, beta_in=None, alpha_in=None, want_penalty=True,
+                   step=None, step_scale=None, hist_id=None, n_hist=None, qmin=-32768, qmax=32767,
+                   want_hist=True, accumulate_hist=False, hist=None):
+        """Allocates the outputs of the fused pass once and returns a callable that enqueues it.
+
+        step: device float32 tensor [n_seg] (GG_STEP_GIVEN); or step_scale: float, step = alpha * scale."""
+        segs = _as_segments(segs)
+        n = len(segs)
+        gsegs = None if grad is None else _as_segments(grad)
+        out = dict(beta=self._new(n, torch.float64), alpha=self._new(n, torch.float64),
+                   sum_abs=self._new(n, torch.float64), sum_sq=self._new(n, torch.float64),
+                   count=self._new(n, torch.int64), flags=self._new(n, torch.int32))
+        out["penalty"] = self._new(n, torch.float64) if want_penalty else None
+        a = FusedArgs()
+        keep = [segs, gsegs, beta_in, alpha_in, step]
+        a.segs, a.n_seg, a.in_dtype = segs.ptr, n, segs.code
+        for k in ("beta", "alpha", "sum_abs", "sum_sq", "count", "flags", "penalty"):
+            setattr(a, k, _ptr(out[k]))
+        a.param_mode = int(param_mode)
+        a.beta_in, a.alpha_in = _ptr(beta_in), _ptr(alpha_in)
+        a.lam, a.reduction = float(lam), int(reduction)
+        a.grad = None if gsegs is None else gsegs.ptr
+        a.grad_dtype = GG_F32 if gsegs is None else gsegs.code
+        a.accumulate_grad = int(bool(accumulate_grad))
+        if want_hist:
+            n_hist = n if n_hist is None else int(n_hist)
+            nb = qmax - qmin + 1
+            if hist is None:
+                hist = torch.zeros((n_hist, nb), dtype=torch.int64, device=self.device)
+            out["hist"] = hist
+            out["entropy_bits"] = self._new(n_hist, torch.float64)
+            out["clamped"] = torch.zeros((n_hist, 2), dtype=torch.int64, device=self.device)
+            if step is not None:
+                a.step_mode, a.step = GG_STEP_GIVEN, _ptr(step)
+                out["step"] = step
+            else:
+                out["step"] = self._new(n, torch.float32)
+                a.step_mode, a.step_scale, a.step_out = GG_STEP_FROM_ALPHA, float(step_scale), _ptr(out["step"])
+            hid = None if hist_id is None else np.ascontiguousarray(hist_id, dtype=np.int32)
+            keep.append(hid)
+            a.hist_id = None if hid is None else hid.ctypes.data
+            a.n_hist, a.qmin, a.qmax = n_hist, int(qmin), int(qmax)
+            a.hist, a.accumulate_hist = _ptr(hist), int(bool(accumulate_hist))
+            a.entropy_bits, a.clamped_lo_hi = _ptr(out["entropy_bits"]), _ptr(out["clamped"])
+
+        def run():
+            self._check(lib().gg_fused(self._h, ctypes.byref(a), _stream_ptr(self.device)))
+            return out
+
+        run.outputs = out
+        run.args = a
+        run._keep = keep
+        return run
+
+    def gg_fused(self, segs, **kw):
+        """One-shot form of make_fused(...)()."""
+        return self.make_fused(segs, **kw)()

@@ -1,0 +1,79 @@
+// Internal declarations shared by the translation units of the library (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gg.h"
+
+namespace gg {
+
+// Elements per tile.  A tile never crosses a segment; a segment of len elements has
+// ceil(len / kTile) tiles and the last one may be ragged.
+constexpr int kTile = 16384;
+constexpr int kStreamThreads = 256;
+// Shared-memory histogram window: symbols [-kWindow/2, kWindow/2) are counted on chip, the
+// (rare) rest goes straight to global memory.
+constexpr int kWindow = 4096;
+
+enum StreamFlags : int { kMoments = 1, kGrad = 2, kHist = 4 };
+
+// Device-side view of a plan: where each tile lives.
+struct TileMap {
+    const void *const *seg_ptr;   // [n_seg] input segments
+    void *const *grad_ptr;        // [n_seg] gradient segments (may be null)
+    const int64_t *seg_len;       // [n_seg]
+    const int32_t *tile_prefix;   // [n_seg + 1] first tile of each segment
+    const int32_t *tile_seg;      // [n_tiles] owning segment of each tile
+    const int32_t *hist_id;       // [n_seg] (null: the segment index)
+    int32_t n_seg;
+    int32_t n_tiles;
+};
+
+// Per-tile partial results (fixed-order reduction happens in the per-segment kernels).
+struct TileScratch {
+    double *s1;       // sum |x|
+    double *s2;       // sum x^2
+    double *pen;      // sum |x| |g|   (penalty = that / beta)
+    uint32_t *bad;    // non-finite entries
+};
+
+struct StreamArgs {
+    TileMap map;
+    TileScratch part;
+    // gradient
+    const double *beta;
+    const double *alpha;
+    double lambda;
+    int mean_reduction;
+    int accumulate;
+    // histogram
+    const float *step;
+    int32_t qmin, qmax;
+    uint64_t *hist;
+    uint64_t *clamped;   // [2 * n_hist] or null
+    uint32_t *flags;     // [n_seg] or null (GG_FLAG_CLAMPED_SYMBOLS is OR-ed in)
+};
+
+struct FitArgs {
+    TileMap map;
+    TileScratch part;
+    double *beta, *alpha, *sum_abs, *sum_sq;
+    int64_t *count;
+    uint32_t *flags;
+    int keep_clamp_bit;   // flags[s] already holds this call's GG_FLAG_CLAMPED_SYMBOLS bit
+    int step_from_alpha;
+    double step_scale;
+    float *step_out;
+};
+
+cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
+                          const StreamArgs &a, cudaStream_t st);
+cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
+cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
+                                    double *penalty, cudaStream_t st);
+cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins,
+                           double *entropy_bits, cudaStream_t st);
+cudaError_t launch_sample(const TileMap &map, gg_dtype dtype, const double *beta, const double *alpha,
+                          uint64_t seed, uint32_t tensor_id0, uint32_t *max_attempts, cudaStream_t st);
+
+}  // namespace gg

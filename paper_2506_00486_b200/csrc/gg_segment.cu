@@ -1,0 +1,163 @@
+// Per-segment and per-histogram kernels of the GG pass: the fixed-order reduction of the tile
+// partials, the moment-ratio inversion (one warp per segment), the penalty sums, and the
+// empirical entropy of a count table.  All arithmetic here is fp64; none of it is bandwidth bound.
+#include "gg_internal.h"
+
+namespace gg {
+namespace {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kSegThreads = 128;   // 4 warps = 4 segments per CTA
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
+// of the density of Eq. 1; increasing in beta from 0 to 3/4.
+__device__ __forceinline__ double log_rho(double beta)
+{
+    return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
+}
+
+// One warp per segment.  Lanes sum the tile partials in a fixed order (strided, then a butterfly,
+// so every lane ends with the same bits), then invert the moment ratio by 33-section search on
+// ln(beta): each round the 32 lanes evaluate log_rho at the interior points of the bracket and a
+// ballot picks the sub-interval with the sign change; ten rounds shrink [ln .05, ln 20] below
+// 1e-14.  The scale follows Eq. 2 with sigma^2 = sum_sq / count.
+__global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
+{
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.map.n_seg) return;
+    const int t0 = a.map.tile_prefix[s], t1 = a.map.tile_prefix[s + 1];
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t bad = 0;
+    for (int t = t0 + lane; t < t1; t += 32) {
+        s1 += a.part.s1[t];
+        s2 += a.part.s2[t];
+        bad += a.part.bad[t];
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    bad = __reduce_add_sync(kFull, bad);
+    const int64_t len = a.map.seg_len[s];
+
+    uint32_t flags = bad ? GG_FLAG_NONFINITE : 0u;
+    double beta = 0.0, alpha = 0.0;
+    if (len <= 0 || !(s2 > 0.0)) {
+        flags |= GG_FLAG_DEGENERATE;
+    } else {
+        const double m1 = s1 / (double)len, m2 = s2 / (double)len;
+        const double log_r = log(m1 * m1 / m2);
+        if (log_r <= log_rho(GG_BETA_LO)) {
+            beta = GG_BETA_LO;
+            flags |= GG_FLAG_BETA_CLAMPED_LO;
+        } else if (log_r >= log_rho(GG_BETA_HI)) {
+            beta = GG_BETA_HI;
+            flags |= GG_FLAG_BETA_CLAMPED_HI;
+        } else {
+            double lo = log(GG_BETA_LO), hi = log(GG_BETA_HI);
+            for (int round = 0; round < 12 && hi - lo > 4e-15; ++round) {
+                const double w = (hi - lo) * (1.0 / 33.0);
+                const double ti = lo + w * (double)(lane + 1);
+                const bool below = log_rho(exp(ti)) < log_r;
+                const int k = __popc(__ballot_sync(kFull, below));   // points 1..k lie below the root
+                hi = lo + w * (double)(k + 1);
+                lo = lo + w * (double)k;
+            }
+            beta = exp(0.5 * (lo + hi));
+        }
+        alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+    }
+    if (lane == 0) {
+        a.beta[s] = beta;
+        a.alpha[s] = alpha;
+        if (a.sum_abs) a.sum_abs[s] = s1;
+        if (a.sum_sq) a.sum_sq[s] = s2;
+        if (a.count) a.count[s] = len;
+        if (a.flags) a.flags[s] = flags | (a.keep_clamp_bit ? (a.flags[s] & GG_FLAG_CLAMPED_SYMBOLS) : 0u);
+        if (a.step_from_alpha && a.step_out) a.step_out[s] = (float)(alpha * a.step_scale);
+    }
+}
+
+// penalty[s] = (1/beta_s) * sum over the segment's tiles of sum |x| |g|
+//            = lambda_s * sum (|x|/alpha_s)^beta_s   since |x| |g| = lambda beta (|x|/alpha)^beta.
+__global__ void __launch_bounds__(kSegThreads)
+penalty_finalize_kernel(const TileMap map, const TileScratch part, const double *beta, double *penalty)
+{
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= map.n_seg) return;
+    double p = 0.0;
+    for (int t = map.tile_prefix[s] + lane; t < map.tile_prefix[s + 1]; t += 32) p += part.pen[t];
+    p = warp_sum(p);
+    if (lane == 0) {
+        const double b = beta[s];
+        penalty[s] = b > 0.0 ? p / b : 0.0;
+    }
+}
+
+// One CTA per histogram: N = sum c, H = log2 N - (1/N) sum_{c>0} c log2 c.
+constexpr int kEntThreads = 256;
+__global__ void __launch_bounds__(kEntThreads)
+entropy_kernel(const uint64_t *hist, int32_t n_bins, double *entropy_bits)
+{
+    __shared__ double shAcc[kEntThreads / 32];
+    __shared__ unsigned long long shTot[kEntThreads / 32];
+    const uint64_t *row = hist + (int64_t)blockIdx.x * n_bins;
+    double acc = 0.0;
+    unsigned long long tot = 0;
+    for (int k = threadIdx.x; k < n_bins; k += kEntThreads) {
+        const uint64_t c = row[k];
+        if (c != 0) {
+            const double cd = (double)c;
+            acc += cd * log2(cd);
+            tot += c;
+        }
+    }
+    acc = warp_sum(acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(kFull, tot, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { shAcc[warp] = acc; shTot[warp] = tot; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double ra = 0.0;
+        unsigned long long rt = 0;
+        for (int w = 0; w < kEntThreads / 32; ++w) { ra += shAcc[w]; rt += shTot[w]; }
+        entropy_bits[blockIdx.x] = rt == 0 ? 0.0 : log2((double)rt) - ra / (double)rt;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_fit(const FitArgs &a, cudaStream_t st)
+{
+    if (a.map.n_seg <= 0) return cudaSuccess;
+    const int per = kSegThreads / 32;
+    fit_kernel<<<(a.map.n_seg + per - 1) / per, kSegThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
+                                    double *penalty, cudaStream_t st)
+{
+    if (map.n_seg <= 0) return cudaSuccess;
+    const int per = kSegThreads / 32;
+    penalty_finalize_kernel<<<(map.n_seg + per - 1) / per, kSegThreads, 0, st>>>(map, part, beta, penalty);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
+                           cudaStream_t st)
+{
+    if (n_hist <= 0) return cudaSuccess;
+    entropy_kernel<<<n_hist, kEntThreads, 0, st>>>(hist, n_bins, entropy_bits);
+    return cudaGetLastError();
+}
+
+}  // namespace gg

@@ -1,0 +1,458 @@
+"""GPU parity: every step of the CUDA pass against the fp64 CPU oracle, element by element, on
+seeded inputs that span several tiles and ragged tails, plus the degenerate cases.
+
+All calls go through the C interface (ctypes binding).  Gradient, penalty and histogram parity
+is always evaluated with the parameter bits the GPU used (its own fit, read back)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import gg_synth
+from oracle import gg_oracle as o
+from parity_util import (ABS_ENTROPY, REL_FIT, REL_PENALTY, assert_grad_close, assert_rel)
+
+pytestmark = pytest.mark.gpu
+
+TILE = 16384
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2506_00486_b200 import Context
+    c = Context(0)
+    yield c
+    c.close()
+
+
+def dev(t):
+    return t.to("cuda:0")
+
+
+def make_segments(dtype, seed=0):
+    """Ragged segment set: sub-tile, exact tile, multi-tile with tail, tiny, misaligned views."""
+    rng = np.random.default_rng(seed)
+    spec = [(0.5, 3e-4, 3 * TILE + 1234), (0.8, 1.0, TILE), (1.0, 0.02, 1), (1.3, 0.014, 7),
+            (2.0, 0.03, 2 * TILE + 5), (1.6, 0.02, 4096), (0.6, 0.004, 70001), (1.0, 0.5, 33)]
+    return [gg_synth.gg_host(rng, b, a, n, dtype) for b, a, n in spec]
+
+
+def misaligned_views(tensors, offsets=(1, 3, 5, 2, 7, 0, 9, 6)):
+    """Device copies whose first element sits `off` elements past a 256-byte boundary."""
+    out = []
+    for t, off in zip(tensors, offsets):
+        buf = torch.zeros(t.numel() + 16, dtype=t.dtype, device="cuda:0")
+        buf[off:off + t.numel()].copy_(t)
+        out.append(buf[off:off + t.numel()])
+    return out
+
+
+# --------------------------------------------------------------------------------------- gg_fit
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("misalign", [False, True])
+def test_fit_parity(ctx, dtype, misalign):
+    xs = make_segments(dtype)
+    xd = misaligned_views(xs) if misalign else [dev(x) for x in xs]
+    out = ctx.gg_fit(xd)
+    torch.cuda.synchronize()
+    for s, x in enumerate(xs):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(x))
+        assert out["count"][s].item() == n
+        assert out["flags"][s].item() == fl
+        assert_rel(out["sum_abs"][s].item(), s1, 1e-7, "sum_abs")
+        assert_rel(out["sum_sq"][s].item(), s2, 1e-7, "sum_sq")
+        if fl & (o.FLAG_BETA_CLAMPED_HI | o.FLAG_BETA_CLAMPED_LO):
+            assert out["beta"][s].item() == b
+        else:
+            assert_rel(out["beta"][s].item(), b, REL_FIT, "beta")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
+
+
+def test_fit_degenerate_and_flags(ctx):
+    xs = [torch.zeros(0), torch.zeros(100), torch.tensor([1.0, -1.0]), torch.tensor([1.0, 2.0, 3.0]),
+          torch.tensor([1.0, float("inf"), -2.0, float("nan"), 3.0] * 50),
+          torch.cat([torch.ones(1), torch.zeros(10 ** 6)])]
+    out = ctx.gg_fit([dev(x) for x in xs])
+    torch.cuda.synchronize()
+    for s, x in enumerate(xs):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(x))
+        assert out["flags"][s].item() == fl, s
+        assert out["count"][s].item() == n
+        assert out["beta"][s].item() == pytest.approx(b, rel=REL_FIT)
+        assert out["alpha"][s].item() == pytest.approx(a, rel=REL_FIT)
+        assert out["sum_abs"][s].item() == pytest.approx(s1, rel=1e-7)
+
+
+def test_fit_over_the_whole_shape_range(ctx):
+    """beta from 0.1 to 8 on large samples: the fitted pair matches the oracle's."""
+    rng = np.random.default_rng(21)
+    betas = [0.1, 0.2, 0.35, 0.5, 0.7, 1.0, 1.4, 2.0, 3.0, 5.0, 8.0]
+    xs = [gg_synth.gg_host(rng, b, 0.05, 200_000, torch.float32) for b in betas]
+    out = ctx.gg_fit([dev(x) for x in xs])
+    torch.cuda.synchronize()
+    for s, x in enumerate(xs):
+        b, a, *_ = o.fit(gg_synth.to_oracle(x))
+        assert_rel(out["beta"][s].item(), b, REL_FIT, f"beta (true {betas[s]})")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, f"alpha (true {betas[s]})")
+
+
+def test_fit_is_deterministic(ctx):
+    xs = [dev(x) for x in make_segments(torch.bfloat16, seed=3)]
+    a = ctx.gg_fit(xs)
+    b = ctx.gg_fit(xs)
+    torch.cuda.synchronize()
+    for k in ("beta", "alpha", "sum_abs", "sum_sq"):
+        assert torch.equal(a[k].view(torch.int64), b[k].view(torch.int64))
+
+
+# ------------------------------------------------------------------------------ gg_penalty_grad
+SPECIALS = [0.0, -0.0, 1e-45, -1e-45, 1e-40, 1.17549435e-38, -1.17549435e-38, 3.0e38, -3.0e38, 1.0, -1.0,
+            2.0, 0.5, 1.4142135, 0.70710678, 1.9999999, 1.0000001]
+
+
+def penalty_case(ctx, x_host, beta, alpha, lam, misalign=False, grad_dtype=torch.float32, reduction=0):
+    from paper_2506_00486_b200 import Segments
+    xd = misaligned_views([x_host], offsets=(3,))[0] if misalign else dev(x_host)
+    gbuf = torch.full((x_host.numel() + 16,), 7.0, dtype=grad_dtype, device="cuda:0")
+    off = 5 if misalign else 0
+    gd = gbuf[off:off + x_host.numel()]
+    bt = torch.tensor([beta], dtype=torch.float64, device="cuda:0")
+    at = torch.tensor([alpha], dtype=torch.float64, device="cuda:0")
+    pen = ctx.gg_penalty_grad(Segments([xd]), bt, at, lam, grad=Segments([gd]), reduction=reduction)
+    torch.cuda.synchronize()
+    # nothing outside the segment was touched
+    assert (gbuf[:off] == 7.0).all() and (gbuf[off + x_host.numel():] == 7.0).all()
+    return pen[0].item(), gd.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("beta,alpha", [(0.5, 3e-4), (0.8, 1.1), (1.0, 0.02), (1.3, 0.014), (1.6, 0.02),
+                                        (2.0, 0.03), (3.0, 0.5), (0.05, 1e-3), (0.1, 0.01),
+                                        (3.7, 0.5), (8.0, 1.0), (20.0, 2.0)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_penalty_grad_parity(ctx, beta, alpha, dtype):
+    rng = np.random.default_rng(int(beta * 1000))
+    n = 2 * TILE + 777
+    x = gg_synth.gg_host(rng, min(beta, 4.0), alpha, n, torch.float32)
+    x[:len(SPECIALS)] = torch.tensor(SPECIALS)
+    # a wide sweep of magnitudes: every binade from 2^-40 to 2^40 around alpha
+    sweep = alpha * np.exp2(rng.uniform(-40, 40, 4000)) * rng.choice([-1.0, 1.0], 4000)
+    x[100:4100] = torch.from_numpy(sweep.astype(np.float32))
+    x = x.to(dtype)
+    lam = 1e-4
+    pen, g = penalty_case(ctx, x, beta, alpha, lam)
+    xo = gg_synth.to_oracle(x)
+    ref_pen, ref_g = o.penalty_grad(xo, beta, alpha, lam)
+    worst = assert_grad_close(g, ref_g)
+    assert worst <= 4
+    if math.isfinite(ref_pen) and ref_pen < 1e300:
+        assert_rel(pen, ref_pen, REL_PENALTY, "penalty")
+
+
+def test_penalty_grad_misaligned_bf16_out_mean_and_accumulate(ctx):
+    from paper_2506_00486_b200 import Segments, GG_MEAN
+    rng = np.random.default_rng(9)
+    n = TILE + 301
+    x = gg_synth.gg_host(rng, 1.3, 0.02, n, torch.bfloat16)
+    xo = gg_synth.to_oracle(x)
+    # misaligned input and output, fp32 gradient
+    pen, g = penalty_case(ctx, x, 1.3, 0.0141, 1e-4, misalign=True)
+    ref_pen, ref_g = o.penalty_grad(xo, 1.3, 0.0141, 1e-4)
+    assert_grad_close(g, ref_g)
+    assert_rel(pen, ref_pen, REL_PENALTY, "penalty")
+    # mean reduction = lambda / len
+    pen, g = penalty_case(ctx, x, 1.3, 0.0141, 1e-4, reduction=GG_MEAN)
+    ref_pen, ref_g = o.penalty_grad(xo, 1.3, 0.0141, 1e-4 / n)
+    assert_grad_close(g, ref_g)
+    assert_rel(pen, ref_pen, REL_PENALTY, "penalty(mean)")
+    # bf16 gradient output: the fp32 result rounded once more (within one bf16 ulp of the oracle)
+    pen, g = penalty_case(ctx, x, 1.3, 0.0141, 1e-4, grad_dtype=torch.bfloat16)
+    ref_bits = o.round_to_bf16_bits(ref_g).astype(np.int64)
+    got_bits = torch.from_numpy(g).to(torch.bfloat16).view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+    assert np.abs((ref_bits & 0x7FFF) - (got_bits & 0x7FFF)).max() <= 1
+    assert ((ref_bits >> 15) == (got_bits >> 15)).all()
+    # accumulate: grad += g
+    xd = dev(x)
+    gd = torch.full((n,), 0.25, dtype=torch.float32, device="cuda:0")
+    bt = torch.tensor([1.3], dtype=torch.float64, device="cuda:0")
+    at = torch.tensor([0.0141], dtype=torch.float64, device="cuda:0")
+    ctx.gg_penalty_grad(Segments([xd]), bt, at, 1e-4, grad=Segments([gd]), accumulate=True)
+    torch.cuda.synchronize()
+    expect = (np.float32(0.25) + ref_g.astype(np.float32)).astype(np.float32)
+    assert np.abs(gd.cpu().numpy() - expect).max() <= 4 * np.spacing(np.float32(0.25))
+
+
+def test_penalty_grad_degenerate_parameters_and_zero_lambda(ctx):
+    x = torch.tensor([1.0, -2.0, 0.0, 3.0])
+    for beta, alpha, lam in ((0.0, 0.0, 1e-4), (1.0, 0.02, 0.0)):
+        pen, g = penalty_case(ctx, x, beta, alpha, lam)
+        assert pen == 0.0 and not g.any()
+    # negative lambda flips the sign
+    pen, g = penalty_case(ctx, x, 1.5, 0.5, -1e-3)
+    ref_pen, ref_g = o.penalty_grad(x.numpy(), 1.5, 0.5, -1e-3)
+    assert_grad_close(g, ref_g)
+    assert_rel(pen, ref_pen, REL_PENALTY, "penalty")
+
+
+# --------------------------------------------------------------------------------- gg_rate_hist
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("step", [1e-3, 0.01, 2.0 ** -10])
+def test_rate_hist_parity(ctx, dtype, step):
+    xs = make_segments(dtype, seed=5)
+    xd = [dev(x) for x in xs]
+    steps = torch.tensor([step * (1 + 0.37 * s) for s in range(len(xs))], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_rate_hist(xd, steps)
+    torch.cuda.synchronize()
+    hist = out["hist"].cpu().numpy()
+    for s, x in enumerate(xs):
+        ref, cl = o.quantise_hist(gg_synth.to_oracle(x), steps[s].item())
+        np.testing.assert_array_equal(hist[s], ref.astype(np.int64))
+        np.testing.assert_array_equal(out["clamped"][s].cpu().numpy(), cl.astype(np.int64))
+        assert abs(out["entropy_bits"][s].item() - o.entropy_bits(ref)) <= ABS_ENTROPY
+
+
+def test_rate_hist_shared_histogram_clamp_window_and_specials(ctx):
+    """Several segments into one table; narrow clamp; symbols outside the on-chip window;
+    inf / nan entries; accumulation across calls."""
+    rng = np.random.default_rng(6)
+    xs = [gg_synth.gg_host(rng, 0.8, 1.0, 40000, torch.bfloat16) for _ in range(3)]
+    xs[1][:6] = torch.tensor([float("inf"), float("-inf"), float("nan"), 1e30, -1e30, 0.0]).to(torch.bfloat16)
+    xs[2] = gg_synth.add_outliers_host(rng, xs[2], 0.01, 25.0)      # symbols +-2500: outside the window
+    xd = [dev(x) for x in xs]
+    steps = torch.tensor([0.01, 0.01, 0.01], dtype=torch.float32, device="cuda:0")
+    for qmin, qmax in ((-32768, 32767), (-100, 50), (3, 9), (-4000, -2100)):
+        out = ctx.gg_rate_hist(xd, steps, hist_id=[0, 1, 0], n_hist=2, qmin=qmin, qmax=qmax)
+        torch.cuda.synchronize()
+        nb = qmax - qmin + 1
+        ref = np.zeros((2, nb), dtype=np.uint64)
+        cl = np.zeros((2, 2), dtype=np.uint64)
+        for s, h in enumerate([0, 1, 0]):
+            o.quantise_hist(gg_synth.to_oracle(xs[s]), 0.01, qmin, qmax, hist=ref[h], clamped=cl[h])
+        np.testing.assert_array_equal(out["hist"].cpu().numpy(), ref.astype(np.int64))
+        np.testing.assert_array_equal(out["clamped"].cpu().numpy(), cl.astype(np.int64))
+        for h in range(2):
+            assert abs(out["entropy_bits"][h].item() - o.entropy_bits(ref[h])) <= ABS_ENTROPY
+    # accumulate on top of an existing table
+    out2 = ctx.gg_rate_hist(xd, steps, hist_id=[0, 1, 0], n_hist=2, qmin=qmin, qmax=qmax,
+                            hist=out["hist"].clone(), accumulate=True)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out2["hist"].cpu().numpy(), 2 * ref.astype(np.int64))
+
+
+def test_rate_hist_all_equal_input(ctx):
+    """Worst case for the shared-memory atomics: every element lands in one bin."""
+    x = torch.full((3 * TILE + 17,), 0.0123, dtype=torch.float32)
+    out = ctx.gg_rate_hist([dev(x)], torch.tensor([1e-3], dtype=torch.float32, device="cuda:0"))
+    torch.cuda.synchronize()
+    ref, _ = o.quantise_hist(x.numpy(), 1e-3)
+    np.testing.assert_array_equal(out["hist"][0].cpu().numpy(), ref.astype(np.int64))
+    assert out["entropy_bits"][0].item() == 0.0
+
+
+# ------------------------------------------------------------------------------------ gg_sample
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_sample_parity(ctx, dtype):
+    betas = [0.1, 0.5, 0.8, 1.0, 1.3, 2.0, 3.0]
+    lens = [5000, TILE + 3, 1, 40000, 2 * TILE, 777, 12345]
+    alphas = [gg_synth.alpha_for_std(0.02, b) for b in betas]
+    outs = [torch.empty(n, dtype=dtype, device="cuda:0") for n in lens]
+    att = ctx.gg_sample(outs, betas, alphas, seed=0x1234567887654321, tensor_id0=40)
+    torch.cuda.synchronize()
+    total = mism = 0
+    for s, (b, a, n) in enumerate(zip(betas, alphas, lens)):
+        ref, ratt = o.sample(b, a, 0x1234567887654321, 40 + s, n, want_attempts=True)
+        assert att[s].item() == int(ratt.max())
+        got = outs[s].cpu()
+        if dtype == torch.float32:
+            refr = ref.astype(np.float32)
+            gotn = got.numpy()
+            diff = np.abs(refr.view(np.int32).astype(np.int64) - gotn.view(np.int32).astype(np.int64))
+        else:
+            refr = o.round_to_bf16_bits(ref).astype(np.int64)
+            gotn = got.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+            diff = np.abs(refr - gotn)
+        assert diff.max() <= 1          # never more than one unit of the storage type
+        np.testing.assert_array_equal(np.signbit(ref), np.signbit(got.float().numpy()))
+        total += n
+        mism += int((diff != 0).sum())
+    # libm and device math may differ in the last fp64 bit: a value that sits on a rounding
+    # boundary of the storage type can land on either side, which is rare
+    assert mism <= max(1, total // 100_000)
+
+
+def test_sample_then_fit_recovers_parameters(ctx):
+    """GG initialisation of scaled Qwen-shaped matrices, then the fit: the recovered shape and
+    scale agree with the nominal ones statistically and with the oracle's fit of the same data."""
+    shapes = gg_synth.scaled_shapes(gg_synth.qwen05b_shapes(), 4)[:9]
+    beta = 1.3
+    alpha = gg_synth.alpha_for_std(0.02, beta)
+    outs = [torch.empty(r * c, dtype=torch.bfloat16, device="cuda:0") for _, r, c in shapes]
+    ctx.gg_sample(outs, [beta] * len(outs), [alpha] * len(outs), seed=1, tensor_id0=0)
+    fit = ctx.gg_fit(outs)
+    torch.cuda.synchronize()
+    for s, t in enumerate(outs):
+        n = t.numel()
+        bh, ah = fit["beta"][s].item(), fit["alpha"][s].item()
+        assert abs(bh - beta) < 5 * 2.5 / math.sqrt(n) + 0.01
+        assert abs(ah / alpha - 1) < 5 * 2.5 / math.sqrt(n) + 0.01
+        b, a, *_ = o.fit(gg_synth.to_oracle(t))
+        assert_rel(bh, b, REL_FIT, "beta")
+        assert_rel(ah, a, REL_FIT, "alpha")
+
+
+# ------------------------------------------------------------------------------------- gg_fused
+def check_fused(out, xs, grads, lam, hist_ids, n_hist, steps=None, step_scale=None, given=None,
+                qmin=-32768, qmax=32767, mean=False):
+    nb = qmax - qmin + 1
+    ref_hist = np.zeros((n_hist, nb), dtype=np.uint64)
+    ref_cl = np.zeros((n_hist, 2), dtype=np.uint64)
+    used_steps = out["step"].cpu().numpy()
+    for s, x in enumerate(xs):
+        xo = gg_synth.to_oracle(x)
+        b, a, s1, s2, n, fl = o.fit(xo)
+        bg, ag = out["beta"][s].item(), out["alpha"][s].item()
+        assert (out["flags"][s].item() & 15) == fl
+        if fl & o.FLAG_DEGENERATE:
+            assert bg == 0.0 and ag == 0.0
+        else:
+            assert_rel(bg, b, REL_FIT, f"beta[{s}]")
+            assert_rel(ag, a, REL_FIT, f"alpha[{s}]")
+        # parameters the gradient used: the GPU's own fit, or the given ones
+        bu, au = (bg, ag) if given is None else given[s]
+        lam_s = lam / max(n, 1) if mean else lam
+        pen, g = o.penalty_grad(xo, bu, au, lam_s)
+        if grads is not None:
+            assert_grad_close(grads[s].float().cpu().numpy(), g)
+        if pen > 0:
+            assert_rel(out["penalty"][s].item(), pen, REL_PENALTY, f"penalty[{s}]")
+        else:
+            assert out["penalty"][s].item() == 0.0
+        if step_scale is not None:
+            assert used_steps[s] == np.float32(ag * step_scale)
+        o.quantise_hist(xo, used_steps[s], qmin, qmax, hist=ref_hist[hist_ids[s]], clamped=ref_cl[hist_ids[s]])
+    np.testing.assert_array_equal(out["hist"].cpu().numpy(), ref_hist.astype(np.int64))
+    np.testing.assert_array_equal(out["clamped"].cpu().numpy(), ref_cl.astype(np.int64))
+    for h in range(n_hist):
+        assert abs(out["entropy_bits"][h].item() - o.entropy_bits(ref_hist[h])) <= ABS_ENTROPY
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fused_fitted_parity(ctx, dtype):
+    from paper_2506_00486_b200 import Segments
+    xs = make_segments(dtype, seed=7) + [torch.zeros(50, dtype=dtype), torch.zeros(0, dtype=dtype)]
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    n = len(xs)
+    steps = torch.full((n,), 2.0 ** -10, dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps)
+    torch.cuda.synchronize()
+    check_fused(out, xs, gd, 1e-4, list(range(n)), n)
+
+
+def test_fused_step_from_alpha_and_shared_histograms(ctx):
+    from paper_2506_00486_b200 import Segments, GG_MEAN
+    xs = make_segments(torch.float32, seed=8)
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    hid = [0, 1, 1, 2, 0, 2, 1, 0]
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=3e-3, step_scale=1 / 16, hist_id=hid, n_hist=3,
+                       reduction=GG_MEAN)
+    torch.cuda.synchronize()
+    check_fused(out, xs, gd, 3e-3, hid, 3, step_scale=1 / 16, mean=True)
+
+
+def test_fused_given_parameters_single_sweep(ctx):
+    """Lagged mode: the gradient uses caller parameters while the same sweep produces the new fit."""
+    from paper_2506_00486_b200 import Segments, GG_PARAMS_GIVEN
+    xs = make_segments(torch.bfloat16, seed=10)
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    n = len(xs)
+    given = [(0.5 + 0.2 * s, 0.01 * (s + 1)) for s in range(n)]
+    bi = torch.tensor([g[0] for g in given], dtype=torch.float64, device="cuda:0")
+    ai = torch.tensor([g[1] for g in given], dtype=torch.float64, device="cuda:0")
+    steps = torch.full((n,), 0.01, dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps, param_mode=GG_PARAMS_GIVEN,
+                       beta_in=bi, alpha_in=ai, qmin=-64, qmax=63)
+    torch.cuda.synchronize()
+    check_fused(out, xs, gd, 1e-4, list(range(n)), n, given=given, qmin=-64, qmax=63)
+    assert (out["flags"].cpu().numpy() & 16).any()       # the narrow clamp was reported
+
+
+def test_config1_single_fp32_tensor(ctx):
+    """1024x1024 fp32 from GG(beta=1, alpha=0.02): fit, penalty gradient (lambda 1e-4) and
+    histogram at step 1e-3 with symbols clamped to int16, as separate calls and fused."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c1()
+    x = w["tensors"][0]
+    xo = gg_synth.to_oracle(x)
+    xd = dev(x)
+    fit = ctx.gg_fit([xd])
+    g = torch.empty_like(xd)
+    pen = ctx.gg_penalty_grad(Segments([xd]), fit["beta"], fit["alpha"], w["lam"], grad=Segments([g]))
+    steps = torch.tensor(w["steps"], dtype=torch.float32, device="cuda:0")
+    rh = ctx.gg_rate_hist([xd], steps)
+    torch.cuda.synchronize()
+    b, a, *_ = o.fit(xo)
+    bg, ag = fit["beta"][0].item(), fit["alpha"][0].item()
+    assert_rel(bg, b, REL_FIT, "beta")
+    assert_rel(ag, a, REL_FIT, "alpha")
+    assert abs(bg - 1.0) < 0.01 and abs(ag / 0.02 - 1) < 0.01      # the generating parameters
+    rp, rg = o.penalty_grad(xo, bg, ag, w["lam"])
+    assert_grad_close(g.cpu().numpy(), rg)
+    assert_rel(pen[0].item(), rp, REL_PENALTY, "penalty")
+    ref, cl = o.quantise_hist(xo, np.float32(1e-3))
+    np.testing.assert_array_equal(rh["hist"][0].cpu().numpy(), ref.astype(np.int64))
+    assert abs(rh["entropy_bits"][0].item() - o.entropy_bits(ref)) <= ABS_ENTROPY
+    g2 = torch.empty_like(xd)
+    out = ctx.gg_fused(Segments([xd]), grad=Segments([g2]), lam=w["lam"], step=steps)
+    torch.cuda.synchronize()
+    check_fused(out, [x], [g2], w["lam"], [0], 1)
+    assert torch.equal(g, g2)
+
+
+def test_config3_activation_rows_scaled(ctx):
+    """Per-token segments of a bf16 activation tensor with outliers, one shared histogram
+    (a [2, 96, 4096] slice of the [8, 2048, 4096] workload shape)."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c3(batch=2, seq=96)
+    x = w["tensor"]
+    xd = dev(x)
+    gd = torch.empty(x.shape, dtype=torch.float32, device="cuda:0")
+    steps = torch.full((w["n_seg"],), w["step"], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments.rows(xd), grad=Segments.rows(gd), lam=w["lam"], step=steps,
+                       hist_id=w["hist_id"], n_hist=1)
+    torch.cuda.synchronize()
+    check_fused(out, list(x), list(gd), w["lam"], w["hist_id"], 1)
+
+
+def test_config4_gradient_buckets_scaled(ctx):
+    """fp32 buckets from GG(beta=0.5), per-bucket alpha log-uniform in [1e-6, 1e-3], step alpha/16
+    (8 buckets of 250 000 instead of 25 000 000 elements)."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c4(bucket=250_000)
+    xs = w["tensors"]
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty_like(x) for x in xd]
+    steps = torch.tensor(w["steps"], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=w["lam"], step=steps)
+    torch.cuda.synchronize()
+    check_fused(out, xs, gd, w["lam"], w["hist_id"], w["n_hist"])
+    for s in range(len(xs)):
+        assert abs(out["beta"][s].item() - 0.5) < 0.02
+
+
+def test_config5_weight_sweep_scaled(ctx):
+    """The Llama-7B-shaped bf16 sweep with every matrix dimension divided by 16: 226 segments in one
+    segmented launch, one histogram per tensor, step 2^-10."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c5_host(divisor=16)
+    xs = w["tensors"]
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    steps = torch.tensor(w["steps"], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=w["lam"], step=steps)
+    torch.cuda.synchronize()
+    check_fused(out, xs, gd, w["lam"], w["hist_id"], w["n_hist"])
