@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the fused GG pass (fit + penalty gradient + symbol histogram + entropy).
+
+One step = one gg_fused call (parameters fitted in the same call) over the whole Llama-7B-shaped
+bf16 weight sweep: 226 tensors, 6.74e9 elements, each GG with its own shape in [0.6, 1.6] and
+standard deviation 0.02; fp32 gradients; one 65536-bin histogram per tensor at step 2^-10.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused GG fit+penalty-grad+histogram pass throughput (algorithmic bytes: input read once + gradient written once)"
+UNIT = "GB/s"
+LAM = 1e-4
+STEP = 2.0 ** -10
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--divisor", type=int, default=1,
+                    help="divide every matrix dimension of the sweep (debugging; 1 = the full workload)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"])
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy kernel)"
+    except Exception:
+        return 6650.0, "fallback (earlier copy measurement on this pool)"
+
+
+def traffic_per_element():
+    """DRAM bytes per element of the second-sweep kernel from the committed ncu capture, if any."""
+    path = os.path.join(ROOT, "profiles", "tail_sweep_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, power, reasons = [], [], [], set()
+        for line in self.file:
+            p = [v.strip() for v in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2])); power.append(float(p[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            # "under load": samples in the upper half of the power range seen
+            lim = (max(power) + min(power)) / 2
+            load = sorted(s for s, w in zip(sm, power) if w >= lim) or sorted(sm)
+            out.update(sm_mhz=load[len(load) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+# ------------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(divisor):
+    """A bounded sample of the workload for the CPU oracle: the first attention matrix of the sweep
+    (4096 x 4096 at full size), generated on the host with the same recipe."""
+    import numpy as np
+    import torch
+    import gg_synth
+    shapes, betas, alphas = gg_synth.workload_c5_params(
+        gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), divisor) if divisor > 1 else None)
+    rng = np.random.default_rng(4)
+    xs = []
+    for i in range(1, 8):        # layer 0: q, k, v, o, gate, up, down
+        _, r, c = shapes[i]
+        xs.append(gg_synth.to_oracle(gg_synth.gg_host(rng, betas[i], alphas[i], r * c, torch.bfloat16)))
+    n = sum(x.size for x in xs)
+    return xs, f"layer 0 of the sweep (7 of 226 bf16 matrices, {n:.3e} of 6.74e9 elements)"
+
+
+def oracle_step(xs):
+    """The whole pass, tensor by tensor, with the oracle as it stands."""
+    from oracle import gg_oracle as o
+    acc = 0.0
+    for x in xs:
+        b, a, *_ = o.fit(x)
+        pen, g = o.penalty_grad(x, b, a, LAM)
+        hist, _ = o.quantise_hist(x, STEP)
+        acc += o.entropy_bits(hist) + pen
+    return acc
+
+
+def time_oracle(xs, steps, warmup):
+    for _ in range(warmup):
+        oracle_step(xs)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(xs)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    alg = sum(x.size for x in xs) * (2 + 4)
+    return alg / dt / 1e9, dt
+
+
+def omp_threads():
+    v = os.environ.get("OMP_NUM_THREADS")
+    return int(v) if v and v.isdigit() else (os.cpu_count() or 1)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import gg_oracle as o
+    o.build()
+    x, what = oracle_sample(args.divisor)
+    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    gbs, dt = time_oracle(x, steps, warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama7b_weight_sweep_bf16 (oracle on a bounded sample)", "sample": what},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "sample": what},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import gg_synth
+    from paper_2506_00486_b200 import Context, Segments
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- workload: every rank holds the whole sweep (segments are independent: weak scaling)
+    shapes = gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), args.divisor) if args.divisor > 1 else None
+    w = gg_synth.workload_c5_device(dev, torch.bfloat16, shapes=shapes, seed=4 + rank)
+    flat, offs, lens = w["flat"], w["offsets"], w["lens"]
+    n_seg, n_elem = len(lens), int(sum(lens))
+    gdtype = torch.float32 if args.grad_dtype == "f32" else torch.bfloat16
+    gflat = torch.empty(flat.numel(), dtype=gdtype, device=dev)
+    segs = Segments.slices(flat, offs, lens)
+    gsegs = Segments.slices(gflat, offs, lens)
+    steps_t = torch.full((n_seg,), STEP, dtype=torch.float32, device=dev)
+    ctx = Context(local)
+    run = ctx.make_fused(segs, grad=gsegs, lam=LAM, step=steps_t)
+    in_bytes = n_elem * 2
+    g_bytes = n_elem * gflat.element_size()
+    alg_bytes = in_bytes + g_bytes
+
+    for _ in range(args.warmup):
+        run()
+    barrier()
+    ctx.timing_enable(True)
+    ctx.timing_read()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = ctx.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        run()
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1) / max(args.steps, 1)
+    launches = ctx.launch_count - launches0
+    ms_first, n_first, ms_tail, n_tail = ctx.timing_read()
+    ctx.timing_enable(False)
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = t.item()
+    value = world * alg_bytes / (ms * 1e-3) / 1e9
+
+    # ---- a quick self-check of the timed outputs (host logic only: no oracle here)
+    out = run.outputs
+    torch.cuda.synchronize()
+    beta_err = max(abs(out["beta"][s].item() - w["beta_true"][s]) for s in range(n_seg))
+    total_counts = int(out["hist"].sum().item())
+
+    # ---- roofline of the dominant kernel (the second sweep: read x, write the gradient, histogram)
+    peak, peak_src = measured_peak()
+    tail_ms = ms_tail / max(n_tail, 1)
+    first_ms = ms_first / max(n_first, 1)
+    achieved = alg_bytes / (tail_ms * 1e-3) / 1e9 if tail_ms > 0 else None
+    tr = traffic_per_element()
+    traffic = None
+    if tr and tr.get("grad_dtype") == args.grad_dtype:
+        traffic = tr["dram_bytes_per_element"] * n_elem
+    roofline = {"bound": "hbm", "kernel": "stream_kernel<bf16, %s, grad|hist> (second sweep)" % args.grad_dtype,
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
+                "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
+                "traffic": traffic, "peak_source": peak_src, "ms_per_launch": tail_ms,
+                "algorithmic_bytes_per_launch": alg_bytes,
+                "first_sweep": {"ms_per_launch": first_ms,
+                                "achieved": in_bytes / (first_ms * 1e-3) / 1e9 if first_ms > 0 else None,
+                                "frac": in_bytes / (first_ms * 1e-3) / 1e9 / peak if first_ms > 0 else None}}
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, ctx, w, world, dev, gdtype, in_bytes, g_bytes, alg_bytes, barrier)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import gg_oracle as o
+        o.build()
+        x, what = oracle_sample(args.divisor)
+        gbs, dt = time_oracle(x, 1, 0)
+        cpu_baseline = {"value": gbs, "unit": UNIT, "cores": omp_threads(), "kind": "oracle",
+                        "sample": what + f"; one pass, {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "llama7b_weight_sweep_bf16" + ("" if args.divisor == 1 else f"/div{args.divisor}"),
+                       "segments": n_seg, "elements": n_elem, "in_dtype": "bf16", "grad_dtype": args.grad_dtype,
+                       "histograms": n_seg, "bins": 65536, "step": STEP, "lambda": LAM, "params": "fitted in the same call",
+                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world} (segments are independent)"},
+            "fraction_of_hbm_peak": {"of_measured_copy_peak": value / world / peak, "of_nominal_8TBs": value / world / 8000.0},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks,
+            "check": {"max_abs_beta_error_vs_generating": beta_err, "histogram_total": total_counts,
+                      "elements": n_elem},
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, ctx, w, world, dev, gdtype, in_bytes, g_bytes, alg_bytes, barrier):
+    import psutil
+    import torch
+    from paper_2506_00486_b200 import Segments
+    local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+    need = in_bytes + g_bytes
+    avail = psutil.virtual_memory().available / max(local_world, 1)
+    if need * 1.25 > avail:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": g_bytes,
+                "skipped": f"host memory: need {need / 1e9:.0f} GB pinned per rank, {avail / 1e9:.0f} GB available"}
+    flat, offs, lens = w["flat"], w["offsets"], w["lens"]
+    n_seg = len(lens)
+    hx = torch.empty(flat.numel(), dtype=flat.dtype, pin_memory=True)
+    hx.copy_(flat)
+    hg = torch.empty(flat.numel(), dtype=gdtype, pin_memory=True)
+    hstep = torch.full((n_seg,), STEP, dtype=torch.float32)
+    runh = ctx.make_fused_host(Segments.slices(hx, offs, lens), grad=Segments.slices(hg, offs, lens),
+                               lam=LAM, step=hstep)
+    runh()                                      # warm-up: allocates the staging buffers and plans
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        runh()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / max(args.e2e_steps, 1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = t.item()
+    out = runh.outputs
+    d2h = g_bytes + out["hist"].numel() * 8 + n_seg * (8 * 6 + 4 + 8 + 16)
+    return {"value": world * alg_bytes / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3, "steps": args.e2e_steps,
+            "h2d_bytes_per_step": in_bytes + n_seg * 4, "d2h_bytes_per_step": int(d2h),
+            "api": "gg_fused_host (pinned host tensors in, gradients + fit + histograms back on the host)"}
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

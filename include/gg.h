@@ -203,6 +203,14 @@ typedef struct {
  * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep). */
 gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *args, void *stream);
 
+/* Optional device timing of the sweeps inside gg_fused (no counterpart in the paper: measurement
+ * support).  While enabled, gg_fused records a CUDA event pair on the caller's stream around its
+ * first sweep (moments, or the single combined sweep of GG_PARAMS_GIVEN) and around its second
+ * sweep (gradient + histogram).  gg_timing_read waits for the recorded events, returns the summed
+ * milliseconds and the number of launches of each kind since the last read, and forgets them. */
+gg_status gg_timing_enable(gg_ctx *ctx, int enable);
+gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double *ms_tail, int64_t *n_tail);
+
 /* The same pass for data that lives in HOST memory: every pointer of `args` that gg_fused documents
  * as device memory (segment data, fit outputs, gradient segments, step, histogram, entropy, ...) is
  * here a host pointer.  The library stages segments through device buffers of its own in chunks of

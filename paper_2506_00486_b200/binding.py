@@ -79,8 +79,11 @@ def lib():
         L.gg_sample.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, u64, u32, _P, _P]
         L.gg_fused.argtypes = [_P, ctypes.POINTER(FusedArgs), _P]
         L.gg_fused_host.argtypes = [_P, ctypes.POINTER(FusedArgs), i64]
+        L.gg_timing_enable.argtypes = [_P, ctypes.c_int]
+        L.gg_timing_read.argtypes = [_P, ctypes.POINTER(d), ctypes.POINTER(i64), ctypes.POINTER(d),
+                                     ctypes.POINTER(i64)]
         for name in ("gg_create", "gg_destroy", "gg_fit", "gg_penalty_grad", "gg_rate_hist", "gg_sample",
-                     "gg_fused", "gg_fused_host"):
+                     "gg_fused", "gg_fused_host", "gg_timing_enable", "gg_timing_read"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -346,3 +349,70 @@ class Context:
     def gg_fused(self, segs, **kw):
         """One-shot form of make_fused(...)()."""
         return self.make_fused(segs, **kw)()
+
+    # ----------------------------------------------------------- gg_fused_host
+    def make_fused_host(self, segs, grad=None, lam=1e-4, reduction=GG_SUM, step=None, step_scale=None,
+                        hist_id=None, n_hist=None, qmin=-32768, qmax=32767, want_hist=True,
+                        chunk_bytes=0, pin=True):
+        """The fused pass on HOST tensors (CPU torch tensors; pinned ones copy asynchronously).
+
+        Allocates the host outputs once (pinned if `pin`) and returns a callable; each call copies
+        the inputs to the device in chunks, runs the pass and returns with all results on the host."""
+        segs = _as_segments(segs)
+        n = len(segs)
+        gsegs = None if grad is None else _as_segments(grad)
+
+        def host(n_, dtype):
+            return torch.empty(n_, dtype=dtype, pin_memory=pin)
+
+        out = dict(beta=host(n, torch.float64), alpha=host(n, torch.float64), sum_abs=host(n, torch.float64),
+                   sum_sq=host(n, torch.float64), count=host(n, torch.int64), flags=host(n, torch.int32),
+                   penalty=host(n, torch.float64))
+        a = FusedArgs()
+        keep = [segs, gsegs, step]
+        a.segs, a.n_seg, a.in_dtype = segs.ptr, n, segs.code
+        for k in ("beta", "alpha", "sum_abs", "sum_sq", "count", "flags", "penalty"):
+            setattr(a, k, _ptr(out[k]))
+        a.param_mode, a.lam, a.reduction = GG_PARAMS_FITTED, float(lam), int(reduction)
+        a.grad = None if gsegs is None else gsegs.ptr
+        a.grad_dtype = GG_F32 if gsegs is None else gsegs.code
+        if want_hist:
+            n_hist = n if n_hist is None else int(n_hist)
+            nb = qmax - qmin + 1
+            out["hist"] = torch.empty((n_hist, nb), dtype=torch.int64, pin_memory=pin)
+            out["entropy_bits"] = host(n_hist, torch.float64)
+            out["clamped"] = torch.empty((n_hist, 2), dtype=torch.int64, pin_memory=pin)
+            if step is not None:
+                a.step_mode, a.step = GG_STEP_GIVEN, _ptr(step)
+                out["step"] = step
+            else:
+                out["step"] = host(n, torch.float32)
+                a.step_mode, a.step_scale, a.step_out = GG_STEP_FROM_ALPHA, float(step_scale), _ptr(out["step"])
+            hid = None if hist_id is None else np.ascontiguousarray(hist_id, dtype=np.int32)
+            keep.append(hid)
+            a.hist_id = None if hid is None else hid.ctypes.data
+            a.n_hist, a.qmin, a.qmax = n_hist, int(qmin), int(qmax)
+            a.hist, a.entropy_bits, a.clamped_lo_hi = _ptr(out["hist"]), _ptr(out["entropy_bits"]), _ptr(out["clamped"])
+
+        def run():
+            self._check(lib().gg_fused_host(self._h, ctypes.byref(a), int(chunk_bytes)))
+            return out
+
+        run.outputs = out
+        run._keep = keep
+        return run
+
+    def gg_fused_host(self, segs, **kw):
+        return self.make_fused_host(segs, **kw)()
+
+    # ------------------------------------------------------------------ timing
+    def timing_enable(self, on=True):
+        self._check(lib().gg_timing_enable(self._h, int(bool(on))))
+
+    def timing_read(self):
+        """(ms of first sweeps, their count, ms of second sweeps, their count) since the last read."""
+        m0, m1 = ctypes.c_double(), ctypes.c_double()
+        n0, n1 = ctypes.c_int64(), ctypes.c_int64()
+        self._check(lib().gg_timing_read(self._h, ctypes.byref(m0), ctypes.byref(n0), ctypes.byref(m1),
+                                         ctypes.byref(n1)))
+        return m0.value, n0.value, m1.value, n1.value

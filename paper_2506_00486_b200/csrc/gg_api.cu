@@ -15,8 +15,8 @@ using namespace gg;
 
 namespace {
 
-constexpr int kMaxPlans = 16;
-constexpr int64_t kDefaultChunkBytes = 512ll << 20;
+constexpr int kMaxPlans = 64;
+constexpr int64_t kDefaultChunkBytes = 1ll << 30;
 
 // A plan is everything that depends only on the layout of a call: segment addresses and lengths,
 // gradient addresses, histogram ids.  It owns the device tables and the per-tile scratch.
@@ -38,6 +38,9 @@ struct gg_ctx {
     uint64_t clock = 0;
     int64_t launches = 0;
     std::string cuda_error;
+    // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
+    bool timing = false;
+    std::vector<cudaEvent_t> ev_first, ev_tail;   // begin, end, begin, end, ...
     // gg_fused_host staging (created on first use)
     struct HostSlot {
         gg_ctx *ctx = nullptr;
@@ -190,6 +193,27 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     return GG_OK;
 }
 
+// Brackets one launch with events when timing is on.
+struct SweepTimer {
+    gg_ctx *ctx; std::vector<cudaEvent_t> *list; cudaStream_t st; bool on;
+    SweepTimer(gg_ctx *c, std::vector<cudaEvent_t> *l, cudaStream_t s) : ctx(c), list(l), st(s), on(c->timing)
+    {
+        if (!on) return;
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+        cudaEventRecord(e, st);
+        list->push_back(e);
+    }
+    ~SweepTimer()
+    {
+        if (!on) return;
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) { cudaEventDestroy(list->back()); list->pop_back(); return; }
+        cudaEventRecord(e, st);
+        list->push_back(e);
+    }
+};
+
 gg_status check_grad(const gg_seg *segs, const gg_seg *grad, int32_t n_seg, int grad_dtype)
 {
     if (!grad) return GG_OK;
@@ -274,6 +298,8 @@ gg_status gg_destroy(gg_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     for (auto &p : ctx->plans) cudaFree(p->dev);
+    for (cudaEvent_t e : ctx->ev_first) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_tail) cudaEventDestroy(e);
     for (auto &sl : ctx->slot) {
         if (sl.ctx) gg_destroy(sl.ctx);
         if (sl.stream) cudaStreamDestroy(sl.stream);
@@ -406,6 +432,40 @@ gg_status gg_sample(gg_ctx *ctx, const gg_seg *out, int32_t n_seg, gg_dtype dtyp
     return GG_OK;
 }
 
+gg_status gg_timing_enable(gg_ctx *ctx, int enable)
+{
+    if (!ctx) return GG_ERR_INVALID_ARG;
+    ctx->timing = enable != 0;
+    return GG_OK;
+}
+
+gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double *ms_tail, int64_t *n_tail)
+{
+    if (!ctx) return GG_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    std::vector<cudaEvent_t> *lists[2] = {&ctx->ev_first, &ctx->ev_tail};
+    double ms[2] = {0.0, 0.0};
+    int64_t cnt[2] = {0, 0};
+    gg_status result = GG_OK;
+    for (int k = 0; k < 2; ++k) {
+        auto &l = *lists[k];
+        for (size_t i = 0; i + 1 < l.size(); i += 2) {
+            float t = 0.0f;
+            cudaError_t e = cudaEventSynchronize(l[i + 1]);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&t, l[i], l[i + 1]);
+            if (e != cudaSuccess) result = cuda_fail(ctx, e);
+            else { ms[k] += (double)t; cnt[k] += 1; }
+        }
+        for (cudaEvent_t e : l) cudaEventDestroy(e);
+        l.clear();
+    }
+    if (ms_first) *ms_first = ms[0];
+    if (n_first) *n_first = cnt[0];
+    if (ms_tail) *ms_tail = ms[1];
+    if (n_tail) *n_tail = cnt[1];
+    return result;
+}
+
 gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
 {
     if (!ctx || !a) return GG_ERR_INVALID_ARG;
@@ -461,12 +521,16 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         const double *beta_used;
         if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
-            GG_CUDA(ctx, launch_stream(kMoments, in_dt, g_dt, false, sa, cs));
+            {
+                SweepTimer tm(ctx, &ctx->ev_first, cs);
+                GG_CUDA(ctx, launch_stream(kMoments, in_dt, g_dt, false, sa, cs));
+            }
             GG_CUDA(ctx, launch_fit(fa, cs));
             ctx->launches += 1 + (p->n_tiles > 0);
             sa.beta = a->beta; sa.alpha = a->alpha;
             sa.step = fa.step_from_alpha ? a->step_out : a->step;
             if (tail_flags) {
+                SweepTimer tm(ctx, &ctx->ev_tail, cs);
                 GG_CUDA(ctx, launch_stream(tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
                 ctx->launches += p->n_tiles > 0;
             }
@@ -479,7 +543,10 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
                 GG_CUDA(ctx, cudaMemsetAsync(a->flags, 0, sizeof(uint32_t) * (size_t)n_seg, cs));
                 fa.keep_clamp_bit = 1;
             }
-            GG_CUDA(ctx, launch_stream(kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
+            {
+                SweepTimer tm(ctx, &ctx->ev_first, cs);
+                GG_CUDA(ctx, launch_stream(kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
+            }
             GG_CUDA(ctx, launch_fit(fa, cs));
             ctx->launches += 1 + (p->n_tiles > 0);
             beta_used = a->beta_in;
@@ -496,10 +563,201 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
     return GG_OK;
 }
 
+// Grows a device buffer (never shrinks).  Blocking; the caller has made sure nothing uses it.
+static gg_status grow(gg_ctx *ctx, void **buf, int64_t *have, int64_t need)
+{
+    if (need <= *have) return GG_OK;
+    if (*buf) { GG_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(*buf); *buf = nullptr; *have = 0; }
+    GG_CUDA(ctx, cudaMalloc(buf, (size_t)need));
+    *have = need;
+    return GG_OK;
+}
+
 gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes)
 {
-    (void)ctx; (void)a; (void)chunk_bytes;
-    return GG_ERR_UNIMPLEMENTED;
+    if (!ctx || !a) return GG_ERR_INVALID_ARG;
+    const int32_t n_seg = a->n_seg;
+    if (n_seg > 0 && (!a->beta || !a->alpha)) return GG_ERR_INVALID_ARG;
+    if (a->param_mode != GG_PARAMS_FITTED && a->param_mode != GG_PARAMS_GIVEN) return GG_ERR_INVALID_ARG;
+    if (a->param_mode == GG_PARAMS_GIVEN && n_seg > 0 && (!a->beta_in || !a->alpha_in)) return GG_ERR_INVALID_ARG;
+    if (a->step_mode != GG_STEP_GIVEN && a->step_mode != GG_STEP_FROM_ALPHA) return GG_ERR_INVALID_ARG;
+    const bool do_hist = a->hist != nullptr;
+    if (do_hist) {
+        if (a->step_mode == GG_STEP_FROM_ALPHA && (a->param_mode != GG_PARAMS_FITTED || !a->step_out))
+            return GG_ERR_INVALID_ARG;
+        if (a->step_mode == GG_STEP_GIVEN && n_seg > 0 && !a->step) return GG_ERR_INVALID_ARG;
+        gg_status hs = check_hist(n_seg, a->hist_id, a->n_hist, a->qmin, a->qmax);
+        if (hs != GG_OK) return hs;
+    }
+    gg_status st = check_segs(a->segs, n_seg, a->in_dtype);
+    if (st != GG_OK) return st;
+    st = check_grad(a->segs, a->grad, n_seg, a->grad_dtype);
+    if (st != GG_OK) return st;
+    if (chunk_bytes <= 0) chunk_bytes = kDefaultChunkBytes;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+
+    const size_t es = esize(a->in_dtype), gs = a->grad ? esize(a->grad_dtype) : 0;
+    // chunks of whole consecutive segments; each segment starts on a 256-byte boundary of the stage
+    struct Chunk { int32_t s0, s1; };
+    std::vector<Chunk> chunks;
+    std::vector<int64_t> in_off((size_t)n_seg), g_off((size_t)n_seg);
+    int64_t max_in = 0, max_g = 0;
+    for (int32_t s = 0; s < n_seg;) {
+        int64_t ib = 0, gb = 0;
+        int32_t e = s;
+        while (e < n_seg) {
+            const int64_t add = (int64_t)align_up((size_t)a->segs[e].len * es, 256);
+            if (e > s && ib + add > chunk_bytes) break;
+            in_off[(size_t)e] = ib; g_off[(size_t)e] = gb;
+            ib += add;
+            gb += (int64_t)align_up((size_t)a->segs[e].len * gs, 256);
+            ++e;
+        }
+        chunks.push_back({s, e});
+        if (ib > max_in) max_in = ib;
+        if (gb > max_g) max_g = gb;
+        s = e;
+    }
+
+    for (auto &sl : ctx->slot) {
+        if (!sl.ctx) { st = gg_create(&sl.ctx, ctx->device); if (st != GG_OK) return st; }
+        if (!sl.stream) GG_CUDA(ctx, cudaStreamCreateWithFlags(&sl.stream, cudaStreamNonBlocking));
+        st = grow(ctx, &sl.in, &sl.in_bytes, max_in > 0 ? max_in : 256);
+        if (st != GG_OK) return st;
+        if (a->grad) { st = grow(ctx, &sl.grad, &sl.grad_bytes, max_g > 0 ? max_g : 256); if (st != GG_OK) return st; }
+    }
+    // device block for per-segment results and histograms
+    const int64_t n_bins = do_hist ? (int64_t)a->qmax - a->qmin + 1 : 0;
+    const int32_t n_hist = do_hist ? a->n_hist : 0;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t nd = (size_t)n_seg;
+    const size_t o_beta = take(8 * nd), o_alpha = take(8 * nd), o_s1 = take(8 * nd), o_s2 = take(8 * nd);
+    const size_t o_cnt = take(8 * nd), o_flags = take(4 * nd), o_pen = take(8 * nd), o_step = take(4 * nd);
+    const size_t o_bin = take(8 * nd), o_ain = take(8 * nd);
+    const size_t o_hist = take(8 * (size_t)n_hist * (size_t)n_bins), o_ent = take(8 * (size_t)n_hist);
+    const size_t o_cl = take(16 * (size_t)n_hist);
+    st = grow(ctx, &ctx->host_dev, &ctx->host_dev_bytes, (int64_t)(off > 0 ? off : 256));
+    if (st != GG_OK) return st;
+    char *d = static_cast<char *>(ctx->host_dev);
+    cudaStream_t s0 = ctx->slot[0].stream, s1 = ctx->slot[1].stream;
+
+    // inputs that every chunk needs, and the histogram's starting state, on stream 0
+    if (a->param_mode == GG_PARAMS_GIVEN && n_seg > 0) {
+        GG_CUDA(ctx, cudaMemcpyAsync(d + o_bin, a->beta_in, 8 * nd, cudaMemcpyHostToDevice, s0));
+        GG_CUDA(ctx, cudaMemcpyAsync(d + o_ain, a->alpha_in, 8 * nd, cudaMemcpyHostToDevice, s0));
+    }
+    if (do_hist && a->step_mode == GG_STEP_GIVEN && n_seg > 0)
+        GG_CUDA(ctx, cudaMemcpyAsync(d + o_step, a->step, 4 * nd, cudaMemcpyHostToDevice, s0));
+    if (do_hist) {
+        const size_t hb = 8 * (size_t)n_hist * (size_t)n_bins;
+        if (a->accumulate_hist) {
+            GG_CUDA(ctx, cudaMemcpyAsync(d + o_hist, a->hist, hb, cudaMemcpyHostToDevice, s0));
+            if (a->clamped_lo_hi)
+                GG_CUDA(ctx, cudaMemcpyAsync(d + o_cl, a->clamped_lo_hi, 16 * (size_t)n_hist, cudaMemcpyHostToDevice, s0));
+            else
+                GG_CUDA(ctx, cudaMemsetAsync(d + o_cl, 0, 16 * (size_t)n_hist, s0));
+        } else {
+            GG_CUDA(ctx, cudaMemsetAsync(d + o_hist, 0, hb, s0));
+            GG_CUDA(ctx, cudaMemsetAsync(d + o_cl, 0, 16 * (size_t)n_hist, s0));
+        }
+    }
+    cudaEvent_t ready = nullptr, done1 = nullptr;
+    GG_CUDA(ctx, cudaEventCreateWithFlags(&ready, cudaEventDisableTiming));
+    GG_CUDA(ctx, cudaEventCreateWithFlags(&done1, cudaEventDisableTiming));
+    gg_status result = GG_OK;
+    cudaError_t ce = cudaEventRecord(ready, s0);
+    if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s1, ready, 0);
+    if (ce != cudaSuccess) result = cuda_fail(ctx, ce);
+
+    std::vector<gg_seg> dsegs, dgrad;
+    std::vector<int32_t> hid;
+    for (size_t c = 0; c < chunks.size() && result == GG_OK; ++c) {
+        auto &sl = ctx->slot[c & 1];
+        const int32_t b = chunks[c].s0, e = chunks[c].s1, m = e - b;
+        dsegs.resize((size_t)m); dgrad.resize((size_t)m); hid.resize((size_t)m);
+        for (int32_t s = b; s < e && result == GG_OK; ++s) {
+            char *din = static_cast<char *>(sl.in) + in_off[(size_t)s];
+            dsegs[(size_t)(s - b)] = gg_seg{din, a->segs[s].len};
+            if (a->segs[s].len > 0) {
+                ce = cudaMemcpyAsync(din, a->segs[s].ptr, (size_t)a->segs[s].len * es, cudaMemcpyHostToDevice, sl.stream);
+                if (ce != cudaSuccess) result = cuda_fail(ctx, ce);
+            }
+            if (a->grad) {
+                char *dg = static_cast<char *>(sl.grad) + g_off[(size_t)s];
+                dgrad[(size_t)(s - b)] = gg_seg{dg, a->segs[s].len};
+                if (a->accumulate_grad && a->segs[s].len > 0 && result == GG_OK) {
+                    ce = cudaMemcpyAsync(dg, a->grad[s].ptr, (size_t)a->segs[s].len * gs, cudaMemcpyHostToDevice, sl.stream);
+                    if (ce != cudaSuccess) result = cuda_fail(ctx, ce);
+                }
+            }
+            hid[(size_t)(s - b)] = a->hist_id ? a->hist_id[s] : s;
+        }
+        if (result != GG_OK) break;
+        gg_fused_args sub = *a;
+        sub.segs = dsegs.data(); sub.n_seg = m;
+        sub.beta = reinterpret_cast<double *>(d + o_beta) + b;
+        sub.alpha = reinterpret_cast<double *>(d + o_alpha) + b;
+        sub.sum_abs = reinterpret_cast<double *>(d + o_s1) + b;
+        sub.sum_sq = reinterpret_cast<double *>(d + o_s2) + b;
+        sub.count = reinterpret_cast<int64_t *>(d + o_cnt) + b;
+        sub.flags = reinterpret_cast<uint32_t *>(d + o_flags) + b;
+        sub.beta_in = reinterpret_cast<const double *>(d + o_bin) + b;
+        sub.alpha_in = reinterpret_cast<const double *>(d + o_ain) + b;
+        sub.grad = a->grad ? dgrad.data() : nullptr;
+        sub.penalty = a->penalty ? reinterpret_cast<double *>(d + o_pen) + b : nullptr;
+        sub.step = reinterpret_cast<const float *>(d + o_step) + b;
+        sub.step_out = reinterpret_cast<float *>(d + o_step) + b;
+        if (do_hist) {
+            sub.hist_id = hid.data();
+            sub.hist = reinterpret_cast<uint64_t *>(d + o_hist);
+            sub.accumulate_hist = 1;
+            sub.entropy_bits = nullptr;
+            sub.clamped_lo_hi = reinterpret_cast<uint64_t *>(d + o_cl);
+        }
+        const int64_t before = sl.ctx->launches;
+        result = gg_fused(sl.ctx, &sub, sl.stream);
+        ctx->launches += sl.ctx->launches - before;
+        if (result == GG_ERR_CUDA) ctx->cuda_error = sl.ctx->cuda_error;
+        for (int32_t s = b; s < e && result == GG_OK && a->grad; ++s) {
+            if (a->segs[s].len == 0) continue;
+            ce = cudaMemcpyAsync(a->grad[s].ptr, static_cast<char *>(sl.grad) + g_off[(size_t)s],
+                                 (size_t)a->segs[s].len * gs, cudaMemcpyDeviceToHost, sl.stream);
+            if (ce != cudaSuccess) result = cuda_fail(ctx, ce);
+        }
+    }
+    // join stream 1 into stream 0, finish the histogram statistics, bring the results back
+    if (result == GG_OK) {
+        ce = cudaEventRecord(done1, s1);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s0, done1, 0);
+        if (ce == cudaSuccess && do_hist && a->entropy_bits && n_hist > 0) {
+            ce = launch_entropy(reinterpret_cast<uint64_t *>(d + o_hist), n_hist, (int32_t)n_bins,
+                                reinterpret_cast<double *>(d + o_ent), s0);
+            ctx->launches += 1;
+        }
+        auto back = [&](void *host, size_t o, size_t bytes) {
+            if (ce == cudaSuccess && host && bytes) ce = cudaMemcpyAsync(host, d + o, bytes, cudaMemcpyDeviceToHost, s0);
+        };
+        back(a->beta, o_beta, 8 * nd); back(a->alpha, o_alpha, 8 * nd);
+        back(a->sum_abs, o_s1, 8 * nd); back(a->sum_sq, o_s2, 8 * nd);
+        back(a->count, o_cnt, 8 * nd); back(a->flags, o_flags, 4 * nd);
+        back(a->penalty, o_pen, 8 * nd);
+        if (do_hist) {
+            if (a->step_mode == GG_STEP_FROM_ALPHA) back(a->step_out, o_step, 4 * nd);
+            back(a->hist, o_hist, 8 * (size_t)n_hist * (size_t)n_bins);
+            back(a->entropy_bits, o_ent, 8 * (size_t)n_hist);
+            back(a->clamped_lo_hi, o_cl, 16 * (size_t)n_hist);
+        }
+        if (ce != cudaSuccess) result = cuda_fail(ctx, ce);
+    }
+    // always drain both streams before returning: host buffers are the caller's again
+    cudaError_t e0 = cudaStreamSynchronize(s0), e1 = cudaStreamSynchronize(s1);
+    cudaEventDestroy(ready);
+    cudaEventDestroy(done1);
+    if (result == GG_OK && e0 != cudaSuccess) result = cuda_fail(ctx, e0);
+    if (result == GG_OK && e1 != cudaSuccess) result = cuda_fail(ctx, e1);
+    return result;
 }
 
 }  // extern "C"

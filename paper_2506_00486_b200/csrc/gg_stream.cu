@@ -203,7 +203,18 @@ __device__ __forceinline__ void process(const float (&x)[KV], float (&g)[KV], Ac
     }
     // short fp32 runs, then fp64: the fp32 part adds at most KV roundings of 2^-24 each
     if constexpr (FLAGS & kMoments) { acc.s1 += (double)m1; acc.s2 += (double)m2; }
-    if constexpr (FLAGS & kGrad) acc.pen += (double)mp;
+    if constexpr (FLAGS & kGrad) {
+        if (mp <= FLT_MAX) {
+            acc.pen += (double)mp;
+        } else {   // a product or a gradient left the fp32 range (or is nan): redo this run in fp64
+            double dp = 0.0;
+            for (int e = 0; e < KV; ++e) {
+                const double ax = (double)fabsf(x[e]);
+                if (ax != 0.0 && gc.mode != 0) dp += ax * exp2(gc.L + gc.b * log2(ax));
+            }
+            acc.pen += dp;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------- the kernel
@@ -352,7 +363,7 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
         if constexpr (GRAD) {
             double rp = 0.0;
             for (int w = 0; w < kWarps; ++w) rp += shRed[2][w];
-            a.part.pen[t] = rp;
+            a.part.pen[t] = gc.sign_flip ? -rp : rp;   // the penalty carries lambda's sign
         }
     }
     if constexpr (HIST) {

@@ -169,6 +169,7 @@ def test_penalty_grad_misaligned_bf16_out_mean_and_accumulate(ctx):
     assert_rel(pen, ref_pen, REL_PENALTY, "penalty(mean)")
     # bf16 gradient output: the fp32 result rounded once more (within one bf16 ulp of the oracle)
     pen, g = penalty_case(ctx, x, 1.3, 0.0141, 1e-4, grad_dtype=torch.bfloat16)
+    ref_pen, ref_g = o.penalty_grad(xo, 1.3, 0.0141, 1e-4)
     ref_bits = o.round_to_bf16_bits(ref_g).astype(np.int64)
     got_bits = torch.from_numpy(g).to(torch.bfloat16).view(torch.int16).numpy().astype(np.int64) & 0xFFFF
     assert np.abs((ref_bits & 0x7FFF) - (got_bits & 0x7FFF)).max() <= 1
