@@ -34,6 +34,7 @@ struct Plan {
 
 struct gg_ctx {
     int device = 0;
+    int sm_count = 148;
     std::vector<std::unique_ptr<Plan>> plans;
     uint64_t clock = 0;
     int64_t launches = 0;
@@ -156,6 +157,8 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     const size_t o_s2 = take(sizeof(double) * (size_t)n_tiles);
     const size_t o_pen = take(sizeof(double) * (size_t)n_tiles);
     const size_t o_bad = take(sizeof(uint32_t) * (size_t)n_tiles);
+    const size_t o_min = take(sizeof(float) * (size_t)n_tiles);
+    const size_t o_max = take(sizeof(float) * (size_t)n_tiles);
     const size_t o_par = take(sizeof(double) * 2 * (size_t)n_seg);
     const size_t total = off > 0 ? off : 256;
 
@@ -186,6 +189,8 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     p->part.s2 = reinterpret_cast<double *>(d + o_s2);
     p->part.pen = reinterpret_cast<double *>(d + o_pen);
     p->part.bad = reinterpret_cast<uint32_t *>(d + o_bad);
+    p->part.xmin = reinterpret_cast<float *>(d + o_min);
+    p->part.xmax = reinterpret_cast<float *>(d + o_max);
     p->params = reinterpret_cast<double *>(d + o_par);
     p->last_use = ctx->clock;
     *out = p.get();
@@ -213,6 +218,16 @@ struct SweepTimer {
         list->push_back(e);
     }
 };
+
+// Picks the kernel for one sweep: bf16 inputs with a gradient or a histogram take the
+// pattern-table kernel, everything else the generic one.
+cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
+                         const StreamArgs &sa, cudaStream_t cs)
+{
+    if (in_dtype == GG_BF16 && (flags & (kGrad | kHist)) != 0)
+        return launch_tail_bf16(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
+    return launch_stream(flags, in_dtype, grad_dtype, has_grad_out, sa, cs);
+}
 
 gg_status check_grad(const gg_seg *segs, const gg_seg *grad, int32_t n_seg, int grad_dtype)
 {
@@ -288,6 +303,7 @@ gg_status gg_create(gg_ctx **out, int device)
     gg_ctx *ctx = new (std::nothrow) gg_ctx;
     if (!ctx) return GG_ERR_NOMEM;
     ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
     *out = ctx;
     return GG_OK;
 }
@@ -328,7 +344,7 @@ gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
     StreamArgs sa{};
     sa.map = p->map;
     sa.part = p->part;
-    GG_CUDA(ctx, launch_stream(kMoments, dtype, GG_F32, false, sa, cs));
+    GG_CUDA(ctx, launch_sweep(ctx, kMoments, dtype, GG_F32, false, sa, cs));
     ctx->launches += p->n_tiles > 0;
     FitArgs fa{};
     fa.map = p->map; fa.part = p->part;
@@ -361,7 +377,7 @@ gg_status gg_penalty_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dty
     sa.map = p->map; sa.part = p->part;
     sa.beta = beta; sa.alpha = alpha; sa.lambda = lambda;
     sa.mean_reduction = reduction == GG_MEAN; sa.accumulate = accumulate;
-    GG_CUDA(ctx, launch_stream(kGrad, in_dtype, grad_dtype, grad != nullptr, sa, cs));
+    GG_CUDA(ctx, launch_sweep(ctx, kGrad, in_dtype, grad_dtype, grad != nullptr, sa, cs));
     ctx->launches += p->n_tiles > 0;
     if (penalty) {
         GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta, penalty, cs));
@@ -395,7 +411,7 @@ gg_status gg_rate_hist(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype 
         StreamArgs sa{};
         sa.map = p->map; sa.part = p->part;
         sa.step = step; sa.qmin = qmin; sa.qmax = qmax; sa.hist = hist; sa.clamped = clamped_lo_hi;
-        GG_CUDA(ctx, launch_stream(kHist, dtype, GG_F32, false, sa, cs));
+        GG_CUDA(ctx, launch_sweep(ctx, kHist, dtype, GG_F32, false, sa, cs));
         ctx->launches += p->n_tiles > 0;
     }
     if (entropy_bits && n_hist > 0) {
@@ -510,20 +526,20 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         sa.map = p->map; sa.part = p->part;
         sa.lambda = a->lambda; sa.mean_reduction = a->reduction == GG_MEAN; sa.accumulate = a->accumulate_grad;
         sa.qmin = a->qmin; sa.qmax = a->qmax; sa.hist = a->hist; sa.clamped = a->clamped_lo_hi;
-        sa.flags = a->flags;
         FitArgs fa{};
         fa.map = p->map; fa.part = p->part;
         fa.beta = a->beta; fa.alpha = a->alpha; fa.sum_abs = a->sum_abs; fa.sum_sq = a->sum_sq;
         fa.count = a->count; fa.flags = a->flags;
         fa.step_from_alpha = do_hist && a->step_mode == GG_STEP_FROM_ALPHA;
         fa.step_scale = a->step_scale; fa.step_out = a->step_out;
+        fa.hist_on = do_hist; fa.step = a->step; fa.qmin = a->qmin; fa.qmax = a->qmax;
 
         const double *beta_used;
         if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
-                GG_CUDA(ctx, launch_stream(kMoments, in_dt, g_dt, false, sa, cs));
+                GG_CUDA(ctx, launch_sweep(ctx, kMoments, in_dt, g_dt, false, sa, cs));
             }
             GG_CUDA(ctx, launch_fit(fa, cs));
             ctx->launches += 1 + (p->n_tiles > 0);
@@ -531,21 +547,16 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             sa.step = fa.step_from_alpha ? a->step_out : a->step;
             if (tail_flags) {
                 SweepTimer tm(ctx, &ctx->ev_tail, cs);
-                GG_CUDA(ctx, launch_stream(tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
+                GG_CUDA(ctx, launch_sweep(ctx, tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
                 ctx->launches += p->n_tiles > 0;
             }
             beta_used = a->beta;
         } else {
-            // one sweep: moments, gradient (given parameters) and histogram together; then the fit,
-            // which keeps the clamp bit that the sweep OR-ed into the zeroed flags.
+            // one sweep: moments, gradient (given parameters) and histogram together; then the fit
             sa.beta = a->beta_in; sa.alpha = a->alpha_in; sa.step = a->step;
-            if (a->flags) {
-                GG_CUDA(ctx, cudaMemsetAsync(a->flags, 0, sizeof(uint32_t) * (size_t)n_seg, cs));
-                fa.keep_clamp_bit = 1;
-            }
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
-                GG_CUDA(ctx, launch_stream(kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
+                GG_CUDA(ctx, launch_sweep(ctx, kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
             }
             GG_CUDA(ctx, launch_fit(fa, cs));
             ctx->launches += 1 + (p->n_tiles > 0);

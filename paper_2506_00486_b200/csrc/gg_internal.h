@@ -35,6 +35,8 @@ struct TileScratch {
     double *s2;       // sum x^2
     double *pen;      // sum |x| |g|   (penalty = that / beta)
     uint32_t *bad;    // non-finite entries
+    float *xmin;      // smallest and largest entry (NaN ignored): decide whether a symbol clamps
+    float *xmax;
 };
 
 struct StreamArgs {
@@ -51,7 +53,6 @@ struct StreamArgs {
     int32_t qmin, qmax;
     uint64_t *hist;
     uint64_t *clamped;   // [2 * n_hist] or null
-    uint32_t *flags;     // [n_seg] or null (GG_FLAG_CLAMPED_SYMBOLS is OR-ed in)
 };
 
 struct FitArgs {
@@ -60,14 +61,21 @@ struct FitArgs {
     double *beta, *alpha, *sum_abs, *sum_sq;
     int64_t *count;
     uint32_t *flags;
-    int keep_clamp_bit;   // flags[s] already holds this call's GG_FLAG_CLAMPED_SYMBOLS bit
     int step_from_alpha;
     double step_scale;
     float *step_out;
+    // when a histogram is part of the call: GG_FLAG_CLAMPED_SYMBOLS from the segment's extremes
+    int hist_on;
+    const float *step;
+    int32_t qmin, qmax;
 };
 
 cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
                           const StreamArgs &a, cudaStream_t st);
+// bf16-input sweeps with a gradient and/or a histogram: persistent CTAs, table look-up gradient,
+// histogram over bf16 bit patterns.  sm_count sizes the grid.
+cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
+                             int sm_count, cudaStream_t st);
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
 cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
                                     double *penalty, cudaStream_t st);

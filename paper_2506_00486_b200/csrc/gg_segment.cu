@@ -36,14 +36,22 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
     const int t0 = a.map.tile_prefix[s], t1 = a.map.tile_prefix[s + 1];
     double s1 = 0.0, s2 = 0.0;
     uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
     for (int t = t0 + lane; t < t1; t += 32) {
         s1 += a.part.s1[t];
         s2 += a.part.s2[t];
         bad += a.part.bad[t];
+        xmin = fminf(xmin, a.part.xmin[t]);
+        xmax = fmaxf(xmax, a.part.xmax[t]);
     }
     s1 = warp_sum(s1);
     s2 = warp_sum(s2);
     bad = __reduce_add_sync(kFull, bad);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xmin = fminf(xmin, __shfl_xor_sync(kFull, xmin, o));
+        xmax = fmaxf(xmax, __shfl_xor_sync(kFull, xmax, o));
+    }
     const int64_t len = a.map.seg_len[s];
 
     uint32_t flags = bad ? GG_FLAG_NONFINITE : 0u;
@@ -79,8 +87,16 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
         if (a.sum_abs) a.sum_abs[s] = s1;
         if (a.sum_sq) a.sum_sq[s] = s2;
         if (a.count) a.count[s] = len;
-        if (a.flags) a.flags[s] = flags | (a.keep_clamp_bit ? (a.flags[s] & GG_FLAG_CLAMPED_SYMBOLS) : 0u);
-        if (a.step_from_alpha && a.step_out) a.step_out[s] = (float)(alpha * a.step_scale);
+        const float step = a.step_from_alpha ? (float)(alpha * a.step_scale) : (a.step ? a.step[s] : 0.0f);
+        if (a.step_from_alpha && a.step_out) a.step_out[s] = step;
+        if (a.hist_on && xmin <= xmax) {
+            // the quantiser is monotone in x, so a symbol clamps iff one of the extremes does
+            const float inv = (float)(1.0 / (double)step);
+            const float tlo = __fmul_rn(xmin, inv), thi = __fmul_rn(xmax, inv);
+            if ((double)floorf(tlo) < (double)a.qmin || (double)floorf(thi) > (double)a.qmax)
+                flags |= GG_FLAG_CLAMPED_SYMBOLS;
+        }
+        if (a.flags) a.flags[s] = flags;
     }
 }
 

@@ -156,6 +156,7 @@ __device__ __forceinline__ float grad_elem(float x, const GradConst &k, const fl
 struct Acc {
     double s1 = 0.0, s2 = 0.0, pen = 0.0;
     uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
 };
 
 struct HistConst {
@@ -193,6 +194,8 @@ __device__ __forceinline__ void process(const float (&x)[KV], float (&g)[KV], Ac
             m1 += af;
             m2 = fmaf(af, af, m2);
             acc.bad += fin ? 0u : 1u;
+            acc.xmin = fminf(acc.xmin, xe);      // fminf / fmaxf return the non-NaN operand
+            acc.xmax = fmaxf(acc.xmax, xe);
         }
         if constexpr (FLAGS & kGrad) {
             const float ge = grad_elem(xe, gc, A, B);
@@ -231,6 +234,7 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
     __shared__ double shL;
     __shared__ double shRed[3][kWarps];
     __shared__ uint32_t shBad[kWarps];
+    __shared__ float shMin[kWarps], shMax[kWarps];
 
     const int tid = threadIdx.x;
     const int t = blockIdx.x;
@@ -346,7 +350,16 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
     if constexpr (MOM) {
         const double w1 = warp_sum(acc.s1), w2 = warp_sum(acc.s2);
         const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, acc.bad);
-        if (lane == 0) { shRed[0][warp] = w1; shRed[1][warp] = w2; shBad[warp] = wb; }
+        float wmin = acc.xmin, wmax = acc.xmax;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            wmin = fminf(wmin, __shfl_xor_sync(0xFFFFFFFFu, wmin, o));
+            wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+        }
+        if (lane == 0) {
+            shRed[0][warp] = w1; shRed[1][warp] = w2; shBad[warp] = wb;
+            shMin[warp] = wmin; shMax[warp] = wmax;
+        }
     }
     if constexpr (GRAD) {
         const double wp = warp_sum(acc.pen);
@@ -357,8 +370,13 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
         if constexpr (MOM) {
             double r1 = 0.0, r2 = 0.0;
             uint32_t rb = 0;
-            for (int w = 0; w < kWarps; ++w) { r1 += shRed[0][w]; r2 += shRed[1][w]; rb += shBad[w]; }
+            float rmin = INFINITY, rmax = -INFINITY;
+            for (int w = 0; w < kWarps; ++w) {
+                r1 += shRed[0][w]; r2 += shRed[1][w]; rb += shBad[w];
+                rmin = fminf(rmin, shMin[w]); rmax = fmaxf(rmax, shMax[w]);
+            }
             a.part.s1[t] = r1; a.part.s2[t] = r2; a.part.bad[t] = rb;
+            a.part.xmin[t] = rmin; a.part.xmax[t] = rmax;
         }
         if constexpr (GRAD) {
             double rp = 0.0;
@@ -376,8 +394,116 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
             if (a.clamped != nullptr)
                 atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + tid,
                           (unsigned long long)shClamp[tid]);
-            if (a.flags != nullptr) atomicOr(&a.flags[s], GG_FLAG_CLAMPED_SYMBOLS);
         }
+    }
+}
+
+// ---------------------------------------------------------------------------- bf16 moments
+// The first sweep over bf16 data reads 2 bytes per element, so at HBM speed an SM has about ten
+// issue slots per element.  This kernel spends about five: the widening and the two sums per
+// element, min/max on packed bf16 pairs, and one packed test per pair for inf/nan (a vector that
+// contains one is redone element by element).
+__device__ __forceinline__ void moments_careful(uint32_t h, float &m1, float &m2, uint32_t &bad)
+{
+    const uint32_t mag = h & 0x7FFFu;
+    const float ax = __uint_as_float(mag << 16);
+    if (mag < 0x7F80u) { m1 += ax; m2 = fmaf(ax, ax, m2); }
+    else bad += 1u;
+}
+
+__global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs a)
+{
+    __shared__ double shRed[2][kWarps];
+    __shared__ uint32_t shBad[kWarps];
+    __shared__ float shMin[kWarps], shMax[kWarps];
+    const int tid = threadIdx.x;
+    const int t = blockIdx.x;
+    const int s = a.map.tile_seg[t];
+    const int64_t len = a.map.seg_len[s];
+    const int64_t off = (int64_t)(t - a.map.tile_prefix[s]) * kTile;
+    const int n = (int)min((int64_t)kTile, len - off);
+    const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
+    int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
+    head = min(head, n);
+    const int nvec = (n - head) / 8;
+    const int tail0 = head + nvec * 8;
+
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
+    for (int i = tid; i < head + (n - tail0); i += kThreads) {
+        const int idx = i < head ? i : tail0 + (i - head);
+        const uint32_t h = (uint32_t)__ldg(x + idx);
+        float m1 = 0.0f, m2 = 0.0f;
+        moments_careful(h, m1, m2, bad);
+        s1 += (double)m1; s2 += (double)m2;
+        xmin = fminf(xmin, __uint_as_float(h << 16));
+        xmax = fmaxf(xmax, __uint_as_float(h << 16));
+    }
+    __nv_bfloat162 mn2 = __floats2bfloat162_rn(INFINITY, INFINITY), mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
+    const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
+    for (int v0 = tid; v0 < nvec; v0 += kThreads * kUnroll) {
+        uint4 raw[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int v = v0 + u * kThreads;
+            if (v < nvec) raw[u] = __ldg(xv + v);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int v = v0 + u * kThreads;
+            if (v < nvec) {
+                const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+                float m1 = 0.0f, m2 = 0.0f;
+                uint32_t probe = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // adding 0x80 to a 15-bit magnitude carries into bit 15 iff the exponent is all ones
+                    probe |= (w[i] & 0x7FFF7FFFu) + 0x00800080u;
+                    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+                    m1 += fabsf(lo);
+                    m1 += fabsf(hi);
+                    m2 = fmaf(lo, lo, m2);
+                    m2 = fmaf(hi, hi, m2);
+                    const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162 *>(&w[i]);
+                    mn2 = __hmin2(mn2, p);      // return the non-NaN operand, like fminf
+                    mx2 = __hmax2(mx2, p);
+                }
+                if (probe & 0x80008000u) {      // an inf or nan in this vector: leave it out of the sums
+                    m1 = 0.0f; m2 = 0.0f;
+                    for (int i = 0; i < 4; ++i) {
+                        moments_careful(w[i] & 0xFFFFu, m1, m2, bad);
+                        moments_careful(w[i] >> 16, m1, m2, bad);
+                    }
+                }
+                s1 += (double)m1;
+                s2 += (double)m2;
+            }
+        }
+    }
+    xmin = fminf(xmin, fminf(__low2float(mn2), __high2float(mn2)));
+    xmax = fmaxf(xmax, fmaxf(__low2float(mx2), __high2float(mx2)));
+
+    const int lane = tid & 31, warp = tid >> 5;
+    const double w1 = warp_sum(s1), w2 = warp_sum(s2);
+    const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, bad);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xmin = fminf(xmin, __shfl_xor_sync(0xFFFFFFFFu, xmin, o));
+        xmax = fmaxf(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, o));
+    }
+    if (lane == 0) { shRed[0][warp] = w1; shRed[1][warp] = w2; shBad[warp] = wb; shMin[warp] = xmin; shMax[warp] = xmax; }
+    __syncthreads();
+    if (tid == 0) {
+        double r1 = 0.0, r2 = 0.0;
+        uint32_t rb = 0;
+        float rmin = INFINITY, rmax = -INFINITY;
+        for (int w = 0; w < kWarps; ++w) {
+            r1 += shRed[0][w]; r2 += shRed[1][w]; rb += shBad[w];
+            rmin = fminf(rmin, shMin[w]); rmax = fmaxf(rmax, shMax[w]);
+        }
+        a.part.s1[t] = r1; a.part.s2[t] = r2; a.part.bad[t] = rb;
+        a.part.xmin[t] = rmin; a.part.xmax[t] = rmax;
     }
 }
 
@@ -406,6 +532,10 @@ cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, boo
                           const StreamArgs &a, cudaStream_t st)
 {
     if (a.map.n_tiles <= 0) return cudaSuccess;
+    if (in_dtype == GG_BF16 && flags == kMoments) {
+        moments_bf16_kernel<<<(unsigned)a.map.n_tiles, kThreads, 0, st>>>(a);
+        return cudaGetLastError();
+    }
     // without a gradient output the gradient type does not matter: use one instantiation
     const bool g16 = has_grad_out && grad_dtype == GG_BF16;
     if (in_dtype == GG_F32)

@@ -1,0 +1,608 @@
+// bf16-input sweep with a gradient and/or a histogram (optionally the moments too), specialised
+// for the fact that a bf16 value is one of 65536 bit patterns.
+//
+// Persistent CTAs each walk one contiguous range of tiles.  Inside a segment that range is one
+// contiguous run of elements, streamed with 128-bit loads issued two iterations ahead.
+//   * gradient: |g| depends only on the 15-bit magnitude pattern.  |g| = A[e] * B[j] with e the
+//     exponent field and j the 7 mantissa bits: A[e] = 2^(L + b (e-127)) (kept as a normal-range
+//     factor times a power of two), B[j] = (1 + j/128)^b, both rounded once from fp64, so the
+//     product is within 1.5 ulp for every shape beta.  For runs of two tiles or more the CTA
+//     expands the 32 binades below 2^6 standard deviations into a 4096-entry table, so an element
+//     costs one shared-memory load.
+//   * histogram: elements are counted by bit pattern (4096 magnitudes x 2 signs in shared memory);
+//     patterns become quantised symbols only when the table is flushed, i.e. when the histogram,
+//     its step or the window changes, or the CTA ends.  Patterns outside the window (zeros, tiny
+//     or huge values) are quantised on the spot into a small symbol window, else straight to
+//     global memory.  Counts are integers, so every order of additions gives the same table.
+//   * in table mode both tables share one window and the element path is branch free: an element
+//     outside the window hits sentinel cells and is redone after its vector.
+#include <cuda_bf16.h>
+#include <float.h>
+
+#include "gg_internal.h"
+
+namespace gg {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kLut = 4096;       // magnitude patterns in the gradient table (32 binades)
+constexpr int kCnt = 4096;       // magnitude patterns in the count table (two cells each: + and -)
+constexpr int kSymWin = 512;     // secondary symbol window [-256, 256)
+constexpr int kCtasPerSm = 4;
+constexpr uint32_t kWinBytes = kLut * 4;
+
+// Constants of the current segment / histogram that only the cold paths need: kept in shared
+// memory so that the streaming loop does not carry them in registers.
+struct Cold {
+    double L, b;               // g = 2^(L + b log2|x|)
+    uint32_t sign_flip;        // 0x80000000 if lambda < 0 (the tables then hold -|g|)
+    int active;                // 0: the gradient is zero everywhere
+    float inv;                 // quantiser: q = floor(x * inv)
+    int32_t qmin, qmax;
+    unsigned long long *row;   // the current histogram, bin 0 = symbol qmin
+    uint32_t c_base;           // first magnitude pattern of the count window
+};
+
+struct Smem {
+    float lut[kLut + 1];            // last cell: sentinel for out-of-window elements (zero)
+    uint32_t cnt[2 * kCnt + 2];     // cell 2 i + s: magnitude pattern c_base + i with sign s; last two: sentinel
+    uint32_t win[kSymWin];
+    float2 A[256];
+    float B[128];
+    double red[3][kWarps];
+    uint32_t bad[kWarps];
+    float mn[kWarps], mx[kWarps];
+    uint32_t clampc[2];
+    Cold cold;
+    int e_top;
+};
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// |g| (with lambda's sign) for a magnitude pattern the A/B tables do not cover: zero, subnormal,
+// inf, nan.
+__device__ __noinline__ float grad_rare(uint32_t mag, const Smem &sm)
+{
+    const float ax = __uint_as_float(mag << 16);
+    if (!sm.cold.active || ax == 0.0f) return 0.0f;
+    const float v = (float)exp2(sm.cold.L + sm.cold.b * log2((double)ax));
+    return __uint_as_float(__float_as_uint(v) ^ sm.cold.sign_flip);
+}
+
+__device__ __forceinline__ float grad_ab(uint32_t mag, const Smem &sm)
+{
+    const uint32_t e = mag >> 7;
+    if (e - 1u < 254u) {
+        const float2 a = sm.A[e];
+        return (a.x * sm.B[mag & 127u]) * a.y;
+    }
+    return grad_rare(mag, sm);
+}
+
+// Quantises one value and adds n to its symbol's count: the shared symbol window when allowed and
+// in reach, else global memory.
+__device__ __forceinline__ void count_symbol(float x, uint32_t n, bool use_window, Smem &sm)
+{
+    const float t = __fmul_rn(x, sm.cold.inv);
+    if (t == t) {                                  // NaN is skipped
+        int q = __float2int_rd(t);                 // floor, saturating
+        const int qmin = sm.cold.qmin, qmax = sm.cold.qmax;
+        if (q < qmin) { q = qmin; atomicAdd(&sm.clampc[0], n); }
+        else if (q > qmax) { q = qmax; atomicAdd(&sm.clampc[1], n); }
+        const uint32_t w = (uint32_t)(q + kSymWin / 2);
+        if (use_window && w < (uint32_t)kSymWin) atomicAdd(&sm.win[w], n);
+        else atomicAdd(&sm.cold.row[q - qmin], (unsigned long long)n);
+    }
+}
+
+__device__ __noinline__ void count_rare(uint32_t xb, Smem &sm) { count_symbol(__uint_as_float(xb), 1u, true, sm); }
+
+struct Acc {
+    double s1 = 0.0, s2 = 0.0, pen = 0.0;
+    uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
+};
+
+struct Run {   // fp32 partials of one short run of elements
+    float m1 = 0.0f, m2 = 0.0f, mp = 0.0f;
+};
+
+// Byte offset of a value's count cell: (pattern index) * 8 + sign * 4.
+__device__ __forceinline__ uint32_t count_cell(uint32_t off4, uint32_t xb) { return (off4 << 1) + ((xb >> 29) & 4u); }
+
+template <int FLAGS>
+__device__ __forceinline__ void moments_elem(uint32_t xb, Acc &acc, Run &r)
+{
+    if constexpr ((FLAGS & kMoments) != 0) {
+        const uint32_t am = xb & 0x7FFFFFFFu;
+        const bool fin = am < 0x7F800000u;
+        const float af = fin ? __uint_as_float(am) : 0.0f;
+        r.m1 += af;
+        r.m2 = fmaf(af, af, r.m2);
+        acc.bad += fin ? 0u : 1u;
+        acc.xmin = fminf(acc.xmin, __uint_as_float(xb));     // fminf / fmaxf return the non-NaN operand
+        acc.xmax = fmaxf(acc.xmax, __uint_as_float(xb));
+    }
+}
+
+// One element given as fp32 bits (a widened bf16: the low 16 bits are zero), table mode.  Branch
+// free: `anyoff` collects the window offsets so one compare per vector finds elements that
+// missed the window; those read and count in the sentinel cells and are redone by fix_rare().
+template <int FLAGS>
+__device__ __forceinline__ float one_table(uint32_t xb, uint32_t base4, Smem &sm, Acc &acc, Run &r, uint32_t &anyoff)
+{
+    moments_elem<FLAGS>(xb, acc, r);
+    const uint32_t am = xb & 0x7FFFFFFFu;
+    uint32_t off = (am >> 14) - base4;              // (magnitude pattern - window base) * 4
+    anyoff |= off;
+    off = min(off, kWinBytes);
+    float ga = 0.0f;
+    if constexpr ((FLAGS & kGrad) != 0)
+        ga = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.lut) + off);
+    if constexpr ((FLAGS & kHist) != 0)
+        atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(off, xb)), 1u);
+    if constexpr ((FLAGS & kGrad) != 0) {
+        r.mp = fmaf(__uint_as_float(am), fabsf(ga), r.mp);
+        return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
+    }
+    return 0.0f;
+}
+
+// Redo of an element that fell outside the table window (zero, tiny, huge, inf, nan).
+template <int FLAGS>
+__device__ __noinline__ float fix_rare(uint32_t xb, Smem &sm, Run &r)
+{
+    float ga = 0.0f;
+    if constexpr ((FLAGS & kGrad) != 0) {
+        ga = grad_ab((xb >> 16) & 0x7FFFu, sm);
+        r.mp = fmaf(__uint_as_float(xb & 0x7FFFFFFFu), fabsf(ga), r.mp);
+    }
+    if constexpr ((FLAGS & kHist) != 0) count_symbol(__uint_as_float(xb), 1u, true, sm);
+    return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+}
+
+// The same element when the gradient table is off (short runs): gradient from the A/B tables,
+// count window wherever it currently sits (base4 = its base * 4).
+template <int FLAGS>
+__device__ __forceinline__ float one_plain(uint32_t xb, uint32_t base4, Smem &sm, Acc &acc, Run &r)
+{
+    moments_elem<FLAGS>(xb, acc, r);
+    const uint32_t am = xb & 0x7FFFFFFFu;
+    float ga = 0.0f;
+    if constexpr ((FLAGS & kGrad) != 0) ga = grad_ab(am >> 16, sm);
+    if constexpr ((FLAGS & kHist) != 0) {
+        const uint32_t off = (am >> 14) - base4;
+        if (off < kWinBytes)
+            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(off, xb)), 1u);
+        else
+            count_rare(xb, sm);
+    }
+    if constexpr ((FLAGS & kGrad) != 0) {
+        r.mp = fmaf(__uint_as_float(am), fabsf(ga), r.mp);
+        return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+    }
+    return 0.0f;
+}
+
+// fp64 penalty terms |x| |g| of up to eight patterns packed in four words (rare path).
+__device__ __noinline__ double pen_rare(uint4 raw, int n, const Smem &sm)
+{
+    if (!sm.cold.active) return 0.0;
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    double dp = 0.0;
+    for (int e = 0; e < n; ++e) {
+        const uint32_t h = (w[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu;
+        const double ax = (double)__uint_as_float(h << 16);
+        if (ax != 0.0) dp += ax * exp2(sm.cold.L + sm.cold.b * log2(ax));
+    }
+    return dp;
+}
+
+template <int FLAGS>
+__device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &acc, const Smem &sm)
+{
+    if constexpr ((FLAGS & kMoments) != 0) { acc.s1 += (double)r.m1; acc.s2 += (double)r.m2; }
+    if constexpr ((FLAGS & kGrad) != 0) {
+        // a product or a gradient that left the fp32 range (or a nan) sends the run to fp64
+        if (r.mp <= FLT_MAX) acc.pen += (double)r.mp;
+        else acc.pen += pen_rare(raw, n, sm);
+    }
+}
+
+template <typename TG>
+__device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumulate)
+{
+    if constexpr (sizeof(TG) == 4) {
+        float4 *p = reinterpret_cast<float4 *>(g);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            if (accumulate) {
+                const float4 old = p[i];
+                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+            }
+            __stcs(p + i, o);     // written once, never re-read by this pass: streaming store
+        }
+    } else {
+        uint32_t w[4];
+        const uint32_t *p = reinterpret_cast<const uint32_t *>(g);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float lo = v[2 * i], hi = v[2 * i + 1];
+            if (accumulate) {
+                const uint32_t old = p[i];
+                lo += __uint_as_float(old << 16);
+                hi += __uint_as_float(old & 0xFFFF0000u);
+            }
+            w[i] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+                   ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+        }
+        __stcs(reinterpret_cast<uint4 *>(g), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+}
+
+// Exponent field of the top binade of a 32-binade window that reaches 2^6 times `scale`.
+__device__ __forceinline__ int window_top_exponent(double scale)
+{
+    int e = 127 + 6;
+    if (scale > 0.0 && scale < 1e300) e = ilogb(scale) + 127 + 6;
+    return max(33, min(254, e));
+}
+
+// Turns the counted patterns into symbols of the current histogram and empties the tables.
+__device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
+{
+    // (callers synchronise before: all counting under the old key is complete)
+    const uint32_t c_base = sm.cold.c_base;
+    for (int p = threadIdx.x; p < 2 * kCnt; p += kThreads) {
+        const uint32_t n = sm.cnt[p];
+        if (n != 0u) {
+            sm.cnt[p] = 0u;
+            const uint32_t h = (c_base + (uint32_t)(p >> 1)) | ((uint32_t)(p & 1) << 15);
+            count_symbol(__uint_as_float(h << 16), n, false, sm);
+        }
+    }
+    for (int i = threadIdx.x; i < kSymWin; i += kThreads) {
+        const uint32_t n = sm.win[i];
+        if (n != 0u) {
+            sm.win[i] = 0u;
+            atomicAdd(&sm.cold.row[(i - kSymWin / 2) - sm.cold.qmin], (unsigned long long)n);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        const uint32_t n = sm.clampc[threadIdx.x];
+        if (n != 0u && clamped != nullptr)
+            atomicAdd(reinterpret_cast<unsigned long long *>(clamped) + 2 * hid + threadIdx.x, (unsigned long long)n);
+        sm.clampc[threadIdx.x] = 0u;
+    }
+    __syncthreads();
+}
+
+template <int FLAGS>
+__device__ __forceinline__ void zero_partials(const TileScratch &part, int t)
+{
+    if constexpr ((FLAGS & kMoments) != 0) {
+        part.s1[t] = 0.0; part.s2[t] = 0.0; part.bad[t] = 0u;
+        part.xmin[t] = INFINITY; part.xmax[t] = -INFINITY;
+    }
+    if constexpr ((FLAGS & kGrad) != 0) part.pen[t] = 0.0;
+}
+
+// Block reduction in a fixed order (butterfly inside each warp, then the warps in sequence) of the
+// partial sums of one run of tiles [t0, t1); the result goes to the slot of t0, zeros to the rest.
+template <int FLAGS>
+__device__ void reduce_partials(const TileScratch &part, int t0, int t1, const Acc &acc, Smem &sm)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if constexpr ((FLAGS & kMoments) != 0) {
+        const double w1 = warp_sum(acc.s1), w2 = warp_sum(acc.s2);
+        const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, acc.bad);
+        float wmin = acc.xmin, wmax = acc.xmax;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            wmin = fminf(wmin, __shfl_xor_sync(0xFFFFFFFFu, wmin, o));
+            wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+        }
+        if (lane == 0) {
+            sm.red[0][warp] = w1; sm.red[1][warp] = w2; sm.bad[warp] = wb;
+            sm.mn[warp] = wmin; sm.mx[warp] = wmax;
+        }
+    }
+    if constexpr ((FLAGS & kGrad) != 0) {
+        const double wp = warp_sum(acc.pen);
+        if (lane == 0) sm.red[2][warp] = wp;
+    }
+    __syncthreads();
+    for (int t = t0 + 1 + tid; t < t1; t += kThreads) zero_partials<FLAGS>(part, t);
+    if (tid == 0) {
+        if constexpr ((FLAGS & kMoments) != 0) {
+            double r1 = 0.0, r2 = 0.0;
+            uint32_t rb = 0;
+            float rmin = INFINITY, rmax = -INFINITY;
+            for (int w = 0; w < kWarps; ++w) {
+                r1 += sm.red[0][w]; r2 += sm.red[1][w]; rb += sm.bad[w];
+                rmin = fminf(rmin, sm.mn[w]); rmax = fmaxf(rmax, sm.mx[w]);
+            }
+            part.s1[t0] = r1; part.s2[t0] = r2; part.bad[t0] = rb;
+            part.xmin[t0] = rmin; part.xmax[t0] = rmax;
+        }
+        if constexpr ((FLAGS & kGrad) != 0) {
+            double rp = 0.0;
+            for (int w = 0; w < kWarps; ++w) rp += sm.red[2][w];
+            part.pen[t0] = sm.cold.sign_flip ? -rp : rp;     // the penalty carries lambda's sign
+        }
+    }
+    __syncthreads();
+}
+
+template <typename TG, int FLAGS, bool TABLE>
+__device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool accumulate, uint32_t base4,
+                                            Smem &sm, Acc &acc)
+{
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    float g[8];
+    Run r;
+    if constexpr (TABLE) {
+        uint32_t anyoff = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            g[2 * i] = one_table<FLAGS>(w[i] << 16, base4, sm, acc, r, anyoff);
+            g[2 * i + 1] = one_table<FLAGS>(w[i] & 0xFFFF0000u, base4, sm, acc, r, anyoff);
+        }
+        if (anyoff >= kWinBytes) {      // some element missed the window
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+                if (((xb & 0x7FFFFFFFu) >> 14) - base4 >= kWinBytes) g[i] = fix_rare<FLAGS>(xb, sm, r);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            g[2 * i] = one_plain<FLAGS>(w[i] << 16, base4, sm, acc, r);
+            g[2 * i + 1] = one_plain<FLAGS>(w[i] & 0xFFFF0000u, base4, sm, acc, r);
+        }
+    }
+    close_run<FLAGS>(raw, 8, r, acc, sm);
+    if constexpr ((FLAGS & kGrad) != 0) {
+        if (gdst != nullptr) store8<TG>(gdst, g, accumulate);
+    }
+}
+
+// One contiguous run of n elements: scalar head up to the first 16-byte boundary of x, 128-bit
+// vector body with loads issued two iterations ahead, scalar tail.  If the gradient's address is
+// not 16-byte aligned at the same element the whole run is scalar.
+template <typename TG, int FLAGS, bool TABLE>
+__device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
+                                              uint32_t base4, Smem &sm, Acc &acc)
+{
+    constexpr bool GRAD = (FLAGS & kGrad) != 0;
+    const int tid = threadIdx.x;
+    int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
+    head = min(head, n);
+    if (gout != nullptr && (reinterpret_cast<uintptr_t>(gout + head) & 15u) != 0) head = n;
+    const int64_t nvec = (n - head) / 8;
+    const int64_t tail0 = head + nvec * 8;
+
+    for (int64_t i = tid; i < head + (n - tail0); i += kThreads) {
+        const int64_t idx = i < head ? i : tail0 + (i - head);
+        const uint32_t h = (uint32_t)__ldg(x + idx);
+        Run r;
+        float g;
+        if constexpr (TABLE) {
+            uint32_t anyoff = 0;
+            g = one_table<FLAGS>(h << 16, base4, sm, acc, r, anyoff);
+            if (anyoff >= kWinBytes) g = fix_rare<FLAGS>(h << 16, sm, r);
+        } else {
+            g = one_plain<FLAGS>(h << 16, base4, sm, acc, r);
+        }
+        close_run<FLAGS>(make_uint4(h, 0u, 0u, 0u), 1, r, acc, sm);
+        if constexpr (GRAD) {
+            if (gout != nullptr) {
+                float v = g;
+                if constexpr (sizeof(TG) == 4) {
+                    if (accumulate) v += gout[idx];
+                    gout[idx] = v;
+                } else {
+                    if (accumulate) v += __uint_as_float((uint32_t)gout[idx] << 16);
+                    gout[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                }
+            }
+        }
+    }
+
+    const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
+    TG *gv = gout != nullptr ? gout + head : nullptr;
+    int64_t v = tid;
+    uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
+    if (v < nvec) r0 = __ldcs(xv + v);                       // read once by this sweep: streaming loads
+    if (v + kThreads < nvec) r1 = __ldcs(xv + v + kThreads);
+    for (; v < nvec; v += kThreads) {
+        uint4 r2 = make_uint4(0u, 0u, 0u, 0u);
+        if (v + 2 * kThreads < nvec) r2 = __ldcs(xv + v + 2 * kThreads);
+        process_vec<TG, FLAGS, TABLE>(r0, gv != nullptr ? gv + v * 8 : nullptr, accumulate, base4, sm, acc);
+        r0 = r1;
+        r1 = r2;
+    }
+}
+
+template <typename TG, int FLAGS>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const StreamArgs a)
+{
+    constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    const int tid = threadIdx.x;
+
+    // contiguous range of tiles for this CTA
+    const int64_t nt = a.map.n_tiles;
+    const int t_begin = (int)(nt * blockIdx.x / gridDim.x);
+    const int t_end = (int)(nt * (blockIdx.x + 1) / gridDim.x);
+
+    if constexpr (HIST) {
+        for (int i = tid; i < 2 * kCnt + 2; i += kThreads) sm.cnt[i] = 0u;
+        for (int i = tid; i < kSymWin; i += kThreads) sm.win[i] = 0u;
+        if (tid < 2) sm.clampc[tid] = 0u;
+    }
+    if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; }
+    int cur_hid = -1;
+    uint32_t cur_inv_bits = 0;
+    bool have_key = false;
+    const bool accumulate = GRAD && a.accumulate != 0;
+    __syncthreads();
+
+    for (int t = t_begin; t < t_end;) {
+        // ---- one run: the tiles of this CTA's range that lie in segment s
+        const int s = a.map.tile_seg[t];
+        const int64_t len = a.map.seg_len[s];
+        const int t_first = a.map.tile_prefix[s];
+        const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
+        bool table_mode = false;
+        uint32_t g_base = 0x8000u;
+
+        if constexpr (GRAD) {
+            const double beta = a.beta[s], alpha = a.alpha[s];
+            const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
+            const bool active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
+            if (tid == 0) {
+                sm.cold.b = beta - 1.0;
+                sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
+                sm.cold.active = active;
+                sm.cold.L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
+                // the standard deviation of the fitted density (Eq. 2-3) places the table window
+                const double sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
+                sm.e_top = window_top_exponent(sd);
+            }
+            __syncthreads();
+            {
+                const double L = sm.cold.L, b = sm.cold.b;
+                const int k = tid;      // kThreads == 256 entries of A
+                float2 v = make_float2(0.0f, 0.0f);
+                if (active && k >= 1 && k <= 254) {
+                    const double e0 = L + b * (double)(k - 127);
+                    double ip = rint(e0);
+                    const double f = exp2(e0 - ip);
+                    ip = fmin(fmax(ip, -400.0), 400.0);
+                    const int ii = (int)ip;
+                    const int i1 = max(-100, min(100, ii));
+                    const int i2 = max(-126, min(126, ii - i1));
+                    v = make_float2((float)ldexp(lam < 0.0 ? -f : f, i1), __int_as_float((i2 + 127) << 23));
+                }
+                sm.A[k] = v;
+                if (k < 128) sm.B[k] = (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0)));
+            }
+            __syncthreads();
+            // expand into the per-pattern table when this CTA stays in the segment for a while
+            table_mode = (t_stop - t) >= 2;
+            if (table_mode) {
+                g_base = (uint32_t)(sm.e_top - 31) << 7;
+                if (tid == 0) sm.lut[kLut] = 0.0f;
+                for (int i = tid; i < kLut; i += kThreads) {
+                    const uint32_t mag = g_base + (uint32_t)i;
+                    const float2 av = sm.A[mag >> 7];
+                    sm.lut[i] = (av.x * sm.B[mag & 127u]) * av.y;
+                }
+            }
+        }
+        uint32_t base4 = g_base << 2;
+        if constexpr (HIST) {
+            const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+            const float step = a.step[s];
+            const float inv = (float)(1.0 / (double)step);
+            const bool new_key = !have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits;
+            // where the count window should sit: with the gradient table when there is one, else
+            // where it is (same key) or around the data's scale (new key)
+            uint32_t want_base = sm.cold.c_base;
+            if (GRAD && table_mode) want_base = g_base;
+            else if (new_key) {
+                int e_top;
+                if constexpr (GRAD) e_top = sm.e_top;
+                else e_top = max(33, min(254, window_top_exponent((double)step) + 5));
+                want_base = (uint32_t)(e_top - 31) << 7;
+            }
+            const bool rebase = new_key || want_base != sm.cold.c_base;
+            __syncthreads();
+            if (rebase) {
+                if (have_key) flush_counts(sm, a.clamped, cur_hid);
+                have_key = true;
+                cur_hid = hid;
+                cur_inv_bits = __float_as_uint(inv);
+                if (tid == 0) {
+                    sm.cold.inv = inv;
+                    sm.cold.qmin = a.qmin;
+                    sm.cold.qmax = a.qmax;
+                    sm.cold.row = reinterpret_cast<unsigned long long *>(a.hist) +
+                                  (int64_t)hid * ((int64_t)a.qmax - (int64_t)a.qmin + 1);
+                    sm.cold.c_base = want_base;
+                }
+            }
+            if constexpr (!GRAD) table_mode = true;    // histogram only: the count window is the table window
+            base4 = want_base << 2;
+        }
+        __syncthreads();
+
+        // ---- stream the run
+        const int64_t off = (int64_t)(t - t_first) * kTile;
+        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
+        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
+        TG *gout = nullptr;
+        if constexpr (GRAD) {
+            if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
+        }
+        Acc acc;
+        if (table_mode) process_range<TG, FLAGS, true>(x, gout, n, accumulate, base4, sm, acc);
+        else process_range<TG, FLAGS, false>(x, gout, n, accumulate, base4, sm, acc);
+
+        if constexpr (MOM || GRAD) reduce_partials<FLAGS>(a.part, t, t_stop, acc, sm);
+        else __syncthreads();
+        t = t_stop;
+    }
+    if constexpr (HIST) {
+        if (have_key) flush_counts(sm, a.clamped, cur_hid);
+    }
+}
+
+template <typename TG, int FLAGS>
+cudaError_t launch_one(const StreamArgs &a, int sm_count, cudaStream_t st)
+{
+    auto kern = tail_bf16_kernel<TG, FLAGS>;
+    // more than 48 KB of dynamic shared memory needs the opt-in (per function and device)
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem));
+    if (e != cudaSuccess) return e;
+    const int grid = (int)min((int64_t)a.map.n_tiles, (int64_t)sm_count * kCtasPerSm);
+    kern<<<grid, kThreads, sizeof(Smem), st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename TG>
+cudaError_t launch_typed(int flags, const StreamArgs &a, int sm_count, cudaStream_t st)
+{
+    switch (flags) {
+    case kGrad: return launch_one<TG, kGrad>(a, sm_count, st);
+    case kHist: return launch_one<TG, kHist>(a, sm_count, st);
+    case kGrad | kHist: return launch_one<TG, kGrad | kHist>(a, sm_count, st);
+    case kMoments | kGrad: return launch_one<TG, kMoments | kGrad>(a, sm_count, st);
+    case kMoments | kHist: return launch_one<TG, kMoments | kHist>(a, sm_count, st);
+    case kMoments | kGrad | kHist: return launch_one<TG, kMoments | kGrad | kHist>(a, sm_count, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
+                             int sm_count, cudaStream_t st)
+{
+    if (a.map.n_tiles <= 0) return cudaSuccess;
+    if (has_grad_out && grad_dtype == GG_BF16) return launch_typed<uint16_t>(flags, a, sm_count, st);
+    return launch_typed<float>(flags, a, sm_count, st);
+}
+
+}  // namespace gg
