@@ -26,7 +26,7 @@ STEP = 2.0 ** -10
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--divisor", type=int, default=1,
@@ -47,12 +47,27 @@ def measured_peak():
         return 6650.0, "fallback (earlier copy measurement on this pool)"
 
 
-def traffic_per_element():
-    """DRAM bytes per element of the second-sweep kernel from the committed ncu capture, if any."""
-    path = os.path.join(ROOT, "profiles", "tail_sweep_traffic.json")
+TAIL_KERNEL_SOURCE = os.path.join(ROOT, "paper_2506_00486_b200", "csrc", "gg_tail_bf16.cu")
+
+
+def traffic_per_element(grad_dtype):
+    """DRAM bytes per element of the second-sweep kernel from the committed ncu capture
+    (profiles/traffic_tail_bf16_kernel.txt: `key = value` lines).  None if there is no capture for this
+    gradient type or if the kernel source has changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "traffic_tail_bf16_kernel.txt")
     try:
+        kv = {}
         with open(path) as f:
-            return json.load(f)
+            for line in f:
+                if "=" in line and not line.lstrip().startswith("#"):
+                    k, v = line.split("=", 1)
+                    kv[k.strip()] = v.strip()
+        with open(TAIL_KERNEL_SOURCE, "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+        if kv.get("kernel_source_sha256") != digest or kv.get("grad_dtype") != grad_dtype:
+            return None
+        return float(kv["dram_bytes_per_element"])
     except Exception:
         return None
 
@@ -68,7 +83,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "200"], stdout=self.file, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -247,11 +262,9 @@ def run_ours(args):
     tail_ms = ms_tail / max(n_tail, 1)
     first_ms = ms_first / max(n_first, 1)
     achieved = alg_bytes / (tail_ms * 1e-3) / 1e9 if tail_ms > 0 else None
-    tr = traffic_per_element()
-    traffic = None
-    if tr and tr.get("grad_dtype") == args.grad_dtype:
-        traffic = tr["dram_bytes_per_element"] * n_elem
-    roofline = {"bound": "hbm", "kernel": "stream_kernel<bf16, %s, grad|hist> (second sweep)" % args.grad_dtype,
+    tr = traffic_per_element(args.grad_dtype)
+    traffic = tr * n_elem if tr is not None else None
+    roofline = {"bound": "hbm", "kernel": "tail_bf16_kernel<%s grad, grad|hist> (second sweep)" % args.grad_dtype,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                 "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
                 "traffic": traffic, "peak_source": peak_src, "ms_per_launch": tail_ms,
