@@ -218,6 +218,32 @@ gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double
  * all results are in host memory.  Pinned host buffers make the copies asynchronous. */
 gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *args, int64_t chunk_bytes);
 
+/* Moments and fit of ONE segment without allocating anything (the paper has no counterpart: this is
+ * gg_fit for callers that cannot allocate).  gg_fit keeps its tile tables and per-tile partial sums in
+ * a plan that the context obtains with cudaMalloc the first time it sees a layout.  Callers that run
+ * while an allocator owns or has frozen the device's memory (a caching pool that must not see side
+ * allocations, a step whose buffer addresses must not move, a plug-in that is given buffers and a
+ * stream and nothing more) cannot afford that.  This call needs no context and calls neither
+ * cudaMalloc, cudaFree nor any allocating routine: its tables and partials live in a fixed array of
+ * about 0.7 MB inside the library image, which every GPU that loads the library holds until exit.
+ *   device    CUDA device that owns `x` and the outputs (compute capability 10.x, index < 64)
+ *   x         device data of type `dtype`, `len` elements, element aligned
+ *   len       0 <= len <= gg_fit_noalloc_max_len() (2^28 elements); a longer segment is refused with
+ *             GG_ERR_WORKSPACE and nothing is enqueued
+ *   beta, alpha, sum_abs, sum_sq, count, flags   device outputs of ONE element each, as in gg_fit
+ *             (sum_abs, sum_sq, count, flags may be NULL)
+ * The results are those of gg_fit on the same segment (same kernels, same summation order).
+ * The first call on a device looks up the array's device address and the device's architecture; make
+ * that first call before any stream capture begins.  Later calls only enqueue three kernels on
+ * `stream`.  All calls on a device share the one array, which keeps the previous call's contents; each
+ * call rewrites every entry it reads, so calls that follow one another on the GPU are independent, but
+ * two calls whose kernels overlap on the GPU (different streams, no ordering between them) race on
+ * the array and give undefined results. */
+gg_status gg_fit_noalloc(int device, const void *x, int64_t len, gg_dtype dtype, double *beta,
+                         double *alpha, double *sum_abs, double *sum_sq, int64_t *count,
+                         uint32_t *flags, void *stream);
+int64_t gg_fit_noalloc_max_len(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -82,6 +82,9 @@ def lib():
         L.gg_timing_enable.argtypes = [_P, ctypes.c_int]
         L.gg_timing_read.argtypes = [_P, ctypes.POINTER(d), ctypes.POINTER(i64), ctypes.POINTER(d),
                                      ctypes.POINTER(i64)]
+        L.gg_fit_noalloc.argtypes = [ctypes.c_int, _P, i64, ctypes.c_int, _P, _P, _P, _P, _P, _P, _P]
+        L.gg_fit_noalloc.restype = ctypes.c_int
+        L.gg_fit_noalloc_max_len.restype = i64
         for name in ("gg_create", "gg_destroy", "gg_fit", "gg_penalty_grad", "gg_rate_hist", "gg_sample",
                      "gg_fused", "gg_fused_host", "gg_timing_enable", "gg_timing_read"):
             getattr(L, name).restype = ctypes.c_int
@@ -99,6 +102,27 @@ def gg_init_alpha(d_in, xi, beta):
 
 def gg_diff_entropy_bits(alpha, beta):
     return lib().gg_diff_entropy_bits(float(alpha), float(beta))
+
+
+def gg_fit_noalloc(x, out=None):
+    """Moments and fit of one contiguous CUDA tensor through the entry point that allocates nothing.
+
+    For callers that cannot allocate device memory at the time of the call, `out` carries the six
+    one-element device tensors (beta, alpha, sum_abs, sum_sq: float64; count: int64; flags: int32)
+    prepared beforehand; without it they are created here with torch (which does allocate)."""
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("need a contiguous CUDA tensor")
+    dev = x.device
+    if out is None:
+        out = dict(beta=torch.empty(1, dtype=torch.float64, device=dev), alpha=torch.empty(1, dtype=torch.float64, device=dev),
+                   sum_abs=torch.empty(1, dtype=torch.float64, device=dev), sum_sq=torch.empty(1, dtype=torch.float64, device=dev),
+                   count=torch.empty(1, dtype=torch.int64, device=dev), flags=torch.empty(1, dtype=torch.int32, device=dev))
+    status = lib().gg_fit_noalloc(dev.index or 0, x.data_ptr() if x.numel() else None, x.numel(), _dtype_code(x.dtype),
+                                  _ptr(out["beta"]), _ptr(out["alpha"]), _ptr(out["sum_abs"]), _ptr(out["sum_sq"]),
+                                  _ptr(out["count"]), _ptr(out["flags"]), _stream_ptr(dev))
+    if status != 0:
+        raise GGError(status, lib().gg_status_str(status).decode())
+    return out
 
 
 def _dtype_code(dt):
