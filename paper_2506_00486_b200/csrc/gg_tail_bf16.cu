@@ -4,18 +4,25 @@
 // Persistent CTAs each walk one contiguous range of tiles.  Inside a segment that range is one
 // contiguous run of elements, streamed with 128-bit loads issued two iterations ahead.
 //   * gradient: |g| depends only on the 15-bit magnitude pattern.  |g| = A[e] * B[j] with e the
-//     exponent field and j the 7 mantissa bits: A[e] = 2^(L + b (e-127)) (kept as a normal-range
-//     factor times a power of two), B[j] = (1 + j/128)^b, both rounded once from fp64, so the
-//     product is within 1.5 ulp for every shape beta.  For runs of two tiles or more the CTA
-//     expands the 32 binades below 2^6 standard deviations into a 4096-entry table, so an element
-//     costs one shared-memory load.
-//   * histogram: elements are counted by bit pattern (4096 magnitudes x 2 signs in shared memory);
-//     patterns become quantised symbols only when the table is flushed, i.e. when the histogram,
-//     its step or the window changes, or the CTA ends.  Patterns outside the window (zeros, tiny
-//     or huge values) are quantised on the spot into a small symbol window, else straight to
-//     global memory.  Counts are integers, so every order of additions gives the same table.
-//   * in table mode both tables share one window and the element path is branch free: an element
-//     outside the window hits sentinel cells and is redone after its vector.
+//     exponent field and j the 7 mantissa bits: A[e] = 2^(L + b (e-127)), B[j] = (1 + j/128)^b,
+//     both rounded once from fp64, so the product is within 1.5 ulp for every shape beta.
+//   * histogram: elements are counted by bit pattern in shared memory; patterns become quantised
+//     symbols only when the table is flushed, i.e. when the histogram, its step or the window
+//     changes, or the CTA ends.  Counts are integers, so every order of additions gives the same
+//     table.
+// The kernel's limit is the shared-memory pipe (one 128-byte wavefront per clock and SM), so the
+// tables are laid out to avoid bank conflicts:
+//   * inside a window of 32 binades below 2^5 standard deviations, A and B are replicated once per
+//     bank (lane l reads word l of a row, so a look-up is one wavefront whatever the data);
+//   * counts have two layouts.  Symbol mode, used when the quantiser is coarse enough that symbols
+//     [-256, 256) hold all but the far tails (256 steps >= 6.5 standard deviations): one row of 32
+//     words per symbol, lane l counts in word l, so the atomic is one wavefront too; the symbol is
+//     floor(x * inv) taken with a round-down add of 1.5 * 2^23.  Pattern mode otherwise: one cell
+//     per bf16 magnitude pattern and sign over the upper 16 binades of the window, four replicas
+//     per cell selected by the low lane bits.
+// The element path inside the windows is branch free; an element outside one (zero, tiny, huge,
+// inf, nan, a far-tail symbol) reads zero or counts in a sentinel cell, and is redone after its
+// vector.
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -24,31 +31,46 @@
 namespace gg {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
-constexpr int kLut = 4096;       // magnitude patterns in the gradient table (32 binades)
-constexpr int kCnt = 4096;       // magnitude patterns in the count table (two cells each: + and -)
-constexpr int kSymWin = 512;     // secondary symbol window [-256, 256)
-constexpr int kCtasPerSm = 4;
-constexpr uint32_t kWinBytes = kLut * 4;
+constexpr int kCtasPerSm = 2;
+constexpr int kGradBinades = 32;                    // binades in the gradient window
+constexpr uint32_t kGradPat = kGradBinades * 128;   // magnitude patterns in it (a power of two)
+constexpr int kCntBinades = 16;                     // pattern-count window: the upper binades of the gradient window
+constexpr uint32_t kCntPat = kCntBinades * 128;
+constexpr int kRep = 4;                             // replicas of every pattern-count cell
+constexpr uint32_t kSymCells = 512;                 // symbol-count window: symbols [-256, 256)
+constexpr uint32_t kMagicBits = 0x4B400000u;        // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
+constexpr uint32_t kSymBase = kMagicBits - kSymCells / 2;
+constexpr int kSymWin = 512;                        // secondary symbol window [-256, 256) of the rare path
+constexpr uint32_t kCntWords = (kSymCells + 1) * 32 > (kCntPat + 1) * 2 * kRep ? (kSymCells + 1) * 32
+                                                                              : (kCntPat + 1) * 2 * kRep;
+enum : int { kModePlain = 0, kModePattern = 1, kModeSymbol = 2 };
 
 // Constants of the current segment / histogram that only the cold paths need: kept in shared
 // memory so that the streaming loop does not carry them in registers.
 struct Cold {
     double L, b;               // g = 2^(L + b log2|x|)
+    double sd;                 // standard deviation of the density the gradient belongs to
     uint32_t sign_flip;        // 0x80000000 if lambda < 0 (the tables then hold -|g|)
     int active;                // 0: the gradient is zero everywhere
     float inv;                 // quantiser: q = floor(x * inv)
     int32_t qmin, qmax;
     unsigned long long *row;   // the current histogram, bin 0 = symbol qmin
-    uint32_t c_base;           // first magnitude pattern of the count window
+    uint32_t c_base;           // first magnitude pattern of the pattern-count window
+    int symbol_mode;           // layout of cnt: 1 = rows of symbols, 0 = cells of patterns
 };
 
 struct Smem {
-    float lut[kLut + 1];            // last cell: sentinel for out-of-window elements (zero)
-    uint32_t cnt[2 * kCnt + 2];     // cell 2 i + s: magnitude pattern c_base + i with sign s; last two: sentinel
+    // pattern mode: cell ((p * 2 + sign) * kRep + r) = magnitude pattern c_base + p, replica r; slot
+    // p = kCntPat is the sentinel that swallows the counts of out-of-window elements.
+    // symbol mode: word (s * 32 + lane) = symbol s - 256 counted by that lane; row s = kSymCells is
+    // the sentinel.
+    uint32_t cnt[kCntWords];
+    float arep[(kGradBinades + 1) * 32];   // row e: A of binade e of the window in every bank; last row: zeros
+    float brep[128 * 32];                  // row j: B[j] in every bank
     uint32_t win[kSymWin];
-    float2 A[256];
+    float2 A[256];                         // every exponent: value = A.x * A.y, A.y a power of two
     float B[128];
     double red[3][kWarps];
     uint32_t bad[kWarps];
@@ -113,8 +135,14 @@ struct Run {   // fp32 partials of one short run of elements
     float m1 = 0.0f, m2 = 0.0f, mp = 0.0f;
 };
 
-// Byte offset of a value's count cell: (pattern index) * 8 + sign * 4.
-__device__ __forceinline__ uint32_t count_cell(uint32_t off4, uint32_t xb) { return (off4 << 1) + ((xb >> 29) & 4u); }
+// Per-thread constants of the element path.
+struct Lane {
+    uint32_t gbase;    // first magnitude pattern of the gradient window
+    uint32_t cbase;    // first magnitude pattern of the pattern-count window
+    uint32_t lane4;    // (lane id) * 4: byte offset of this lane's bank inside a replicated row
+    uint32_t rep4;     // (lane id mod kRep) * 4: byte offset of this lane's pattern-count replica
+    float inv;         // quantiser scale (symbol mode)
+};
 
 template <int FLAGS>
 __device__ __forceinline__ void moments_elem(uint32_t xb, Acc &acc, Run &r)
@@ -131,22 +159,60 @@ __device__ __forceinline__ void moments_elem(uint32_t xb, Acc &acc, Run &r)
     }
 }
 
-// One element given as fp32 bits (a widened bf16: the low 16 bits are zero), table mode.  Branch
-// free: `anyoff` collects the window offsets so one compare per vector finds elements that
-// missed the window; those read and count in the sentinel cells and are redone by fix_rare().
-template <int FLAGS>
-__device__ __forceinline__ float one_table(uint32_t xb, uint32_t base4, Smem &sm, Acc &acc, Run &r, uint32_t &anyoff)
+// Byte offset of a value's pattern-count cell (without the replica): (p * 2 + sign) * kRep * 4.
+__device__ __forceinline__ uint32_t count_cell(uint32_t p, uint32_t xb)
+{
+    return (p << 5) + ((xb >> 27) & 16u);
+}
+
+// Row of a value in the symbol-count table: floor(x * inv) + 256 as an unsigned number, so that
+// every symbol outside [-256, 256), and inf and nan, give a row >= kSymCells.
+__device__ __forceinline__ uint32_t symbol_row(uint32_t xb, float inv)
+{
+    const float t = __fmul_rn(__uint_as_float(xb), inv);
+    // for |t| < 2^22 the sum lies in [2^23, 2^24) where floats are the integers: rounding down gives floor
+    return __float_as_uint(__fadd_rd(t, __uint_as_float(kMagicBits))) - kSymBase;
+}
+
+// Where the miss thresholds of the two windows sit in the collected index bits.
+template <int MODE>
+__device__ __forceinline__ bool any_miss(uint32_t anyg, uint32_t anyc)
+{
+    return (anyg >= kGradPat) | (anyc >= (MODE == kModeSymbol ? kSymCells : kCntPat));
+}
+
+// One element given as fp32 bits (a widened bf16: the low 16 bits are zero), window modes.  Branch
+// free: `anyg` / `anyc` collect the window indices so one compare per vector finds elements that
+// missed a window; those read a zero gradient or count in the sentinel cells and are redone by the
+// fix-up below.
+template <int FLAGS, int MODE>
+__device__ __forceinline__ float one_window(uint32_t xb, const Lane &ln, Smem &sm, Acc &acc, Run &r, uint32_t &anyg,
+                                            uint32_t &anyc)
 {
     moments_elem<FLAGS>(xb, acc, r);
     const uint32_t am = xb & 0x7FFFFFFFu;
-    uint32_t off = (am >> 14) - base4;              // (magnitude pattern - window base) * 4
-    anyoff |= off;
-    off = min(off, kWinBytes);
     float ga = 0.0f;
-    if constexpr ((FLAGS & kGrad) != 0)
-        ga = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.lut) + off);
-    if constexpr ((FLAGS & kHist) != 0)
-        atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(off, xb)), 1u);
+    if constexpr ((FLAGS & kGrad) != 0) {
+        uint32_t p = (am >> 16) - ln.gbase;              // index of the magnitude pattern in the window
+        anyg |= p;
+        p = min(p, kGradPat);
+        const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.arep) + ((p & ~127u) | ln.lane4));
+        const float b = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.brep) + (((p & 127u) << 7) | ln.lane4));
+        ga = a * b;
+    }
+    if constexpr ((FLAGS & kHist) != 0) {
+        if constexpr (MODE == kModeSymbol) {
+            uint32_t row = symbol_row(xb, ln.inv);
+            anyc |= row;
+            row = min(row, kSymCells);
+            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + ((row << 7) | ln.lane4)), 1u);
+        } else {
+            uint32_t p = (am >> 16) - ln.cbase;
+            anyc |= p;
+            p = min(p, kCntPat);
+            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(p, xb) + ln.rep4), 1u);
+        }
+    }
     if constexpr ((FLAGS & kGrad) != 0) {
         r.mp = fmaf(__uint_as_float(am), fabsf(ga), r.mp);
         return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
@@ -154,32 +220,45 @@ __device__ __forceinline__ float one_table(uint32_t xb, uint32_t base4, Smem &sm
     return 0.0f;
 }
 
-// Redo of an element that fell outside the table window (zero, tiny, huge, inf, nan).
-template <int FLAGS>
-__device__ __noinline__ float fix_rare(uint32_t xb, Smem &sm, Run &r)
+// Gradient of an element outside the gradient window (zero, tiny, huge, inf, nan).
+__device__ __noinline__ float fix_grad(uint32_t xb, Smem &sm, Run &r)
 {
-    float ga = 0.0f;
-    if constexpr ((FLAGS & kGrad) != 0) {
-        ga = grad_ab((xb >> 16) & 0x7FFFu, sm);
-        r.mp = fmaf(__uint_as_float(xb & 0x7FFFFFFFu), fabsf(ga), r.mp);
-    }
-    if constexpr ((FLAGS & kHist) != 0) count_symbol(__uint_as_float(xb), 1u, true, sm);
+    const float ga = grad_ab((xb >> 16) & 0x7FFFu, sm);
+    r.mp = fmaf(__uint_as_float(xb & 0x7FFFFFFFu), fabsf(ga), r.mp);
     return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
 }
 
-// The same element when the gradient table is off (short runs): gradient from the A/B tables,
-// count window wherever it currently sits (base4 = its base * 4).
+// Redo of whatever part of an element missed its window; g is the gradient from the first pass.
+template <int FLAGS, int MODE>
+__device__ __forceinline__ float fix_elem(uint32_t xb, float g, const Lane &ln, Smem &sm, Run &r)
+{
+    const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
+    if constexpr ((FLAGS & kGrad) != 0) {
+        if (mag - ln.gbase >= kGradPat) g = fix_grad(xb, sm, r);
+    }
+    if constexpr ((FLAGS & kHist) != 0) {
+        bool miss;
+        if constexpr (MODE == kModeSymbol) miss = symbol_row(xb, ln.inv) >= kSymCells;
+        else miss = mag - ln.cbase >= kCntPat;
+        if (miss) count_rare(xb, sm);
+    }
+    return g;
+}
+
+// The same element when the replicated tables are off (a gradient whose factors leave the fp32
+// range inside the window, or no gradient at all): gradient from the A/B tables of all
+// exponents, pattern-count window as usual.
 template <int FLAGS>
-__device__ __forceinline__ float one_plain(uint32_t xb, uint32_t base4, Smem &sm, Acc &acc, Run &r)
+__device__ __forceinline__ float one_plain(uint32_t xb, const Lane &ln, Smem &sm, Acc &acc, Run &r)
 {
     moments_elem<FLAGS>(xb, acc, r);
     const uint32_t am = xb & 0x7FFFFFFFu;
     float ga = 0.0f;
     if constexpr ((FLAGS & kGrad) != 0) ga = grad_ab(am >> 16, sm);
     if constexpr ((FLAGS & kHist) != 0) {
-        const uint32_t off = (am >> 14) - base4;
-        if (off < kWinBytes)
-            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(off, xb)), 1u);
+        const uint32_t p = (am >> 16) - ln.cbase;
+        if (p < kCntPat)
+            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(p, xb) + ln.rep4), 1u);
         else
             count_rare(xb, sm);
     }
@@ -215,10 +294,19 @@ __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &
     }
 }
 
+// Eight gradient values to g.  `wide`: g is 32-byte aligned, so fp32 output goes out as one
+// 256-bit store per thread (a full 32-byte sector per lane, 1 KB contiguous per warp).
 template <typename TG>
-__device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumulate)
+__device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumulate, bool wide)
 {
     if constexpr (sizeof(TG) == 4) {
+        if (wide && !accumulate) {
+            // written once, never re-read by this pass: streaming (evict-first) store
+            asm volatile("st.global.cs.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(g), "f"(v[0]), "f"(v[1]),
+                         "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                         : "memory");
+            return;
+        }
         float4 *p = reinterpret_cast<float4 *>(g);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -227,7 +315,7 @@ __device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumula
                 const float4 old = p[i];
                 o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
             }
-            __stcs(p + i, o);     // written once, never re-read by this pass: streaming store
+            __stcs(p + i, o);
         }
     } else {
         uint32_t w[4];
@@ -247,25 +335,44 @@ __device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumula
     }
 }
 
-// Exponent field of the top binade of a 32-binade window that reaches 2^6 times `scale`.
-__device__ __forceinline__ int window_top_exponent(double scale)
+// Exponent field of the top binade of a window of `binades` binades that reaches 2^(above+1) times
+// `scale`.
+__device__ __forceinline__ int window_top_exponent(double scale, int above, int binades)
 {
-    int e = 127 + 6;
-    if (scale > 0.0 && scale < 1e300) e = ilogb(scale) + 127 + 6;
-    return max(33, min(254, e));
+    int e = 127 + above;
+    if (scale > 0.0 && scale < 1e300) e = ilogb(scale) + 127 + above;
+    return max(binades, min(254, e));
 }
 
-// Turns the counted patterns into symbols of the current histogram and empties the tables.
+// Adds the counted cells to the current histogram and empties the tables.
 __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
 {
     // (callers synchronise before: all counting under the old key is complete)
-    const uint32_t c_base = sm.cold.c_base;
-    for (int p = threadIdx.x; p < 2 * kCnt; p += kThreads) {
-        const uint32_t n = sm.cnt[p];
-        if (n != 0u) {
-            sm.cnt[p] = 0u;
-            const uint32_t h = (c_base + (uint32_t)(p >> 1)) | ((uint32_t)(p & 1) << 15);
-            count_symbol(__uint_as_float(h << 16), n, false, sm);
+    if (sm.cold.symbol_mode) {
+        const int lane = threadIdx.x & 31;
+        for (uint32_t row = threadIdx.x >> 5; row <= kSymCells; row += kWarps) {
+            const uint32_t v = sm.cnt[row * 32 + lane];
+            const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, v);
+            if (n != 0u) {
+                sm.cnt[row * 32 + lane] = 0u;
+                // symbols [-256, 256) lie inside [qmin, qmax] in this mode; the sentinel row is only emptied
+                if (lane == 0 && row < kSymCells)
+                    atomicAdd(&sm.cold.row[((int)row - (int)(kSymCells / 2)) - sm.cold.qmin], (unsigned long long)n);
+            }
+        }
+    } else {
+        const uint32_t c_base = sm.cold.c_base;
+        for (uint32_t c = threadIdx.x; c < (kCntPat + 1) * 2; c += kThreads) {   // c = p * 2 + sign
+            uint4 *cell = reinterpret_cast<uint4 *>(sm.cnt) + c;
+            const uint4 v = *cell;
+            const uint32_t n = v.x + v.y + v.z + v.w;
+            if (n != 0u) {
+                *cell = make_uint4(0u, 0u, 0u, 0u);
+                if (c < kCntPat * 2) {          // the sentinel slot is only emptied
+                    const uint32_t h = (c_base + (c >> 1)) | ((c & 1u) << 15);
+                    count_symbol(__uint_as_float(h << 16), n, false, sm);
+                }
+            }
         }
     }
     for (int i = threadIdx.x; i < kSymWin; i += kThreads) {
@@ -342,46 +449,46 @@ __device__ void reduce_partials(const TileScratch &part, int t0, int t1, const A
     __syncthreads();
 }
 
-template <typename TG, int FLAGS, bool TABLE>
-__device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool accumulate, uint32_t base4,
+template <typename TG, int FLAGS, int MODE>
+__device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool accumulate, bool wide, const Lane &ln,
                                             Smem &sm, Acc &acc)
 {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     float g[8];
     Run r;
-    if constexpr (TABLE) {
-        uint32_t anyoff = 0;
+    if constexpr (MODE != kModePlain) {
+        uint32_t anyg = 0, anyc = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            g[2 * i] = one_table<FLAGS>(w[i] << 16, base4, sm, acc, r, anyoff);
-            g[2 * i + 1] = one_table<FLAGS>(w[i] & 0xFFFF0000u, base4, sm, acc, r, anyoff);
+            g[2 * i] = one_window<FLAGS, MODE>(w[i] << 16, ln, sm, acc, r, anyg, anyc);
+            g[2 * i + 1] = one_window<FLAGS, MODE>(w[i] & 0xFFFF0000u, ln, sm, acc, r, anyg, anyc);
         }
-        if (anyoff >= kWinBytes) {      // some element missed the window
+        if (any_miss<MODE>(anyg, anyc)) {      // some element missed a window
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-                if (((xb & 0x7FFFFFFFu) >> 14) - base4 >= kWinBytes) g[i] = fix_rare<FLAGS>(xb, sm, r);
+                g[i] = fix_elem<FLAGS, MODE>(xb, g[i], ln, sm, r);
             }
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            g[2 * i] = one_plain<FLAGS>(w[i] << 16, base4, sm, acc, r);
-            g[2 * i + 1] = one_plain<FLAGS>(w[i] & 0xFFFF0000u, base4, sm, acc, r);
+            g[2 * i] = one_plain<FLAGS>(w[i] << 16, ln, sm, acc, r);
+            g[2 * i + 1] = one_plain<FLAGS>(w[i] & 0xFFFF0000u, ln, sm, acc, r);
         }
     }
     close_run<FLAGS>(raw, 8, r, acc, sm);
     if constexpr ((FLAGS & kGrad) != 0) {
-        if (gdst != nullptr) store8<TG>(gdst, g, accumulate);
+        if (gdst != nullptr) store8<TG>(gdst, g, accumulate, wide);
     }
 }
 
 // One contiguous run of n elements: scalar head up to the first 16-byte boundary of x, 128-bit
 // vector body with loads issued two iterations ahead, scalar tail.  If the gradient's address is
 // not 16-byte aligned at the same element the whole run is scalar.
-template <typename TG, int FLAGS, bool TABLE>
+template <typename TG, int FLAGS, int MODE>
 __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
-                                              uint32_t base4, Smem &sm, Acc &acc)
+                                              const Lane &ln, Smem &sm, Acc &acc)
 {
     constexpr bool GRAD = (FLAGS & kGrad) != 0;
     const int tid = threadIdx.x;
@@ -396,12 +503,12 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
         const uint32_t h = (uint32_t)__ldg(x + idx);
         Run r;
         float g;
-        if constexpr (TABLE) {
-            uint32_t anyoff = 0;
-            g = one_table<FLAGS>(h << 16, base4, sm, acc, r, anyoff);
-            if (anyoff >= kWinBytes) g = fix_rare<FLAGS>(h << 16, sm, r);
+        if constexpr (MODE != kModePlain) {
+            uint32_t anyg = 0, anyc = 0;
+            g = one_window<FLAGS, MODE>(h << 16, ln, sm, acc, r, anyg, anyc);
+            if (any_miss<MODE>(anyg, anyc)) g = fix_elem<FLAGS, MODE>(h << 16, g, ln, sm, r);
         } else {
-            g = one_plain<FLAGS>(h << 16, base4, sm, acc, r);
+            g = one_plain<FLAGS>(h << 16, ln, sm, acc, r);
         }
         close_run<FLAGS>(make_uint4(h, 0u, 0u, 0u), 1, r, acc, sm);
         if constexpr (GRAD) {
@@ -418,18 +525,22 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
         }
     }
 
-    const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
-    TG *gv = gout != nullptr ? gout + head : nullptr;
-    int64_t v = tid;
+    // (a CTA's run never exceeds device memory / grid size elements: 32-bit vector indices suffice)
+    const uint4 *xv = reinterpret_cast<const uint4 *>(x + head) + tid;
+    TG *gv = gout != nullptr ? gout + head + (int64_t)tid * 8 : nullptr;
+    const bool wide = (reinterpret_cast<uintptr_t>(gv) & 31u) == 0;
+    const int nv = (int)nvec;
     uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
-    if (v < nvec) r0 = __ldcs(xv + v);                       // read once by this sweep: streaming loads
-    if (v + kThreads < nvec) r1 = __ldcs(xv + v + kThreads);
-    for (; v < nvec; v += kThreads) {
+    if (tid < nv) r0 = __ldcs(xv);                           // read once by this sweep: streaming loads
+    if (tid + kThreads < nv) r1 = __ldcs(xv + kThreads);
+    for (int v = tid; v < nv; v += kThreads) {
         uint4 r2 = make_uint4(0u, 0u, 0u, 0u);
-        if (v + 2 * kThreads < nvec) r2 = __ldcs(xv + v + 2 * kThreads);
-        process_vec<TG, FLAGS, TABLE>(r0, gv != nullptr ? gv + v * 8 : nullptr, accumulate, base4, sm, acc);
+        if (v + 2 * kThreads < nv) r2 = __ldcs(xv + 2 * kThreads);
+        process_vec<TG, FLAGS, MODE>(r0, gv, accumulate, wide, ln, sm, acc);
         r0 = r1;
         r1 = r2;
+        xv += kThreads;
+        if (gv != nullptr) gv += kThreads * 8;
     }
 }
 
@@ -447,15 +558,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
     const int t_end = (int)(nt * (blockIdx.x + 1) / gridDim.x);
 
     if constexpr (HIST) {
-        for (int i = tid; i < 2 * kCnt + 2; i += kThreads) sm.cnt[i] = 0u;
+        for (int i = tid; i < (int)kCntWords; i += kThreads) sm.cnt[i] = 0u;
         for (int i = tid; i < kSymWin; i += kThreads) sm.win[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
-    if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; }
-    int cur_hid = -1;
+    if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.symbol_mode = 0; sm.cold.sd = 0.0; }
+    int cur_hid = -1, cur_mode = kModePattern;
     uint32_t cur_inv_bits = 0;
     bool have_key = false;
     const bool accumulate = GRAD && a.accumulate != 0;
+    Lane ln;
+    ln.lane4 = (uint32_t)(tid & 31) * 4u;
+    ln.rep4 = (uint32_t)(tid & (kRep - 1)) * 4u;
+    ln.gbase = 0x8000u;
+    ln.cbase = 0x8000u;
+    ln.inv = 0.0f;
     __syncthreads();
 
     for (int t = t_begin; t < t_end;) {
@@ -464,7 +581,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         const int64_t len = a.map.seg_len[s];
         const int t_first = a.map.tile_prefix[s];
         const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
-        bool table_mode = false;
+        int mode = kModePlain;
         uint32_t g_base = 0x8000u;
 
         if constexpr (GRAD) {
@@ -476,15 +593,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                 sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
                 sm.cold.active = active;
                 sm.cold.L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
-                // the standard deviation of the fitted density (Eq. 2-3) places the table window
-                const double sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
-                sm.e_top = window_top_exponent(sd);
+                // the standard deviation of the fitted density (Eq. 2-3) places the window
+                sm.cold.sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
+                sm.e_top = window_top_exponent(sm.cold.sd, 4, kGradBinades);
             }
             __syncthreads();
-            {
-                const double L = sm.cold.L, b = sm.cold.b;
-                const int k = tid;      // kThreads == 256 entries of A
-                float2 v = make_float2(0.0f, 0.0f);
+            const double L = sm.cold.L, b = sm.cold.b;
+            if (tid < 256) {
+                const int k = tid;
+                float2 v = make_float2(0.0f, 1.0f);
                 if (active && k >= 1 && k <= 254) {
                     const double e0 = L + b * (double)(k - 127);
                     double ip = rint(e0);
@@ -496,44 +613,56 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                     v = make_float2((float)ldexp(lam < 0.0 ? -f : f, i1), __int_as_float((i2 + 127) << 23));
                 }
                 sm.A[k] = v;
-                if (k < 128) sm.B[k] = (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0)));
+            } else if (tid < 384) {
+                const int k = tid - 256;
+                sm.B[k] = (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0)));
             }
+            g_base = (uint32_t)(sm.e_top - (kGradBinades - 1)) << 7;
             __syncthreads();
-            // expand into the per-pattern table when this CTA stays in the segment for a while
-            table_mode = (t_stop - t) >= 2;
-            if (table_mode) {
-                g_base = (uint32_t)(sm.e_top - 31) << 7;
-                if (tid == 0) sm.lut[kLut] = 0.0f;
-                for (int i = tid; i < kLut; i += kThreads) {
-                    const uint32_t mag = g_base + (uint32_t)i;
-                    const float2 av = sm.A[mag >> 7];
-                    sm.lut[i] = (av.x * sm.B[mag & 127u]) * av.y;
-                }
+            // The replicated tables hold A[e].x alone, so they serve only if no exponent of the
+            // window needs the power-of-two factor A[e].y (|L + b (e-127)| <= 100: products of the
+            // two table entries then stay in the normal fp32 range).
+            bool row_ok = true;
+            if (tid < kGradBinades) row_ok = sm.A[(g_base >> 7) + tid].y == 1.0f;
+            if (__syncthreads_and(active && row_ok) != 0) {
+                mode = kModePattern;
+                for (int i = tid; i < (kGradBinades + 1) * 32; i += kThreads)
+                    sm.arep[i] = (i >> 5) < kGradBinades ? sm.A[(g_base >> 7) + (i >> 5)].x : 0.0f;
+                for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
             }
         }
-        uint32_t base4 = g_base << 2;
+        ln.gbase = g_base;
         if constexpr (HIST) {
             const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
             const float step = a.step[s];
             const float inv = (float)(1.0 / (double)step);
-            const bool new_key = !have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits;
-            // where the count window should sit: with the gradient table when there is one, else
-            // where it is (same key) or around the data's scale (new key)
+            // where the pattern-count window should sit: on the upper binades of the gradient window
+            // when there is one, else where it is (same key) or from four binades below the step
+            // upwards (new key)
             uint32_t want_base = sm.cold.c_base;
-            if (GRAD && table_mode) want_base = g_base;
-            else if (new_key) {
-                int e_top;
-                if constexpr (GRAD) e_top = sm.e_top;
-                else e_top = max(33, min(254, window_top_exponent((double)step) + 5));
-                want_base = (uint32_t)(e_top - 31) << 7;
+            if constexpr (GRAD) {
+                want_base = g_base + (kGradPat - kCntPat);
+                // symbol mode: the replicated tables are on, symbols [-256, 256) are not clamped, and
+                // they reach 6.5 standard deviations
+                if (mode == kModePattern && a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 &&
+                    step > 0.0f && (double)(kSymCells / 2) * (double)step >= 6.5 * sm.cold.sd && inv < 3.0e38f)
+                    mode = kModeSymbol;
+            } else {
+                mode = kModePattern;        // histogram only: nothing but the pattern-count window
+                if (!have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits)
+                    want_base = (uint32_t)(window_top_exponent((double)step, 11, kCntBinades) - (kCntBinades - 1)) << 7;
             }
-            const bool rebase = new_key || want_base != sm.cold.c_base;
+            const int want_layout = mode == kModeSymbol ? kModeSymbol : kModePattern;
+            const bool new_key = !have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits ||
+                                 want_layout != cur_mode;
+            const bool rebase = new_key || (want_layout == kModePattern && want_base != sm.cold.c_base);
             __syncthreads();
             if (rebase) {
                 if (have_key) flush_counts(sm, a.clamped, cur_hid);
                 have_key = true;
                 cur_hid = hid;
                 cur_inv_bits = __float_as_uint(inv);
+                cur_mode = want_layout;
                 if (tid == 0) {
                     sm.cold.inv = inv;
                     sm.cold.qmin = a.qmin;
@@ -541,10 +670,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                     sm.cold.row = reinterpret_cast<unsigned long long *>(a.hist) +
                                   (int64_t)hid * ((int64_t)a.qmax - (int64_t)a.qmin + 1);
                     sm.cold.c_base = want_base;
+                    sm.cold.symbol_mode = want_layout == kModeSymbol;
                 }
             }
-            if constexpr (!GRAD) table_mode = true;    // histogram only: the count window is the table window
-            base4 = want_base << 2;
+            ln.cbase = want_base;
+            ln.inv = inv;
         }
         __syncthreads();
 
@@ -557,8 +687,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
         }
         Acc acc;
-        if (table_mode) process_range<TG, FLAGS, true>(x, gout, n, accumulate, base4, sm, acc);
-        else process_range<TG, FLAGS, false>(x, gout, n, accumulate, base4, sm, acc);
+        if constexpr (GRAD && HIST) {
+            if (mode == kModeSymbol) process_range<TG, FLAGS, kModeSymbol>(x, gout, n, accumulate, ln, sm, acc);
+            else if (mode == kModePattern) process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
+            else process_range<TG, FLAGS, kModePlain>(x, gout, n, accumulate, ln, sm, acc);
+        } else {
+            if (mode == kModePattern) process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
+            else process_range<TG, FLAGS, kModePlain>(x, gout, n, accumulate, ln, sm, acc);
+        }
 
         if constexpr (MOM || GRAD) reduce_partials<FLAGS>(a.part, t, t_stop, acc, sm);
         else __syncthreads();
