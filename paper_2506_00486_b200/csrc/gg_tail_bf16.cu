@@ -2,7 +2,7 @@
 // for the fact that a bf16 value is one of 65536 bit patterns.
 //
 // Persistent CTAs each walk one contiguous range of tiles.  Inside a segment that range is one
-// contiguous run of elements, streamed with 128-bit loads issued two iterations ahead.
+// contiguous run of elements, streamed as 128-bit vectors.
 //   * gradient: |g| depends only on the 15-bit magnitude pattern.  |g| = A[e] * B[j] with e the
 //     exponent field and j the 7 mantissa bits: A[e] = 2^(L + b (e-127)), B[j] = (1 + j/128)^b,
 //     both rounded once from fp64, so the product is within 1.5 ulp for every shape beta.
@@ -15,11 +15,13 @@
 //   * inside a window of 32 binades below 2^5 standard deviations, A and B are replicated once per
 //     bank (lane l reads word l of a row, so a look-up is one wavefront whatever the data);
 //   * counts have two layouts.  Symbol mode, used when the quantiser is coarse enough that symbols
-//     [-256, 256) hold all but the far tails (256 steps >= 6.5 standard deviations): one row of 32
+//     [-192, 192) hold all but the far tails (192 steps >= 6.5 standard deviations): one row of 32
 //     words per symbol, lane l counts in word l, so the atomic is one wavefront too; the symbol is
 //     floor(x * inv) taken with a round-down add of 1.5 * 2^23.  Pattern mode otherwise: one cell
-//     per bf16 magnitude pattern and sign over the upper 16 binades of the window, four replicas
-//     per cell selected by the low lane bits.
+//     per bf16 magnitude pattern and sign over the upper 16 binades of the window, two replicas
+//     per cell selected by the lowest lane bit.
+// Input vectors reach each thread through a private ring of shared-memory slots filled by
+// asynchronous copies issued kDepth iterations ahead: bytes in flight cost no registers.
 // The element path inside the windows is branch free; an element outside one (zero, tiny, huge,
 // inf, nan, a far-tail symbol) reads zero or counts in a sentinel cell, and is redone after its
 // vector.
@@ -38,8 +40,9 @@ constexpr int kGradBinades = 32;                    // binades in the gradient w
 constexpr uint32_t kGradPat = kGradBinades * 128;   // magnitude patterns in it (a power of two)
 constexpr int kCntBinades = 16;                     // pattern-count window: the upper binades of the gradient window
 constexpr uint32_t kCntPat = kCntBinades * 128;
-constexpr int kRep = 4;                             // replicas of every pattern-count cell
-constexpr uint32_t kSymCells = 512;                 // symbol-count window: symbols [-256, 256)
+constexpr int kRep = 2;                             // replicas of every pattern-count cell
+constexpr uint32_t kSymCells = 384;                 // symbol-count window: symbols [-192, 192)
+constexpr int kDepth = 4;                           // input vectors staged ahead per thread
 constexpr uint32_t kMagicBits = 0x4B400000u;        // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr uint32_t kSymBase = kMagicBits - kSymCells / 2;
 constexpr int kSymWin = 512;                        // secondary symbol window [-256, 256) of the rare path
@@ -64,9 +67,10 @@ struct Cold {
 struct Smem {
     // pattern mode: cell ((p * 2 + sign) * kRep + r) = magnitude pattern c_base + p, replica r; slot
     // p = kCntPat is the sentinel that swallows the counts of out-of-window elements.
-    // symbol mode: word (s * 32 + lane) = symbol s - 256 counted by that lane; row s = kSymCells is
-    // the sentinel.
+    // symbol mode: word (s * 32 + lane) = symbol s - kSymCells/2 counted by that lane; row s = kSymCells
+    // is the sentinel.
     uint32_t cnt[kCntWords];
+    uint4 stage[kDepth][kThreads];         // per-thread ring of input vectors in flight
     float arep[(kGradBinades + 1) * 32];   // row e: A of binade e of the window in every bank; last row: zeros
     float brep[128 * 32];                  // row j: B[j] in every bank
     uint32_t win[kSymWin];
@@ -162,11 +166,12 @@ __device__ __forceinline__ void moments_elem(uint32_t xb, Acc &acc, Run &r)
 // Byte offset of a value's pattern-count cell (without the replica): (p * 2 + sign) * kRep * 4.
 __device__ __forceinline__ uint32_t count_cell(uint32_t p, uint32_t xb)
 {
-    return (p << 5) + ((xb >> 27) & 16u);
+    static_assert(kRep == 2, "cell stride");
+    return (p << 4) + ((xb >> 28) & 8u);
 }
 
-// Row of a value in the symbol-count table: floor(x * inv) + 256 as an unsigned number, so that
-// every symbol outside [-256, 256), and inf and nan, give a row >= kSymCells.
+// Row of a value in the symbol-count table: floor(x * inv) + kSymCells/2 as an unsigned number, so that
+// every symbol outside the window, and inf and nan, give a row >= kSymCells.
 __device__ __forceinline__ uint32_t symbol_row(uint32_t xb, float inv)
 {
     const float t = __fmul_rn(__uint_as_float(xb), inv);
@@ -182,7 +187,7 @@ __device__ __forceinline__ bool any_miss(uint32_t anyg, uint32_t anyc)
 }
 
 // One element given as fp32 bits (a widened bf16: the low 16 bits are zero), window modes.  Branch
-// free: `anyg` / `anyc` collect the window indices so one compare per vector finds elements that
+// free: `anyg` (bitwise or) and `anyc` (maximum) collect the window indices so one compare per vector finds elements that
 // missed a window; those read a zero gradient or count in the sentinel cells and are redone by the
 // fix-up below.
 template <int FLAGS, int MODE>
@@ -203,12 +208,12 @@ __device__ __forceinline__ float one_window(uint32_t xb, const Lane &ln, Smem &s
     if constexpr ((FLAGS & kHist) != 0) {
         if constexpr (MODE == kModeSymbol) {
             uint32_t row = symbol_row(xb, ln.inv);
-            anyc |= row;
+            anyc = max(anyc, row);
             row = min(row, kSymCells);
             atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + ((row << 7) | ln.lane4)), 1u);
         } else {
             uint32_t p = (am >> 16) - ln.cbase;
-            anyc |= p;
+            anyc = max(anyc, p);
             p = min(p, kCntPat);
             atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(p, xb) + ln.rep4), 1u);
         }
@@ -355,7 +360,7 @@ __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
             const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, v);
             if (n != 0u) {
                 sm.cnt[row * 32 + lane] = 0u;
-                // symbols [-256, 256) lie inside [qmin, qmax] in this mode; the sentinel row is only emptied
+                // the window's symbols lie inside [qmin, qmax] in this mode; the sentinel row is only emptied
                 if (lane == 0 && row < kSymCells)
                     atomicAdd(&sm.cold.row[((int)row - (int)(kSymCells / 2)) - sm.cold.qmin], (unsigned long long)n);
             }
@@ -363,11 +368,11 @@ __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
     } else {
         const uint32_t c_base = sm.cold.c_base;
         for (uint32_t c = threadIdx.x; c < (kCntPat + 1) * 2; c += kThreads) {   // c = p * 2 + sign
-            uint4 *cell = reinterpret_cast<uint4 *>(sm.cnt) + c;
-            const uint4 v = *cell;
-            const uint32_t n = v.x + v.y + v.z + v.w;
+            uint2 *cell = reinterpret_cast<uint2 *>(sm.cnt) + c;
+            const uint2 v = *cell;
+            const uint32_t n = v.x + v.y;
             if (n != 0u) {
-                *cell = make_uint4(0u, 0u, 0u, 0u);
+                *cell = make_uint2(0u, 0u);
                 if (c < kCntPat * 2) {          // the sentinel slot is only emptied
                     const uint32_t h = (c_base + (c >> 1)) | ((c & 1u) << 15);
                     count_symbol(__uint_as_float(h << 16), n, false, sm);
@@ -484,7 +489,7 @@ __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool acc
 }
 
 // One contiguous run of n elements: scalar head up to the first 16-byte boundary of x, 128-bit
-// vector body with loads issued two iterations ahead, scalar tail.  If the gradient's address is
+// vector body fed through the asynchronous-copy ring, scalar tail.  If the gradient's address is
 // not 16-byte aligned at the same element the whole run is scalar.
 template <typename TG, int FLAGS, int MODE>
 __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
@@ -526,22 +531,37 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     }
 
     // (a CTA's run never exceeds device memory / grid size elements: 32-bit vector indices suffice)
+    // Each thread owns slot [d][tid] of every stage d: it fills them with asynchronous 16-byte
+    // copies (one commit group per iteration, empty past the end so that the group count stays in
+    // step) and reads a slot back once the group that filled it has landed.
     const uint4 *xv = reinterpret_cast<const uint4 *>(x + head) + tid;
     TG *gv = gout != nullptr ? gout + head + (int64_t)tid * 8 : nullptr;
     const bool wide = (reinterpret_cast<uintptr_t>(gv) & 31u) == 0;
     const int nv = (int)nvec;
-    uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
-    if (tid < nv) r0 = __ldcs(xv);                           // read once by this sweep: streaming loads
-    if (tid + kThreads < nv) r1 = __ldcs(xv + kThreads);
+    const uint32_t slot0 = (uint32_t)__cvta_generic_to_shared(&sm.stage[0][tid]);
+    constexpr uint32_t kStageBytes = sizeof(uint4) * kThreads;
+#pragma unroll
+    for (int d = 0; d < kDepth - 1; ++d) {
+        if (tid + d * kThreads < nv)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + d * kStageBytes), "l"(xv + d * kThreads) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    uint32_t rd = 0, wr = (kDepth - 1) * kStageBytes;      // byte offsets of the slot to read / to fill next
     for (int v = tid; v < nv; v += kThreads) {
-        uint4 r2 = make_uint4(0u, 0u, 0u, 0u);
-        if (v + 2 * kThreads < nv) r2 = __ldcs(xv + 2 * kThreads);
+        // fill the slot emptied by the previous iteration (its value is in registers since then)
+        if (v + (kDepth - 1) * kThreads < nv)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + wr), "l"(xv + (kDepth - 1) * kThreads) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
+        uint4 r0;
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r0.x), "=r"(r0.y), "=r"(r0.z), "=r"(r0.w) : "r"(slot0 + rd) : "memory");
         process_vec<TG, FLAGS, MODE>(r0, gv, accumulate, wide, ln, sm, acc);
-        r0 = r1;
-        r1 = r2;
+        rd = rd + kStageBytes == kDepth * kStageBytes ? 0u : rd + kStageBytes;
+        wr = wr + kStageBytes == kDepth * kStageBytes ? 0u : wr + kStageBytes;
         xv += kThreads;
         if (gv != nullptr) gv += kThreads * 8;
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 template <typename TG, int FLAGS>
@@ -642,7 +662,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             uint32_t want_base = sm.cold.c_base;
             if constexpr (GRAD) {
                 want_base = g_base + (kGradPat - kCntPat);
-                // symbol mode: the replicated tables are on, symbols [-256, 256) are not clamped, and
+                // symbol mode: the replicated tables are on, the window's symbols are not clamped, and
                 // they reach 6.5 standard deviations
                 if (mode == kModePattern && a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 &&
                     step > 0.0f && (double)(kSymCells / 2) * (double)step >= 6.5 * sm.cold.sd && inv < 3.0e38f)
