@@ -6,25 +6,28 @@
 //   * gradient: |g| depends only on the 15-bit magnitude pattern.  |g| = A[e] * B[j] with e the
 //     exponent field and j the 7 mantissa bits: A[e] = 2^(L + b (e-127)), B[j] = (1 + j/128)^b,
 //     both rounded once from fp64, so the product is within 1.5 ulp for every shape beta.
-//   * histogram: elements are counted by bit pattern in shared memory; patterns become quantised
-//     symbols only when the table is flushed, i.e. when the histogram, its step or the window
-//     changes, or the CTA ends.  Counts are integers, so every order of additions gives the same
-//     table.
-// The kernel's limit is the shared-memory pipe (one 128-byte wavefront per clock and SM), so the
-// tables are laid out to avoid bank conflicts:
-//   * inside a window of 32 binades below 2^5 standard deviations, A and B are replicated once per
-//     bank (lane l reads word l of a row, so a look-up is one wavefront whatever the data);
-//   * counts have two layouts.  Symbol mode, used when the quantiser is coarse enough that symbols
-//     [-192, 192) hold all but the far tails (192 steps >= 6.5 standard deviations): one row of 32
-//     words per symbol, lane l counts in word l, so the atomic is one wavefront too; the symbol is
-//     floor(x * inv) taken with a round-down add of 1.5 * 2^23.  Pattern mode otherwise: one cell
-//     per bf16 magnitude pattern and sign over the upper 16 binades of the window, two replicas
-//     per cell selected by the lowest lane bit.
+//   * histogram: elements are counted in shared memory, by quantised symbol when the quantiser is
+//     coarse and by bit pattern otherwise; patterns become symbols only when the table is flushed,
+//     i.e. when the histogram, its step or the window changes, or the CTA ends.  Counts are
+//     integers, so every order of additions gives the same table.
+// The kernel's limits are instruction issue and the shared-memory pipe (one 128-byte wavefront per
+// clock and SM), so the element path is kept to two table reads, one atomic and about twenty
+// instructions, with tables laid out against bank conflicts:
+//   * A is indexed by the exponent field: the lanes of a warp hold a handful of neighbouring
+//     exponents, which fall in different banks or in the same word.  B is indexed by the random
+//     mantissa bits and is therefore replicated once per bank (lane l reads word l of row j).
+//     Exponents whose A cannot be a single normal fp32 factor (zero/subnormal, inf/nan, far
+//     binades) hold NaN; the NaN reaches the penalty partial of the vector, whose range check
+//     then sends the vector to the exact path.
+//   * counts have two layouts.  Symbol mode, used when symbols [-192, 192) hold all but the far
+//     tails (192 steps >= 6.5 standard deviations): one row of 32 words per symbol, lane l counts
+//     in word l; the symbol is floor(x * inv) taken with a round-down add of 1.5 * 2^23.  Pattern
+//     mode otherwise: one cell per bf16 magnitude pattern and sign over 16 binades below 2^5
+//     standard deviations, two replicas per cell selected by the lowest lane bit.
+//     An element outside the count window (a far-tail symbol, a tiny or huge pattern, inf, nan)
+//     counts in a sentinel cell and is redone after its vector.
 // Input vectors reach each thread through a private ring of shared-memory slots filled by
 // asynchronous copies issued kDepth iterations ahead: bytes in flight cost no registers.
-// The element path inside the windows is branch free; an element outside one (zero, tiny, huge,
-// inf, nan, a far-tail symbol) reads zero or counts in a sentinel cell, and is redone after its
-// vector.
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -36,19 +39,17 @@ namespace {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kCtasPerSm = 2;
-constexpr int kGradBinades = 32;                    // binades in the gradient window
-constexpr uint32_t kGradPat = kGradBinades * 128;   // magnitude patterns in it (a power of two)
-constexpr int kCntBinades = 16;                     // pattern-count window: the upper binades of the gradient window
-constexpr uint32_t kCntPat = kCntBinades * 128;
+constexpr int kDepth = 4;                           // input vectors staged ahead per thread
+constexpr int kCntBinades = 16;                     // pattern-count window
+constexpr uint32_t kCntPat = kCntBinades * 128;     // magnitude patterns in it
 constexpr int kRep = 2;                             // replicas of every pattern-count cell
 constexpr uint32_t kSymCells = 384;                 // symbol-count window: symbols [-192, 192)
-constexpr int kDepth = 4;                           // input vectors staged ahead per thread
 constexpr uint32_t kMagicBits = 0x4B400000u;        // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr uint32_t kSymBase = kMagicBits - kSymCells / 2;
 constexpr int kSymWin = 512;                        // secondary symbol window [-256, 256) of the rare path
-constexpr uint32_t kCntWords = (kSymCells + 1) * 32 > (kCntPat + 1) * 2 * kRep ? (kSymCells + 1) * 32
+constexpr uint32_t kCntWords = (kSymCells + 2) * 32 > (kCntPat + 1) * 2 * kRep ? (kSymCells + 2) * 32
                                                                               : (kCntPat + 1) * 2 * kRep;
-enum : int { kModePlain = 0, kModePattern = 1, kModeSymbol = 2 };
+enum : int { kModePattern = 1, kModeSymbol = 2 };
 
 // Constants of the current segment / histogram that only the cold paths need: kept in shared
 // memory so that the streaming loop does not carry them in registers.
@@ -67,15 +68,14 @@ struct Cold {
 struct Smem {
     // pattern mode: cell ((p * 2 + sign) * kRep + r) = magnitude pattern c_base + p, replica r; slot
     // p = kCntPat is the sentinel that swallows the counts of out-of-window elements.
-    // symbol mode: word (s * 32 + lane) = symbol s - kSymCells/2 counted by that lane; row s = kSymCells
-    // is the sentinel.
+    // symbol mode: word ((s + 1) * 32 + lane) = symbol s - kSymCells/2 counted by that lane; the rows
+    // before and after the window (s = -1 and s = kSymCells) are the sentinels of the two tails.
     uint32_t cnt[kCntWords];
-    uint4 stage[kDepth][kThreads];         // per-thread ring of input vectors in flight
-    float arep[(kGradBinades + 1) * 32];   // row e: A of binade e of the window in every bank; last row: zeros
-    float brep[128 * 32];                  // row j: B[j] in every bank
-    uint32_t win[kSymWin];
-    float2 A[256];                         // every exponent: value = A.x * A.y, A.y a power of two
+    uint4 stage[kDepth][kThreads];   // per-thread ring of input vectors in flight
+    float brep[128 * 32];            // row j: B[j] in every bank
+    float2 A[256];                   // every exponent: value = A.x * A.y, A.y a power of two
     float B[128];
+    uint32_t win[kSymWin];
     double red[3][kWarps];
     uint32_t bad[kWarps];
     float mn[kWarps], mx[kWarps];
@@ -83,6 +83,22 @@ struct Smem {
     Cold cold;
     int e_top;
 };
+
+// A[e] as one factor (with lambda's sign), NaN where that is not possible.  Static shared memory:
+// its address is a compile-time constant, so a look-up is an index and a load.
+__shared__ float s_a1[256];
+
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ void red_inc(uint32_t addr)
+{
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
+}
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -101,7 +117,8 @@ __device__ __noinline__ float grad_rare(uint32_t mag, const Smem &sm)
     return __uint_as_float(__float_as_uint(v) ^ sm.cold.sign_flip);
 }
 
-__device__ __forceinline__ float grad_ab(uint32_t mag, const Smem &sm)
+// The gradient of any magnitude pattern from the two-factor tables (exact path).
+__device__ __noinline__ float grad_exact(uint32_t mag, const Smem &sm)
 {
     const uint32_t e = mag >> 7;
     if (e - 1u < 254u) {
@@ -141,10 +158,11 @@ struct Run {   // fp32 partials of one short run of elements
 
 // Per-thread constants of the element path.
 struct Lane {
-    uint32_t gbase;    // first magnitude pattern of the gradient window
     uint32_t cbase;    // first magnitude pattern of the pattern-count window
-    uint32_t lane4;    // (lane id) * 4: byte offset of this lane's bank inside a replicated row
-    uint32_t rep4;     // (lane id mod kRep) * 4: byte offset of this lane's pattern-count replica
+    // 32-bit shared-memory addresses of this lane's word in the first row of each table
+    uint32_t b_addr;   // brep + lane * 4
+    uint32_t s_addr;   // symbol mode: row of symbol -kSymCells/2 in cnt, + lane * 4
+    uint32_t p_addr;   // pattern mode: cnt + (lane mod kRep) * 4
     float inv;         // quantiser scale (symbol mode)
 };
 
@@ -163,15 +181,8 @@ __device__ __forceinline__ void moments_elem(uint32_t xb, Acc &acc, Run &r)
     }
 }
 
-// Byte offset of a value's pattern-count cell (without the replica): (p * 2 + sign) * kRep * 4.
-__device__ __forceinline__ uint32_t count_cell(uint32_t p, uint32_t xb)
-{
-    static_assert(kRep == 2, "cell stride");
-    return (p << 4) + ((xb >> 28) & 8u);
-}
-
-// Row of a value in the symbol-count table: floor(x * inv) + kSymCells/2 as an unsigned number, so that
-// every symbol outside the window, and inf and nan, give a row >= kSymCells.
+// Row of a value in the symbol-count table: floor(x * inv) + kSymCells/2 as an unsigned number, so
+// that every symbol outside the window, and inf and nan, give a row >= kSymCells.
 __device__ __forceinline__ uint32_t symbol_row(uint32_t xb, float inv)
 {
     const float t = __fmul_rn(__uint_as_float(xb), inv);
@@ -179,67 +190,73 @@ __device__ __forceinline__ uint32_t symbol_row(uint32_t xb, float inv)
     return __float_as_uint(__fadd_rd(t, __uint_as_float(kMagicBits))) - kSymBase;
 }
 
-// Where the miss thresholds of the two windows sit in the collected index bits.
-template <int MODE>
-__device__ __forceinline__ bool any_miss(uint32_t anyg, uint32_t anyc)
+// One element of a 32-bit word w holding two bf16 values: HALF 0 is the low half, 1 the high half.
+// Branch free.  Gradient: a NaN entry of s_a1 (an exponent outside the single-factor range) makes
+// the vector's penalty partial NaN, which the caller checks once per vector.  Count: `anyc` keeps
+// the largest |x * inv| (symbol mode) or window index (pattern mode) so that one compare per
+// vector finds elements that missed the window; those count in the sentinel cells.
+template <int FLAGS, int MODE, int HALF>
+__device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, Run &r, uint32_t &anyc)
 {
-    return (anyg >= kGradPat) | (anyc >= (MODE == kModeSymbol ? kSymCells : kCntPat));
-}
-
-// One element given as fp32 bits (a widened bf16: the low 16 bits are zero), window modes.  Branch
-// free: `anyg` (bitwise or) and `anyc` (maximum) collect the window indices so one compare per vector finds elements that
-// missed a window; those read a zero gradient or count in the sentinel cells and are redone by the
-// fix-up below.
-template <int FLAGS, int MODE>
-__device__ __forceinline__ float one_window(uint32_t xb, const Lane &ln, Smem &sm, Acc &acc, Run &r, uint32_t &anyg,
-                                            uint32_t &anyc)
-{
+    const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);     // the value as fp32 bits
     moments_elem<FLAGS>(xb, acc, r);
-    const uint32_t am = xb & 0x7FFFFFFFu;
     float ga = 0.0f;
     if constexpr ((FLAGS & kGrad) != 0) {
-        uint32_t p = (am >> 16) - ln.gbase;              // index of the magnitude pattern in the window
-        anyg |= p;
-        p = min(p, kGradPat);
-        const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.arep) + ((p & ~127u) | ln.lane4));
-        const float b = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(sm.brep) + (((p & 127u) << 7) | ln.lane4));
-        ga = a * b;
+        const uint32_t e4 = HALF ? ((w >> 21) & 0x3FCu) : ((w >> 5) & 0x3FCu);     // exponent field * 4
+        const uint32_t j = HALF ? ((w >> 16) & 127u) : (w & 127u);
+        const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(s_a1) + e4);
+        ga = a * lds_f32(j * 128u + ln.b_addr);
     }
     if constexpr ((FLAGS & kHist) != 0) {
         if constexpr (MODE == kModeSymbol) {
-            uint32_t row = symbol_row(xb, ln.inv);
-            anyc = max(anyc, row);
-            row = min(row, kSymCells);
-            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + ((row << 7) | ln.lane4)), 1u);
+            // t clamped to just outside the window: the floor of the clamped value lands on a sentinel
+            // row for either tail (and for nan, which the maximum replaces by the lower bound)
+            const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
+            anyc = max(anyc, __float_as_uint(t) & 0x7FFFFFFFu);
+            const float tc = fminf(fmaxf(t, -(float)(kSymCells / 2) - 0.5f), (float)(kSymCells / 2));
+            // for |t| < 2^22 the sum lies in [2^23, 2^24) where floats are the integers: rounding down gives floor
+            const uint32_t fb = __float_as_uint(__fadd_rd(tc, __uint_as_float(kMagicBits)));
+            red_inc(fb * 128u + ln.s_addr);     // (s_addr already holds minus 128 times the bits of symbol -kSymCells/2)
         } else {
-            uint32_t p = (am >> 16) - ln.cbase;
+            static_assert(kRep == 2, "cell stride");
+            const uint32_t mag = HALF ? ((w >> 16) & 0x7FFFu) : (w & 0x7FFFu);
+            uint32_t p = mag - ln.cbase;
             anyc = max(anyc, p);
             p = min(p, kCntPat);
-            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(p, xb) + ln.rep4), 1u);
+            const uint32_t sign8 = HALF ? ((w >> 28) & 8u) : ((w >> 12) & 8u);
+            red_inc(p * 16u + sign8 + ln.p_addr);
         }
     }
     if constexpr ((FLAGS & kGrad) != 0) {
-        r.mp = fmaf(__uint_as_float(am), fabsf(ga), r.mp);
+        r.mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), r.mp);
         return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
     }
     return 0.0f;
 }
 
-// Gradient of an element outside the gradient window (zero, tiny, huge, inf, nan).
-__device__ __noinline__ float fix_grad(uint32_t xb, Smem &sm, Run &r)
+// (symbol mode: some |t| >= kSymCells/2, or a nan, whose bits are larger still; the exact test is
+// redone per element by fix_elem)
+template <int MODE>
+__device__ __forceinline__ bool count_miss(uint32_t anyc)
 {
-    const float ga = grad_ab((xb >> 16) & 0x7FFFu, sm);
-    r.mp = fmaf(__uint_as_float(xb & 0x7FFFFFFFu), fabsf(ga), r.mp);
-    return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+    if constexpr (MODE == kModeSymbol) return anyc >= __float_as_uint((float)(kSymCells / 2));
+    return anyc >= kCntPat;
 }
 
-// Redo of whatever part of an element missed its window; g is the gradient from the first pass.
+// Redo of whatever part of an element (given as fp32 bits) the branch-free path could not do; g is
+// the gradient from the first pass.  grad_bad: the vector's penalty partial left the fp32 range.
 template <int FLAGS, int MODE>
-__device__ __forceinline__ float fix_elem(uint32_t xb, float g, const Lane &ln, Smem &sm, Run &r)
+__device__ __forceinline__ float fix_elem(uint32_t xb, float g, bool grad_bad, const Lane &ln, Smem &sm)
 {
     const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
     if constexpr ((FLAGS & kGrad) != 0) {
-        if (mag - ln.gbase >= kGradPat) g = fix_grad(xb, sm, r);
+        if (grad_bad) {
+            const float a = s_a1[mag >> 7];
+            if (a != a) {     // this element read a NaN marker: zero needs no table, the rest the exact path
+                const float ga = mag == 0u ? 0.0f : grad_exact(mag, sm);
+                g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+            }
+        }
     }
     if constexpr ((FLAGS & kHist) != 0) {
         bool miss;
@@ -248,30 +265,6 @@ __device__ __forceinline__ float fix_elem(uint32_t xb, float g, const Lane &ln, 
         if (miss) count_rare(xb, sm);
     }
     return g;
-}
-
-// The same element when the replicated tables are off (a gradient whose factors leave the fp32
-// range inside the window, or no gradient at all): gradient from the A/B tables of all
-// exponents, pattern-count window as usual.
-template <int FLAGS>
-__device__ __forceinline__ float one_plain(uint32_t xb, const Lane &ln, Smem &sm, Acc &acc, Run &r)
-{
-    moments_elem<FLAGS>(xb, acc, r);
-    const uint32_t am = xb & 0x7FFFFFFFu;
-    float ga = 0.0f;
-    if constexpr ((FLAGS & kGrad) != 0) ga = grad_ab(am >> 16, sm);
-    if constexpr ((FLAGS & kHist) != 0) {
-        const uint32_t p = (am >> 16) - ln.cbase;
-        if (p < kCntPat)
-            atomicAdd(reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(sm.cnt) + count_cell(p, xb) + ln.rep4), 1u);
-        else
-            count_rare(xb, sm);
-    }
-    if constexpr ((FLAGS & kGrad) != 0) {
-        r.mp = fmaf(__uint_as_float(am), fabsf(ga), r.mp);
-        return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
-    }
-    return 0.0f;
 }
 
 // fp64 penalty terms |x| |g| of up to eight patterns packed in four words (rare path).
@@ -293,7 +286,7 @@ __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &
 {
     if constexpr ((FLAGS & kMoments) != 0) { acc.s1 += (double)r.m1; acc.s2 += (double)r.m2; }
     if constexpr ((FLAGS & kGrad) != 0) {
-        // a product or a gradient that left the fp32 range (or a nan) sends the run to fp64
+        // a product or a gradient that left the fp32 range, or a NaN marker, sends the run to fp64
         if (r.mp <= FLT_MAX) acc.pen += (double)r.mp;
         else acc.pen += pen_rare(raw, n, sm);
     }
@@ -340,13 +333,12 @@ __device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumula
     }
 }
 
-// Exponent field of the top binade of a window of `binades` binades that reaches 2^(above+1) times
-// `scale`.
-__device__ __forceinline__ int window_top_exponent(double scale, int above, int binades)
+// Exponent field of the top binade of the pattern-count window: the binade of 2^above times `scale`.
+__device__ __forceinline__ int window_top_exponent(double scale, int above)
 {
     int e = 127 + above;
     if (scale > 0.0 && scale < 1e300) e = ilogb(scale) + 127 + above;
-    return max(binades, min(254, e));
+    return max(kCntBinades, min(254, e));
 }
 
 // Adds the counted cells to the current histogram and empties the tables.
@@ -355,14 +347,14 @@ __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
     // (callers synchronise before: all counting under the old key is complete)
     if (sm.cold.symbol_mode) {
         const int lane = threadIdx.x & 31;
-        for (uint32_t row = threadIdx.x >> 5; row <= kSymCells; row += kWarps) {
+        for (uint32_t row = threadIdx.x >> 5; row < kSymCells + 2; row += kWarps) {   // row 0 and the last: sentinels
             const uint32_t v = sm.cnt[row * 32 + lane];
             const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, v);
             if (n != 0u) {
                 sm.cnt[row * 32 + lane] = 0u;
-                // the window's symbols lie inside [qmin, qmax] in this mode; the sentinel row is only emptied
-                if (lane == 0 && row < kSymCells)
-                    atomicAdd(&sm.cold.row[((int)row - (int)(kSymCells / 2)) - sm.cold.qmin], (unsigned long long)n);
+                // the window's symbols lie inside [qmin, qmax] in this mode; the sentinel rows are only emptied
+                if (lane == 0 && row >= 1 && row <= kSymCells)
+                    atomicAdd(&sm.cold.row[((int)row - 1 - (int)(kSymCells / 2)) - sm.cold.qmin], (unsigned long long)n);
             }
         }
     } else {
@@ -454,36 +446,31 @@ __device__ void reduce_partials(const TileScratch &part, int t0, int t1, const A
     __syncthreads();
 }
 
+
 template <typename TG, int FLAGS, int MODE>
 __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool accumulate, bool wide, const Lane &ln,
                                             Smem &sm, Acc &acc)
 {
+    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     float g[8];
     Run r;
-    if constexpr (MODE != kModePlain) {
-        uint32_t anyg = 0, anyc = 0;
+    uint32_t anyc = 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            g[2 * i] = one_window<FLAGS, MODE>(w[i] << 16, ln, sm, acc, r, anyg, anyc);
-            g[2 * i + 1] = one_window<FLAGS, MODE>(w[i] & 0xFFFF0000u, ln, sm, acc, r, anyg, anyc);
-        }
-        if (any_miss<MODE>(anyg, anyc)) {      // some element missed a window
+    for (int i = 0; i < 4; ++i) {
+        g[2 * i] = one_elem<FLAGS, MODE, 0>(w[i], ln, acc, r, anyc);
+        g[2 * i + 1] = one_elem<FLAGS, MODE, 1>(w[i], ln, acc, r, anyc);
+    }
+    const bool grad_bad = GRAD && !(r.mp <= FLT_MAX);
+    if (grad_bad || (HIST && count_miss<MODE>(anyc))) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-                g[i] = fix_elem<FLAGS, MODE>(xb, g[i], ln, sm, r);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            g[2 * i] = one_plain<FLAGS>(w[i] << 16, ln, sm, acc, r);
-            g[2 * i + 1] = one_plain<FLAGS>(w[i] & 0xFFFF0000u, ln, sm, acc, r);
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+            g[i] = fix_elem<FLAGS, MODE>(xb, g[i], grad_bad, ln, sm);
         }
     }
     close_run<FLAGS>(raw, 8, r, acc, sm);
-    if constexpr ((FLAGS & kGrad) != 0) {
+    if constexpr (GRAD) {
         if (gdst != nullptr) store8<TG>(gdst, g, accumulate, wide);
     }
 }
@@ -495,7 +482,7 @@ template <typename TG, int FLAGS, int MODE>
 __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
                                               const Lane &ln, Smem &sm, Acc &acc)
 {
-    constexpr bool GRAD = (FLAGS & kGrad) != 0;
+    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     const int tid = threadIdx.x;
     int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
     head = min(head, n);
@@ -507,14 +494,10 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
         const int64_t idx = i < head ? i : tail0 + (i - head);
         const uint32_t h = (uint32_t)__ldg(x + idx);
         Run r;
-        float g;
-        if constexpr (MODE != kModePlain) {
-            uint32_t anyg = 0, anyc = 0;
-            g = one_window<FLAGS, MODE>(h << 16, ln, sm, acc, r, anyg, anyc);
-            if (any_miss<MODE>(anyg, anyc)) g = fix_elem<FLAGS, MODE>(h << 16, g, ln, sm, r);
-        } else {
-            g = one_plain<FLAGS>(h << 16, ln, sm, acc, r);
-        }
+        uint32_t anyc = 0;
+        float g = one_elem<FLAGS, MODE, 0>(h, ln, acc, r, anyc);
+        const bool grad_bad = GRAD && !(r.mp <= FLT_MAX);
+        if (grad_bad || (HIST && count_miss<MODE>(anyc))) g = fix_elem<FLAGS, MODE>(h << 16, g, grad_bad, ln, sm);
         close_run<FLAGS>(make_uint4(h, 0u, 0u, 0u), 1, r, acc, sm);
         if constexpr (GRAD) {
             if (gout != nullptr) {
@@ -588,9 +571,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
     bool have_key = false;
     const bool accumulate = GRAD && a.accumulate != 0;
     Lane ln;
-    ln.lane4 = (uint32_t)(tid & 31) * 4u;
-    ln.rep4 = (uint32_t)(tid & (kRep - 1)) * 4u;
-    ln.gbase = 0x8000u;
+    ln.b_addr = (uint32_t)__cvta_generic_to_shared(sm.brep) + (uint32_t)(tid & 31) * 4u;
+    // row r of the symbol table is reached as bits(floor(t) + magic) * 128 + s_addr (mod 2^32)
+    ln.s_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + 128u + (uint32_t)(tid & 31) * 4u - kSymBase * 128u;
+    ln.p_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + (uint32_t)(tid & (kRep - 1)) * 4u;
     ln.cbase = 0x8000u;
     ln.inv = 0.0f;
     __syncthreads();
@@ -601,21 +585,20 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         const int64_t len = a.map.seg_len[s];
         const int t_first = a.map.tile_prefix[s];
         const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
-        int mode = kModePlain;
-        uint32_t g_base = 0x8000u;
+        int mode = kModePattern;
+        bool active = false;
 
         if constexpr (GRAD) {
             const double beta = a.beta[s], alpha = a.alpha[s];
             const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
-            const bool active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
+            active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
             if (tid == 0) {
                 sm.cold.b = beta - 1.0;
                 sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
                 sm.cold.active = active;
                 sm.cold.L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
-                // the standard deviation of the fitted density (Eq. 2-3) places the window
+                // the standard deviation of the fitted density (Eq. 2-3) places the count windows
                 sm.cold.sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
-                sm.e_top = window_top_exponent(sm.cold.sd, 4, kGradBinades);
             }
             __syncthreads();
             const double L = sm.cold.L, b = sm.cold.b;
@@ -633,56 +616,46 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                     v = make_float2((float)ldexp(lam < 0.0 ? -f : f, i1), __int_as_float((i2 + 127) << 23));
                 }
                 sm.A[k] = v;
+                // One factor serves an exponent if its power-of-two part is 1 (|L + b (e-127)| <= 100:
+                // the product with B then stays in the normal fp32 range).  Zero/subnormal (e = 0),
+                // inf/nan (e = 255) and the far exponents get the marker.  Without a gradient all is zero.
+                float one = 0.0f;
+                if (active) one = (k >= 1 && k <= 254 && v.y == 1.0f) ? v.x : __int_as_float(0x7FC00000);
+                s_a1[k] = one;
             } else if (tid < 384) {
                 const int k = tid - 256;
-                sm.B[k] = (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0)));
+                sm.B[k] = active ? (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0))) : 1.0f;
             }
-            g_base = (uint32_t)(sm.e_top - (kGradBinades - 1)) << 7;
             __syncthreads();
-            // The replicated tables hold A[e].x alone, so they serve only if no exponent of the
-            // window needs the power-of-two factor A[e].y (|L + b (e-127)| <= 100: products of the
-            // two table entries then stay in the normal fp32 range).
-            bool row_ok = true;
-            if (tid < kGradBinades) row_ok = sm.A[(g_base >> 7) + tid].y == 1.0f;
-            if (__syncthreads_and(active && row_ok) != 0) {
-                mode = kModePattern;
-                for (int i = tid; i < (kGradBinades + 1) * 32; i += kThreads)
-                    sm.arep[i] = (i >> 5) < kGradBinades ? sm.A[(g_base >> 7) + (i >> 5)].x : 0.0f;
-                for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
-            }
+            for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
         }
-        ln.gbase = g_base;
         if constexpr (HIST) {
             const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
             const float step = a.step[s];
             const float inv = (float)(1.0 / (double)step);
-            // where the pattern-count window should sit: on the upper binades of the gradient window
-            // when there is one, else where it is (same key) or from four binades below the step
-            // upwards (new key)
+            const bool same_key = have_key && hid == cur_hid && __float_as_uint(inv) == cur_inv_bits;
+            // where the pattern-count window should sit: 16 binades below 2^5 standard deviations when
+            // the scale of the data is known, else where it is (same key) or from four binades below
+            // the step upwards (new key)
             uint32_t want_base = sm.cold.c_base;
-            if constexpr (GRAD) {
-                want_base = g_base + (kGradPat - kCntPat);
-                // symbol mode: the replicated tables are on, the window's symbols are not clamped, and
-                // they reach 6.5 standard deviations
-                if (mode == kModePattern && a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 &&
-                    step > 0.0f && (double)(kSymCells / 2) * (double)step >= 6.5 * sm.cold.sd && inv < 3.0e38f)
+            const double sd = GRAD ? sm.cold.sd : 0.0;
+            if (sd > 0.0) {
+                want_base = (uint32_t)(window_top_exponent(sd, 4) - (kCntBinades - 1)) << 7;
+                // symbol mode: the window's symbols are not clamped and reach 6.5 standard deviations
+                if (a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 && step > 0.0f &&
+                    (double)(kSymCells / 2) * (double)step >= 6.5 * sd && inv < 3.0e38f)
                     mode = kModeSymbol;
-            } else {
-                mode = kModePattern;        // histogram only: nothing but the pattern-count window
-                if (!have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits)
-                    want_base = (uint32_t)(window_top_exponent((double)step, 11, kCntBinades) - (kCntBinades - 1)) << 7;
+            } else if (!same_key) {
+                want_base = (uint32_t)(window_top_exponent((double)step, 11) - (kCntBinades - 1)) << 7;
             }
-            const int want_layout = mode == kModeSymbol ? kModeSymbol : kModePattern;
-            const bool new_key = !have_key || hid != cur_hid || __float_as_uint(inv) != cur_inv_bits ||
-                                 want_layout != cur_mode;
-            const bool rebase = new_key || (want_layout == kModePattern && want_base != sm.cold.c_base);
+            const bool rebase = !same_key || mode != cur_mode || (mode == kModePattern && want_base != sm.cold.c_base);
             __syncthreads();
             if (rebase) {
                 if (have_key) flush_counts(sm, a.clamped, cur_hid);
                 have_key = true;
                 cur_hid = hid;
                 cur_inv_bits = __float_as_uint(inv);
-                cur_mode = want_layout;
+                cur_mode = mode;
                 if (tid == 0) {
                     sm.cold.inv = inv;
                     sm.cold.qmin = a.qmin;
@@ -690,7 +663,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                     sm.cold.row = reinterpret_cast<unsigned long long *>(a.hist) +
                                   (int64_t)hid * ((int64_t)a.qmax - (int64_t)a.qmin + 1);
                     sm.cold.c_base = want_base;
-                    sm.cold.symbol_mode = want_layout == kModeSymbol;
+                    sm.cold.symbol_mode = mode == kModeSymbol;
                 }
             }
             ln.cbase = want_base;
@@ -709,11 +682,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         Acc acc;
         if constexpr (GRAD && HIST) {
             if (mode == kModeSymbol) process_range<TG, FLAGS, kModeSymbol>(x, gout, n, accumulate, ln, sm, acc);
-            else if (mode == kModePattern) process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
-            else process_range<TG, FLAGS, kModePlain>(x, gout, n, accumulate, ln, sm, acc);
+            else process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
         } else {
-            if (mode == kModePattern) process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
-            else process_range<TG, FLAGS, kModePlain>(x, gout, n, accumulate, ln, sm, acc);
+            process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
         }
 
         if constexpr (MOM || GRAD) reduce_partials<FLAGS>(a.part, t, t_stop, acc, sm);
