@@ -23,6 +23,7 @@ constexpr int64_t kDefaultChunkBytes = 1ll << 30;
 struct Plan {
     std::string key;
     int32_t n_seg = 0, n_tiles = 0;
+    int64_t max_len = 0;          // longest segment
     void *dev = nullptr;          // one allocation holding all tables and scratch
     TileMap map{};
     TileScratch part{};
@@ -39,6 +40,7 @@ struct gg_ctx {
     uint64_t clock = 0;
     int64_t launches = 0;
     std::string cuda_error;
+    double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
     std::vector<cudaEvent_t> ev_first, ev_tail;   // begin, end, begin, end, ...
@@ -142,6 +144,7 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
         prefix[(size_t)s + 1] = prefix[(size_t)s] + (int32_t)((segs[s].len + kTile - 1) / kTile);
     const int32_t n_tiles = prefix[(size_t)n_seg];
     p->n_tiles = n_tiles;
+    for (int32_t s = 0; s < n_seg; ++s) p->max_len = segs[s].len > p->max_len ? segs[s].len : p->max_len;
 
     // layout of the single device block
     size_t off = 0;
@@ -304,6 +307,19 @@ gg_status gg_create(gg_ctx **out, int device)
     if (!ctx) return GG_ERR_NOMEM;
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
+    {
+        DeviceGuard guard(device);
+        cudaError_t se = guard.ok ? cudaMalloc(reinterpret_cast<void **>(&ctx->seed), sizeof(double) * (kSeedCells + 1))
+                                  : cudaErrorInvalidDevice;
+        if (se == cudaSuccess) se = launch_fit_seed_table(ctx->seed, nullptr);
+        if (se == cudaSuccess) se = cudaStreamSynchronize(nullptr);
+        if (se != cudaSuccess) {
+            cudaGetLastError();
+            if (ctx->seed) cudaFree(ctx->seed);
+            delete ctx;
+            return se == cudaErrorMemoryAllocation ? GG_ERR_NOMEM : GG_ERR_CUDA;
+        }
+    }
     *out = ctx;
     return GG_OK;
 }
@@ -323,6 +339,7 @@ gg_status gg_destroy(gg_ctx *ctx)
         if (sl.grad) cudaFree(sl.grad);
     }
     if (ctx->host_dev) cudaFree(ctx->host_dev);
+    if (ctx->seed) cudaFree(ctx->seed);
     delete ctx;
     return GG_OK;
 }
@@ -535,7 +552,27 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         fa.hist_on = do_hist; fa.step = a->step; fa.qmin = a->qmin; fa.qmax = a->qmax;
 
         const double *beta_used;
-        if (a->param_mode == GG_PARAMS_FITTED) {
+        // Many short bf16 segments with fitted parameters: one kernel, one warp per segment, does the
+        // whole pass (below a few dozen segments the two-sweep path fills the GPU better).
+        const bool small_path = a->param_mode == GG_PARAMS_FITTED && in_dt == GG_BF16 && p->max_len <= kSmallSegMax &&
+                                n_seg >= 64;
+        if (small_path) {
+            SmallArgs ka{};
+            ka.map = p->map;
+            ka.beta = a->beta; ka.alpha = a->alpha; ka.sum_abs = a->sum_abs; ka.sum_sq = a->sum_sq;
+            ka.count = a->count; ka.flags = a->flags; ka.penalty = a->penalty;
+            ka.lambda = a->lambda; ka.mean_reduction = a->reduction == GG_MEAN; ka.accumulate = a->accumulate_grad;
+            ka.do_grad = want_pg; ka.do_hist = do_hist;
+            ka.step = a->step; ka.step_from_alpha = fa.step_from_alpha; ka.step_scale = a->step_scale;
+            ka.step_out = a->step_out;
+            ka.qmin = a->qmin; ka.qmax = a->qmax; ka.hist = a->hist; ka.clamped = a->clamped_lo_hi;
+            ka.seed = ctx->seed;
+            {
+                SweepTimer tm(ctx, &ctx->ev_first, cs);
+                GG_CUDA(ctx, launch_small_bf16(g_dt, ka, ctx->sm_count, cs));
+            }
+            ctx->launches += 1;
+        } else if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
@@ -562,7 +599,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             ctx->launches += 1 + (p->n_tiles > 0);
             beta_used = a->beta_in;
         }
-        if (a->penalty) {
+        if (a->penalty && !small_path) {
             GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta_used, a->penalty, cs));
             ctx->launches += 1;
         }

@@ -76,6 +76,33 @@ cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, boo
 // histogram over bf16 bit patterns.  sm_count sizes the grid.
 cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
                              int sm_count, cudaStream_t st);
+// Whole pass for short bf16 segments: one warp per segment does the moments, the fit, the gradient
+// and the histogram while the segment is still in cache, so DRAM sees one read and one write.
+constexpr int kSmallSegMax = 16384;   // longest segment the kernel takes (elements)
+constexpr int kSeedCells = 2048;      // cells of the ln(beta) grid that seeds the moment-ratio inversion
+struct SmallArgs {
+    TileMap map;                       // seg_ptr, grad_ptr, seg_len, hist_id, n_seg are used
+    double *beta, *alpha, *sum_abs, *sum_sq;
+    int64_t *count;
+    uint32_t *flags;
+    double *penalty;                   // may be null
+    double lambda;
+    int mean_reduction, accumulate;
+    int do_grad;                       // gradient and penalty wanted
+    int do_hist;
+    const float *step;                 // given steps (null with step_from_alpha)
+    int step_from_alpha;
+    double step_scale;
+    float *step_out;
+    int32_t qmin, qmax;
+    uint64_t *hist;
+    uint64_t *clamped;
+    const double *seed;                // [kSeedCells + 1]: ln rho on the grid of ln beta (launch_fit_seed_table)
+};
+cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st);
+// Fills seed[0 .. kSeedCells] with ln rho(beta_i), ln beta_i evenly spaced over [ln GG_BETA_LO, ln GG_BETA_HI].
+cudaError_t launch_fit_seed_table(double *seed, cudaStream_t st);
+
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
 cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
                                     double *penalty, cudaStream_t st);

@@ -1,0 +1,500 @@
+// The whole pass for short bf16 segments (per-token activation rows and the like): one warp per
+// segment.  The warp reads its segment once for the moments, inverts the moment ratio itself,
+// builds the segment's two gradient tables, and reads the segment a second time, while it is
+// still in L1/L2, for the gradient and the histogram.  DRAM sees the input once and the gradient
+// once; nothing is staged between kernels and no per-tile scratch is used.
+//
+//   * fit: the root of ln rho(beta) = ln r is bracketed by a binary search in a table of ln rho over
+//     a grid of ln beta (built once per context), then narrowed by three rounds of 33-section (the 32
+//     lanes evaluate the interior points, a ballot picks the sub-interval) and finished by linear
+//     interpolation between the two lane values that straddle the root: error ~1e-11 relative.
+//   * gradient: |g| = A[e] * B[j] as in the long-segment kernel, with per-warp tables: A for the 64
+//     exponents around the segment's scale as one fp32 factor, NaN elsewhere; a NaN sends the
+//     element to the fp64 evaluation, which also adds its penalty term in fp64.
+//   * histogram: a CTA-wide pattern-count table serves the segments whose histogram and step equal
+//     those of the CTA's first segment (the common case: many rows, one histogram); other segments
+//     add to global memory element by element.
+#include <cuda_bf16.h>
+#include <float.h>
+
+#include "gg_internal.h"
+
+namespace gg {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kCtasPerSm = 2;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kCntBinades = 16;
+constexpr uint32_t kCntPat = kCntBinades * 128;
+constexpr int kTabExp = 64;          // exponents covered by a warp's A table
+
+struct WarpTab {
+    float a1[kTabExp];   // A of exponent e_lo + i as one factor (with lambda's sign), NaN if not possible
+    float B[128];
+};
+
+struct Smem {
+    uint32_t cnt[(kCntPat + 1) * 2];   // cell p * 2 + sign: magnitude pattern c_base + p
+    WarpTab tab[kWarps];
+    double log2m[128];                 // log2(1 + j/128): the same for every segment
+    // the CTA's histogram key
+    int key_hid;
+    uint32_t key_inv_bits;
+    uint32_t c_base;
+    int key_on;
+};
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double log_rho(double beta)
+{
+    return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
+}
+
+__global__ void seed_table_kernel(double *seed)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > kSeedCells) return;
+    const double lo = log(GG_BETA_LO), hi = log(GG_BETA_HI);
+    seed[i] = log_rho(exp(lo + (hi - lo) * ((double)i / (double)kSeedCells)));
+}
+
+// Moment-ratio inversion by one warp; every lane returns the same beta.  log_r lies strictly
+// between ln rho(GG_BETA_LO) and ln rho(GG_BETA_HI).
+__device__ double invert_ratio(double log_r, const double *seed, int lane)
+{
+    // largest grid index whose ln rho is below the target (ln rho increases with beta)
+    int i0 = 0, i1 = kSeedCells;
+    while (i1 - i0 > 1) {
+        const int m = (i0 + i1) >> 1;
+        if (__ldg(seed + m) < log_r) i0 = m; else i1 = m;
+    }
+    const double u0 = log(GG_BETA_LO), h = (log(GG_BETA_HI) - log(GG_BETA_LO)) / (double)kSeedCells;
+    // one cell of margin on each side absorbs rounding differences between the table and the
+    // evaluations below
+    double lo = u0 + h * (double)max(i0 - 1, 0), hi = u0 + h * (double)min(i1 + 1, kSeedCells);
+    double f_lo = 0.0, f_hi = 0.0, w = 0.0;
+    int k = 0;
+    for (int round = 0; round < 3; ++round) {
+        w = (hi - lo) * (1.0 / 33.0);
+        const double f = log_rho(exp(lo + w * (double)(lane + 1))) - log_r;
+        k = __popc(__ballot_sync(kFull, f < 0.0));          // points 1..k lie below the root
+        // values at the ends of the chosen sub-interval, where a lane has them
+        f_lo = __shfl_sync(kFull, f, max(k - 1, 0));
+        f_hi = __shfl_sync(kFull, f, min(k, 31));
+        hi = lo + w * (double)(k + 1);
+        lo = lo + w * (double)k;
+    }
+    double u = 0.5 * (lo + hi);
+    if (k >= 1 && k <= 31 && f_hi > f_lo) u = lo + w * (-f_lo / (f_hi - f_lo));   // secant inside the sub-interval
+    return exp(u);
+}
+
+// The gradient magnitude (with lambda's sign) in fp64 for one magnitude pattern: the exact path.
+// Its penalty term |x| |g| is added to `pen` before the gradient is rounded to fp32 (which may
+// underflow or overflow).
+__device__ __noinline__ float grad_fp64(uint32_t mag, double L, double b, bool active, uint32_t sign_flip, double &pen)
+{
+    const float ax = __uint_as_float(mag << 16);
+    if (!active || ax == 0.0f) return 0.0f;
+    const double g = exp2(L + b * log2((double)ax));
+    pen += (double)ax * g;
+    return __uint_as_float(__float_as_uint((float)g) ^ sign_flip);
+}
+
+template <typename TG>
+__device__ __forceinline__ float load_grad(const TG *g)
+{
+    if constexpr (sizeof(TG) == 4) return *g;
+    else return __uint_as_float((uint32_t)*g << 16);
+}
+
+template <typename TG>
+__device__ __forceinline__ void store_grad(TG *g, float v)
+{
+    if constexpr (sizeof(TG) == 4) *g = v;
+    else *g = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+
+// Per-segment constants of the second pass.
+struct SegConst {
+    double L, b;
+    bool active;
+    uint32_t sign_flip;
+    int e_lo;             // first exponent of the warp's A table
+    // histogram
+    bool hist, fast;      // fast: the CTA table serves this segment
+    float inv;
+    int32_t qmin, qmax;
+    unsigned long long *row;
+    uint32_t c_base;
+};
+
+// One element (fp32 bits of a widened bf16): gradient value and penalty term, and the count.
+template <bool GRAD, bool HIST>
+__device__ __forceinline__ float small_elem(uint32_t xb, const SegConst &k, const WarpTab &tab, Smem &sm, float &mp,
+                                            double &pen, uint32_t (&clampc)[2])
+{
+    const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
+    float g = 0.0f;
+    if constexpr (GRAD) {
+        const uint32_t ei = (mag >> 7) - (uint32_t)k.e_lo;
+        float ga = ei < (uint32_t)kTabExp ? tab.a1[ei] * tab.B[mag & 127u] : __int_as_float(0x7FC00000);
+        if (ga != ga) ga = grad_fp64(mag, k.L, k.b, k.active, k.sign_flip, pen);
+        else mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);     // (table products are normal fp32 numbers)
+        g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+    }
+    if constexpr (HIST) {
+        if (k.hist) {
+            const uint32_t p = mag - k.c_base;
+            if (k.fast && p < kCntPat) {
+                atomicAdd(&sm.cnt[p * 2u + (xb >> 31)], 1u);
+            } else {
+                const float t = __fmul_rn(__uint_as_float(xb), k.inv);
+                if (t == t) {                               // NaN is skipped
+                    int q = __float2int_rd(t);              // floor, saturating
+                    if (q < k.qmin) { q = k.qmin; clampc[0] += 1u; }
+                    else if (q > k.qmax) { q = k.qmax; clampc[1] += 1u; }
+                    atomicAdd(&k.row[q - k.qmin], 1ull);
+                }
+            }
+        }
+    }
+    return g;
+}
+
+// Exponent field of the top binade of the CTA's pattern-count window: 2^11 steps.
+__device__ __forceinline__ int window_top_exponent(double step)
+{
+    int e = 127 + 11;
+    if (step > 0.0 && step < 1e300) e = ilogb(step) + 127 + 11;
+    return max(kCntBinades, min(254, e));
+}
+
+template <typename TG, bool GRAD, bool HIST>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const SmallArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_seg = a.map.n_seg;
+    const int64_t n_bins = (int64_t)a.qmax - (int64_t)a.qmin + 1;
+
+    if constexpr (HIST) {
+        for (int i = tid; i < (int)((kCntPat + 1) * 2); i += kThreads) sm.cnt[i] = 0u;
+    }
+    if (tid < 128) sm.log2m[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
+    if (tid == 0) {
+        // the CTA's histogram key: that of the first segment it handles, when steps are given
+        sm.key_on = 0;
+        const int s0 = blockIdx.x * kWarps;
+        if (HIST && a.do_hist && !a.step_from_alpha && s0 < n_seg) {
+            const float step = a.step[s0];
+            sm.key_hid = a.map.hist_id ? a.map.hist_id[s0] : s0;
+            sm.key_inv_bits = __float_as_uint((float)(1.0 / (double)step));
+            sm.c_base = (uint32_t)(window_top_exponent((double)step) - (kCntBinades - 1)) << 7;
+            sm.key_on = 1;
+        }
+    }
+    __syncthreads();
+    WarpTab &tab = sm.tab[warp];
+
+    for (int s = blockIdx.x * kWarps + warp; s < n_seg; s += gridDim.x * kWarps) {
+        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]);
+        const int len = (int)a.map.seg_len[s];
+        TG *gout = nullptr;
+        if constexpr (GRAD) {
+            if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]);
+        }
+        // scalar head up to the first 16-byte boundary of x, 128-bit vector body, scalar tail; if the
+        // gradient is not 16-byte aligned at the same element the whole segment is scalar
+        int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
+        head = min(head, len);
+        if (gout != nullptr && (reinterpret_cast<uintptr_t>(gout + head) & 15u) != 0) head = len;
+        const int nvec = (len - head) / 8;
+        const int tail0 = head + nvec * 8;
+        const int n_scalar = head + (len - tail0);
+        const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
+
+        // ---- first pass: moments (fp32 runs of 8, then fp64), extremes, non-finite count
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t bad = 0;
+        float xmin = INFINITY, xmax = -INFINITY;
+        for (int i = lane; i < n_scalar; i += 32) {
+            const int idx = i < head ? i : tail0 + (i - head);
+            const uint32_t xb = (uint32_t)__ldg(x + idx) << 16;
+            const uint32_t am = xb & 0x7FFFFFFFu;
+            if (am < 0x7F800000u) { s1 += (double)__uint_as_float(am); s2 += (double)__uint_as_float(am) * (double)__uint_as_float(am); }
+            else bad += 1u;
+            xmin = fminf(xmin, __uint_as_float(xb));
+            xmax = fmaxf(xmax, __uint_as_float(xb));
+        }
+        for (int v = lane; v < nvec; v += 32) {
+            const uint4 raw = __ldg(xv + v);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+            float m1 = 0.0f, m2 = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+                const uint32_t am = xb & 0x7FFFFFFFu;
+                const bool fin = am < 0x7F800000u;
+                const float af = fin ? __uint_as_float(am) : 0.0f;
+                m1 += af;
+                m2 = fmaf(af, af, m2);
+                bad += fin ? 0u : 1u;
+                xmin = fminf(xmin, __uint_as_float(xb));
+                xmax = fmaxf(xmax, __uint_as_float(xb));
+            }
+            if (m2 <= FLT_MAX) {
+                s1 += (double)m1;
+                s2 += (double)m2;
+            } else {     // a square or a sum left the fp32 range: this vector again in fp64
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t am = ((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16)) & 0x7FFFFFFFu;
+                    if (am < 0x7F800000u) {
+                        const double ax = (double)__uint_as_float(am);
+                        s1 += ax;
+                        s2 += ax * ax;
+                    }
+                }
+            }
+        }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        bad = __reduce_add_sync(kFull, bad);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            xmin = fminf(xmin, __shfl_xor_sync(kFull, xmin, o));
+            xmax = fmaxf(xmax, __shfl_xor_sync(kFull, xmax, o));
+        }
+
+        // ---- fit (every lane holds the same values)
+        uint32_t flags = bad ? GG_FLAG_NONFINITE : 0u;
+        double beta = 0.0, alpha = 0.0;
+        if (len <= 0 || !(s2 > 0.0)) {
+            flags |= GG_FLAG_DEGENERATE;
+        } else {
+            const double m1 = s1 / (double)len, m2 = s2 / (double)len;
+            const double log_r = log(m1 * m1 / m2);
+            if (log_r <= __ldg(a.seed)) {
+                beta = GG_BETA_LO;
+                flags |= GG_FLAG_BETA_CLAMPED_LO;
+            } else if (log_r >= __ldg(a.seed + kSeedCells)) {
+                beta = GG_BETA_HI;
+                flags |= GG_FLAG_BETA_CLAMPED_HI;
+            } else {
+                beta = invert_ratio(log_r, a.seed, lane);
+            }
+            alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+        }
+        float step = 0.0f;
+        if (HIST && a.do_hist) {
+            step = a.step_from_alpha ? (float)(alpha * a.step_scale) : a.step[s];
+            if (xmin <= xmax) {
+                // the quantiser is monotone in x, so a symbol clamps iff one of the extremes does
+                const float inv = (float)(1.0 / (double)step);
+                const float tlo = __fmul_rn(xmin, inv), thi = __fmul_rn(xmax, inv);
+                if ((double)floorf(tlo) < (double)a.qmin || (double)floorf(thi) > (double)a.qmax)
+                    flags |= GG_FLAG_CLAMPED_SYMBOLS;
+            }
+        }
+        if (lane == 0) {
+            a.beta[s] = beta;
+            a.alpha[s] = alpha;
+            if (a.sum_abs) a.sum_abs[s] = s1;
+            if (a.sum_sq) a.sum_sq[s] = s2;
+            if (a.count) a.count[s] = len;
+            if (a.flags) a.flags[s] = flags;
+            if (HIST && a.do_hist && a.step_from_alpha && a.step_out) a.step_out[s] = step;
+        }
+
+        // ---- constants and tables of the second pass
+        SegConst k{};
+        if constexpr (GRAD) {
+            const double lam = a.mean_reduction ? a.lambda / (double)max(len, 1) : a.lambda;
+            k.active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
+            k.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
+            k.b = beta - 1.0;
+            k.L = k.active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
+            // the table's 64 exponents: 40 binades below the standard deviation's to 23 above
+            int e_c = 127;
+            if (k.active) e_c = ilogb(sqrt(s2 / (double)len)) + 127;
+            k.e_lo = max(1, min(254 - (kTabExp - 1), e_c - 40));
+            __syncwarp();       // the previous segment's second pass is done with the tables
+#pragma unroll
+            for (int i = lane; i < kTabExp; i += 32) {
+                float v = 0.0f;
+                if (k.active) {
+                    // one fp32 factor serves if |L + b (e-127)| <= 100: its product with B stays a normal
+                    // number; the same bound on L + beta (e-127) keeps the penalty terms |x| |g| normal too
+                    const double de = (double)(k.e_lo + i - 127);
+                    const double e0 = k.L + k.b * de;
+                    const bool ok = fabs(e0) <= 100.0 && fabs(e0 + de) <= 100.0;
+                    v = ok ? (float)(lam < 0.0 ? -exp2(e0) : exp2(e0)) : __int_as_float(0x7FC00000);
+                }
+                tab.a1[i] = v;
+            }
+#pragma unroll
+            for (int j = lane; j < 128; j += 32) tab.B[j] = k.active ? (float)exp2(k.b * sm.log2m[j]) : 1.0f;
+            __syncwarp();
+        }
+        if constexpr (HIST) {
+            k.hist = a.do_hist != 0;
+            if (k.hist) {
+                const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+                k.inv = (float)(1.0 / (double)step);
+                k.qmin = a.qmin;
+                k.qmax = a.qmax;
+                k.row = reinterpret_cast<unsigned long long *>(a.hist) + (int64_t)hid * n_bins;
+                k.fast = sm.key_on && hid == sm.key_hid && __float_as_uint(k.inv) == sm.key_inv_bits;
+                k.c_base = sm.c_base;
+            }
+        }
+
+        // ---- second pass: gradient, penalty partial, counts (the segment is in L1/L2 now)
+        if (GRAD || (HIST && k.hist)) {
+            double pen = 0.0;
+            uint32_t clampc[2] = {0u, 0u};
+            const bool accumulate = GRAD && a.accumulate != 0;
+            for (int i = lane; i < n_scalar; i += 32) {
+                const int idx = i < head ? i : tail0 + (i - head);
+                const uint32_t h = (uint32_t)__ldg(x + idx);
+                float mp = 0.0f;
+                float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
+                if constexpr (GRAD) {
+                    pen += (double)mp;
+                    if (gout != nullptr) {
+                        if (accumulate) g += load_grad<TG>(gout + idx);
+                        store_grad<TG>(gout + idx, g);
+                    }
+                }
+            }
+            for (int v = lane; v < nvec; v += 32) {
+                const uint4 raw = __ldg(xv + v);
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                float g[8];
+                float mp = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+                    g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
+                }
+                if constexpr (GRAD) {
+                    pen += (double)mp;
+                    if (gout != nullptr) {
+                        TG *gp = gout + head + v * 8;
+                        if constexpr (sizeof(TG) == 4) {
+                            float4 *p4 = reinterpret_cast<float4 *>(gp);
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                float4 o = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
+                                if (accumulate) {
+                                    const float4 old = p4[q];
+                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                }
+                                __stcs(p4 + q, o);
+                            }
+                        } else {
+                            uint32_t o[4];
+                            const uint32_t *p1 = reinterpret_cast<const uint32_t *>(gp);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                float lo = g[2 * q], hi = g[2 * q + 1];
+                                if (accumulate) {
+                                    const uint32_t old = p1[q];
+                                    lo += __uint_as_float(old << 16);
+                                    hi += __uint_as_float(old & 0xFFFF0000u);
+                                }
+                                o[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+                                       ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+                            }
+                            __stcs(reinterpret_cast<uint4 *>(gp), make_uint4(o[0], o[1], o[2], o[3]));
+                        }
+                    }
+                }
+            }
+            if constexpr (GRAD) {
+                pen = warp_sum(pen);
+                if (lane == 0 && a.penalty) {
+                    // sum |x| |g| = |lambda| beta sum (|x|/alpha)^beta; the penalty carries lambda's sign
+                    a.penalty[s] = beta > 0.0 ? (k.sign_flip ? -pen : pen) / beta : 0.0;
+                }
+            }
+            if constexpr (HIST) {
+                if (k.hist && a.clamped != nullptr) {
+                    const uint32_t c0 = __reduce_add_sync(kFull, clampc[0]), c1 = __reduce_add_sync(kFull, clampc[1]);
+                    const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+                    if (lane == 0 && c0) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid, (unsigned long long)c0);
+                    if (lane == 0 && c1) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + 1, (unsigned long long)c1);
+                }
+            }
+        } else if (GRAD && lane == 0 && a.penalty) {
+            a.penalty[s] = 0.0;
+        }
+    }
+
+    // ---- the CTA's pattern counts become symbols of its histogram
+    if constexpr (HIST) {
+        __syncthreads();
+        if (sm.key_on) {
+            const float inv = __uint_as_float(sm.key_inv_bits);
+            unsigned long long *row = reinterpret_cast<unsigned long long *>(a.hist) + (int64_t)sm.key_hid * n_bins;
+            for (uint32_t c = tid; c < kCntPat * 2; c += kThreads) {
+                const uint32_t n = sm.cnt[c];
+                if (n == 0u) continue;
+                const uint32_t h = (sm.c_base + (c >> 1)) | ((c & 1u) << 15);
+                const float t = __fmul_rn(__uint_as_float(h << 16), inv);     // (window patterns are finite)
+                int q = __float2int_rd(t);
+                if (q < a.qmin) {
+                    q = a.qmin;
+                    if (a.clamped) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * sm.key_hid, (unsigned long long)n);
+                } else if (q > a.qmax) {
+                    q = a.qmax;
+                    if (a.clamped) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * sm.key_hid + 1, (unsigned long long)n);
+                }
+                atomicAdd(&row[q - a.qmin], (unsigned long long)n);
+            }
+        }
+    }
+}
+
+template <typename TG>
+cudaError_t launch_typed(const SmallArgs &a, int sm_count, cudaStream_t st)
+{
+    const int grid = (int)min((int64_t)(a.map.n_seg + kWarps - 1) / kWarps, (int64_t)sm_count * kCtasPerSm);
+    auto go = [&](auto kern) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem));
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kThreads, sizeof(Smem), st>>>(a);
+        return cudaGetLastError();
+    };
+    if (a.do_grad && a.do_hist) return go(small_bf16_kernel<TG, true, true>);
+    if (a.do_grad) return go(small_bf16_kernel<TG, true, false>);
+    if (a.do_hist) return go(small_bf16_kernel<TG, false, true>);
+    return go(small_bf16_kernel<TG, false, false>);
+}
+
+}  // namespace
+
+cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st)
+{
+    if (a.map.n_seg <= 0) return cudaSuccess;
+    if (a.do_grad && a.map.grad_ptr != nullptr && grad_dtype == GG_BF16) return launch_typed<uint16_t>(a, sm_count, st);
+    return launch_typed<float>(a, sm_count, st);
+}
+
+cudaError_t launch_fit_seed_table(double *seed, cudaStream_t st)
+{
+    seed_table_kernel<<<(kSeedCells + 1 + 255) / 256, 256, 0, st>>>(seed);
+    return cudaGetLastError();
+}
+
+}  // namespace gg

@@ -429,6 +429,79 @@ def test_config3_activation_rows_scaled(ctx):
     check_fused(out, list(x), list(gd), w["lam"], w["hist_id"], 1)
 
 
+def short_segments(seed, n_seg=150):
+    """Many short bf16 segments of ragged lengths (1 .. 9000), a few of them empty, zero or tiny."""
+    rng = np.random.default_rng(seed)
+    xs = []
+    for s in range(n_seg):
+        n = int(rng.integers(1, 9000))
+        beta = float(rng.uniform(0.5, 2.5))
+        xs.append(gg_synth.gg_host(rng, beta, 10.0 ** rng.uniform(-3, 0.5), n, torch.bfloat16))
+    xs[3] = torch.zeros(0, dtype=torch.bfloat16)
+    xs[4] = torch.zeros(77, dtype=torch.bfloat16)
+    xs[5] = torch.tensor([1.0, -1.0], dtype=torch.bfloat16)
+    xs[6][:8] = torch.tensor([0.0, -0.0, 1e-40, -1e-39, 3e38, -3e38, 1e-30, 1e20]).to(torch.bfloat16)
+    return xs
+
+
+def test_fused_many_short_segments_fit_only_with_nonfinite_entries(ctx):
+    from paper_2506_00486_b200 import Segments
+    xs = short_segments(32, n_seg=80)
+    xs[7][:3] = torch.tensor([float("inf"), float("nan"), float("-inf")]).to(torch.bfloat16)
+    out = ctx.gg_fused(Segments([dev(x) for x in xs]), want_penalty=False, want_hist=False)
+    torch.cuda.synchronize()
+    for s, x in enumerate(xs):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(x))
+        assert out["flags"][s].item() == fl and out["count"][s].item() == n
+        if fl & o.FLAG_DEGENERATE:
+            assert out["beta"][s].item() == 0.0 and out["alpha"][s].item() == 0.0
+            continue
+        assert_rel(out["sum_abs"][s].item(), s1, 1e-7, "sum_abs")
+        assert_rel(out["sum_sq"][s].item(), s2, 1e-7, "sum_sq")
+        assert_rel(out["beta"][s].item(), b, REL_FIT, f"beta[{s}]")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, f"alpha[{s}]")
+
+
+@pytest.mark.parametrize("variant", ["shared_hist", "own_hist_step_from_alpha", "misaligned_bf16_grad_mean"])
+def test_fused_many_short_segments(ctx, variant):
+    """The one-warp-per-segment path: shared histogram (CTA count table), per-segment histograms with
+    steps taken from the fit (element-wise global counts), misaligned data with bf16 gradients."""
+    from paper_2506_00486_b200 import Segments, GG_MEAN
+    xs = short_segments(31)
+    n = len(xs)
+    if variant == "misaligned_bf16_grad_mean":
+        xd = misaligned_views(xs, offsets=[(3 * s) % 8 for s in range(n)])
+        gd = [torch.empty(x.numel(), dtype=torch.bfloat16, device="cuda:0") for x in xs]
+        steps = torch.full((n,), 0.01, dtype=torch.float32, device="cuda:0")
+        hid = [s % 3 for s in range(n)]
+        out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=2e-3, step=steps, hist_id=hid, n_hist=3,
+                           reduction=GG_MEAN, qmin=-300, qmax=200)
+        torch.cuda.synchronize()
+        # bf16 gradients: compare after rounding the oracle's values to bf16 (one bf16 ulp)
+        check_fused(out, xs, None, 2e-3, hid, 3, qmin=-300, qmax=200, mean=True)
+        for s, x in enumerate(xs):
+            if x.numel() == 0:
+                continue
+            xo = gg_synth.to_oracle(x)
+            _, g = o.penalty_grad(xo, out["beta"][s].item(), out["alpha"][s].item(), 2e-3 / x.numel())
+            ref = o.round_to_bf16_bits(g).astype(np.int64)
+            got = gd[s].cpu().view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+            fin = np.isfinite(g)
+            assert np.abs((ref & 0x7FFF) - (got & 0x7FFF))[fin].max(initial=0) <= 1
+        return
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    if variant == "shared_hist":
+        steps = torch.full((n,), 2.0 ** -7, dtype=torch.float32, device="cuda:0")
+        out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps, hist_id=[0] * n, n_hist=1)
+        torch.cuda.synchronize()
+        check_fused(out, xs, gd, 1e-4, [0] * n, 1)
+    else:
+        out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step_scale=1 / 8, qmin=-2000, qmax=1999)
+        torch.cuda.synchronize()
+        check_fused(out, xs, gd, 1e-4, list(range(n)), n, step_scale=1 / 8, qmin=-2000, qmax=1999)
+
+
 def test_config4_gradient_buckets_scaled(ctx):
     """fp32 buckets from GG(beta=0.5), per-bucket alpha log-uniform in [1e-6, 1e-3], step alpha/16
     (8 buckets of 250 000 instead of 25 000 000 elements)."""
