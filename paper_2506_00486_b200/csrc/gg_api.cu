@@ -40,6 +40,8 @@ struct gg_ctx {
     uint64_t clock = 0;
     int64_t launches = 0;
     std::string cuda_error;
+    double *ent_part = nullptr;   // scratch of the entropy kernels: 2 * kEntSplit doubles per histogram
+    int64_t ent_hists = 0;
     double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
@@ -232,6 +234,20 @@ cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype gra
     return launch_stream(flags, in_dtype, grad_dtype, has_grad_out, sa, cs);
 }
 
+// Entropy of n_hist count tables; grows the context's scratch (blocking) the first time a call needs more.
+gg_status run_entropy(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
+                      cudaStream_t cs)
+{
+    if (n_hist > ctx->ent_hists) {
+        if (ctx->ent_part) { GG_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(ctx->ent_part); ctx->ent_part = nullptr; ctx->ent_hists = 0; }
+        GG_CUDA(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->ent_part), sizeof(double) * 2 * kEntSplit * (size_t)n_hist));
+        ctx->ent_hists = n_hist;
+    }
+    GG_CUDA(ctx, launch_entropy(hist, n_hist, n_bins, entropy_bits, ctx->ent_part, cs));
+    ctx->launches += 2;
+    return GG_OK;
+}
+
 gg_status check_grad(const gg_seg *segs, const gg_seg *grad, int32_t n_seg, int grad_dtype)
 {
     if (!grad) return GG_OK;
@@ -309,7 +325,7 @@ gg_status gg_create(gg_ctx **out, int device)
     ctx->sm_count = prop.multiProcessorCount;
     {
         DeviceGuard guard(device);
-        cudaError_t se = guard.ok ? cudaMalloc(reinterpret_cast<void **>(&ctx->seed), sizeof(double) * (kSeedCells + 1))
+        cudaError_t se = guard.ok ? cudaMalloc(reinterpret_cast<void **>(&ctx->seed), sizeof(double) * 2 * (kSeedCells + 1))
                                   : cudaErrorInvalidDevice;
         if (se == cudaSuccess) se = launch_fit_seed_table(ctx->seed, nullptr);
         if (se == cudaSuccess) se = cudaStreamSynchronize(nullptr);
@@ -340,6 +356,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     }
     if (ctx->host_dev) cudaFree(ctx->host_dev);
     if (ctx->seed) cudaFree(ctx->seed);
+    if (ctx->ent_part) cudaFree(ctx->ent_part);
     delete ctx;
     return GG_OK;
 }
@@ -366,7 +383,7 @@ gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
     FitArgs fa{};
     fa.map = p->map; fa.part = p->part;
     fa.beta = beta; fa.alpha = alpha; fa.sum_abs = sum_abs; fa.sum_sq = sum_sq;
-    fa.count = count; fa.flags = flags;
+    fa.count = count; fa.flags = flags; fa.seed = ctx->seed;
     GG_CUDA(ctx, launch_fit(fa, cs));
     ctx->launches += 1;
     return GG_OK;
@@ -432,8 +449,8 @@ gg_status gg_rate_hist(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype 
         ctx->launches += p->n_tiles > 0;
     }
     if (entropy_bits && n_hist > 0) {
-        GG_CUDA(ctx, launch_entropy(hist, n_hist, n_bins, entropy_bits, cs));
-        ctx->launches += 1;
+        st = run_entropy(ctx, hist, n_hist, n_bins, entropy_bits, cs);
+        if (st != GG_OK) return st;
     }
     return GG_OK;
 }
@@ -546,7 +563,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         FitArgs fa{};
         fa.map = p->map; fa.part = p->part;
         fa.beta = a->beta; fa.alpha = a->alpha; fa.sum_abs = a->sum_abs; fa.sum_sq = a->sum_sq;
-        fa.count = a->count; fa.flags = a->flags;
+        fa.count = a->count; fa.flags = a->flags; fa.seed = ctx->seed;
         fa.step_from_alpha = do_hist && a->step_mode == GG_STEP_FROM_ALPHA;
         fa.step_scale = a->step_scale; fa.step_out = a->step_out;
         fa.hist_on = do_hist; fa.step = a->step; fa.qmin = a->qmin; fa.qmax = a->qmax;
@@ -605,8 +622,8 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         }
     }
     if (do_hist && a->entropy_bits && a->n_hist > 0) {
-        GG_CUDA(ctx, launch_entropy(a->hist, a->n_hist, n_bins, a->entropy_bits, cs));
-        ctx->launches += 1;
+        gg_status es = run_entropy(ctx, a->hist, a->n_hist, n_bins, a->entropy_bits, cs);
+        if (es != GG_OK) return es;
     }
     return GG_OK;
 }
@@ -780,9 +797,9 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
         ce = cudaEventRecord(done1, s1);
         if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s0, done1, 0);
         if (ce == cudaSuccess && do_hist && a->entropy_bits && n_hist > 0) {
-            ce = launch_entropy(reinterpret_cast<uint64_t *>(d + o_hist), n_hist, (int32_t)n_bins,
-                                reinterpret_cast<double *>(d + o_ent), s0);
-            ctx->launches += 1;
+            if (run_entropy(ctx, reinterpret_cast<uint64_t *>(d + o_hist), n_hist, (int32_t)n_bins,
+                            reinterpret_cast<double *>(d + o_ent), s0) != GG_OK)
+                ce = cudaErrorUnknown;
         }
         auto back = [&](void *host, size_t o, size_t bytes) {
             if (ce == cudaSuccess && host && bytes) ce = cudaMemcpyAsync(host, d + o, bytes, cudaMemcpyDeviceToHost, s0);

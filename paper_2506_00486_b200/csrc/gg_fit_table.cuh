@@ -1,0 +1,59 @@
+// Moment-ratio inversion from a table (shared by the per-segment fit kernel and the short-segment
+// kernel).
+//
+// The table holds, on kSeedCells cells of a uniform grid of u = ln(beta) over
+// [ln GG_BETA_LO, ln GG_BETA_HI], the two smooth functions the fit needs:
+//     Y(u) = ln rho(beta) = 2 lgamma(2/beta) - lgamma(1/beta) - lgamma(3/beta)    (increasing in u)
+//     Z(u) = ln(alpha / sigma) = (lgamma(1/beta) - lgamma(3/beta)) / 2             (Eq. 2)
+// Given ln r, the cell with Y[i] <= ln r < Y[i+1] is found by bisection of the table, and u is the
+// root of the cubic through the four nodes around the cell (Newton from the linear guess).  With
+// 2048 cells the cubic is within 1e-11 of Y and Z over the whole range, so beta and alpha come out
+// to about 1e-10 relative without a single lgamma at fit time.
+#pragma once
+#include "gg_internal.h"
+
+namespace gg {
+
+// Values and derivatives of the cubic Lagrange basis on the nodes -1, 0, 1, 2.
+__device__ __forceinline__ void cubic_basis(double t, double (&w)[4], double (&d)[4])
+{
+    const double a = t + 1.0, b = t, c = t - 1.0, e = t - 2.0;
+    w[0] = -b * c * e * (1.0 / 6.0);
+    w[1] = a * c * e * 0.5;
+    w[2] = -a * b * e * 0.5;
+    w[3] = a * b * c * (1.0 / 6.0);
+    d[0] = -(c * e + b * e + b * c) * (1.0 / 6.0);
+    d[1] = (c * e + a * e + a * c) * 0.5;
+    d[2] = -(b * e + a * e + a * b) * 0.5;
+    d[3] = (b * c + a * c + a * b) * (1.0 / 6.0);
+}
+
+// table: Y[0 .. kSeedCells] followed by Z[0 .. kSeedCells].  log_r must lie strictly between Y[0] and
+// Y[kSeedCells].  Returns beta and writes ln(alpha / sigma).
+__device__ __forceinline__ double invert_ratio_table(double log_r, const double *table, double *ln_alpha_over_sigma)
+{
+    const double *Y = table, *Z = table + (kSeedCells + 1);
+    int i0 = 0, i1 = kSeedCells;            // Y[i0] <= log_r < Y[i1]
+    while (i1 - i0 > 1) {
+        const int m = (i0 + i1) >> 1;
+        if (__ldg(Y + m) <= log_r) i0 = m; else i1 = m;
+    }
+    const int j = max(0, min(kSeedCells - 3, i0 - 1));     // first node of the four-point stencil
+    const double y0 = __ldg(Y + j), y1 = __ldg(Y + j + 1), y2 = __ldg(Y + j + 2), y3 = __ldg(Y + j + 3);
+    const double ya = __ldg(Y + i0), yb = __ldg(Y + i0 + 1);
+    double t = (double)(i0 - j - 1) + (log_r - ya) / (yb - ya);
+    double w[4], d[4];
+#pragma unroll
+    for (int it = 0; it < 3; ++it) {
+        cubic_basis(t, w, d);
+        const double f = w[0] * y0 + w[1] * y1 + w[2] * y2 + w[3] * y3 - log_r;
+        const double fp = d[0] * y0 + d[1] * y1 + d[2] * y2 + d[3] * y3;
+        t -= f / fp;
+    }
+    cubic_basis(t, w, d);
+    *ln_alpha_over_sigma = w[0] * __ldg(Z + j) + w[1] * __ldg(Z + j + 1) + w[2] * __ldg(Z + j + 2) + w[3] * __ldg(Z + j + 3);
+    const double u0 = log(GG_BETA_LO), h = (log(GG_BETA_HI) - log(GG_BETA_LO)) / (double)kSeedCells;
+    return exp(u0 + h * ((double)(j + 1) + t));
+}
+
+}  // namespace gg

@@ -61,6 +61,7 @@ struct FitArgs {
     double *beta, *alpha, *sum_abs, *sum_sq;
     int64_t *count;
     uint32_t *flags;
+    const double *seed;       // the fit table (launch_fit_seed_table), or null: search with lgamma evaluations
     int step_from_alpha;
     double step_scale;
     float *step_out;
@@ -97,17 +98,20 @@ struct SmallArgs {
     int32_t qmin, qmax;
     uint64_t *hist;
     uint64_t *clamped;
-    const double *seed;                // [kSeedCells + 1]: ln rho on the grid of ln beta (launch_fit_seed_table)
+    const double *seed;                // the fit table (launch_fit_seed_table)
 };
 cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st);
-// Fills seed[0 .. kSeedCells] with ln rho(beta_i), ln beta_i evenly spaced over [ln GG_BETA_LO, ln GG_BETA_HI].
-cudaError_t launch_fit_seed_table(double *seed, cudaStream_t st);
+// Fills the fit table, 2 * (kSeedCells + 1) doubles: ln rho(beta_i) and then ln(alpha/sigma)(beta_i), ln beta_i
+// evenly spaced over [ln GG_BETA_LO, ln GG_BETA_HI].
+cudaError_t launch_fit_seed_table(double *table, cudaStream_t st);
 
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
 cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
                                     double *penalty, cudaStream_t st);
-cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins,
-                           double *entropy_bits, cudaStream_t st);
+// scratch: 2 * kEntSplit * n_hist doubles
+constexpr int kEntSplit = 16;
+cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
+                           double *scratch, cudaStream_t st);
 cudaError_t launch_sample(const TileMap &map, gg_dtype dtype, const double *beta, const double *alpha,
                           uint64_t seed, uint32_t tensor_id0, uint32_t *max_attempts, cudaStream_t st);
 

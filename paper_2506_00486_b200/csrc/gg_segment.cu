@@ -1,6 +1,7 @@
 // Per-segment and per-histogram kernels of the GG pass: the fixed-order reduction of the tile
 // partials, the moment-ratio inversion (one warp per segment), the penalty sums, and the
 // empirical entropy of a count table.  All arithmetic here is fp64; none of it is bandwidth bound.
+#include "gg_fit_table.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -24,7 +25,8 @@ __device__ __forceinline__ double log_rho(double beta)
 }
 
 // One warp per segment.  Lanes sum the tile partials in a fixed order (strided, then a butterfly,
-// so every lane ends with the same bits), then invert the moment ratio by 33-section search on
+// so every lane ends with the same bits), then invert the moment ratio: from the context's fit
+// table when there is one, else by 33-section search on
 // ln(beta): each round the 32 lanes evaluate log_rho at the interior points of the bracket and a
 // ballot picks the sub-interval with the sign change; ten rounds shrink [ln .05, ln 20] below
 // 1e-14.  The scale follows Eq. 2 with sigma^2 = sum_sq / count.
@@ -61,6 +63,22 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
     } else {
         const double m1 = s1 / (double)len, m2 = s2 / (double)len;
         const double log_r = log(m1 * m1 / m2);
+        if (a.seed != nullptr) {
+            // table look-up and cubic interpolation (no lgamma at fit time)
+            double lnz;
+            if (log_r <= __ldg(a.seed)) {
+                beta = GG_BETA_LO;
+                lnz = __ldg(a.seed + kSeedCells + 1);
+                flags |= GG_FLAG_BETA_CLAMPED_LO;
+            } else if (log_r >= __ldg(a.seed + kSeedCells)) {
+                beta = GG_BETA_HI;
+                lnz = __ldg(a.seed + 2 * kSeedCells + 1);
+                flags |= GG_FLAG_BETA_CLAMPED_HI;
+            } else {
+                beta = invert_ratio_table(log_r, a.seed, &lnz);
+            }
+            alpha = sqrt(m2) * exp(lnz);
+        } else {
         if (log_r <= log_rho(GG_BETA_LO)) {
             beta = GG_BETA_LO;
             flags |= GG_FLAG_BETA_CLAMPED_LO;
@@ -80,6 +98,7 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
             beta = exp(0.5 * (lo + hi));
         }
         alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+        }
     }
     if (lane == 0) {
         a.beta[s] = beta;
@@ -117,17 +136,22 @@ penalty_finalize_kernel(const TileMap map, const TileScratch part, const double 
     }
 }
 
-// One CTA per histogram: N = sum c, H = log2 N - (1/N) sum_{c>0} c log2 c.
+// Entropy of a count table, H = log2 N - (1/N) sum_{c>0} c log2 c, in two steps so that one large
+// table keeps many SMs busy: kEntSplit CTAs per histogram each reduce a slice of the bins to
+// (sum c log2 c, sum c) in a fixed order, then one thread per histogram adds the slices in order.
 constexpr int kEntThreads = 256;
 __global__ void __launch_bounds__(kEntThreads)
-entropy_kernel(const uint64_t *hist, int32_t n_bins, double *entropy_bits)
+entropy_partial_kernel(const uint64_t *hist, int32_t n_bins, double *part)
 {
     __shared__ double shAcc[kEntThreads / 32];
     __shared__ unsigned long long shTot[kEntThreads / 32];
-    const uint64_t *row = hist + (int64_t)blockIdx.x * n_bins;
+    const int h = blockIdx.x / kEntSplit, slice = blockIdx.x % kEntSplit;
+    const uint64_t *row = hist + (int64_t)h * n_bins;
+    const int per = (n_bins + kEntSplit - 1) / kEntSplit;
+    const int k0 = slice * per, k1 = min(n_bins, k0 + per);
     double acc = 0.0;
     unsigned long long tot = 0;
-    for (int k = threadIdx.x; k < n_bins; k += kEntThreads) {
+    for (int k = k0 + threadIdx.x; k < k1; k += kEntThreads) {
         const uint64_t c = row[k];
         if (c != 0) {
             const double cd = (double)c;
@@ -145,8 +169,18 @@ entropy_kernel(const uint64_t *hist, int32_t n_bins, double *entropy_bits)
         double ra = 0.0;
         unsigned long long rt = 0;
         for (int w = 0; w < kEntThreads / 32; ++w) { ra += shAcc[w]; rt += shTot[w]; }
-        entropy_bits[blockIdx.x] = rt == 0 ? 0.0 : log2((double)rt) - ra / (double)rt;
+        part[2 * blockIdx.x] = ra;
+        part[2 * blockIdx.x + 1] = (double)rt;      // (exact below 2^53 symbols)
     }
+}
+
+__global__ void entropy_final_kernel(const double *part, int32_t n_hist, double *entropy_bits)
+{
+    const int h = blockIdx.x * blockDim.x + threadIdx.x;
+    if (h >= n_hist) return;
+    double ra = 0.0, rt = 0.0;
+    for (int s = 0; s < kEntSplit; ++s) { ra += part[2 * (h * kEntSplit + s)]; rt += part[2 * (h * kEntSplit + s) + 1]; }
+    entropy_bits[h] = rt == 0.0 ? 0.0 : log2(rt) - ra / rt;
 }
 
 }  // namespace
@@ -169,10 +203,13 @@ cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part,
 }
 
 cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
-                           cudaStream_t st)
+                           double *scratch, cudaStream_t st)
 {
     if (n_hist <= 0) return cudaSuccess;
-    entropy_kernel<<<n_hist, kEntThreads, 0, st>>>(hist, n_bins, entropy_bits);
+    entropy_partial_kernel<<<n_hist * kEntSplit, kEntThreads, 0, st>>>(hist, n_bins, scratch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    entropy_final_kernel<<<(n_hist + 127) / 128, 128, 0, st>>>(scratch, n_hist, entropy_bits);
     return cudaGetLastError();
 }
 

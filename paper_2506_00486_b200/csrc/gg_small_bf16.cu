@@ -4,10 +4,8 @@
 // still in L1/L2, for the gradient and the histogram.  DRAM sees the input once and the gradient
 // once; nothing is staged between kernels and no per-tile scratch is used.
 //
-//   * fit: the root of ln rho(beta) = ln r is bracketed by a binary search in a table of ln rho over
-//     a grid of ln beta (built once per context), then narrowed by three rounds of 33-section (the 32
-//     lanes evaluate the interior points, a ballot picks the sub-interval) and finished by linear
-//     interpolation between the two lane values that straddle the root: error ~1e-11 relative.
+//   * fit: beta and alpha come from a table of ln rho and ln(alpha/sigma) over a grid of ln beta
+//     (built once per context) by cubic interpolation: no lgamma at fit time.
 //   * gradient: |g| = A[e] * B[j] as in the long-segment kernel, with per-warp tables: A for the 64
 //     exponents around the segment's scale as one fp32 factor, NaN elsewhere; a NaN sends the
 //     element to the fp64 evaluation, which also adds its penalty term in fp64.
@@ -17,6 +15,7 @@
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include "gg_fit_table.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -58,43 +57,14 @@ __device__ __forceinline__ double log_rho(double beta)
     return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
 }
 
-__global__ void seed_table_kernel(double *seed)
+__global__ void seed_table_kernel(double *table)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i > kSeedCells) return;
     const double lo = log(GG_BETA_LO), hi = log(GG_BETA_HI);
-    seed[i] = log_rho(exp(lo + (hi - lo) * ((double)i / (double)kSeedCells)));
-}
-
-// Moment-ratio inversion by one warp; every lane returns the same beta.  log_r lies strictly
-// between ln rho(GG_BETA_LO) and ln rho(GG_BETA_HI).
-__device__ double invert_ratio(double log_r, const double *seed, int lane)
-{
-    // largest grid index whose ln rho is below the target (ln rho increases with beta)
-    int i0 = 0, i1 = kSeedCells;
-    while (i1 - i0 > 1) {
-        const int m = (i0 + i1) >> 1;
-        if (__ldg(seed + m) < log_r) i0 = m; else i1 = m;
-    }
-    const double u0 = log(GG_BETA_LO), h = (log(GG_BETA_HI) - log(GG_BETA_LO)) / (double)kSeedCells;
-    // one cell of margin on each side absorbs rounding differences between the table and the
-    // evaluations below
-    double lo = u0 + h * (double)max(i0 - 1, 0), hi = u0 + h * (double)min(i1 + 1, kSeedCells);
-    double f_lo = 0.0, f_hi = 0.0, w = 0.0;
-    int k = 0;
-    for (int round = 0; round < 3; ++round) {
-        w = (hi - lo) * (1.0 / 33.0);
-        const double f = log_rho(exp(lo + w * (double)(lane + 1))) - log_r;
-        k = __popc(__ballot_sync(kFull, f < 0.0));          // points 1..k lie below the root
-        // values at the ends of the chosen sub-interval, where a lane has them
-        f_lo = __shfl_sync(kFull, f, max(k - 1, 0));
-        f_hi = __shfl_sync(kFull, f, min(k, 31));
-        hi = lo + w * (double)(k + 1);
-        lo = lo + w * (double)k;
-    }
-    double u = 0.5 * (lo + hi);
-    if (k >= 1 && k <= 31 && f_hi > f_lo) u = lo + w * (-f_lo / (f_hi - f_lo));   // secant inside the sub-interval
-    return exp(u);
+    const double beta = exp(lo + (hi - lo) * ((double)i / (double)kSeedCells));
+    table[i] = log_rho(beta);
+    table[kSeedCells + 1 + i] = 0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta));
 }
 
 // The gradient magnitude (with lambda's sign) in fp64 for one magnitude pattern: the exact path.
@@ -137,8 +107,21 @@ struct SegConst {
     uint32_t c_base;
 };
 
+// Quantises one value and counts its symbol in global memory (elements the CTA table does not serve).
+__device__ __noinline__ void count_global(uint32_t xb, const SegConst &k, uint32_t (&clampc)[2])
+{
+    const float t = __fmul_rn(__uint_as_float(xb), k.inv);
+    if (t == t) {                               // NaN is skipped
+        int q = __float2int_rd(t);              // floor, saturating
+        if (q < k.qmin) { q = k.qmin; clampc[0] += 1u; }
+        else if (q > k.qmax) { q = k.qmax; clampc[1] += 1u; }
+        atomicAdd(&k.row[q - k.qmin], 1ull);
+    }
+}
+
 // One element (fp32 bits of a widened bf16): gradient value and penalty term, and the count.
-template <bool GRAD, bool HIST>
+// HIST: 0 = no histogram, 1 = the CTA table serves the segment, 2 = it does not.
+template <bool GRAD, int HIST>
 __device__ __forceinline__ float small_elem(uint32_t xb, const SegConst &k, const WarpTab &tab, Smem &sm, float &mp,
                                             double &pen, uint32_t (&clampc)[2])
 {
@@ -151,21 +134,12 @@ __device__ __forceinline__ float small_elem(uint32_t xb, const SegConst &k, cons
         else mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);     // (table products are normal fp32 numbers)
         g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
     }
-    if constexpr (HIST) {
-        if (k.hist) {
-            const uint32_t p = mag - k.c_base;
-            if (k.fast && p < kCntPat) {
-                atomicAdd(&sm.cnt[p * 2u + (xb >> 31)], 1u);
-            } else {
-                const float t = __fmul_rn(__uint_as_float(xb), k.inv);
-                if (t == t) {                               // NaN is skipped
-                    int q = __float2int_rd(t);              // floor, saturating
-                    if (q < k.qmin) { q = k.qmin; clampc[0] += 1u; }
-                    else if (q > k.qmax) { q = k.qmax; clampc[1] += 1u; }
-                    atomicAdd(&k.row[q - k.qmin], 1ull);
-                }
-            }
-        }
+    if constexpr (HIST == 1) {
+        const uint32_t p = mag - k.c_base;
+        if (p < kCntPat) atomicAdd(&sm.cnt[p * 2u + (xb >> 31)], 1u);
+        else count_global(xb, k, clampc);
+    } else if constexpr (HIST == 2) {
+        count_global(xb, k, clampc);
     }
     return g;
 }
@@ -176,6 +150,95 @@ __device__ __forceinline__ int window_top_exponent(double step)
     int e = 127 + 11;
     if (step > 0.0 && step < 1e300) e = ilogb(step) + 127 + 11;
     return max(kCntBinades, min(254, e));
+}
+
+// Second pass over one segment by one warp.
+template <typename TG, bool GRAD, int HIST>
+__device__ __forceinline__ void second_pass(const SmallArgs &a, int s, const uint16_t *x, TG *gout, int head, int nvec,
+                                            int tail0, int n_scalar, double beta, const SegConst &k, const WarpTab &tab,
+                                            Smem &sm)
+{
+    const int lane = threadIdx.x & 31;
+    const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
+    if (GRAD || HIST != 0) {
+            double pen = 0.0;
+            uint32_t clampc[2] = {0u, 0u};
+            const bool accumulate = GRAD && a.accumulate != 0;
+            for (int i = lane; i < n_scalar; i += 32) {
+                const int idx = i < head ? i : tail0 + (i - head);
+                const uint32_t h = (uint32_t)__ldg(x + idx);
+                float mp = 0.0f;
+                float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
+                if constexpr (GRAD) {
+                    pen += (double)mp;
+                    if (gout != nullptr) {
+                        if (accumulate) g += load_grad<TG>(gout + idx);
+                        store_grad<TG>(gout + idx, g);
+                    }
+                }
+            }
+            for (int v = lane; v < nvec; v += 32) {
+                const uint4 raw = __ldg(xv + v);
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                float g[8];
+                float mp = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+                    g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
+                }
+                if constexpr (GRAD) {
+                    pen += (double)mp;
+                    if (gout != nullptr) {
+                        TG *gp = gout + head + v * 8;
+                        if constexpr (sizeof(TG) == 4) {
+                            float4 *p4 = reinterpret_cast<float4 *>(gp);
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                float4 o = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
+                                if (accumulate) {
+                                    const float4 old = p4[q];
+                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                }
+                                __stcs(p4 + q, o);
+                            }
+                        } else {
+                            uint32_t o[4];
+                            const uint32_t *p1 = reinterpret_cast<const uint32_t *>(gp);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                float lo = g[2 * q], hi = g[2 * q + 1];
+                                if (accumulate) {
+                                    const uint32_t old = p1[q];
+                                    lo += __uint_as_float(old << 16);
+                                    hi += __uint_as_float(old & 0xFFFF0000u);
+                                }
+                                o[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+                                       ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+                            }
+                            __stcs(reinterpret_cast<uint4 *>(gp), make_uint4(o[0], o[1], o[2], o[3]));
+                        }
+                    }
+                }
+            }
+            if constexpr (GRAD) {
+                pen = warp_sum(pen);
+                if (lane == 0 && a.penalty) {
+                    // sum |x| |g| = |lambda| beta sum (|x|/alpha)^beta; the penalty carries lambda's sign
+                    a.penalty[s] = beta > 0.0 ? (k.sign_flip ? -pen : pen) / beta : 0.0;
+                }
+            }
+            if constexpr (HIST != 0) {
+                if (a.clamped != nullptr) {
+                    const uint32_t c0 = __reduce_add_sync(kFull, clampc[0]), c1 = __reduce_add_sync(kFull, clampc[1]);
+                    const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+                    if (lane == 0 && c0) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid, (unsigned long long)c0);
+                    if (lane == 0 && c1) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + 1, (unsigned long long)c1);
+                }
+            }
+        } else if (GRAD && lane == 0 && a.penalty) {
+            a.penalty[s] = 0.0;
+        }
 }
 
 template <typename TG, bool GRAD, bool HIST>
@@ -284,16 +347,19 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
         } else {
             const double m1 = s1 / (double)len, m2 = s2 / (double)len;
             const double log_r = log(m1 * m1 / m2);
+            double lnz;
             if (log_r <= __ldg(a.seed)) {
                 beta = GG_BETA_LO;
+                lnz = __ldg(a.seed + kSeedCells + 1);
                 flags |= GG_FLAG_BETA_CLAMPED_LO;
             } else if (log_r >= __ldg(a.seed + kSeedCells)) {
                 beta = GG_BETA_HI;
+                lnz = __ldg(a.seed + 2 * kSeedCells + 1);
                 flags |= GG_FLAG_BETA_CLAMPED_HI;
             } else {
-                beta = invert_ratio(log_r, a.seed, lane);
+                beta = invert_ratio_table(log_r, a.seed, &lnz);
             }
-            alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+            alpha = sqrt(m2) * exp(lnz);       // Eq. 2 with sigma^2 = sum_sq / count
         }
         float step = 0.0f;
         if (HIST && a.do_hist) {
@@ -360,84 +426,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
         }
 
         // ---- second pass: gradient, penalty partial, counts (the segment is in L1/L2 now)
-        if (GRAD || (HIST && k.hist)) {
-            double pen = 0.0;
-            uint32_t clampc[2] = {0u, 0u};
-            const bool accumulate = GRAD && a.accumulate != 0;
-            for (int i = lane; i < n_scalar; i += 32) {
-                const int idx = i < head ? i : tail0 + (i - head);
-                const uint32_t h = (uint32_t)__ldg(x + idx);
-                float mp = 0.0f;
-                float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
-                if constexpr (GRAD) {
-                    pen += (double)mp;
-                    if (gout != nullptr) {
-                        if (accumulate) g += load_grad<TG>(gout + idx);
-                        store_grad<TG>(gout + idx, g);
-                    }
-                }
-            }
-            for (int v = lane; v < nvec; v += 32) {
-                const uint4 raw = __ldg(xv + v);
-                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-                float g[8];
-                float mp = 0.0f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-                    g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
-                }
-                if constexpr (GRAD) {
-                    pen += (double)mp;
-                    if (gout != nullptr) {
-                        TG *gp = gout + head + v * 8;
-                        if constexpr (sizeof(TG) == 4) {
-                            float4 *p4 = reinterpret_cast<float4 *>(gp);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                float4 o = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
-                                if (accumulate) {
-                                    const float4 old = p4[q];
-                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                                }
-                                __stcs(p4 + q, o);
-                            }
-                        } else {
-                            uint32_t o[4];
-                            const uint32_t *p1 = reinterpret_cast<const uint32_t *>(gp);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                float lo = g[2 * q], hi = g[2 * q + 1];
-                                if (accumulate) {
-                                    const uint32_t old = p1[q];
-                                    lo += __uint_as_float(old << 16);
-                                    hi += __uint_as_float(old & 0xFFFF0000u);
-                                }
-                                o[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
-                                       ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
-                            }
-                            __stcs(reinterpret_cast<uint4 *>(gp), make_uint4(o[0], o[1], o[2], o[3]));
-                        }
-                    }
-                }
-            }
-            if constexpr (GRAD) {
-                pen = warp_sum(pen);
-                if (lane == 0 && a.penalty) {
-                    // sum |x| |g| = |lambda| beta sum (|x|/alpha)^beta; the penalty carries lambda's sign
-                    a.penalty[s] = beta > 0.0 ? (k.sign_flip ? -pen : pen) / beta : 0.0;
-                }
-            }
-            if constexpr (HIST) {
-                if (k.hist && a.clamped != nullptr) {
-                    const uint32_t c0 = __reduce_add_sync(kFull, clampc[0]), c1 = __reduce_add_sync(kFull, clampc[1]);
-                    const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
-                    if (lane == 0 && c0) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid, (unsigned long long)c0);
-                    if (lane == 0 && c1) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + 1, (unsigned long long)c1);
-                }
-            }
-        } else if (GRAD && lane == 0 && a.penalty) {
-            a.penalty[s] = 0.0;
+        if constexpr (HIST) {
+            if (!k.hist) second_pass<TG, GRAD, 0>(a, s, x, gout, head, nvec, tail0, n_scalar, beta, k, tab, sm);
+            else if (k.fast) second_pass<TG, GRAD, 1>(a, s, x, gout, head, nvec, tail0, n_scalar, beta, k, tab, sm);
+            else second_pass<TG, GRAD, 2>(a, s, x, gout, head, nvec, tail0, n_scalar, beta, k, tab, sm);
+        } else {
+            second_pass<TG, GRAD, 0>(a, s, x, gout, head, nvec, tail0, n_scalar, beta, k, tab, sm);
         }
     }
 
