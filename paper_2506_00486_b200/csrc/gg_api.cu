@@ -42,6 +42,7 @@ struct gg_ctx {
     std::string cuda_error;
     double *ent_part = nullptr;   // scratch of the entropy kernels: 2 * kEntSplit doubles per histogram
     int64_t ent_hists = 0;
+    uint32_t *small_counts = nullptr;   // scratch of the short-segment kernel: one slot of count cells per CTA
     double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
@@ -356,6 +357,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     }
     if (ctx->host_dev) cudaFree(ctx->host_dev);
     if (ctx->seed) cudaFree(ctx->seed);
+    if (ctx->small_counts) cudaFree(ctx->small_counts);
     if (ctx->ent_part) cudaFree(ctx->ent_part);
     delete ctx;
     return GG_OK;
@@ -584,11 +586,15 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             ka.step_out = a->step_out;
             ka.qmin = a->qmin; ka.qmax = a->qmax; ka.hist = a->hist; ka.clamped = a->clamped_lo_hi;
             ka.seed = ctx->seed;
+            if (do_hist && ctx->small_counts == nullptr)      // (first use: a blocking allocation, like a plan)
+                GG_CUDA(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->small_counts),
+                                        sizeof(uint32_t) * kSmallSlotWords * (size_t)ctx->sm_count * 2));
+            ka.cta_counts = ctx->small_counts;
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
                 GG_CUDA(ctx, launch_small_bf16(g_dt, ka, ctx->sm_count, cs));
             }
-            ctx->launches += 1;
+            ctx->launches += 1 + (do_hist ? 1 : 0);
         } else if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
             {

@@ -28,6 +28,9 @@ constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kCntBinades = 16;
 constexpr uint32_t kCntPat = kCntBinades * 128;
 constexpr int kTabExp = 64;          // exponents covered by a warp's A table
+constexpr uint32_t kCells = (kCntPat + 1) * 2;   // count cells of a CTA: the window's patterns and the two "below" cells
+static_assert(kCells + 4 <= (uint32_t)kSmallSlotWords, "scratch slot");
+constexpr int kMaxSlots = 1024;      // CTAs of one launch whose tables the flush kernel can take
 
 struct WarpTab {
     float a1[kTabExp];   // A of exponent e_lo + i as one factor (with lambda's sign), NaN if not possible
@@ -35,7 +38,9 @@ struct WarpTab {
 };
 
 struct Smem {
-    uint32_t cnt[(kCntPat + 1) * 2];   // cell p * 2 + sign: magnitude pattern c_base + p
+    // cell p * 2 + sign: magnitude pattern c_base + p; the last two cells count the values below the
+    // window (all of symbol 0, or -1 if negative) when the window starts at or below one step
+    uint32_t cnt[kCells];
     WarpTab tab[kWarps];
     double log2m[128];                 // log2(1 + j/128): the same for every segment
     // the CTA's histogram key
@@ -43,6 +48,7 @@ struct Smem {
     uint32_t key_inv_bits;
     uint32_t c_base;
     int key_on;
+    int below_ok;                      // values below the window quantise to 0 / -1
 };
 
 __device__ __forceinline__ double warp_sum(double v)
@@ -67,16 +73,13 @@ __global__ void seed_table_kernel(double *table)
     table[kSeedCells + 1 + i] = 0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta));
 }
 
-// The gradient magnitude (with lambda's sign) in fp64 for one magnitude pattern: the exact path.
-// Its penalty term |x| |g| is added to `pen` before the gradient is rounded to fp32 (which may
-// underflow or overflow).
-__device__ __noinline__ float grad_fp64(uint32_t mag, double L, double b, bool active, uint32_t sign_flip, double &pen)
+// The gradient magnitude in fp64 for one magnitude pattern: the exact path.  The caller adds its
+// penalty term |x| |g| before rounding the gradient to fp32 (which may underflow or overflow).
+__device__ __noinline__ double grad_fp64(uint32_t mag, double L, double b, bool active)
 {
     const float ax = __uint_as_float(mag << 16);
-    if (!active || ax == 0.0f) return 0.0f;
-    const double g = exp2(L + b * log2((double)ax));
-    pen += (double)ax * g;
-    return __uint_as_float(__float_as_uint((float)g) ^ sign_flip);
+    if (!active || ax == 0.0f) return 0.0;
+    return exp2(L + b * log2((double)ax));
 }
 
 template <typename TG>
@@ -105,18 +108,23 @@ struct SegConst {
     int32_t qmin, qmax;
     unsigned long long *row;
     uint32_t c_base;
+    bool below_ok;
 };
 
 // Quantises one value and counts its symbol in global memory (elements the CTA table does not serve).
-__device__ __noinline__ void count_global(uint32_t xb, const SegConst &k, uint32_t (&clampc)[2])
+// Returns 1 / 2 if the symbol was clamped at the low / high end, else 0.  (Everything by value: a
+// structure passed by reference to a function that is not inlined would live in local memory.)
+__device__ __noinline__ int count_global(uint32_t xb, float inv, int32_t qmin, int32_t qmax, unsigned long long *row)
 {
-    const float t = __fmul_rn(__uint_as_float(xb), k.inv);
+    const float t = __fmul_rn(__uint_as_float(xb), inv);
+    int clamped = 0;
     if (t == t) {                               // NaN is skipped
         int q = __float2int_rd(t);              // floor, saturating
-        if (q < k.qmin) { q = k.qmin; clampc[0] += 1u; }
-        else if (q > k.qmax) { q = k.qmax; clampc[1] += 1u; }
-        atomicAdd(&k.row[q - k.qmin], 1ull);
+        if (q < qmin) { q = qmin; clamped = 1; }
+        else if (q > qmax) { q = qmax; clamped = 2; }
+        atomicAdd(&row[q - qmin], 1ull);
     }
+    return clamped;
 }
 
 // One element (fp32 bits of a widened bf16): gradient value and penalty term, and the count.
@@ -130,16 +138,26 @@ __device__ __forceinline__ float small_elem(uint32_t xb, const SegConst &k, cons
     if constexpr (GRAD) {
         const uint32_t ei = (mag >> 7) - (uint32_t)k.e_lo;
         float ga = ei < (uint32_t)kTabExp ? tab.a1[ei] * tab.B[mag & 127u] : __int_as_float(0x7FC00000);
-        if (ga != ga) ga = grad_fp64(mag, k.L, k.b, k.active, k.sign_flip, pen);
-        else mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);     // (table products are normal fp32 numbers)
+        if (ga != ga) {
+            const double gd = grad_fp64(mag, k.L, k.b, k.active);      // |g| before rounding to fp32
+            pen += (double)__uint_as_float(mag << 16) * gd;
+            ga = __uint_as_float(__float_as_uint((float)gd) ^ k.sign_flip);
+        } else {
+            mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);     // (table products are normal fp32 numbers)
+        }
         g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
     }
     if constexpr (HIST == 1) {
         const uint32_t p = mag - k.c_base;
         if (p < kCntPat) atomicAdd(&sm.cnt[p * 2u + (xb >> 31)], 1u);
-        else count_global(xb, k, clampc);
+        else if (k.below_ok && mag < k.c_base) atomicAdd(&sm.cnt[kCntPat * 2u + (mag != 0u ? (xb >> 31) : 0u)], 1u);
+        else {
+            const int c = count_global(xb, k.inv, k.qmin, k.qmax, k.row);
+            if (c) clampc[c - 1] += 1u;
+        }
     } else if constexpr (HIST == 2) {
-        count_global(xb, k, clampc);
+        const int c = count_global(xb, k.inv, k.qmin, k.qmax, k.row);
+        if (c) clampc[c - 1] += 1u;
     }
     return g;
 }
@@ -177,8 +195,16 @@ __device__ __forceinline__ void second_pass(const SmallArgs &a, int s, const uin
                     }
                 }
             }
+            // (loads run three vectors ahead of their use: the pass is bound by cache latency otherwise)
+            uint4 q0 = make_uint4(0u, 0u, 0u, 0u), q1 = q0, q2 = q0;
+            if (lane < nvec) q0 = __ldg(xv + lane);
+            if (lane + 32 < nvec) q1 = __ldg(xv + lane + 32);
+            if (lane + 64 < nvec) q2 = __ldg(xv + lane + 64);
             for (int v = lane; v < nvec; v += 32) {
-                const uint4 raw = __ldg(xv + v);
+                const uint4 raw = q0;
+                q0 = q1;
+                q1 = q2;
+                if (v + 96 < nvec) q2 = __ldg(xv + v + 96);
                 const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
                 float g[8];
                 float mp = 0.0f;
@@ -251,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
     const int64_t n_bins = (int64_t)a.qmax - (int64_t)a.qmin + 1;
 
     if constexpr (HIST) {
-        for (int i = tid; i < (int)((kCntPat + 1) * 2); i += kThreads) sm.cnt[i] = 0u;
+        for (int i = tid; i < (int)kCells; i += kThreads) sm.cnt[i] = 0u;
     }
     if (tid < 128) sm.log2m[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
     if (tid == 0) {
@@ -262,7 +288,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
             const float step = a.step[s0];
             sm.key_hid = a.map.hist_id ? a.map.hist_id[s0] : s0;
             sm.key_inv_bits = __float_as_uint((float)(1.0 / (double)step));
-            sm.c_base = (uint32_t)(window_top_exponent((double)step) - (kCntBinades - 1)) << 7;
+            const int e_top = window_top_exponent((double)step);
+            sm.c_base = (uint32_t)(e_top - (kCntBinades - 1)) << 7;
+            // the window starts 2^-4 steps up unless its position had to be clamped
+            sm.below_ok = step > 0.0f && e_top == ilogb((double)step) + 127 + 11;
             sm.key_on = 1;
         }
     }
@@ -299,8 +328,18 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
             xmin = fminf(xmin, __uint_as_float(xb));
             xmax = fmaxf(xmax, __uint_as_float(xb));
         }
-        for (int v = lane; v < nvec; v += 32) {
-            const uint4 raw = __ldg(xv + v);
+        for (int v0 = lane; v0 < nvec; v0 += 128) {
+            // four independent loads per trip
+            uint4 r4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                r4[u] = make_uint4(0u, 0u, 0u, 0u);      // (zeros add nothing to the sums or the extremes' validity)
+                if (v0 + 32 * u < nvec) r4[u] = __ldg(xv + v0 + 32 * u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+            if (v0 + 32 * u >= nvec) break;
+            const uint4 raw = r4[u];
             const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
             float m1 = 0.0f, m2 = 0.0f;
 #pragma unroll
@@ -328,6 +367,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                         s2 += ax * ax;
                     }
                 }
+            }
             }
         }
         s1 = warp_sum(s1);
@@ -422,6 +462,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                 k.row = reinterpret_cast<unsigned long long *>(a.hist) + (int64_t)hid * n_bins;
                 k.fast = sm.key_on && hid == sm.key_hid && __float_as_uint(k.inv) == sm.key_inv_bits;
                 k.c_base = sm.c_base;
+                k.below_ok = sm.below_ok != 0;
             }
         }
 
@@ -435,45 +476,96 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
         }
     }
 
-    // ---- the CTA's pattern counts become symbols of its histogram
+    // ---- the CTA's pattern counts go to its slot of the scratch; small_flush_kernel turns them into
+    // symbols.  (Adding them to the histogram from here would make every CTA hit the same few
+    // thousand addresses with 64-bit atomics at the same time, which serialises.)
     if constexpr (HIST) {
         __syncthreads();
-        if (sm.key_on) {
-            const float inv = __uint_as_float(sm.key_inv_bits);
-            unsigned long long *row = reinterpret_cast<unsigned long long *>(a.hist) + (int64_t)sm.key_hid * n_bins;
-            for (uint32_t c = tid; c < kCntPat * 2; c += kThreads) {
-                const uint32_t n = sm.cnt[c];
-                if (n == 0u) continue;
-                const uint32_t h = (sm.c_base + (c >> 1)) | ((c & 1u) << 15);
-                const float t = __fmul_rn(__uint_as_float(h << 16), inv);     // (window patterns are finite)
-                int q = __float2int_rd(t);
-                if (q < a.qmin) {
-                    q = a.qmin;
-                    if (a.clamped) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * sm.key_hid, (unsigned long long)n);
-                } else if (q > a.qmax) {
-                    q = a.qmax;
-                    if (a.clamped) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * sm.key_hid + 1, (unsigned long long)n);
-                }
-                atomicAdd(&row[q - a.qmin], (unsigned long long)n);
-            }
+        uint32_t *slot = a.cta_counts + (size_t)blockIdx.x * kSmallSlotWords;
+        for (uint32_t c = tid; c < kCells; c += kThreads) slot[c] = sm.key_on ? sm.cnt[c] : 0u;
+        if (tid == 0) {
+            slot[kCells + 0] = (uint32_t)sm.key_on;
+            slot[kCells + 1] = (uint32_t)sm.key_hid;
+            slot[kCells + 2] = sm.key_inv_bits;
+            slot[kCells + 3] = sm.c_base;
         }
+    }
+}
+
+// One thread per count cell walks the CTA slots in order and adds up the runs of slots that share a
+// key (histogram, step, window); each run becomes one symbol and one 64-bit addition.  With one key
+// for the whole call, the usual case, that is one addition per cell.
+__global__ void small_flush_kernel(const uint32_t *__restrict__ cta_counts, int n_slots, int32_t qmin, int32_t qmax, uint64_t *hist,
+                                   uint64_t *clamped)
+{
+    // the slots' keys first, into shared memory: scanning them from global memory would be one
+    // dependent cache miss per slot
+    __shared__ uint32_t sh_key[kMaxSlots][4];
+    for (int b = threadIdx.x; b < n_slots; b += blockDim.x) {
+        const uint32_t *key = cta_counts + (size_t)b * kSmallSlotWords + kCells;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sh_key[b][q] = __ldg(key + q);
+    }
+    __syncthreads();
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= kCells) return;
+    const int64_t n_bins = (int64_t)qmax - (int64_t)qmin + 1;
+    unsigned long long run = 0;
+    uint32_t k_hid = 0, k_inv = 0, k_base = 0;
+    auto emit = [&]() {
+        if (run == 0) return;
+        int q;
+        if (c < kCntPat * 2) {
+            const uint32_t h = (k_base + (c >> 1)) | ((c & 1u) << 15);
+            q = __float2int_rd(__fmul_rn(__uint_as_float(h << 16), __uint_as_float(k_inv)));   // (window patterns are finite)
+        } else {
+            q = c == kCntPat * 2 ? 0 : -1;      // the values below the window
+        }
+        unsigned long long *cl = reinterpret_cast<unsigned long long *>(clamped);
+        if (q < qmin) { q = qmin; if (cl) atomicAdd(cl + 2 * k_hid, run); }
+        else if (q > qmax) { q = qmax; if (cl) atomicAdd(cl + 2 * k_hid + 1, run); }
+        atomicAdd(reinterpret_cast<unsigned long long *>(hist) + (int64_t)k_hid * n_bins + (q - qmin), run);
+        run = 0;
+    };
+    // (the keys are the same words for every thread: cached; the sums over a run are independent
+    // loads, unrolled so that many are in flight)
+    int b = 0;
+    while (b < n_slots) {
+        if (sh_key[b][0] == 0u) { ++b; continue; }                        // this CTA had no table (its cells are zeros)
+        k_hid = sh_key[b][1]; k_inv = sh_key[b][2]; k_base = sh_key[b][3];
+        int e = b + 1;
+        for (; e < n_slots; ++e) {
+            if (sh_key[e][0] != 0u && (sh_key[e][1] != k_hid || sh_key[e][2] != k_inv || sh_key[e][3] != k_base)) break;
+        }
+        int i = b;
+        for (; i + 16 <= e; i += 16) {
+            uint32_t t[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) t[u] = __ldg(cta_counts + (size_t)(i + u) * kSmallSlotWords + c);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) run += t[u];
+        }
+        for (; i < e; ++i) run += __ldg(cta_counts + (size_t)i * kSmallSlotWords + c);
+        emit();
+        b = e;
     }
 }
 
 template <typename TG>
 cudaError_t launch_typed(const SmallArgs &a, int sm_count, cudaStream_t st)
 {
-    const int grid = (int)min((int64_t)(a.map.n_seg + kWarps - 1) / kWarps, (int64_t)sm_count * kCtasPerSm);
+    const int grid = small_grid(a.map.n_seg, sm_count);
     auto go = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem));
         if (e != cudaSuccess) return e;
         kern<<<grid, kThreads, sizeof(Smem), st>>>(a);
         return cudaGetLastError();
     };
-    if (a.do_grad && a.do_hist) return go(small_bf16_kernel<TG, true, true>);
-    if (a.do_grad) return go(small_bf16_kernel<TG, true, false>);
-    if (a.do_hist) return go(small_bf16_kernel<TG, false, true>);
-    return go(small_bf16_kernel<TG, false, false>);
+    if (!a.do_hist) return a.do_grad ? go(small_bf16_kernel<TG, true, false>) : go(small_bf16_kernel<TG, false, false>);
+    cudaError_t e = a.do_grad ? go(small_bf16_kernel<TG, true, true>) : go(small_bf16_kernel<TG, false, true>);
+    if (e != cudaSuccess) return e;
+    small_flush_kernel<<<(kCells + 255) / 256, 256, 0, st>>>(a.cta_counts, grid, a.qmin, a.qmax, a.hist, a.clamped);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -483,6 +575,11 @@ cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_co
     if (a.map.n_seg <= 0) return cudaSuccess;
     if (a.do_grad && a.map.grad_ptr != nullptr && grad_dtype == GG_BF16) return launch_typed<uint16_t>(a, sm_count, st);
     return launch_typed<float>(a, sm_count, st);
+}
+
+int small_grid(int32_t n_seg, int sm_count)
+{
+    return (int)min(min((int64_t)(n_seg + kWarps - 1) / kWarps, (int64_t)sm_count * kCtasPerSm), (int64_t)kMaxSlots);
 }
 
 cudaError_t launch_fit_seed_table(double *seed, cudaStream_t st)

@@ -347,7 +347,10 @@ __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
     // (callers synchronise before: all counting under the old key is complete)
     if (sm.cold.symbol_mode) {
         const int lane = threadIdx.x & 31;
-        for (uint32_t row = threadIdx.x >> 5; row < kSymCells + 2; row += kWarps) {   // row 0 and the last: sentinels
+        // (every CTA starts at another row / cell: CTAs that flush into one histogram at the same time
+        // would otherwise walk its addresses in step and serialise on them)
+        for (uint32_t r0 = threadIdx.x >> 5; r0 < kSymCells + 2; r0 += kWarps) {   // row 0 and the last: sentinels
+            const uint32_t row = (r0 + blockIdx.x * 13u) % (kSymCells + 2);
             const uint32_t v = sm.cnt[row * 32 + lane];
             const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, v);
             if (n != 0u) {
@@ -359,7 +362,8 @@ __device__ void flush_counts(Smem &sm, uint64_t *clamped, int hid)
         }
     } else {
         const uint32_t c_base = sm.cold.c_base;
-        for (uint32_t c = threadIdx.x; c < (kCntPat + 1) * 2; c += kThreads) {   // c = p * 2 + sign
+        for (uint32_t i = threadIdx.x; i < (kCntPat + 1) * 2; i += kThreads) {
+            const uint32_t c = (i + blockIdx.x * 61u) % ((kCntPat + 1) * 2);     // c = p * 2 + sign
             uint2 *cell = reinterpret_cast<uint2 *>(sm.cnt) + c;
             const uint2 v = *cell;
             const uint32_t n = v.x + v.y;
