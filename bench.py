@@ -188,6 +188,23 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------- whole-job figures over ranks
+def max_over_ranks(value, world, device="cpu"):
+    """The largest of the ranks' values (every rank gets it): the job is as slow as its slowest rank."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_gbs(world, bytes_per_rank, ms):
+    """Replicas are independent (weak scaling): the job moves world * bytes_per_rank in the slowest rank's time."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------------- GPU arm
 def run_ours(args):
     import torch
@@ -245,11 +262,8 @@ def run_ours(args):
     ms_first, n_first, ms_tail, n_tail = ctx.timing_read()
     ctx.timing_enable(False)
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = t.item()
-    value = world * alg_bytes / (ms * 1e-3) / 1e9
+    ms = max_over_ranks(ms, world, dev)
+    value = whole_job_gbs(world, alg_bytes, ms)
 
     # ---- a quick self-check of the timed outputs (host logic only: no oracle here)
     out = run.outputs
@@ -333,14 +347,10 @@ def run_e2e(args, ctx, w, world, dev, gdtype, in_bytes, g_bytes, alg_bytes, barr
         runh()
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / max(args.e2e_steps, 1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([dt], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = t.item()
+    dt = max_over_ranks(dt, world, dev)
     out = runh.outputs
     d2h = g_bytes + out["hist"].numel() * 8 + n_seg * (8 * 6 + 4 + 8 + 16)
-    return {"value": world * alg_bytes / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3, "steps": args.e2e_steps,
+    return {"value": whole_job_gbs(world, alg_bytes, dt * 1e3), "unit": UNIT, "ms_per_step": dt * 1e3, "steps": args.e2e_steps,
             "h2d_bytes_per_step": in_bytes + n_seg * 4, "d2h_bytes_per_step": int(d2h),
             "api": "gg_fused_host (pinned host tensors in, gradients + fit + histograms back on the host)"}
 
