@@ -28,6 +28,7 @@
 #include <math.h>
 #include <stdint.h>
 #include <string.h>
+#include <stdlib.h>
 
 #define GGO_BETA_LO 0.05
 #define GGO_BETA_HI 20.0
@@ -345,4 +346,153 @@ void ggo_sample_debug(double beta, uint64_t seed, uint32_t tensor_id, uint64_t i
     *z_out = z;
     *lhs_out = log(ggo_u01(r[2]));
     *rhs_out = w > 0.0 ? 0.5 * z * z + d * (1.0 - v + log(v)) : -INFINITY;
+}
+
+/* ------------------------------------------- Exponential-Golomb rate (Eq. 6-7) */
+
+/* Eq. 6: the signed symbol to the unsigned one that is coded: q < 0 -> -2q, 0 -> 0, q > 0 -> 2q - 1. */
+uint64_t ggo_map(int64_t q)
+{
+    if (q < 0) return (uint64_t)(-2 * q);
+    if (q == 0) return 0;
+    return (uint64_t)(2 * q - 1);
+}
+
+/* Length in bits of the k-th order Exponential-Golomb code of m >= 0:
+ * 2 floor(log2(m + 2^k)) - k + 1.  (Eq. 7 prints this with its floor written as a straight-through
+ * operator and the "- k + 1" outside the mean; read as the standard code length.)  The floor of
+ * the logarithm is the position of the highest set bit, found by shifting. */
+int32_t ggo_eg_length(uint64_t m, int32_t k)
+{
+    uint64_t v = m + ((uint64_t)1 << k);
+    int32_t fl = -1;
+    while (v) { v >>= 1; ++fl; }
+    return 2 * fl - k + 1;
+}
+
+/* Eq. 7 for one tensor, element by element: quantise (the fp32-defined floor quantiser above, with
+ * the clamp), map, take the code length, average.  n = 0 gives 0. */
+double ggo_eg_rate(const float *x, int64_t n, float step, int32_t qmin, int32_t qmax, int32_t k)
+{
+    const float inv = (float)(1.0 / (double)step);
+    long double bits = 0.0L;
+    int64_t counted = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        const float t = x[i] * inv;
+        double f = floor((double)t);
+        if (isnan(f)) continue;
+        int64_t q;
+        if (f < (double)qmin) q = qmin; else if (f > (double)qmax) q = qmax; else q = (int64_t)f;
+        bits += (long double)ggo_eg_length(ggo_map(q), k);
+        ++counted;
+    }
+    return counted ? (double)(bits / (long double)counted) : 0.0;
+}
+
+/* The same rate from a count table (bin b holds symbol qmin + b). */
+double ggo_eg_rate_hist(const uint64_t *hist, int64_t n_bins, int32_t qmin, int32_t k)
+{
+    long double bits = 0.0L, total = 0.0L;
+    for (int64_t b = 0; b < n_bins; ++b) {
+        if (!hist[b]) continue;
+        bits += (long double)hist[b] * (long double)ggo_eg_length(ggo_map((int64_t)qmin + b), k);
+        total += (long double)hist[b];
+    }
+    return total > 0.0L ? (double)(bits / total) : 0.0;
+}
+
+/* Gradient of lambda * R with respect to the elements, the paper's
+ *     dR/dG = 2^(n+2) / (N ln 2) * Sign(G) / Map(Quant(G))
+ * with 2^n = 1/step, N the element count, and the denominator read as m + 2^k (the derivative of
+ * 2 log2(m + 2^k); the printed form leaves 2^k out and divides by zero at m = 0):
+ *     g_i = lambda * 4 / (step N ln 2) * sign(x_i) / (Map(q_i) + 2^k),   sign(0) = 0.
+ * The scaling 1/step is the quantiser's fp32 inv, so that both sides use the same number. */
+void ggo_eg_rate_grad(const float *x, int64_t n, float step, int32_t qmin, int32_t qmax, int32_t k,
+                      double lambda, double *grad)
+{
+    const float inv = (float)(1.0 / (double)step);
+    const double c = n > 0 ? lambda * 4.0 * (double)inv / ((double)n * log(2.0)) : 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        const float t = x[i] * inv;
+        double f = floor((double)t);
+        double g = 0.0;
+        if (!isnan(f) && x[i] != 0.0f) {
+            int64_t q;
+            if (f < (double)qmin) q = qmin; else if (f > (double)qmax) q = qmax; else q = (int64_t)f;
+            g = c / (double)(ggo_map(q) + ((uint64_t)1 << k));
+            if (x[i] < 0.0f) g = -g;
+        }
+        grad[i] = g;
+    }
+}
+
+/* ------------------------------------------------ Huffman and fixed-length bits */
+
+static int ggo_cmp_u64(const void *a, const void *b)
+{
+    const uint64_t x = *(const uint64_t *)a, y = *(const uint64_t *)b;
+    return x < y ? -1 : x > y;
+}
+
+/* Average length in bits of a Huffman code for the counts (textbook construction: repeatedly merge
+ * the two lightest nodes; the average length is the sum of the merged weights over the total).
+ * One occupied bin gives 0 bits.  work: scratch of 2 * n_bins uint64. */
+double ggo_huffman_bits(const uint64_t *hist, int64_t n_bins, uint64_t *work)
+{
+    int64_t n = 0;
+    long double total = 0.0L;
+    for (int64_t b = 0; b < n_bins; ++b) if (hist[b]) { work[n++] = hist[b]; total += (long double)hist[b]; }
+    if (n <= 1) return 0.0;
+    qsort(work, (size_t)n, sizeof(uint64_t), ggo_cmp_u64);
+    /* two queues: leaves work[0..n) in ascending order, merged nodes in creation order (also ascending) */
+    uint64_t *merged = work + n_bins;
+    int64_t li = 0, mi = 0, mn = 0;
+    long double sum = 0.0L;
+    for (int64_t step = 0; step < n - 1; ++step) {
+        uint64_t pick[2];
+        for (int j = 0; j < 2; ++j) {
+            if (mi >= mn || (li < n && work[li] <= merged[mi])) pick[j] = work[li++];
+            else pick[j] = merged[mi++];
+        }
+        merged[mn++] = pick[0] + pick[1];
+        sum += (long double)(pick[0] + pick[1]);
+    }
+    return (double)(sum / total);
+}
+
+/* Bits of a fixed-length code over the occupied symbol range: ceil(log2(max - min + 1)); an empty
+ * table or a single symbol gives 0.  (The paper reports FL without defining it; its values are
+ * whole numbers of bits.) */
+int32_t ggo_fixed_length_bits(const uint64_t *hist, int64_t n_bins)
+{
+    int64_t lo = -1, hi = -1;
+    for (int64_t b = 0; b < n_bins; ++b) if (hist[b]) { if (lo < 0) lo = b; hi = b; }
+    if (lo < 0) return 0;
+    uint64_t span = (uint64_t)(hi - lo);   /* symbols - 1 */
+    int32_t bits = 0;
+    while (span) { span >>= 1; ++bits; }
+    return bits;
+}
+
+/* --------------------------------------------------- GCT elementwise update (Algorithm 2) */
+
+/* One step of gradient constrained training for one tensor, the three elementwise lines of
+ * Algorithm 2 in their printed order, in fp64:
+ *     h_i    = ( -(1/eta) g_i / (ghat_prev_i + eps) + 1/eta ) * [t >= 2]
+ *     ghat_i = g_i + lambda * dR/dg_i * h_i        (dR/dg: ggo_eg_rate_grad with lambda = 1)
+ *     w_i   <- w_i - eta * ghat_i
+ * eps is added to the signed previous gradient exactly as printed.  ghat_out is what the next step
+ * needs as ghat_prev. */
+void ggo_gct_step(const float *g, const double *ghat_prev, const double *w, int64_t n, float step,
+                  int32_t qmin, int32_t qmax, int32_t k, double eta, double lambda, double eps,
+                  int64_t t, double *drdg_work, double *ghat_out, double *w_out)
+{
+    ggo_eg_rate_grad(g, n, step, qmin, qmax, k, 1.0, drdg_work);
+    for (int64_t i = 0; i < n; ++i) {
+        double h = 0.0;
+        if (t >= 2) h = -(1.0 / eta) * (double)g[i] / (ghat_prev[i] + eps) + 1.0 / eta;
+        const double gh = (double)g[i] + lambda * drdg_work[i] * h;
+        ghat_out[i] = gh;
+        w_out[i] = w[i] - eta * gh;
+    }
 }

@@ -73,6 +73,22 @@ def lib():
         L.ggo_sample.argtypes = [d, d, u64, u32, u64, i64, P, P]
         L.ggo_sample_debug.restype = None
         L.ggo_sample_debug.argtypes = [d, u64, u32, u64, u32, P, P, P]
+        L.ggo_map.restype = u64
+        L.ggo_map.argtypes = [i64]
+        L.ggo_eg_length.restype = i32
+        L.ggo_eg_length.argtypes = [u64, i32]
+        L.ggo_eg_rate.restype = d
+        L.ggo_eg_rate.argtypes = [P, i64, f32, i32, i32, i32]
+        L.ggo_eg_rate_hist.restype = d
+        L.ggo_eg_rate_hist.argtypes = [P, i64, i32, i32]
+        L.ggo_eg_rate_grad.restype = None
+        L.ggo_eg_rate_grad.argtypes = [P, i64, f32, i32, i32, i32, d, P]
+        L.ggo_huffman_bits.restype = d
+        L.ggo_huffman_bits.argtypes = [P, i64, P]
+        L.ggo_fixed_length_bits.restype = i32
+        L.ggo_fixed_length_bits.argtypes = [P, i64]
+        L.ggo_gct_step.restype = None
+        L.ggo_gct_step.argtypes = [P, P, P, i64, f32, i32, i32, i32, d, d, d, i64, P, P, P]
         _lib = L
     return _lib
 
@@ -150,6 +166,60 @@ def quantise(x, step, qmin=-32768, qmax=32767):
 def entropy_bits(hist):
     h = np.ascontiguousarray(hist, dtype=np.uint64)
     return lib().ggo_entropy_bits(h.ctypes.data, h.size)
+
+
+# ------------------------------------------------ code lengths (Eq. 6-7)
+def map_unsigned(q): return int(lib().ggo_map(int(q)))
+def eg_length(m, k=0): return int(lib().ggo_eg_length(int(m), int(k)))
+
+
+def eg_rate(x, step, k=0, qmin=-32768, qmax=32767):
+    """Mean k-th order Exponential-Golomb code length of the quantised elements, bits."""
+    a, p = _f32(x)
+    return lib().ggo_eg_rate(p, a.size, np.float32(step).item(), int(qmin), int(qmax), int(k))
+
+
+def eg_rate_hist(hist, k=0, qmin=-32768):
+    h = np.ascontiguousarray(hist, dtype=np.uint64)
+    return lib().ggo_eg_rate_hist(h.ctypes.data, h.size, int(qmin), int(k))
+
+
+def eg_rate_grad(x, step, lam, k=0, qmin=-32768, qmax=32767):
+    a, p = _f32(x)
+    g = np.empty(a.size, dtype=np.float64)
+    lib().ggo_eg_rate_grad(p, a.size, np.float32(step).item(), int(qmin), int(qmax), int(k), float(lam),
+                           g.ctypes.data)
+    return g
+
+
+def huffman_bits(hist):
+    h = np.ascontiguousarray(hist, dtype=np.uint64)
+    work = np.empty(2 * h.size, dtype=np.uint64)
+    return lib().ggo_huffman_bits(h.ctypes.data, h.size, work.ctypes.data)
+
+
+def fixed_length_bits(hist):
+    h = np.ascontiguousarray(hist, dtype=np.uint64)
+    return int(lib().ggo_fixed_length_bits(h.ctypes.data, h.size))
+
+
+def compression_ratio(bits, fixed_bits):
+    """C = 1 - bits / FL: the saving of a variable-length code against the fixed-length one."""
+    return 1.0 - float(bits) / float(fixed_bits)
+
+
+def gct_step(g, ghat_prev, w, step, eta, lam, eps, t, k=0, qmin=-32768, qmax=32767):
+    """(ghat, w_new) of one GCT step (Algorithm 2), fp64."""
+    a, p = _f32(g)
+    gp = np.ascontiguousarray(ghat_prev, dtype=np.float64)
+    ww = np.ascontiguousarray(w, dtype=np.float64)
+    work = np.empty(a.size, dtype=np.float64)
+    gh = np.empty(a.size, dtype=np.float64)
+    wn = np.empty(a.size, dtype=np.float64)
+    lib().ggo_gct_step(p, gp.ctypes.data, ww.ctypes.data, a.size, np.float32(step).item(), int(qmin), int(qmax),
+                       int(k), float(eta), float(lam), float(eps), int(t), work.ctypes.data, gh.ctypes.data,
+                       wn.ctypes.data)
+    return gh, wn
 
 
 def philox4x32_10(ctr, key):
