@@ -203,6 +203,61 @@ typedef struct {
  * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep). */
 gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *args, void *stream);
 
+/* ---- code lengths: the rate the paper defines (Eq. 6-7) and its reporting metrics ------------- */
+
+/* Average k-th order Exponential-Golomb code length of each histogram, bits per symbol: the rate
+ * function R of Eq. 7.  A symbol q is first mapped to an unsigned one (Eq. 6: q < 0 -> -2q,
+ * 0 -> 0, q > 0 -> 2q - 1) and an unsigned m costs 2 floor(log2(m + 2^k)) - k + 1 bits.  Exact
+ * 64-bit integer arithmetic up to the final division; an empty histogram gives 0.
+ *   hist     device uint64[n_hist * (qmax-qmin+1)], bin 0 = symbol qmin (as written by gg_rate_hist)
+ *   k        order of the code, 0 <= k <= 30
+ *   eg_bits  device double[n_hist] output */
+gg_status gg_eg_rate(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t qmin, int32_t qmax,
+                     int32_t k, double *eg_bits, void *stream);
+
+/* Elementwise gradient of lambda * R (the paper's dR/dG = 2^(n+2)/(N ln 2) Sign(G)/Map(Quant(G)),
+ * with 2^n = 1/step, N the element count of the segment, and the denominator taken as
+ * Map(q) + 2^k, the derivative of 2 log2(m + 2^k); the printed form omits 2^k and is undefined at
+ * m = 0):
+ *     g_i = lambda * 4 inv / (N ln 2) * sign(x_i) / (Map(q_i) + 2^k),   g = 0 at x = 0 and at nan
+ * with inv and q_i those of the quantiser of gg_rate_hist.
+ *   step   device float[n_segs]
+ *   grad   host array of n_seg segments (device data of grad_dtype, same lengths), required
+ *   accumulate   0: grad = g;  1: grad += g */
+gg_status gg_eg_rate_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
+                          const float *step, int32_t k, double lambda, int32_t qmin, int32_t qmax,
+                          const gg_seg *grad, gg_dtype grad_dtype, int accumulate, void *stream);
+
+/* Reporting metrics of the paper's tables from histograms: Exponential-Golomb, Huffman and
+ * fixed-length bits per symbol ("EG", "HM", "FL" of Section 5.1).  HM is the average length of a
+ * Huffman code for the counts (0 for fewer than two occupied bins); FL is
+ * ceil(log2(largest occupied symbol - smallest + 1)).  The histograms are copied to the host and
+ * the call returns after `stream` has finished the work before it: this is a reporting call, not
+ * part of a training step.
+ *   eg_bits, hm_bits, fl_bits   HOST double[n_hist] outputs (each may be NULL) */
+gg_status gg_code_stats(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t qmin, int32_t qmax,
+                        int32_t k, double *eg_bits, double *hm_bits, double *fl_bits, void *stream);
+
+/* Compression ratio of a variable-length code against the fixed-length one, C = 1 - bits / FL
+ * (the C_EG and C_HM columns of the paper's tables). */
+double gg_compression_ratio(double bits, double fixed_length_bits);
+
+/* One step of gradient constrained training for a list of tensors, the elementwise lines of
+ * Algorithm 2 in one streaming pass (three reads, two writes per element):
+ *     h      = ( -(1/eta) g / (ghat + eps) + 1/eta ) * [t >= 2]      (curvature estimate)
+ *     ghat  <- g + lambda * dR/dg * h                                 (stored for the next step)
+ *     w     <- w - eta * ghat
+ * with dR/dg the gradient of gg_eg_rate_grad for lambda = 1.  Arithmetic is fp64, storage fp32.
+ *   g      host array of n_seg segments (device data of g_dtype): this step's gradients
+ *   ghat   host array of n_seg segments (device float32, same lengths): in: the equivalent gradients
+ *          of the previous step (not read when t < 2); out: this step's
+ *   w      host array of n_seg segments (device float32, same lengths): the weights, updated in place
+ *   step   device float[n_seg]: quantiser steps
+ *   t      the training step, 1-based */
+gg_status gg_gct_step(gg_ctx *ctx, const gg_seg *g, int32_t n_seg, gg_dtype g_dtype, const gg_seg *ghat,
+                      const gg_seg *w, const float *step, int32_t k, int32_t qmin, int32_t qmax,
+                      double eta, double lambda, double eps, int64_t t, void *stream);
+
 /* Optional device timing of the sweeps inside gg_fused (no counterpart in the paper: measurement
  * support).  While enabled, gg_fused records a CUDA event pair on the caller's stream around its
  * first sweep (moments, or the single combined sweep of GG_PARAMS_GIVEN) and around its second

@@ -85,6 +85,14 @@ def lib():
         L.gg_fit_noalloc.argtypes = [ctypes.c_int, _P, i64, ctypes.c_int, _P, _P, _P, _P, _P, _P, _P]
         L.gg_fit_noalloc.restype = ctypes.c_int
         L.gg_fit_noalloc_max_len.restype = i64
+        L.gg_eg_rate.argtypes = [_P, _P, i32, i32, i32, i32, _P, _P]
+        L.gg_eg_rate_grad.argtypes = [_P, _P, i32, ctypes.c_int, _P, i32, d, i32, i32, _P, ctypes.c_int, ctypes.c_int, _P]
+        L.gg_code_stats.argtypes = [_P, _P, i32, i32, i32, i32, _P, _P, _P, _P]
+        L.gg_gct_step.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, _P, i32, i32, i32, d, d, d, i64, _P]
+        L.gg_compression_ratio.argtypes = [d, d]
+        L.gg_compression_ratio.restype = d
+        for name in ("gg_eg_rate", "gg_eg_rate_grad", "gg_code_stats", "gg_gct_step"):
+            getattr(L, name).restype = ctypes.c_int
         for name in ("gg_create", "gg_destroy", "gg_fit", "gg_penalty_grad", "gg_rate_hist", "gg_sample",
                      "gg_fused", "gg_fused_host", "gg_timing_enable", "gg_timing_read"):
             getattr(L, name).restype = ctypes.c_int
@@ -123,6 +131,10 @@ def gg_fit_noalloc(x, out=None):
     if status != 0:
         raise GGError(status, lib().gg_status_str(status).decode())
     return out
+
+
+def gg_compression_ratio(bits, fixed_length_bits):
+    return lib().gg_compression_ratio(float(bits), float(fixed_length_bits))
 
 
 def _dtype_code(dt):
@@ -428,6 +440,38 @@ class Context:
 
     def gg_fused_host(self, segs, **kw):
         return self.make_fused_host(segs, **kw)()
+
+    # ------------------------------------------------------------ code lengths
+    def gg_eg_rate(self, hist, k=0, qmin=-32768, qmax=32767):
+        """Average Exponential-Golomb code length per histogram (device float64)."""
+        n_hist = hist.shape[0]
+        out = self._new(n_hist, torch.float64)
+        self._check(lib().gg_eg_rate(self._h, _ptr(hist), n_hist, int(qmin), int(qmax), int(k), _ptr(out),
+                                     _stream_ptr(self.device)))
+        return out
+
+    def gg_eg_rate_grad(self, segs, step, lam, grad, k=0, qmin=-32768, qmax=32767, accumulate=False):
+        """Writes the gradient of lam * (Exponential-Golomb rate) into the `grad` segments."""
+        segs, gsegs = _as_segments(segs), _as_segments(grad)
+        self._check(lib().gg_eg_rate_grad(self._h, segs.ptr, len(segs), segs.code, _ptr(step), int(k), float(lam),
+                                          int(qmin), int(qmax), gsegs.ptr, gsegs.code, int(bool(accumulate)),
+                                          _stream_ptr(self.device)))
+
+    def gg_code_stats(self, hist, k=0, qmin=-32768, qmax=32767):
+        """EG, Huffman and fixed-length bits per histogram as numpy arrays (synchronises the stream)."""
+        n_hist = hist.shape[0]
+        eg, hm, fl = (np.empty(n_hist, dtype=np.float64) for _ in range(3))
+        self._check(lib().gg_code_stats(self._h, _ptr(hist), n_hist, int(qmin), int(qmax), int(k), eg.ctypes.data,
+                                        hm.ctypes.data, fl.ctypes.data, _stream_ptr(self.device)))
+        return dict(eg_bits=eg, hm_bits=hm, fl_bits=fl)
+
+    def gg_gct_step(self, g, ghat, w, step, eta, lam, eps, t, k=0, qmin=-32768, qmax=32767):
+        """One GCT step in place: `ghat` (float32 segments) and `w` (float32 segments) are updated."""
+        gs, hs, ws = _as_segments(g), _as_segments(ghat), _as_segments(w)
+        if hs.dtype != torch.float32 or ws.dtype != torch.float32:
+            raise TypeError("ghat and w are float32")
+        self._check(lib().gg_gct_step(self._h, gs.ptr, len(gs), gs.code, hs.ptr, ws.ptr, _ptr(step), int(k), int(qmin),
+                                      int(qmax), float(eta), float(lam), float(eps), int(t), _stream_ptr(self.device)))
 
     # ------------------------------------------------------------------ timing
     def timing_enable(self, on=True):

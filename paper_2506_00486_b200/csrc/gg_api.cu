@@ -832,3 +832,151 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ code lengths and the GCT step
+#include <algorithm>
+
+namespace {
+
+// Average Huffman code length of the non-zero counts: sort, then merge the two lightest nodes with
+// two queues (leaves in ascending order, merged nodes in creation order).
+double huffman_bits(const uint64_t *row, int64_t n_bins, std::vector<uint64_t> &leaves, std::vector<uint64_t> &merged)
+{
+    leaves.clear();
+    long double total = 0.0L;
+    for (int64_t b = 0; b < n_bins; ++b)
+        if (row[b]) { leaves.push_back(row[b]); total += (long double)row[b]; }
+    const size_t n = leaves.size();
+    if (n <= 1) return 0.0;
+    std::sort(leaves.begin(), leaves.end());
+    merged.assign(n, 0);
+    size_t li = 0, mi = 0, mn = 0;
+    long double sum = 0.0L;
+    for (size_t it = 0; it + 1 < n; ++it) {
+        uint64_t pick[2];
+        for (int j = 0; j < 2; ++j) {
+            if (mi >= mn || (li < n && leaves[li] <= merged[mi])) pick[j] = leaves[li++];
+            else pick[j] = merged[mi++];
+        }
+        merged[mn++] = pick[0] + pick[1];
+        sum += (long double)(pick[0] + pick[1]);
+    }
+    return (double)(sum / total);
+}
+
+int eg_length_host(uint64_t m, int k)
+{
+    uint64_t v = m + (1ull << k);
+    int fl = -1;
+    while (v) { v >>= 1; ++fl; }
+    return 2 * fl - k + 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+double gg_compression_ratio(double bits, double fixed_length_bits) { return 1.0 - bits / fixed_length_bits; }
+
+gg_status gg_eg_rate(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t qmin, int32_t qmax, int32_t k,
+                     double *eg_bits, void *stream)
+{
+    if (!ctx || !hist || !eg_bits || k < 0 || k > 30) return GG_ERR_INVALID_ARG;
+    gg_status st = check_hist(0, nullptr, 0, qmin, qmax);
+    if (st != GG_OK || n_hist < 0) return GG_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+    GG_CUDA(ctx, launch_eg_rate(hist, n_hist, qmax - qmin + 1, qmin, k, eg_bits, static_cast<cudaStream_t>(stream)));
+    ctx->launches += n_hist > 0;
+    return GG_OK;
+}
+
+gg_status gg_eg_rate_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype, const float *step, int32_t k,
+                          double lambda, int32_t qmin, int32_t qmax, const gg_seg *grad, gg_dtype grad_dtype,
+                          int accumulate, void *stream)
+{
+    if (!ctx || !grad || (n_seg > 0 && !step) || k < 0 || k > 30 || qmax < qmin) return GG_ERR_INVALID_ARG;
+    gg_status st = check_segs(segs, n_seg, dtype);
+    if (st != GG_OK) return st;
+    st = check_grad(segs, grad, n_seg, grad_dtype);
+    if (st != GG_OK) return st;
+    if (n_seg == 0) return GG_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+    Plan *p = nullptr;
+    st = get_plan(ctx, segs, n_seg, dtype, grad, grad_dtype, nullptr, &p);
+    if (st != GG_OK) return st;
+    GG_CUDA(ctx, launch_eg_grad(p->map, dtype, grad_dtype, step, qmin, qmax, k, lambda, accumulate,
+                                static_cast<cudaStream_t>(stream)));
+    ctx->launches += p->n_tiles > 0;
+    return GG_OK;
+}
+
+gg_status gg_code_stats(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t qmin, int32_t qmax, int32_t k,
+                        double *eg_bits, double *hm_bits, double *fl_bits, void *stream)
+{
+    if (!ctx || !hist || n_hist < 0 || k < 0 || k > 30 || qmax < qmin) return GG_ERR_INVALID_ARG;
+    if ((int64_t)qmax - (int64_t)qmin + 1 > (1ll << 24)) return GG_ERR_INVALID_ARG;
+    if (n_hist == 0) return GG_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+    const int64_t n_bins = (int64_t)qmax - qmin + 1;
+    std::vector<uint64_t> host;
+    try { host.resize((size_t)n_hist * (size_t)n_bins); } catch (...) { return GG_ERR_NOMEM; }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    GG_CUDA(ctx, cudaMemcpyAsync(host.data(), hist, sizeof(uint64_t) * host.size(), cudaMemcpyDeviceToHost, cs));
+    GG_CUDA(ctx, cudaStreamSynchronize(cs));
+    std::vector<uint64_t> leaves, merged;
+    for (int32_t h = 0; h < n_hist; ++h) {
+        const uint64_t *row = host.data() + (size_t)h * (size_t)n_bins;
+        if (eg_bits) {
+            long double bits = 0.0L, total = 0.0L;
+            for (int64_t b = 0; b < n_bins; ++b) {
+                if (!row[b]) continue;
+                const int64_t q = (int64_t)qmin + b;
+                const uint64_t m = q < 0 ? (uint64_t)(-2 * q) : (q == 0 ? 0 : (uint64_t)(2 * q - 1));
+                bits += (long double)row[b] * (long double)eg_length_host(m, k);
+                total += (long double)row[b];
+            }
+            eg_bits[h] = total > 0.0L ? (double)(bits / total) : 0.0;
+        }
+        if (hm_bits) hm_bits[h] = huffman_bits(row, n_bins, leaves, merged);
+        if (fl_bits) {
+            int64_t lo = -1, hi = -1;
+            for (int64_t b = 0; b < n_bins; ++b) if (row[b]) { if (lo < 0) lo = b; hi = b; }
+            uint64_t span = lo < 0 ? 0 : (uint64_t)(hi - lo);
+            int bits = 0;
+            while (span) { span >>= 1; ++bits; }
+            fl_bits[h] = (double)bits;
+        }
+    }
+    return GG_OK;
+}
+
+gg_status gg_gct_step(gg_ctx *ctx, const gg_seg *g, int32_t n_seg, gg_dtype g_dtype, const gg_seg *ghat, const gg_seg *w,
+                      const float *step, int32_t k, int32_t qmin, int32_t qmax, double eta, double lambda, double eps,
+                      int64_t t, void *stream)
+{
+    if (!ctx || !ghat || !w || (n_seg > 0 && !step) || k < 0 || k > 30 || qmax < qmin || !(eta > 0.0)) return GG_ERR_INVALID_ARG;
+    gg_status st = check_segs(g, n_seg, g_dtype);
+    if (st != GG_OK) return st;
+    st = check_grad(g, ghat, n_seg, GG_F32);
+    if (st != GG_OK) return st;
+    st = check_grad(g, w, n_seg, GG_F32);
+    if (st != GG_OK) return st;
+    if (n_seg == 0) return GG_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+    Plan *pg = nullptr, *pw = nullptr;
+    st = get_plan(ctx, g, n_seg, g_dtype, ghat, GG_F32, nullptr, &pg);
+    if (st != GG_OK) return st;
+    st = get_plan(ctx, w, n_seg, GG_F32, nullptr, 0, nullptr, &pw);      // (for its device table of the weight addresses)
+    if (st != GG_OK) return st;
+    GG_CUDA(ctx, launch_gct_step(pg->map, const_cast<void *const *>(reinterpret_cast<const void *const *>(pw->map.seg_ptr)),
+                                 g_dtype, step, qmin, qmax, k, eta, lambda, eps, t >= 2 ? 1 : 0,
+                                 static_cast<cudaStream_t>(stream)));
+    ctx->launches += pg->n_tiles > 0;
+    return GG_OK;
+}
+
+}  // extern "C"

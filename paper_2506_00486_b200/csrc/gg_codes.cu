@@ -1,0 +1,169 @@
+// Code-length side of the rate model: the Exponential-Golomb rate of Eq. 6-7 from a symbol histogram,
+// its elementwise gradient, and the elementwise update of gradient constrained training
+// (Algorithm 2).  All three are streaming or O(bins) kernels; none is a contraction.
+#include <cuda_bf16.h>
+
+#include "gg_internal.h"
+
+namespace gg {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+// Eq. 6: signed symbol -> unsigned symbol.
+__device__ __forceinline__ uint32_t map_unsigned(int32_t q)
+{
+    return q < 0 ? (uint32_t)(-2 * (int64_t)q) : (q == 0 ? 0u : (uint32_t)(2 * (int64_t)q - 1));
+}
+
+// Length of the k-th order Exponential-Golomb code of m: 2 floor(log2(m + 2^k)) - k + 1.
+__device__ __forceinline__ int eg_length(uint32_t m, int k)
+{
+    const unsigned long long v = (unsigned long long)m + (1ull << k);
+    return 2 * (63 - __clzll((long long)v)) - k + 1;
+}
+
+// One CTA per histogram: sum of count * length and sum of counts in 64-bit integers (exact, so the
+// order of the additions does not matter), then the mean.
+__global__ void __launch_bounds__(kThreads) eg_rate_kernel(const uint64_t *hist, int32_t n_bins, int32_t qmin, int32_t k,
+                                                           double *eg_bits)
+{
+    __shared__ unsigned long long shBits[kThreads / 32], shTot[kThreads / 32];
+    const uint64_t *row = hist + (int64_t)blockIdx.x * n_bins;
+    unsigned long long bits = 0, tot = 0;
+    for (int b = threadIdx.x; b < n_bins; b += kThreads) {
+        const unsigned long long c = row[b];
+        if (c != 0) {
+            bits += c * (unsigned long long)eg_length(map_unsigned(qmin + b), k);
+            tot += c;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        bits += __shfl_xor_sync(kFull, bits, o);
+        tot += __shfl_xor_sync(kFull, tot, o);
+    }
+    if ((threadIdx.x & 31) == 0) { shBits[threadIdx.x >> 5] = bits; shTot[threadIdx.x >> 5] = tot; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long rb = 0, rt = 0;
+        for (int w = 0; w < kThreads / 32; ++w) { rb += shBits[w]; rt += shTot[w]; }
+        eg_bits[blockIdx.x] = rt ? (double)rb / (double)rt : 0.0;
+    }
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<uint16_t>(uint16_t v) { return __uint_as_float((uint32_t)v << 16); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ uint16_t from_f32<uint16_t>(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
+
+// The unsigned symbol of x plus 2^k, as the quantiser defines it (fp32 product, floor, clamp), or 0
+// when x is zero or nan (no gradient there).
+__device__ __forceinline__ uint32_t eg_denominator(float x, float inv, int32_t qmin, int32_t qmax, int k)
+{
+    const float t = __fmul_rn(x, inv);
+    if (!(t == t) || x == 0.0f) return 0u;
+    const int q = max(qmin, min(qmax, __float2int_rd(t)));      // floor, saturating, then the clamp
+    return map_unsigned(q) + (1u << k);
+}
+
+// Gradient of lambda * R (Eq. 7) for every element: one CTA per tile.
+//     g = lambda * 4 inv / (N ln 2) * sign(x) / (Map(q) + 2^k)
+// The per-segment factor is formed in fp64 and rounded once; the division is one fp32 rounding.
+template <typename TIn, typename TG>
+__global__ void __launch_bounds__(kThreads) eg_grad_kernel(const TileMap map, const float *step, int32_t qmin, int32_t qmax,
+                                                           int32_t k, double lambda, int accumulate)
+{
+    const int t = blockIdx.x;
+    const int s = map.tile_seg[t];
+    const int64_t len = map.seg_len[s];
+    const int64_t off = (int64_t)(t - map.tile_prefix[s]) * kTile;
+    const int n = (int)min((int64_t)kTile, len - off);
+    const TIn *x = reinterpret_cast<const TIn *>(map.seg_ptr[s]) + off;
+    TG *g = reinterpret_cast<TG *>(map.grad_ptr[s]) + off;
+    const float inv = (float)(1.0 / (double)step[s]);
+    const float c = (float)(lambda * 4.0 * (double)inv / ((double)len * 0.6931471805599453094));
+    for (int i = threadIdx.x; i < n; i += kThreads) {
+        const float xv = to_f32<TIn>(x[i]);
+        const uint32_t den = eg_denominator(xv, inv, qmin, qmax, k);
+        float v = 0.0f;
+        if (den != 0u) {
+            v = __fdiv_rn(c, (float)den);       // (den is exact in fp32 up to 2^24: symbols of any 16-bit alphabet)
+            if (xv < 0.0f) v = -v;
+        }
+        if (accumulate) v += to_f32<TG>(g[i]);
+        g[i] = from_f32<TG>(v);
+    }
+}
+
+// Algorithm 2, the three elementwise lines, one CTA per tile; fp64 arithmetic (the curvature estimate
+// 1 - g / ghat_prev cancels, and five streams of four bytes leave room for it), fp32 storage.
+template <typename TIn>
+__global__ void __launch_bounds__(kThreads) gct_step_kernel(const TileMap map, void *const *w_ptr, const float *step,
+                                                            int32_t qmin, int32_t qmax, int32_t k, double eta, double lambda,
+                                                            double eps, int apply_h)
+{
+    const int t = blockIdx.x;
+    const int s = map.tile_seg[t];
+    const int64_t len = map.seg_len[s];
+    const int64_t off = (int64_t)(t - map.tile_prefix[s]) * kTile;
+    const int n = (int)min((int64_t)kTile, len - off);
+    const TIn *g = reinterpret_cast<const TIn *>(map.seg_ptr[s]) + off;
+    float *ghat = reinterpret_cast<float *>(map.grad_ptr[s]) + off;
+    float *w = reinterpret_cast<float *>(w_ptr[s]) + off;
+    const float inv = (float)(1.0 / (double)step[s]);
+    const double c = 4.0 * (double)inv / ((double)len * 0.6931471805599453094);
+    const double inv_eta = 1.0 / eta;
+    for (int i = threadIdx.x; i < n; i += kThreads) {
+        const float gf = to_f32<TIn>(g[i]);
+        const double gd = (double)gf;
+        double gh = gd;
+        if (apply_h) {
+            const uint32_t den = eg_denominator(gf, inv, qmin, qmax, k);
+            if (den != 0u) {
+                const double drdg = (gf < 0.0f ? -c : c) / (double)den;
+                const double h = -inv_eta * gd / ((double)ghat[i] + eps) + inv_eta;
+                gh = gd + lambda * drdg * h;
+            }
+        }
+        ghat[i] = (float)gh;
+        w[i] = (float)((double)w[i] - eta * gh);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_eg_rate(const uint64_t *hist, int32_t n_hist, int32_t n_bins, int32_t qmin, int32_t k, double *eg_bits,
+                           cudaStream_t st)
+{
+    if (n_hist <= 0) return cudaSuccess;
+    eg_rate_kernel<<<n_hist, kThreads, 0, st>>>(hist, n_bins, qmin, k, eg_bits);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_eg_grad(const TileMap &map, gg_dtype in_dtype, gg_dtype grad_dtype, const float *step, int32_t qmin,
+                           int32_t qmax, int32_t k, double lambda, int accumulate, cudaStream_t st)
+{
+    if (map.n_tiles <= 0) return cudaSuccess;
+    const dim3 grid((unsigned)map.n_tiles), block(kThreads);
+    if (in_dtype == GG_F32 && grad_dtype == GG_F32) eg_grad_kernel<float, float><<<grid, block, 0, st>>>(map, step, qmin, qmax, k, lambda, accumulate);
+    else if (in_dtype == GG_F32) eg_grad_kernel<float, uint16_t><<<grid, block, 0, st>>>(map, step, qmin, qmax, k, lambda, accumulate);
+    else if (grad_dtype == GG_F32) eg_grad_kernel<uint16_t, float><<<grid, block, 0, st>>>(map, step, qmin, qmax, k, lambda, accumulate);
+    else eg_grad_kernel<uint16_t, uint16_t><<<grid, block, 0, st>>>(map, step, qmin, qmax, k, lambda, accumulate);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gct_step(const TileMap &map, void *const *w_ptr, gg_dtype g_dtype, const float *step, int32_t qmin,
+                            int32_t qmax, int32_t k, double eta, double lambda, double eps, int apply_h, cudaStream_t st)
+{
+    if (map.n_tiles <= 0) return cudaSuccess;
+    const dim3 grid((unsigned)map.n_tiles), block(kThreads);
+    if (g_dtype == GG_F32) gct_step_kernel<float><<<grid, block, 0, st>>>(map, w_ptr, step, qmin, qmax, k, eta, lambda, eps, apply_h);
+    else gct_step_kernel<uint16_t><<<grid, block, 0, st>>>(map, w_ptr, step, qmin, qmax, k, eta, lambda, eps, apply_h);
+    return cudaGetLastError();
+}
+
+}  // namespace gg

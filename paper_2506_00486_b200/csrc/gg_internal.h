@@ -115,6 +115,13 @@ cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part,
 constexpr int kEntSplit = 16;
 cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
                            double *scratch, cudaStream_t st);
+cudaError_t launch_eg_rate(const uint64_t *hist, int32_t n_hist, int32_t n_bins, int32_t qmin, int32_t k, double *eg_bits,
+                           cudaStream_t st);
+cudaError_t launch_eg_grad(const TileMap &map, gg_dtype in_dtype, gg_dtype grad_dtype, const float *step, int32_t qmin,
+                           int32_t qmax, int32_t k, double lambda, int accumulate, cudaStream_t st);
+// map: the gradient segments with the stored equivalent gradients (fp32) as grad_ptr; w_ptr: the weights (fp32)
+cudaError_t launch_gct_step(const TileMap &map, void *const *w_ptr, gg_dtype g_dtype, const float *step, int32_t qmin,
+                            int32_t qmax, int32_t k, double eta, double lambda, double eps, int apply_h, cudaStream_t st);
 cudaError_t launch_sample(const TileMap &map, gg_dtype dtype, const double *beta, const double *alpha,
                           uint64_t seed, uint32_t tensor_id0, uint32_t *max_attempts, cudaStream_t st);
 
