@@ -70,7 +70,40 @@ __device__ __forceinline__ uint32_t eg_denominator(float x, float inv, int32_t q
     return map_unsigned(q) + (1u << k);
 }
 
-// Gradient of lambda * R (Eq. 7) for every element: one CTA per tile.
+// Four consecutive elements at p (aligned to four elements) or one element, as fp32.
+template <typename T> struct Vec4;
+template <> struct Vec4<float> {
+    static __device__ __forceinline__ void load(const float *p, float (&v)[4])
+    {
+        const float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&v)[4])
+    {
+        __stcs(reinterpret_cast<float4 *>(p), make_float4(v[0], v[1], v[2], v[3]));
+    }
+};
+template <> struct Vec4<uint16_t> {
+    static __device__ __forceinline__ void load(const uint16_t *p, float (&v)[4])
+    {
+        const uint2 t = __ldcs(reinterpret_cast<const uint2 *>(p));
+        v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xFFFF0000u);
+        v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ void store(uint16_t *p, const float (&v)[4])
+    {
+        uint2 t;
+        t.x = (uint32_t)from_f32<uint16_t>(v[0]) | ((uint32_t)from_f32<uint16_t>(v[1]) << 16);
+        t.y = (uint32_t)from_f32<uint16_t>(v[2]) | ((uint32_t)from_f32<uint16_t>(v[3]) << 16);
+        __stcs(reinterpret_cast<uint2 *>(p), t);
+    }
+};
+
+template <typename T>
+__device__ __forceinline__ bool aligned4(const T *p) { return (reinterpret_cast<uintptr_t>(p) & (4 * sizeof(T) - 1)) == 0; }
+
+// Gradient of lambda * R (Eq. 7) for every element: one CTA per tile, four elements per thread and
+// trip when the tile's addresses allow vector accesses.
 //     g = lambda * 4 inv / (N ln 2) * sign(x) / (Map(q) + 2^k)
 // The per-segment factor is formed in fp64 and rounded once; the division is one fp32 rounding.
 template <typename TIn, typename TG>
@@ -86,21 +119,32 @@ __global__ void __launch_bounds__(kThreads) eg_grad_kernel(const TileMap map, co
     TG *g = reinterpret_cast<TG *>(map.grad_ptr[s]) + off;
     const float inv = (float)(1.0 / (double)step[s]);
     const float c = (float)(lambda * 4.0 * (double)inv / ((double)len * 0.6931471805599453094));
-    for (int i = threadIdx.x; i < n; i += kThreads) {
-        const float xv = to_f32<TIn>(x[i]);
+    auto one = [&](float xv, float old) {
         const uint32_t den = eg_denominator(xv, inv, qmin, qmax, k);
         float v = 0.0f;
         if (den != 0u) {
             v = __fdiv_rn(c, (float)den);       // (den is exact in fp32 up to 2^24: symbols of any 16-bit alphabet)
             if (xv < 0.0f) v = -v;
         }
-        if (accumulate) v += to_f32<TG>(g[i]);
-        g[i] = from_f32<TG>(v);
+        return accumulate ? v + old : v;
+    };
+    const int nvec = (aligned4(x) && aligned4(g)) ? n / 4 : 0;
+    for (int v = threadIdx.x; v < nvec; v += kThreads) {
+        float xv[4], gv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        Vec4<TIn>::load(x + 4 * v, xv);
+        if (accumulate) Vec4<TG>::load(g + 4 * v, gv);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gv[i] = one(xv[i], gv[i]);
+        Vec4<TG>::store(g + 4 * v, gv);
     }
+    for (int i = 4 * nvec + threadIdx.x; i < n; i += kThreads)
+        g[i] = from_f32<TG>(one(to_f32<TIn>(x[i]), accumulate ? to_f32<TG>(g[i]) : 0.0f));
 }
 
-// Algorithm 2, the three elementwise lines, one CTA per tile; fp64 arithmetic (the curvature estimate
-// 1 - g / ghat_prev cancels, and five streams of four bytes leave room for it), fp32 storage.
+// Algorithm 2, the three elementwise lines, one CTA per tile.  The curvature estimate
+// 1 - g / (ghat_prev + eps) cancels, so that quotient and what follows are fp64 (one fp64 division
+// per element fits under the time the five streams of four bytes take); the reciprocal of dR/dg's
+// integer denominator is an fp32 reciprocal refined by one fp64 Newton step.  Storage fp32.
 template <typename TIn>
 __global__ void __launch_bounds__(kThreads) gct_step_kernel(const TileMap map, void *const *w_ptr, const float *step,
                                                             int32_t qmin, int32_t qmax, int32_t k, double eta, double lambda,
@@ -115,23 +159,37 @@ __global__ void __launch_bounds__(kThreads) gct_step_kernel(const TileMap map, v
     float *ghat = reinterpret_cast<float *>(map.grad_ptr[s]) + off;
     float *w = reinterpret_cast<float *>(w_ptr[s]) + off;
     const float inv = (float)(1.0 / (double)step[s]);
-    const double c = 4.0 * (double)inv / ((double)len * 0.6931471805599453094);
+    const double c = lambda * 4.0 * (double)inv / ((double)len * 0.6931471805599453094);
     const double inv_eta = 1.0 / eta;
-    for (int i = threadIdx.x; i < n; i += kThreads) {
-        const float gf = to_f32<TIn>(g[i]);
+    auto one = [&](float gf, float &gh_io, float &w_io) {
         const double gd = (double)gf;
         double gh = gd;
         if (apply_h) {
             const uint32_t den = eg_denominator(gf, inv, qmin, qmax, k);
             if (den != 0u) {
-                const double drdg = (gf < 0.0f ? -c : c) / (double)den;
-                const double h = -inv_eta * gd / ((double)ghat[i] + eps) + inv_eta;
-                gh = gd + lambda * drdg * h;
+                // 1 / den: an fp32 reciprocal and one Newton step in fp64 (error ~1e-14), cheaper than a division
+                const double r0 = (double)__frcp_rn((float)den);
+                const double rcp = r0 * fma(-(double)den, r0, 2.0);
+                const double rate_term = (gf < 0.0f ? -c : c) * rcp;     // lambda dR/dg
+                const double h = inv_eta - inv_eta * gd / ((double)gh_io + eps);
+                gh = fma(rate_term, h, gd);
             }
         }
-        ghat[i] = (float)gh;
-        w[i] = (float)((double)w[i] - eta * gh);
+        gh_io = (float)gh;
+        w_io = (float)fma(-eta, gh, (double)w_io);
+    };
+    const int nvec = (aligned4(g) && aligned4(ghat) && aligned4(w)) ? n / 4 : 0;
+    for (int v = threadIdx.x; v < nvec; v += kThreads) {
+        float gv[4], hv[4], wv[4];
+        Vec4<TIn>::load(g + 4 * v, gv);
+        Vec4<float>::load(ghat + 4 * v, hv);
+        Vec4<float>::load(w + 4 * v, wv);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) one(gv[i], hv[i], wv[i]);
+        Vec4<float>::store(ghat + 4 * v, hv);
+        Vec4<float>::store(w + 4 * v, wv);
     }
+    for (int i = 4 * nvec + threadIdx.x; i < n; i += kThreads) one(to_f32<TIn>(g[i]), ghat[i], w[i]);
 }
 
 }  // namespace

@@ -205,7 +205,17 @@ __device__ __forceinline__ void process(const float (&x)[KV], float (&g)[KV], Ac
         if constexpr (FLAGS & kHist) hist_elem(xe, hc, win, clampc);
     }
     // short fp32 runs, then fp64: the fp32 part adds at most KV roundings of 2^-24 each
-    if constexpr (FLAGS & kMoments) { acc.s1 += (double)m1; acc.s2 += (double)m2; }
+    if constexpr (FLAGS & kMoments) {
+        if (m2 <= FLT_MAX) {
+            acc.s1 += (double)m1;
+            acc.s2 += (double)m2;
+        } else {     // a square or a sum beyond the fp32 range: this run again in fp64
+            for (int e = 0; e < KV; ++e) {
+                const double ax = (double)fabsf(x[e]);
+                if (ax <= (double)FLT_MAX) { acc.s1 += ax; acc.s2 += ax * ax; }
+            }
+        }
+    }
     if constexpr (FLAGS & kGrad) {
         if (mp <= FLT_MAX) {
             acc.pen += (double)mp;
@@ -403,11 +413,11 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
 // issue slots per element.  This kernel spends about five: the widening and the two sums per
 // element, min/max on packed bf16 pairs, and one packed test per pair for inf/nan (a vector that
 // contains one is redone element by element).
-__device__ __forceinline__ void moments_careful(uint32_t h, float &m1, float &m2, uint32_t &bad)
+__device__ __forceinline__ void moments_careful(uint32_t h, double &m1, double &m2, uint32_t &bad)
 {
     const uint32_t mag = h & 0x7FFFu;
-    const float ax = __uint_as_float(mag << 16);
-    if (mag < 0x7F80u) { m1 += ax; m2 = fmaf(ax, ax, m2); }
+    const double ax = (double)__uint_as_float(mag << 16);
+    if (mag < 0x7F80u) { m1 += ax; m2 = fma(ax, ax, m2); }     // (fp64: a square above 3.4e38 must not become inf)
     else bad += 1u;
 }
 
@@ -434,9 +444,7 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
     for (int i = tid; i < head + (n - tail0); i += kThreads) {
         const int idx = i < head ? i : tail0 + (i - head);
         const uint32_t h = (uint32_t)__ldg(x + idx);
-        float m1 = 0.0f, m2 = 0.0f;
-        moments_careful(h, m1, m2, bad);
-        s1 += (double)m1; s2 += (double)m2;
+        moments_careful(h, s1, s2, bad);
         xmin = fminf(xmin, __uint_as_float(h << 16));
         xmax = fmaxf(xmax, __uint_as_float(h << 16));
     }
@@ -469,15 +477,17 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
                     mn2 = __hmin2(mn2, p);      // return the non-NaN operand, like fminf
                     mx2 = __hmax2(mx2, p);
                 }
-                if (probe & 0x80008000u) {      // an inf or nan in this vector: leave it out of the sums
-                    m1 = 0.0f; m2 = 0.0f;
+                if ((probe & 0x80008000u) || !(m2 <= FLT_MAX)) {
+                    // an inf or nan in this vector (left out of the sums), or a square or a sum beyond the
+                    // fp32 range: the vector again, element by element in fp64
                     for (int i = 0; i < 4; ++i) {
-                        moments_careful(w[i] & 0xFFFFu, m1, m2, bad);
-                        moments_careful(w[i] >> 16, m1, m2, bad);
+                        moments_careful(w[i] & 0xFFFFu, s1, s2, bad);
+                        moments_careful(w[i] >> 16, s1, s2, bad);
                     }
+                } else {
+                    s1 += (double)m1;
+                    s2 += (double)m2;
                 }
-                s1 += (double)m1;
-                s2 += (double)m2;
             }
         }
     }

@@ -284,7 +284,22 @@ __device__ __noinline__ double pen_rare(uint4 raw, int n, const Smem &sm)
 template <int FLAGS>
 __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &acc, const Smem &sm)
 {
-    if constexpr ((FLAGS & kMoments) != 0) { acc.s1 += (double)r.m1; acc.s2 += (double)r.m2; }
+    if constexpr ((FLAGS & kMoments) != 0) {
+        if (r.m2 <= FLT_MAX) {
+            acc.s1 += (double)r.m1;
+            acc.s2 += (double)r.m2;
+        } else {     // a square or a sum beyond the fp32 range: this run again in fp64
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+            for (int e = 0; e < n; ++e) {
+                const uint32_t h = (w[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu;
+                if (h < 0x7F80u) {
+                    const double ax = (double)__uint_as_float(h << 16);
+                    acc.s1 += ax;
+                    acc.s2 += ax * ax;
+                }
+            }
+        }
+    }
     if constexpr ((FLAGS & kGrad) != 0) {
         // a product or a gradient that left the fp32 range, or a NaN marker, sends the run to fp64
         if (r.mp <= FLT_MAX) acc.pen += (double)r.mp;

@@ -86,6 +86,25 @@ def test_fit_degenerate_and_flags(ctx):
         assert out["sum_abs"][s].item() == pytest.approx(s1, rel=1e-7)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fit_with_magnitudes_whose_squares_leave_the_fp32_range(ctx, dtype):
+    """|x| above 1.8e19 squares to more than fp32 holds; the moments must still be those of the oracle."""
+    rng = np.random.default_rng(17)
+    x = gg_synth.gg_host(rng, 0.7, 1e22, 3 * TILE + 50, torch.float32)
+    x[::97] = 3.0e38
+    x[5::89] = -2.5e38
+    x = x.to(dtype)
+    out = ctx.gg_fit([dev(x), dev(x[:1000])])
+    torch.cuda.synchronize()
+    for s, xs in enumerate((x, x[:1000])):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(xs))
+        assert out["flags"][s].item() == fl
+        assert_rel(out["sum_abs"][s].item(), s1, 1e-7, "sum_abs")
+        assert_rel(out["sum_sq"][s].item(), s2, 1e-7, "sum_sq")
+        assert_rel(out["beta"][s].item(), b, REL_FIT, "beta")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
+
+
 def test_fit_over_the_whole_shape_range(ctx):
     """beta from 0.1 to 8 on large samples: the fitted pair matches the oracle's."""
     rng = np.random.default_rng(21)
