@@ -411,8 +411,9 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
 // ---------------------------------------------------------------------------- bf16 moments
 // The first sweep over bf16 data reads 2 bytes per element, so at HBM speed an SM has about ten
 // issue slots per element.  This kernel spends about five: the widening and the two sums per
-// element, min/max on packed bf16 pairs, and one packed test per pair for inf/nan (a vector that
-// contains one is redone element by element).
+// element and min/max on packed bf16 pairs; a vector whose fp32 sum of squares comes out inf or nan
+// (it holds an inf or a nan, or values whose squares leave the fp32 range) is redone element by
+// element in fp64.
 __device__ __forceinline__ void moments_careful(uint32_t h, double &m1, double &m2, uint32_t &bad)
 {
     const uint32_t mag = h & 0x7FFFu;
@@ -463,11 +464,8 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
             if (v < nvec) {
                 const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
                 float m1 = 0.0f, m2 = 0.0f;
-                uint32_t probe = 0;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    // adding 0x80 to a 15-bit magnitude carries into bit 15 iff the exponent is all ones
-                    probe |= (w[i] & 0x7FFF7FFFu) + 0x00800080u;
                     const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
                     m1 += fabsf(lo);
                     m1 += fabsf(hi);
@@ -477,9 +475,10 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
                     mn2 = __hmin2(mn2, p);      // return the non-NaN operand, like fminf
                     mx2 = __hmax2(mx2, p);
                 }
-                if ((probe & 0x80008000u) || !(m2 <= FLT_MAX)) {
-                    // an inf or nan in this vector (left out of the sums), or a square or a sum beyond the
-                    // fp32 range: the vector again, element by element in fp64
+                if (!(m2 <= FLT_MAX)) {
+                    // the sum of squares is inf or nan: an inf or nan in this vector (to be left out of the
+                    // sums), or a square or a sum beyond the fp32 range: the vector again, element by element
+                    // in fp64
                     for (int i = 0; i < 4; ++i) {
                         moments_careful(w[i] & 0xFFFFu, s1, s2, bad);
                         moments_careful(w[i] >> 16, s1, s2, bad);
