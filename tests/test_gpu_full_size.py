@@ -1,0 +1,138 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration the benchmark times.
+What the oracle can do in seconds is compared element by element on sampled tensors / rows; the
+rest is checked through properties that hold at any size (histogram totals, counts, the generating
+parameters)."""
+import numpy as np
+import pytest
+import torch
+
+import gg_synth
+from oracle import gg_oracle as o
+from parity_util import ABS_ENTROPY, REL_FIT, REL_PENALTY, assert_grad_close, assert_rel
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2506_00486_b200 import Context
+    c = Context(0)
+    yield c
+    c.close()
+
+
+def check_segment(x_host, g_dev, out, s, lam, step, hist_row=None):
+    xo = gg_synth.to_oracle(x_host)
+    b, a, s1, s2, n, fl = o.fit(xo)
+    bg, ag = out["beta"][s].item(), out["alpha"][s].item()
+    assert (out["flags"][s].item() & 15) == fl and out["count"][s].item() == n
+    assert_rel(bg, b, REL_FIT, f"beta[{s}]")
+    assert_rel(ag, a, REL_FIT, f"alpha[{s}]")
+    pen, g = o.penalty_grad(xo, bg, ag, lam)
+    assert_grad_close(g_dev.float().cpu().numpy().reshape(-1), g)
+    assert_rel(out["penalty"][s].item(), pen, REL_PENALTY, f"penalty[{s}]")
+    if hist_row is not None:
+        ref, _ = o.quantise_hist(xo, step)
+        np.testing.assert_array_equal(hist_row.cpu().numpy(), ref.astype(np.int64))
+        return ref
+    return None
+
+
+def test_config5_llama7b_sweep_full_size(ctx):
+    """The whole 6.74e9-element sweep as bench.py runs it; three tensors (an attention matrix, an MLP
+    matrix, the output head) against the oracle in full, every tensor through its invariants."""
+    from paper_2506_00486_b200 import Segments
+    dev = torch.device("cuda", 0)
+    w = gg_synth.workload_c5_device(dev, torch.bfloat16, seed=4)
+    flat, offs, lens = w["flat"], w["offsets"], w["lens"]
+    n_seg = len(lens)
+    gflat = torch.empty(flat.numel(), dtype=torch.float32, device=dev)
+    steps = torch.full((n_seg,), 2.0 ** -10, dtype=torch.float32, device=dev)
+    run = ctx.make_fused(Segments.slices(flat, offs, lens), grad=Segments.slices(gflat, offs, lens), lam=1e-4, step=steps)
+    out = run()
+    out = run()             # a second call over the cached plan must give the same tables
+    torch.cuda.synchronize()
+    totals = out["hist"].sum(dim=1).cpu().numpy()
+    np.testing.assert_array_equal(totals, np.asarray(lens))
+    np.testing.assert_array_equal(out["count"].cpu().numpy(), np.asarray(lens))
+    beta = out["beta"].cpu().numpy()
+    assert np.abs(beta - np.asarray(w["beta_true"])).max() < 0.01          # the generating shapes, statistically
+    assert (out["flags"].cpu().numpy() == 0).all()
+    for s in (1, 5, n_seg - 1):
+        sl = slice(offs[s], offs[s] + lens[s])
+        ref = check_segment(flat[sl].cpu(), gflat[sl], out, s, 1e-4, 2.0 ** -10, out["hist"][s])
+        assert abs(out["entropy_bits"][s].item() - o.entropy_bits(ref)) <= ABS_ENTROPY
+    del flat, gflat, run, out
+    torch.cuda.empty_cache()
+
+
+def test_config3_activations_full_size(ctx):
+    """bf16 [8, 2048, 4096] with outliers, per-token segments, one shared histogram: the histogram in
+    full, 48 sampled rows element by element."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c3()
+    x = w["tensor"]
+    xd = x.to("cuda:0")
+    gd = torch.empty(x.shape, dtype=torch.float32, device="cuda:0")
+    steps = torch.full((w["n_seg"],), w["step"], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments.rows(xd), grad=Segments.rows(gd), lam=w["lam"], step=steps,
+                       hist_id=w["hist_id"], n_hist=1)
+    torch.cuda.synchronize()
+    ref, cl = o.quantise_hist(gg_synth.to_oracle(x), w["step"])
+    np.testing.assert_array_equal(out["hist"][0].cpu().numpy(), ref.astype(np.int64))
+    np.testing.assert_array_equal(out["clamped"][0].cpu().numpy(), cl.astype(np.int64))
+    assert abs(out["entropy_bits"][0].item() - o.entropy_bits(ref)) <= ABS_ENTROPY
+    rows = np.random.default_rng(0).choice(w["n_seg"], 48, replace=False)
+    for s in rows:
+        check_segment(x[s], gd[s], out, int(s), w["lam"], w["step"])
+    b = out["beta"].cpu().numpy()
+    assert np.isfinite(b).all() and (b > 0.3).all() and (b < 1.5).all()     # outliers pull the fitted shape below 0.8
+
+
+def test_config4_gradient_buckets_full_size(ctx):
+    """8 fp32 buckets of 25 M elements, step = alpha / 16 from each bucket's own fit: two buckets against
+    the oracle in full, all through their invariants."""
+    from paper_2506_00486_b200 import Segments
+    w = gg_synth.workload_c4()
+    xs = w["tensors"]
+    xd = [x.to("cuda:0") for x in xs]
+    gd = [torch.empty_like(x) for x in xd]
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=w["lam"], step_scale=1 / 16)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out["hist"].sum(dim=1).cpu().numpy(), [x.numel() for x in xs])
+    for s in range(len(xs)):
+        assert abs(out["beta"][s].item() - 0.5) < 0.01
+        assert out["step"][s].item() == np.float32(out["alpha"][s].item() / 16)
+    for s in (0, 5):
+        ref = check_segment(xs[s], gd[s], out, s, w["lam"], out["step"][s].item(), out["hist"][s])
+        H = o.entropy_bits(ref)
+        assert abs(out["entropy_bits"][s].item() - H) <= ABS_ENTROPY
+        # bits per element near the fine-step formula h(alpha, beta) - log2(step) (loose: beta = 0.5 is sharply peaked)
+        assert abs(H - (o.diff_entropy_nats(out["alpha"][s].item(), out["beta"][s].item()) / np.log(2)
+                        - np.log2(out["step"][s].item()))) < 0.5
+
+
+def test_config2_qwen_initialisation_full_size(ctx):
+    """gg_sample of the 169 Qwen-0.5B-shaped bf16 matrices (beta 1.3, std 0.02, seed 1), then gg_fit:
+    three matrices against the oracle's sampler in full, the recovered parameters of all of them."""
+    shapes = gg_synth.qwen05b_shapes()
+    beta, alpha = 1.3, gg_synth.alpha_for_std(0.02, 1.3)
+    outs = [torch.empty(r * c, dtype=torch.bfloat16, device="cuda:0") for _, r, c in shapes]
+    att = ctx.gg_sample(outs, [beta] * len(outs), [alpha] * len(outs), seed=1, tensor_id0=0)
+    fit = ctx.gg_fit(outs)
+    torch.cuda.synchronize()
+    assert att.max().item() <= 64
+    n = np.array([t.numel() for t in outs], dtype=np.float64)
+    assert (np.abs(fit["beta"].cpu().numpy() - beta) < 5 * 2.5 / np.sqrt(n) + 0.01).all()
+    assert (np.abs(fit["alpha"].cpu().numpy() / alpha - 1) < 5 * 2.5 / np.sqrt(n) + 0.01).all()
+    for s in (2, 5, 168):          # a key projection, a gate projection, the last down projection
+        ref = o.sample(beta, alpha, 1, s, outs[s].numel())
+        refb = o.round_to_bf16_bits(ref).astype(np.int64)
+        got = outs[s].cpu().view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+        diff = np.abs(refb - got)
+        assert diff.max() <= 1 and int((diff != 0).sum()) <= max(1, got.size // 100_000)
+        b, a, *_ = o.fit(gg_synth.to_oracle(outs[s].cpu()))
+        assert_rel(fit["beta"][s].item(), b, REL_FIT, "beta")
+        assert_rel(fit["alpha"][s].item(), a, REL_FIT, "alpha")
