@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <memory>
 #include <new>
 #include <string>
@@ -834,7 +835,6 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
 }  // extern "C"
 
 // ------------------------------------------------------------------ code lengths and the GCT step
-#include <algorithm>
 
 namespace {
 

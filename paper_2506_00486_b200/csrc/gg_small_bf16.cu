@@ -176,95 +176,92 @@ __device__ __forceinline__ void second_pass(const SmallArgs &a, int s, const uin
                                             int tail0, int n_scalar, double beta, const SegConst &k, const WarpTab &tab,
                                             Smem &sm)
 {
+    if constexpr (!GRAD && HIST == 0) return;     // a fit-only call has no second pass
     const int lane = threadIdx.x & 31;
     const uint4 *xv = reinterpret_cast<const uint4 *>(x + head);
-    if (GRAD || HIST != 0) {
-            double pen = 0.0;
-            uint32_t clampc[2] = {0u, 0u};
-            const bool accumulate = GRAD && a.accumulate != 0;
-            for (int i = lane; i < n_scalar; i += 32) {
-                const int idx = i < head ? i : tail0 + (i - head);
-                const uint32_t h = (uint32_t)__ldg(x + idx);
-                float mp = 0.0f;
-                float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
-                if constexpr (GRAD) {
-                    pen += (double)mp;
-                    if (gout != nullptr) {
-                        if (accumulate) g += load_grad<TG>(gout + idx);
-                        store_grad<TG>(gout + idx, g);
-                    }
-                }
+    double pen = 0.0;
+    uint32_t clampc[2] = {0u, 0u};
+    const bool accumulate = GRAD && a.accumulate != 0;
+    for (int i = lane; i < n_scalar; i += 32) {
+        const int idx = i < head ? i : tail0 + (i - head);
+        const uint32_t h = (uint32_t)__ldg(x + idx);
+        float mp = 0.0f;
+        float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
+        if constexpr (GRAD) {
+            pen += (double)mp;
+            if (gout != nullptr) {
+                if (accumulate) g += load_grad<TG>(gout + idx);
+                store_grad<TG>(gout + idx, g);
             }
-            // (loads run three vectors ahead of their use: the pass is bound by cache latency otherwise)
-            uint4 q0 = make_uint4(0u, 0u, 0u, 0u), q1 = q0, q2 = q0;
-            if (lane < nvec) q0 = __ldg(xv + lane);
-            if (lane + 32 < nvec) q1 = __ldg(xv + lane + 32);
-            if (lane + 64 < nvec) q2 = __ldg(xv + lane + 64);
-            for (int v = lane; v < nvec; v += 32) {
-                const uint4 raw = q0;
-                q0 = q1;
-                q1 = q2;
-                if (v + 96 < nvec) q2 = __ldg(xv + v + 96);
-                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-                float g[8];
-                float mp = 0.0f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-                    g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
-                }
-                if constexpr (GRAD) {
-                    pen += (double)mp;
-                    if (gout != nullptr) {
-                        TG *gp = gout + head + v * 8;
-                        if constexpr (sizeof(TG) == 4) {
-                            float4 *p4 = reinterpret_cast<float4 *>(gp);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                float4 o = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
-                                if (accumulate) {
-                                    const float4 old = p4[q];
-                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                                }
-                                __stcs(p4 + q, o);
-                            }
-                        } else {
-                            uint32_t o[4];
-                            const uint32_t *p1 = reinterpret_cast<const uint32_t *>(gp);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                float lo = g[2 * q], hi = g[2 * q + 1];
-                                if (accumulate) {
-                                    const uint32_t old = p1[q];
-                                    lo += __uint_as_float(old << 16);
-                                    hi += __uint_as_float(old & 0xFFFF0000u);
-                                }
-                                o[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
-                                       ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
-                            }
-                            __stcs(reinterpret_cast<uint4 *>(gp), make_uint4(o[0], o[1], o[2], o[3]));
-                        }
-                    }
-                }
-            }
-            if constexpr (GRAD) {
-                pen = warp_sum(pen);
-                if (lane == 0 && a.penalty) {
-                    // sum |x| |g| = |lambda| beta sum (|x|/alpha)^beta; the penalty carries lambda's sign
-                    a.penalty[s] = beta > 0.0 ? (k.sign_flip ? -pen : pen) / beta : 0.0;
-                }
-            }
-            if constexpr (HIST != 0) {
-                if (a.clamped != nullptr) {
-                    const uint32_t c0 = __reduce_add_sync(kFull, clampc[0]), c1 = __reduce_add_sync(kFull, clampc[1]);
-                    const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
-                    if (lane == 0 && c0) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid, (unsigned long long)c0);
-                    if (lane == 0 && c1) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + 1, (unsigned long long)c1);
-                }
-            }
-        } else if (GRAD && lane == 0 && a.penalty) {
-            a.penalty[s] = 0.0;
         }
+    }
+    // (loads run three vectors ahead of their use: the pass is bound by cache latency otherwise)
+    uint4 q0 = make_uint4(0u, 0u, 0u, 0u), q1 = q0, q2 = q0;
+    if (lane < nvec) q0 = __ldg(xv + lane);
+    if (lane + 32 < nvec) q1 = __ldg(xv + lane + 32);
+    if (lane + 64 < nvec) q2 = __ldg(xv + lane + 64);
+    for (int v = lane; v < nvec; v += 32) {
+        const uint4 raw = q0;
+        q0 = q1;
+        q1 = q2;
+        if (v + 96 < nvec) q2 = __ldg(xv + v + 96);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        float g[8];
+        float mp = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+            g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
+        }
+        if constexpr (GRAD) {
+            pen += (double)mp;
+            if (gout != nullptr) {
+                TG *gp = gout + head + v * 8;
+                if constexpr (sizeof(TG) == 4) {
+                    float4 *p4 = reinterpret_cast<float4 *>(gp);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        float4 o = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
+                        if (accumulate) {
+                            const float4 old = p4[q];
+                            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                        }
+                        __stcs(p4 + q, o);
+                    }
+                } else {
+                    uint32_t o[4];
+                    const uint32_t *p1 = reinterpret_cast<const uint32_t *>(gp);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float lo = g[2 * q], hi = g[2 * q + 1];
+                        if (accumulate) {
+                            const uint32_t old = p1[q];
+                            lo += __uint_as_float(old << 16);
+                            hi += __uint_as_float(old & 0xFFFF0000u);
+                        }
+                        o[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+                               ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+                    }
+                    __stcs(reinterpret_cast<uint4 *>(gp), make_uint4(o[0], o[1], o[2], o[3]));
+                }
+            }
+        }
+    }
+    if constexpr (GRAD) {
+        pen = warp_sum(pen);
+        if (lane == 0 && a.penalty) {
+            // sum |x| |g| = |lambda| beta sum (|x|/alpha)^beta; the penalty carries lambda's sign
+            a.penalty[s] = beta > 0.0 ? (k.sign_flip ? -pen : pen) / beta : 0.0;
+        }
+    }
+    if constexpr (HIST != 0) {
+        if (a.clamped != nullptr) {
+            const uint32_t c0 = __reduce_add_sync(kFull, clampc[0]), c1 = __reduce_add_sync(kFull, clampc[1]);
+            const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+            if (lane == 0 && c0) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid, (unsigned long long)c0);
+            if (lane == 0 && c1) atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + 2 * hid + 1, (unsigned long long)c1);
+        }
+    }
 }
 
 template <typename TG, bool GRAD, bool HIST>
