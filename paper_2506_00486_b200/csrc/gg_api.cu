@@ -233,6 +233,8 @@ cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype gra
 {
     if (in_dtype == GG_BF16 && (flags & (kGrad | kHist)) != 0)
         return launch_tail_bf16(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
+    if (in_dtype == GG_F32 && (flags & kMoments) == 0 && flags != 0)
+        return launch_tail_f32(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
     return launch_stream(flags, in_dtype, grad_dtype, has_grad_out, sa, cs);
 }
 

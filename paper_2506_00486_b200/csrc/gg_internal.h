@@ -108,6 +108,10 @@ cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_co
 // evenly spaced over [ln GG_BETA_LO, ln GG_BETA_HI].
 cudaError_t launch_fit_seed_table(double *table, cudaStream_t st);
 
+// fp32-input sweeps with a gradient and/or a histogram but no moments (flags in kGrad, kHist, kGrad | kHist):
+// persistent CTAs, table + series gradient, symbol counts in shared memory.
+cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a, int sm_count,
+                            cudaStream_t st);
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
 cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
                                     double *penalty, cudaStream_t st);
