@@ -101,7 +101,7 @@ struct SmallArgs {
     const double *seed;                // the fit table (launch_fit_seed_table)
     uint32_t *cta_counts;              // scratch, kSmallSlotWords words per CTA (small_grid CTAs); needed with do_hist
 };
-constexpr int kSmallSlotWords = 4104;  // a CTA's count cells and its histogram key
+constexpr int kSmallSlotWords = 8200;  // a CTA's count cells and its histogram key
 int small_grid(int32_t n_seg, int sm_count);   // CTAs launch_small_bf16 uses
 cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st);
 // Fills the fit table, 2 * (kSeedCells + 1) doubles: ln rho(beta_i) and then ln(alpha/sigma)(beta_i), ln beta_i

@@ -25,20 +25,23 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kCtasPerSm = 2;
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kCntBinades = 16;
+constexpr int kCntBinades = 32;
 constexpr uint32_t kCntPat = kCntBinades * 128;
-constexpr int kTabExp = 64;          // exponents covered by a warp's A table
-constexpr uint32_t kCells = (kCntPat + 1) * 2;   // count cells of a CTA: the window's patterns and the two "below" cells
+constexpr int kTabExp = 64;          // exponents around the segment's scale whose A is evaluated
+// count cells of a CTA: two per pattern of the window (sign), the sentinel pair that swallows the
+// first-pass counts of values outside the window, and the pair for values below the window
+constexpr uint32_t kSentinel = kCntPat * 2, kBelow = kCntPat * 2 + 2;
+constexpr uint32_t kCells = kCntPat * 2 + 4;
 static_assert(kCells + 4 <= (uint32_t)kSmallSlotWords, "scratch slot");
 constexpr int kMaxSlots = 1024;      // CTAs of one launch whose tables the flush kernel can take
 
 struct WarpTab {
-    float a1[kTabExp];   // A of exponent e_lo + i as one factor (with lambda's sign), NaN if not possible
+    float a1[256];       // A[e] as one factor (with lambda's sign); NaN where that is not possible or not evaluated
     float B[128];
 };
 
 struct Smem {
-    // cell p * 2 + sign: magnitude pattern c_base + p; the last two cells count the values below the
+    // cell p * 2 + sign: magnitude pattern c_base + p; then the sentinel pair; then the values below the
     // window (all of symbol 0, or -1 if negative) when the window starts at or below one step
     uint32_t cnt[kCells];
     WarpTab tab[kWarps];
@@ -50,6 +53,18 @@ struct Smem {
     int key_on;
     int below_ok;                      // values below the window quantise to 0 / -1
 };
+
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ void red_inc(uint32_t addr)
+{
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
+}
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -127,37 +142,68 @@ __device__ __noinline__ int count_global(uint32_t xb, float inv, int32_t qmin, i
     return clamped;
 }
 
-// One element (fp32 bits of a widened bf16): gradient value and penalty term, and the count.
-// HIST: 0 = no histogram, 1 = the CTA table serves the segment, 2 = it does not.
-template <bool GRAD, int HIST>
-__device__ __forceinline__ float small_elem(uint32_t xb, const SegConst &k, const WarpTab &tab, Smem &sm, float &mp,
-                                            double &pen, uint32_t (&clampc)[2])
+// One element of a 32-bit word w holding two bf16 values (HALF 0: low half, 1: high half).  Branch
+// free.  Gradient: a NaN entry of the warp's A table makes the vector's penalty partial NaN, which
+// the caller checks once per vector.  Count (HIST 1: the CTA table serves the segment): `anyc` keeps
+// the largest window index so that one compare per vector finds values outside the window; those
+// count in the sentinel cells.  HIST 2 (the table does not serve the segment) counts in global memory.
+template <bool GRAD, int HIST, int HALF>
+__device__ __forceinline__ float small_elem(uint32_t w, const SegConst &k, uint32_t a_addr, uint32_t b_addr, uint32_t cnt_addr,
+                                            float &mp, uint32_t &anyc, uint32_t (&clampc)[2])
 {
-    const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
+    const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);
     float g = 0.0f;
     if constexpr (GRAD) {
-        const uint32_t ei = (mag >> 7) - (uint32_t)k.e_lo;
-        float ga = ei < (uint32_t)kTabExp ? tab.a1[ei] * tab.B[mag & 127u] : __int_as_float(0x7FC00000);
-        if (ga != ga) {
-            const double gd = grad_fp64(mag, k.L, k.b, k.active);      // |g| before rounding to fp32
-            pen += (double)__uint_as_float(mag << 16) * gd;
-            ga = __uint_as_float(__float_as_uint((float)gd) ^ k.sign_flip);
-        } else {
-            mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);     // (table products are normal fp32 numbers)
-        }
+        const uint32_t e4 = HALF ? ((w >> 21) & 0x3FCu) : ((w >> 5) & 0x3FCu);     // exponent field * 4
+        const uint32_t j4 = HALF ? ((w >> 14) & 0x1FCu) : ((w << 2) & 0x1FCu);     // mantissa bits * 4
+        const float ga = lds_f32(a_addr + e4) * lds_f32(b_addr + j4);
+        mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);
         g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
     }
     if constexpr (HIST == 1) {
-        const uint32_t p = mag - k.c_base;
-        if (p < kCntPat) atomicAdd(&sm.cnt[p * 2u + (xb >> 31)], 1u);
-        else if (k.below_ok && mag < k.c_base) atomicAdd(&sm.cnt[kCntPat * 2u + (mag != 0u ? (xb >> 31) : 0u)], 1u);
-        else {
-            const int c = count_global(xb, k.inv, k.qmin, k.qmax, k.row);
-            if (c) clampc[c - 1] += 1u;
-        }
+        const uint32_t mag = HALF ? ((w >> 16) & 0x7FFFu) : (w & 0x7FFFu);
+        uint32_t p = mag - k.c_base;
+        anyc = max(anyc, p);
+        p = min(p, kCntPat);
+        const uint32_t sign4 = HALF ? ((w >> 29) & 4u) : ((w >> 13) & 4u);
+        red_inc(cnt_addr + p * 8u + sign4);
     } else if constexpr (HIST == 2) {
         const int c = count_global(xb, k.inv, k.qmin, k.qmax, k.row);
         if (c) clampc[c - 1] += 1u;
+    }
+    return g;
+}
+
+// Redo of whatever part of an element (fp32 bits) the branch-free path could not do; g is its
+// gradient from the first pass.  grad_bad: the vector's penalty partial is not a finite number, so
+// the whole vector's penalty terms are added here instead, in fp64.
+template <bool GRAD, int HIST>
+__device__ __forceinline__ float small_fix(uint32_t xb, float g, bool grad_bad, const SegConst &k, const WarpTab &tab, Smem &sm,
+                                           double &pen, uint32_t (&clampc)[2])
+{
+    const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
+    if constexpr (GRAD) {
+        if (grad_bad) {
+            const float a = tab.a1[mag >> 7];
+            const double ax = (double)__uint_as_float(mag << 16);
+            if (a != a) {     // this element read a NaN marker: the fp64 evaluation
+                const double gd = grad_fp64(mag, k.L, k.b, k.active);
+                pen += ax * gd;
+                g = __uint_as_float(__float_as_uint((float)gd) ^ k.sign_flip ^ (xb & 0x80000000u));
+            } else {
+                pen += ax * (double)fabsf(g);
+            }
+        }
+    }
+    if constexpr (HIST == 1) {
+        if (mag - k.c_base >= kCntPat) {
+            if (k.below_ok && mag < k.c_base) {
+                atomicAdd(&sm.cnt[kBelow + (mag != 0u ? (xb >> 31) : 0u)], 1u);
+            } else {
+                const int c = count_global(xb, k.inv, k.qmin, k.qmax, k.row);
+                if (c) clampc[c - 1] += 1u;
+            }
+        }
     }
     return g;
 }
@@ -182,13 +228,19 @@ __device__ __forceinline__ void second_pass(const SmallArgs &a, int s, const uin
     double pen = 0.0;
     uint32_t clampc[2] = {0u, 0u};
     const bool accumulate = GRAD && a.accumulate != 0;
+    // 32-bit shared addresses of the warp's tables and of the CTA's count cells
+    const uint32_t a_addr = (uint32_t)__cvta_generic_to_shared(tab.a1), b_addr = (uint32_t)__cvta_generic_to_shared(tab.B);
+    const uint32_t cnt_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt);
     for (int i = lane; i < n_scalar; i += 32) {
         const int idx = i < head ? i : tail0 + (i - head);
         const uint32_t h = (uint32_t)__ldg(x + idx);
         float mp = 0.0f;
-        float g = small_elem<GRAD, HIST>(h << 16, k, tab, sm, mp, pen, clampc);
+        uint32_t anyc = 0;
+        float g = small_elem<GRAD, HIST, 0>(h, k, a_addr, b_addr, cnt_addr, mp, anyc, clampc);
+        const bool grad_bad = GRAD && !(mp <= FLT_MAX);
+        if (grad_bad || (HIST == 1 && anyc >= kCntPat)) g = small_fix<GRAD, HIST>(h << 16, g, grad_bad, k, tab, sm, pen, clampc);
         if constexpr (GRAD) {
-            pen += (double)mp;
+            if (!grad_bad) pen += (double)mp;
             if (gout != nullptr) {
                 if (accumulate) g += load_grad<TG>(gout + idx);
                 store_grad<TG>(gout + idx, g);
@@ -208,13 +260,24 @@ __device__ __forceinline__ void second_pass(const SmallArgs &a, int s, const uin
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
         float g[8];
         float mp = 0.0f;
+        uint32_t anyc = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-            g[i] = small_elem<GRAD, HIST>(xb, k, tab, sm, mp, pen, clampc);
+        for (int i = 0; i < 4; ++i) {
+            g[2 * i] = small_elem<GRAD, HIST, 0>(w[i], k, a_addr, b_addr, cnt_addr, mp, anyc, clampc);
+            g[2 * i + 1] = small_elem<GRAD, HIST, 1>(w[i], k, a_addr, b_addr, cnt_addr, mp, anyc, clampc);
+        }
+        // (table products are normal numbers whose terms |x| |g| stay far inside the fp32 range, so a
+        // partial that is not finite means a NaN marker was read)
+        const bool grad_bad = GRAD && !(mp <= FLT_MAX);
+        if (grad_bad || (HIST == 1 && anyc >= kCntPat)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
+                g[i] = small_fix<GRAD, HIST>(xb, g[i], grad_bad, k, tab, sm, pen, clampc);
+            }
         }
         if constexpr (GRAD) {
-            pen += (double)mp;
+            if (!grad_bad) pen += (double)mp;
             if (gout != nullptr) {
                 TG *gp = gout + head + v * 8;
                 if constexpr (sizeof(TG) == 4) {
@@ -432,18 +495,18 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
             if (k.active) e_c = ilogb(sqrt(s2 / (double)len)) + 127;
             k.e_lo = max(1, min(254 - (kTabExp - 1), e_c - 40));
             __syncwarp();       // the previous segment's second pass is done with the tables
-#pragma unroll
-            for (int i = lane; i < kTabExp; i += 32) {
-                float v = 0.0f;
-                if (k.active) {
+            // A for the kTabExp exponents from 40 binades below the standard deviation's upwards, NaN for
+            // the rest (zero/subnormal, inf/nan and far binades go to the fp64 evaluation)
+            for (int e = lane; e < 256; e += 32) {
+                float v = k.active ? __int_as_float(0x7FC00000) : 0.0f;
+                if (k.active && (uint32_t)(e - k.e_lo) < (uint32_t)kTabExp) {
                     // one fp32 factor serves if |L + b (e-127)| <= 100: its product with B stays a normal
                     // number; the same bound on L + beta (e-127) keeps the penalty terms |x| |g| normal too
-                    const double de = (double)(k.e_lo + i - 127);
+                    const double de = (double)(e - 127);
                     const double e0 = k.L + k.b * de;
-                    const bool ok = fabs(e0) <= 100.0 && fabs(e0 + de) <= 100.0;
-                    v = ok ? (float)(lam < 0.0 ? -exp2(e0) : exp2(e0)) : __int_as_float(0x7FC00000);
+                    if (fabs(e0) <= 100.0 && fabs(e0 + de) <= 100.0) v = (float)(lam < 0.0 ? -exp2(e0) : exp2(e0));
                 }
-                tab.a1[i] = v;
+                tab.a1[e] = v;
             }
 #pragma unroll
             for (int j = lane; j < 128; j += 32) tab.B[j] = k.active ? (float)exp2(k.b * sm.log2m[j]) : 1.0f;
@@ -498,25 +561,29 @@ __global__ void small_flush_kernel(const uint32_t *__restrict__ cta_counts, int 
     // the slots' keys first, into shared memory: scanning them from global memory would be one
     // dependent cache miss per slot
     __shared__ uint32_t sh_key[kMaxSlots][4];
-    for (int b = threadIdx.x; b < n_slots; b += blockDim.x) {
+    for (int b = threadIdx.y * blockDim.x + threadIdx.x; b < n_slots; b += blockDim.x * blockDim.y) {
         const uint32_t *key = cta_counts + (size_t)b * kSmallSlotWords + kCells;
 #pragma unroll
         for (int q = 0; q < 4; ++q) sh_key[b][q] = __ldg(key + q);
     }
     __syncthreads();
+    // thread (x, y): cell blockIdx.x * blockDim.x + x, the y-th of blockDim.y contiguous parts of the slots
+    // (additions commute, so every part may emit its own runs)
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= kCells) return;
+    if (c >= kCells || c == kSentinel || c == kSentinel + 1) return;     // (the sentinel pair is not counted)
+    const int per_part = (n_slots + (int)blockDim.y - 1) / (int)blockDim.y;
+    const int b_first = (int)threadIdx.y * per_part, b_last = min(n_slots, b_first + per_part);
     const int64_t n_bins = (int64_t)qmax - (int64_t)qmin + 1;
     unsigned long long run = 0;
     uint32_t k_hid = 0, k_inv = 0, k_base = 0;
     auto emit = [&]() {
         if (run == 0) return;
         int q;
-        if (c < kCntPat * 2) {
+        if (c < kSentinel) {
             const uint32_t h = (k_base + (c >> 1)) | ((c & 1u) << 15);
             q = __float2int_rd(__fmul_rn(__uint_as_float(h << 16), __uint_as_float(k_inv)));   // (window patterns are finite)
         } else {
-            q = c == kCntPat * 2 ? 0 : -1;      // the values below the window
+            q = c == kBelow ? 0 : -1;           // the values below the window
         }
         unsigned long long *cl = reinterpret_cast<unsigned long long *>(clamped);
         if (q < qmin) { q = qmin; if (cl) atomicAdd(cl + 2 * k_hid, run); }
@@ -526,12 +593,12 @@ __global__ void small_flush_kernel(const uint32_t *__restrict__ cta_counts, int 
     };
     // (the keys are the same words for every thread: cached; the sums over a run are independent
     // loads, unrolled so that many are in flight)
-    int b = 0;
-    while (b < n_slots) {
+    int b = b_first;
+    while (b < b_last) {
         if (sh_key[b][0] == 0u) { ++b; continue; }                        // this CTA had no table (its cells are zeros)
         k_hid = sh_key[b][1]; k_inv = sh_key[b][2]; k_base = sh_key[b][3];
         int e = b + 1;
-        for (; e < n_slots; ++e) {
+        for (; e < b_last; ++e) {
             if (sh_key[e][0] != 0u && (sh_key[e][1] != k_hid || sh_key[e][2] != k_inv || sh_key[e][3] != k_base)) break;
         }
         int i = b;
@@ -561,7 +628,7 @@ cudaError_t launch_typed(const SmallArgs &a, int sm_count, cudaStream_t st)
     if (!a.do_hist) return a.do_grad ? go(small_bf16_kernel<TG, true, false>) : go(small_bf16_kernel<TG, false, false>);
     cudaError_t e = a.do_grad ? go(small_bf16_kernel<TG, true, true>) : go(small_bf16_kernel<TG, false, true>);
     if (e != cudaSuccess) return e;
-    small_flush_kernel<<<(kCells + 255) / 256, 256, 0, st>>>(a.cta_counts, grid, a.qmin, a.qmax, a.hist, a.clamped);
+    small_flush_kernel<<<(kCells + 31) / 32, dim3(32, 8), 0, st>>>(a.cta_counts, grid, a.qmin, a.qmax, a.hist, a.clamped);
     return cudaGetLastError();
 }
 
