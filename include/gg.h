@@ -273,6 +273,49 @@ gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double
  * all results are in host memory.  Pinned host buffers make the copies asynchronous. */
 gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *args, int64_t chunk_bytes);
 
+/* ---- channel-wise (strided) segments ------------------------------------------------------------ */
+
+/* Arguments of the fused pass over the COLUMNS of a row-major matrix: segment c is the column
+ * x[0 * ld + c], x[1 * ld + c], ..., x[(rows-1) * ld + c] (one GG per channel of an activation or
+ * input channel of a weight matrix; rows of a matrix are contiguous segments and go through
+ * gg_fused).  The paper fits one GG per tensor; per-channel fits are this library's generalisation
+ * of the same pass and every formula is that of gg_fit, gg_penalty_grad and gg_rate_hist.
+ * All columns are quantised with one step into ONE histogram (the rate of the whole tensor). */
+typedef struct {
+    const void *x;               /* device, bf16, element (r, c) at x[r * ld + c]             */
+    int64_t     rows, cols, ld;  /* ld >= cols, in elements                                   */
+    int32_t     in_dtype;        /* GG_BF16 (GG_F32 is refused with GG_ERR_DTYPE)             */
+    /* fit outputs, device [cols]; beta and alpha are required                                */
+    double   *beta, *alpha, *sum_abs, *sum_sq;
+    int64_t  *count;
+    uint32_t *flags;
+    /* penalty and gradient with the fitted parameters of each column                         */
+    double    lambda;
+    int32_t   reduction;         /* GG_SUM or GG_MEAN (lambda / rows)                         */
+    void     *grad;              /* device matrix of grad_dtype, element (r, c) at            */
+    int64_t   grad_ld;           /*   grad[r * grad_ld + c]; NULL: no gradient                */
+    int32_t   grad_dtype;
+    int32_t   accumulate_grad;
+    double   *penalty;           /* device [cols] or NULL                                     */
+    /* quantiser, histogram, entropy                                                          */
+    float     step;              /* one step for the matrix                                   */
+    int32_t   qmin, qmax;
+    uint64_t *hist;              /* device [qmax-qmin+1]; NULL skips the histogram step       */
+    int32_t   accumulate_hist;
+    double   *entropy_bits;      /* device [1] or NULL                                        */
+    uint64_t *clamped_lo_hi;     /* device [2] or NULL                                        */
+} gg_channel_args;
+
+/* moments -> fit -> penalty + gradient + histogram -> entropy for every column of the matrix, all
+ * enqueued on `stream`: the matrix is read twice (row-major, coalesced: a strip of 64 columns is
+ * 128 contiguous bytes of every row), the second time from L2 when it fits there.  Results per
+ * column equal those of gg_fused on the gathered column within the same tolerances; sums over a
+ * column are reduced in a fixed order.  GG_FLAG_CLAMPED_SYMBOLS is set per column when a histogram
+ * is taken.  The first call with a larger matrix than any before allocates scratch (blocking).
+ * Errors: GG_ERR_DTYPE for fp32 input, GG_ERR_INVALID_ARG for ld < cols, negative sizes, a missing
+ * required pointer or qmin > qmax, GG_ERR_ALIGNMENT for x or grad not element aligned. */
+gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *args, void *stream);
+
 /* Moments and fit of ONE segment without allocating anything (the paper has no counterpart: this is
  * gg_fit for callers that cannot allocate).  gg_fit keeps its tile tables and per-tile partial sums in
  * a plan that the context obtains with cudaMalloc the first time it sees a layout.  Callers that run

@@ -39,6 +39,20 @@ class FusedArgs(ctypes.Structure):
     ]
 
 
+class ChannelArgs(ctypes.Structure):
+    """Mirror of gg_channel_args."""
+    _fields_ = [
+        ("x", _P), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("ld", ctypes.c_int64),
+        ("in_dtype", ctypes.c_int32),
+        ("beta", _P), ("alpha", _P), ("sum_abs", _P), ("sum_sq", _P), ("count", _P), ("flags", _P),
+        ("lam", ctypes.c_double), ("reduction", ctypes.c_int32),
+        ("grad", _P), ("grad_ld", ctypes.c_int64), ("grad_dtype", ctypes.c_int32),
+        ("accumulate_grad", ctypes.c_int32), ("penalty", _P),
+        ("step", ctypes.c_float), ("qmin", ctypes.c_int32), ("qmax", ctypes.c_int32),
+        ("hist", _P), ("accumulate_hist", ctypes.c_int32), ("entropy_bits", _P), ("clamped_lo_hi", _P),
+    ]
+
+
 class GGError(RuntimeError):
     def __init__(self, status, text):
         super().__init__(f"gg status {status}: {text}")
@@ -79,6 +93,8 @@ def lib():
         L.gg_sample.argtypes = [_P, _P, i32, ctypes.c_int, _P, _P, u64, u32, _P, _P]
         L.gg_fused.argtypes = [_P, ctypes.POINTER(FusedArgs), _P]
         L.gg_fused_host.argtypes = [_P, ctypes.POINTER(FusedArgs), i64]
+        L.gg_fused_channels.argtypes = [_P, ctypes.POINTER(ChannelArgs), _P]
+        L.gg_fused_channels.restype = ctypes.c_int
         L.gg_timing_enable.argtypes = [_P, ctypes.c_int]
         L.gg_timing_read.argtypes = [_P, ctypes.POINTER(d), ctypes.POINTER(i64), ctypes.POINTER(d),
                                      ctypes.POINTER(i64)]
@@ -385,6 +401,55 @@ class Context:
     def gg_fused(self, segs, **kw):
         """One-shot form of make_fused(...)()."""
         return self.make_fused(segs, **kw)()
+
+    # ------------------------------------------------------- gg_fused_channels
+    def make_fused_channels(self, x, grad=None, lam=1e-4, reduction=GG_SUM, accumulate_grad=False,
+                            want_penalty=True, step=None, qmin=-32768, qmax=32767, accumulate_hist=False,
+                            hist=None):
+        """The fused pass over the COLUMNS of the 2-D tensor x (rows may be strided: x.stride(1) == 1).
+
+        Allocates the per-column outputs once and returns a callable that enqueues the pass.
+        step: float, one quantiser step for the matrix; None skips the histogram."""
+        if x.dim() != 2 or (x.shape[1] > 1 and x.stride(1) != 1):
+            raise ValueError("x must be 2-D with contiguous rows")
+        rows, cols = x.shape
+        out = dict(beta=self._new(cols, torch.float64), alpha=self._new(cols, torch.float64),
+                   sum_abs=self._new(cols, torch.float64), sum_sq=self._new(cols, torch.float64),
+                   count=self._new(cols, torch.int64), flags=self._new(cols, torch.int32))
+        out["penalty"] = self._new(cols, torch.float64) if want_penalty else None
+        a = ChannelArgs()
+        a.x, a.rows, a.cols, a.ld, a.in_dtype = _ptr(x), rows, cols, (x.stride(0) if rows > 1 else cols), _dtype_code(x.dtype)
+        for k in ("beta", "alpha", "sum_abs", "sum_sq", "count", "flags", "penalty"):
+            setattr(a, k, _ptr(out[k]))
+        a.lam, a.reduction = float(lam), int(reduction)
+        if grad is not None:
+            if grad.shape != x.shape or (cols > 1 and grad.stride(1) != 1):
+                raise ValueError("grad must have the shape of x and contiguous rows")
+            a.grad, a.grad_ld, a.grad_dtype = _ptr(grad), (grad.stride(0) if rows > 1 else cols), _dtype_code(grad.dtype)
+        a.accumulate_grad = int(bool(accumulate_grad))
+        if step is not None:
+            nb = qmax - qmin + 1
+            if hist is None:
+                hist = torch.zeros(nb, dtype=torch.int64, device=self.device)
+            out["hist"] = hist
+            out["entropy_bits"] = self._new(1, torch.float64)
+            out["clamped"] = torch.zeros(2, dtype=torch.int64, device=self.device)
+            a.step, a.qmin, a.qmax = float(step), int(qmin), int(qmax)
+            a.hist, a.accumulate_hist = _ptr(hist), int(bool(accumulate_hist))
+            a.entropy_bits, a.clamped_lo_hi = _ptr(out["entropy_bits"]), _ptr(out["clamped"])
+
+        def run():
+            self._check(lib().gg_fused_channels(self._h, ctypes.byref(a), _stream_ptr(self.device)))
+            return out
+
+        run.outputs = out
+        run.args = a
+        run._keep = [x, grad, hist]
+        return run
+
+    def gg_fused_channels(self, x, **kw):
+        """One-shot form of make_fused_channels(...)()."""
+        return self.make_fused_channels(x, **kw)()
 
     # ----------------------------------------------------------- gg_fused_host
     def make_fused_host(self, segs, grad=None, lam=1e-4, reduction=GG_SUM, step=None, step_scale=None,

@@ -1,5 +1,6 @@
 // Host side of the library: contexts, cached plans (tile maps + scratch), argument checks and
 // the C entry points declared in gg.h.  No kernel lives here.
+#include <float.h>
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
@@ -44,6 +45,8 @@ struct gg_ctx {
     double *ent_part = nullptr;   // scratch of the entropy kernels: 2 * kEntSplit doubles per histogram
     int64_t ent_hists = 0;
     uint32_t *small_counts = nullptr;   // scratch of the short-segment kernel: one slot of count cells per CTA
+    void *chan_buf = nullptr;     // scratch of gg_fused_channels (partials per row block and column)
+    int64_t chan_bytes = 0;
     double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
@@ -361,6 +364,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     if (ctx->host_dev) cudaFree(ctx->host_dev);
     if (ctx->seed) cudaFree(ctx->seed);
     if (ctx->small_counts) cudaFree(ctx->small_counts);
+    if (ctx->chan_buf) cudaFree(ctx->chan_buf);
     if (ctx->ent_part) cudaFree(ctx->ent_part);
     delete ctx;
     return GG_OK;
@@ -644,6 +648,86 @@ static gg_status grow(gg_ctx *ctx, void **buf, int64_t *have, int64_t need)
     if (*buf) { GG_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(*buf); *buf = nullptr; *have = 0; }
     GG_CUDA(ctx, cudaMalloc(buf, (size_t)need));
     *have = need;
+    return GG_OK;
+}
+
+gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
+{
+    if (!ctx || !a) return GG_ERR_INVALID_ARG;
+    if (a->in_dtype != GG_BF16) return GG_ERR_DTYPE;
+    if (a->rows < 0 || a->cols < 0 || a->ld < a->cols) return GG_ERR_INVALID_ARG;
+    if (a->cols > 0 && (!a->beta || !a->alpha)) return GG_ERR_INVALID_ARG;
+    if (a->rows > 0 && a->cols > 0 && !a->x) return GG_ERR_INVALID_ARG;
+    if (a->reduction != GG_SUM && a->reduction != GG_MEAN) return GG_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(a->x) % 2 != 0) return GG_ERR_ALIGNMENT;
+    if (a->grad) {
+        if (!dtype_ok(a->grad_dtype)) return GG_ERR_DTYPE;
+        if (a->grad_ld < a->cols) return GG_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(a->grad) % esize(a->grad_dtype) != 0) return GG_ERR_ALIGNMENT;
+    }
+    const bool do_hist = a->hist != nullptr;
+    if (do_hist) {
+        if (a->qmax < a->qmin || (int64_t)a->qmax - (int64_t)a->qmin + 1 > (1ll << 24)) return GG_ERR_INVALID_ARG;
+        if (!(a->step > 0.0f) || !(a->step <= FLT_MAX)) return GG_ERR_INVALID_ARG;
+    }
+    const int64_t n_mom = (a->rows + kChanMomRows - 1) / kChanMomRows;
+    if (n_mom > 65535 || a->cols > (1ll << 31) - kChanStrip) return GG_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return GG_ERR_CUDA;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const int32_t n_bins = do_hist ? a->qmax - a->qmin + 1 : 0;
+    if (do_hist && !a->accumulate_hist) {
+        GG_CUDA(ctx, cudaMemsetAsync(a->hist, 0, sizeof(uint64_t) * (size_t)n_bins, cs));
+        if (a->clamped_lo_hi) GG_CUDA(ctx, cudaMemsetAsync(a->clamped_lo_hi, 0, sizeof(uint64_t) * 2, cs));
+    }
+    if (a->cols > 0) {
+        const bool want_pg = a->grad != nullptr || a->penalty != nullptr;
+        ChanArgs ka{};
+        ka.x = static_cast<const uint16_t *>(a->x);
+        ka.rows = a->rows; ka.cols = a->cols; ka.ld = a->ld;
+        ka.grad = a->grad; ka.grad_ld = a->grad_ld; ka.accumulate = a->accumulate_grad;
+        ka.n_mom_blocks = (int32_t)n_mom;
+        ka.n_slices = chan_slices(a->rows, a->cols, ctx->sm_count);
+        // scratch: doubles first, then the 32-bit arrays
+        const size_t nc = (size_t)a->cols, nm = (size_t)n_mom * nc, ns = (size_t)ka.n_slices * nc;
+        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + nc;
+        void *buf = ctx->chan_buf;
+        gg_status st = grow(ctx, &buf, &ctx->chan_bytes, (int64_t)(n_dbl * 8 + n_w32 * 4));
+        ctx->chan_buf = buf;
+        if (st != GG_OK) return st;
+        double *d = static_cast<double *>(ctx->chan_buf);
+        ka.s1 = d; ka.s2 = d + nm; ka.L = d + 2 * nm; ka.b = ka.L + nc; ka.pen = ka.b + nc;
+        uint32_t *w = reinterpret_cast<uint32_t *>(d + n_dbl);
+        ka.bad = w;
+        ka.xmin = reinterpret_cast<float *>(w + nm);
+        ka.xmax = reinterpret_cast<float *>(w + 2 * nm);
+        ka.amax = reinterpret_cast<float *>(w + 3 * nm);
+        ka.beta = a->beta; ka.alpha = a->alpha; ka.sum_abs = a->sum_abs; ka.sum_sq = a->sum_sq;
+        ka.count = a->count; ka.flags = a->flags; ka.penalty = a->penalty;
+        ka.seed = ctx->seed;
+        ka.lambda = a->reduction == GG_MEAN && a->rows > 0 ? a->lambda / (double)a->rows : a->lambda;
+        ka.do_grad = want_pg; ka.do_hist = do_hist;
+        ka.step = a->step; ka.qmin = a->qmin; ka.qmax = a->qmax; ka.hist = a->hist; ka.clamped = a->clamped_lo_hi;
+        {
+            SweepTimer tm(ctx, &ctx->ev_first, cs);
+            GG_CUDA(ctx, launch_chan_moments(ka, cs));
+        }
+        GG_CUDA(ctx, launch_chan_fit(ka, cs));
+        ctx->launches += 1 + (a->rows > 0);
+        if ((want_pg || do_hist) && a->rows > 0) {
+            SweepTimer tm(ctx, &ctx->ev_tail, cs);
+            GG_CUDA(ctx, launch_chan_tail((gg_dtype)a->grad_dtype, ka, ctx->sm_count, cs));
+            ctx->launches += 1;
+        }
+        if (a->penalty) {
+            if (a->rows <= 0) GG_CUDA(ctx, cudaMemsetAsync(a->penalty, 0, sizeof(double) * nc, cs));
+            else { GG_CUDA(ctx, launch_chan_penalty(ka, cs)); ctx->launches += 1; }
+        }
+    }
+    if (do_hist && a->entropy_bits) {
+        gg_status es = run_entropy(ctx, a->hist, 1, n_bins, a->entropy_bits, cs);
+        if (es != GG_OK) return es;
+    }
     return GG_OK;
 }
 

@@ -56,4 +56,31 @@ __device__ __forceinline__ double invert_ratio_table(double log_r, const double 
     return exp(u0 + h * ((double)(j + 1) + t));
 }
 
+// The fit of one segment from its sums: beta from the moment ratio, alpha from Eq. 2 with
+// sigma^2 = sum_sq / len.  Returns the GG_FLAG_* bits of the fit (degenerate, clamped).
+__device__ __forceinline__ uint32_t fit_from_sums(double s1, double s2, int64_t len, const double *table, double *beta,
+                                                  double *alpha)
+{
+    *beta = 0.0;
+    *alpha = 0.0;
+    if (len <= 0 || !(s2 > 0.0)) return GG_FLAG_DEGENERATE;
+    const double m1 = s1 / (double)len, m2 = s2 / (double)len;
+    const double log_r = log(m1 * m1 / m2);
+    uint32_t flags = 0u;
+    double lnz;
+    if (log_r <= __ldg(table)) {
+        *beta = GG_BETA_LO;
+        lnz = __ldg(table + kSeedCells + 1);
+        flags = GG_FLAG_BETA_CLAMPED_LO;
+    } else if (log_r >= __ldg(table + kSeedCells)) {
+        *beta = GG_BETA_HI;
+        lnz = __ldg(table + 2 * kSeedCells + 1);
+        flags = GG_FLAG_BETA_CLAMPED_HI;
+    } else {
+        *beta = invert_ratio_table(log_r, table, &lnz);
+    }
+    *alpha = sqrt(m2) * exp(lnz);
+    return flags;
+}
+
 }  // namespace gg

@@ -17,6 +17,15 @@ constexpr int kWindow = 4096;
 
 enum StreamFlags : int { kMoments = 1, kGrad = 2, kHist = 4 };
 
+// Moments are summed in fp32 over a short run of elements and then added in fp64.  The fp32 sums m1 = sum |x|
+// and m2 = sum x^2 of a run can stand for the exact ones unless a square left the fp32 range: upwards
+// (m2 is inf or nan; an inf or nan entry ends here too) or downwards, into the subnormals (then m2 is tiny;
+// a run of zeros is the harmless case of that).  Runs that fail the test are summed again in fp64.
+__device__ __forceinline__ bool run_sums_exact_enough(float m1, float m2)
+{
+    return m2 <= 3.402823466e+38f && (m2 >= 1e-30f || m1 == 0.0f);
+}
+
 // Device-side view of a plan: where each tile lives.
 struct TileMap {
     const void *const *seg_ptr;   // [n_seg] input segments
@@ -112,6 +121,41 @@ cudaError_t launch_fit_seed_table(double *table, cudaStream_t st);
 // persistent CTAs, table + series gradient, symbol counts in shared memory.
 cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a, int sm_count,
                             cudaStream_t st);
+// Column segments of a row-major bf16 matrix (gg_fused_channels).  Scratch arrays are indexed
+// [row block][column]; the moments kernel and the second kernel cut the rows differently.
+constexpr int kChanStrip = 64;        // columns per strip: 128 contiguous bytes of a row
+constexpr int kChanMomRows = 256;     // rows per CTA of the moments kernel
+struct ChanArgs {
+    const uint16_t *x;
+    int64_t rows, cols, ld;
+    void *grad;                        // may be null
+    int64_t grad_ld;
+    int accumulate;
+    int32_t n_mom_blocks;              // ceil(rows / kChanMomRows)
+    int32_t n_slices;                  // row slices per strip in the second kernel
+    double *s1, *s2;                   // [n_mom_blocks * cols] partial sums
+    uint32_t *bad;
+    float *xmin, *xmax;
+    double *L, *b;                     // [cols]: |g| = 2^(L + b log2|x|); L is NaN for a column without gradient
+    float *amax;                       // [cols] largest finite magnitude
+    double *pen;                       // [n_slices * cols] partial sums of |x| |g|
+    double *beta, *alpha, *sum_abs, *sum_sq;
+    int64_t *count;
+    uint32_t *flags;
+    double *penalty;                   // may be null
+    const double *seed;                // the fit table
+    double lambda;                     // already divided by rows for GG_MEAN
+    int do_grad, do_hist;
+    float step;
+    int32_t qmin, qmax;
+    uint64_t *hist;
+    uint64_t *clamped;                 // [2] or null
+};
+cudaError_t launch_chan_moments(const ChanArgs &a, cudaStream_t st);
+cudaError_t launch_chan_fit(const ChanArgs &a, cudaStream_t st);
+int chan_slices(int64_t rows, int64_t cols, int sm_count);      // n_slices the second kernel should use
+cudaError_t launch_chan_tail(gg_dtype grad_dtype, const ChanArgs &a, int sm_count, cudaStream_t st);
+cudaError_t launch_chan_penalty(const ChanArgs &a, cudaStream_t st);
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
 cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
                                     double *penalty, cudaStream_t st);

@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                 xmin = fminf(xmin, __uint_as_float(xb));
                 xmax = fmaxf(xmax, __uint_as_float(xb));
             }
-            if (m2 <= FLT_MAX) {
+            if (run_sums_exact_enough(m1, m2)) {
                 s1 += (double)m1;
                 s2 += (double)m2;
             } else {     // a square or a sum left the fp32 range: this vector again in fp64

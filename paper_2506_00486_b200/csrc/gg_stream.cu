@@ -206,10 +206,10 @@ __device__ __forceinline__ void process(const float (&x)[KV], float (&g)[KV], Ac
     }
     // short fp32 runs, then fp64: the fp32 part adds at most KV roundings of 2^-24 each
     if constexpr (FLAGS & kMoments) {
-        if (m2 <= FLT_MAX) {
+        if (run_sums_exact_enough(m1, m2)) {
             acc.s1 += (double)m1;
             acc.s2 += (double)m2;
-        } else {     // a square or a sum beyond the fp32 range: this run again in fp64
+        } else {     // a square or a sum outside the fp32 range: this run again in fp64
             for (int e = 0; e < KV; ++e) {
                 const double ax = (double)fabsf(x[e]);
                 if (ax <= (double)FLT_MAX) { acc.s1 += ax; acc.s2 += ax * ax; }
@@ -475,10 +475,9 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
                     mn2 = __hmin2(mn2, p);      // return the non-NaN operand, like fminf
                     mx2 = __hmax2(mx2, p);
                 }
-                if (!(m2 <= FLT_MAX)) {
-                    // the sum of squares is inf or nan: an inf or nan in this vector (to be left out of the
-                    // sums), or a square or a sum beyond the fp32 range: the vector again, element by element
-                    // in fp64
+                if (!run_sums_exact_enough(m1, m2)) {
+                    // an inf or nan in this vector (to be left out of the sums), or squares outside the fp32
+                    // range: the vector again, element by element in fp64
                     for (int i = 0; i < 4; ++i) {
                         moments_careful(w[i] & 0xFFFFu, s1, s2, bad);
                         moments_careful(w[i] >> 16, s1, s2, bad);

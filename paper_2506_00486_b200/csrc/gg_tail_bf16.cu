@@ -285,10 +285,10 @@ template <int FLAGS>
 __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &acc, const Smem &sm)
 {
     if constexpr ((FLAGS & kMoments) != 0) {
-        if (r.m2 <= FLT_MAX) {
+        if (run_sums_exact_enough(r.m1, r.m2)) {
             acc.s1 += (double)r.m1;
             acc.s2 += (double)r.m2;
-        } else {     // a square or a sum beyond the fp32 range: this run again in fp64
+        } else {     // a square or a sum outside the fp32 range: this run again in fp64
             const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
             for (int e = 0; e < n; ++e) {
                 const uint32_t h = (w[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu;

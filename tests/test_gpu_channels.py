@@ -1,0 +1,190 @@
+"""GPU parity of the channel-wise pass: every column of a row-major matrix is one segment.  The oracle
+has no notion of strides: each column is gathered on the host and goes through the same oracle calls
+as a contiguous segment."""
+import numpy as np
+import pytest
+import torch
+
+import gg_synth
+from oracle import gg_oracle as o
+from parity_util import ABS_ENTROPY, REL_FIT, REL_PENALTY, assert_grad_close, assert_rel
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2506_00486_b200 import Context
+    c = Context(0)
+    yield c
+    c.close()
+
+
+def channel_matrix(rows, cols, seed, wide_scales=True):
+    """bf16 [rows, cols]: column c is GG(beta_c, alpha_c) with its own shape and scale."""
+    rng = np.random.default_rng(seed)
+    x = torch.empty((rows, cols), dtype=torch.bfloat16)
+    for c in range(cols):
+        beta = float(rng.uniform(0.4, 2.5))
+        alpha = 10.0 ** rng.uniform(-4, 1) if wide_scales else 0.05 * (1 + c % 7)
+        x[:, c] = gg_synth.gg_host(rng, beta, alpha, rows, torch.bfloat16)
+    return x
+
+
+def check_channels(out, x, grad, lam, step=None, qmin=-32768, qmax=32767, mean=False, grad_before=None,
+                   hist_before=None, cols=None):
+    rows, ncol = x.shape
+    nb = qmax - qmin + 1
+    ref_hist = np.zeros(nb, dtype=np.uint64) if hist_before is None else hist_before.astype(np.uint64).copy()
+    ref_cl = np.zeros(2, dtype=np.uint64)
+    for c in (range(ncol) if cols is None else cols):
+        xo = gg_synth.to_oracle(x[:, c].contiguous())
+        b, a, s1, s2, n, fl = o.fit(xo)
+        bg, ag = out["beta"][c].item(), out["alpha"][c].item()
+        assert (out["flags"][c].item() & 15) == fl, f"flags[{c}]"
+        assert out["count"][c].item() == n
+        if fl & o.FLAG_DEGENERATE:
+            assert bg == 0.0 and ag == 0.0
+        else:
+            assert_rel(out["sum_abs"][c].item(), s1, 1e-7, f"sum_abs[{c}]")
+            assert_rel(out["sum_sq"][c].item(), s2, 1e-7, f"sum_sq[{c}]")
+            assert_rel(bg, b, REL_FIT, f"beta[{c}]")
+            assert_rel(ag, a, REL_FIT, f"alpha[{c}]")
+        lam_c = lam / max(n, 1) if mean else lam
+        pen, g = o.penalty_grad(xo, bg, ag, lam_c)
+        if grad is not None:
+            got = grad[:, c]
+            if grad.dtype == torch.bfloat16:
+                if grad_before is not None:
+                    with np.errstate(invalid="ignore", over="ignore"):
+                        g = (g.astype(np.float32) + grad_before[:, c].float().numpy()).astype(np.float64)
+                ref = o.round_to_bf16_bits(g).astype(np.int64)
+                gb = got.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+                fin = np.isfinite(g)
+                assert np.abs((ref & 0x7FFF) - (gb & 0x7FFF))[fin].max(initial=0) <= 1, f"grad[:, {c}]"
+            else:
+                assert grad_before is None
+                nan = np.isnan(g)                      # a nan entry gives a nan gradient: any nan will do
+                assert np.isnan(got.numpy()[nan]).all()
+                assert_grad_close(got.numpy()[~nan], g[~nan])
+        if out["penalty"] is not None:
+            if not np.isfinite(pen):                   # inf or nan entries: the sum is not a number either
+                assert not np.isfinite(out["penalty"][c].item())
+            elif pen != 0:
+                assert_rel(out["penalty"][c].item(), pen, REL_PENALTY, f"penalty[{c}]")
+            else:
+                assert out["penalty"][c].item() == 0.0
+        if step is not None and cols is None:
+            cl = np.zeros(2, dtype=np.uint64)
+            o.quantise_hist(xo, np.float32(step), qmin, qmax, hist=ref_hist, clamped=cl)
+            ref_cl += cl
+            assert bool(out["flags"][c].item() & 16) == bool(cl.sum() > 0), f"clamp flag[{c}]"
+    if step is not None and cols is None:
+        np.testing.assert_array_equal(out["hist"].cpu().numpy(), ref_hist.astype(np.int64))
+        np.testing.assert_array_equal(out["clamped"].cpu().numpy(), ref_cl.astype(np.int64))
+        assert abs(out["entropy_bits"][0].item() - o.entropy_bits(ref_hist)) <= ABS_ENTROPY
+
+
+def cpu(out):
+    return {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in out.items()}
+
+
+def test_channels_ragged_padded_with_special_columns(ctx):
+    """Three full strips and a ragged one, rows that fill no whole block, padded rows (ld > cols),
+    scales 1e-4 .. 10 inside one strip, and columns of zeros, specials, tiny and huge values."""
+    rows, cols, ld = 1500, 200, 208
+    x = channel_matrix(rows, cols, seed=41)
+    x[:, 5] = 0
+    x[:, 6] = torch.where(torch.arange(rows) % 2 == 0, x[:, 6], torch.zeros(()).to(torch.bfloat16))   # half exact zeros
+    x[:9, 7] = torch.tensor([0.0, -0.0, 1e-40, -1e-39, 3e38, -3e38, 1e-30, 1e20, -1e-20]).to(torch.bfloat16)
+    x[:3, 8] = torch.tensor([float("inf"), float("nan"), float("-inf")]).to(torch.bfloat16)
+    x[:, 70] = (x[:, 70].float() * 1e-25).to(torch.bfloat16)       # far below the strip's exponent window
+    x[:, 130] = (x[:, 130].float() * 1e20).to(torch.bfloat16)      # pushes the window up for its strip
+    buf = torch.full((rows, ld), 7.0, dtype=torch.bfloat16, device="cuda:0")
+    buf[:, :cols].copy_(x)
+    gbuf = torch.full((rows, ld), -1.0, dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused_channels(buf[:, :cols], grad=gbuf[:, :cols], lam=1e-4, step=2.0 ** -7)
+    torch.cuda.synchronize()
+    assert torch.all(gbuf[:, cols:] == -1.0)                      # the padding is not written
+    check_channels(cpu(out), x, gbuf[:, :cols].cpu(), 1e-4, step=2.0 ** -7)
+
+
+def test_channels_odd_width_bf16_grad_mean_accumulate_and_clamp(ctx):
+    """Odd column count and odd leading dimension (scalar loads and stores), bf16 gradient added to
+    what is there, mean reduction, negative lambda, a clamp narrower than the count window, counts
+    added to an existing histogram."""
+    from paper_2506_00486_b200 import GG_MEAN
+    rows, cols, ld = 777, 131, 133
+    x = channel_matrix(rows, cols, seed=42, wide_scales=False)
+    buf = torch.zeros((rows, ld), dtype=torch.bfloat16, device="cuda:0")
+    buf[:, :cols].copy_(x)
+    g0 = (torch.randn((rows, cols), generator=torch.Generator().manual_seed(1)) * 1e-4).to(torch.bfloat16)
+    gbuf = torch.zeros((rows, ld), dtype=torch.bfloat16, device="cuda:0")
+    gbuf[:, :cols].copy_(g0)
+    qmin, qmax = -300, 200
+    h0 = torch.arange(qmax - qmin + 1, dtype=torch.int64)
+    hist = h0.to("cuda:0")
+    out = ctx.gg_fused_channels(buf[:, :cols], grad=gbuf[:, :cols], lam=-2e-3, reduction=GG_MEAN, accumulate_grad=True,
+                                step=0.01, qmin=qmin, qmax=qmax, accumulate_hist=True, hist=hist)
+    torch.cuda.synchronize()
+    check_channels(cpu(out), x, gbuf[:, :cols].cpu(), -2e-3, step=0.01, qmin=qmin, qmax=qmax, mean=True,
+                   grad_before=g0, hist_before=h0.numpy())
+
+
+def test_channels_fit_only_and_empty_shapes(ctx):
+    x = channel_matrix(300, 70, seed=43)
+    out = ctx.gg_fused_channels(x.to("cuda:0"), want_penalty=False)
+    torch.cuda.synchronize()
+    check_channels(cpu(out), x, None, 0.0)
+    # no rows: every column degenerate; no columns: nothing to do
+    out = ctx.gg_fused_channels(torch.empty((0, 5), dtype=torch.bfloat16, device="cuda:0"), step=0.5)
+    torch.cuda.synchronize()
+    assert torch.all(out["beta"] == 0) and torch.all(out["flags"] == 1) and torch.all(out["penalty"] == 0)
+    assert out["hist"].sum().item() == 0 and out["entropy_bits"][0].item() == 0.0
+    out = ctx.gg_fused_channels(torch.empty((4, 0), dtype=torch.bfloat16, device="cuda:0"), step=0.5)
+    torch.cuda.synchronize()
+    assert out["beta"].numel() == 0
+    # one row: |x| is the whole sample, the ratio is 1 and beta clamps high
+    one = torch.tensor([[0.5, -2.0, 0.0]], dtype=torch.bfloat16)
+    g = torch.empty((1, 3), dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused_channels(one.to("cuda:0"), grad=g, step=0.25)
+    torch.cuda.synchronize()
+    check_channels(cpu(out), one, g.cpu(), 1e-4, step=0.25)
+
+
+def test_channels_rejects_what_it_does_not_take(ctx):
+    from paper_2506_00486_b200 import GGError
+    with pytest.raises(GGError):
+        ctx.gg_fused_channels(torch.zeros((4, 4), dtype=torch.float32, device="cuda:0"))
+    with pytest.raises(GGError):
+        ctx.gg_fused_channels(torch.zeros((4, 4), dtype=torch.bfloat16, device="cuda:0"), step=0.0)
+
+
+def test_channels_activation_shaped_matrix_sampled_columns(ctx):
+    """[8192 tokens, 4096 channels] bf16 with channel-dependent scale and 0.1 % outliers: several row
+    slices per strip.  Sampled columns against the oracle element by element; for the whole matrix the
+    histogram against torch's own floor and bincount, and column sums against torch reductions."""
+    rows, cols = 8192, 4096
+    gen = torch.Generator(device="cuda:0").manual_seed(44)
+    a = gg_synth.alpha_for_std(1.0, 0.8)
+    x = gg_synth.gg_device(gen, 0.8, a, rows * cols, torch.bfloat16, torch.device("cuda:0")).view(rows, cols)
+    scale = torch.exp2(torch.arange(cols, device="cuda:0") % 9 - 4.0).to(torch.bfloat16)
+    x = (x * scale).contiguous()
+    gg_synth.add_outliers_device(gen, x, 1e-3, 20.0)
+    g = torch.empty((rows, cols), dtype=torch.float32, device="cuda:0")
+    step = 0.01
+    out = ctx.gg_fused_channels(x, grad=g, lam=1e-4, step=step)
+    torch.cuda.synchronize()
+    xf = x.float()
+    inv = torch.tensor(1.0 / step, dtype=torch.float64).float().item()
+    q = torch.floor(xf * inv).clamp_(-32768, 32767).to(torch.int64) + 32768
+    ref = torch.bincount(q.view(-1), minlength=65536)
+    assert torch.equal(out["hist"], ref)
+    assert out["hist"].sum().item() == rows * cols
+    torch.testing.assert_close(out["sum_abs"], xf.double().abs().sum(0), rtol=1e-7, atol=0)
+    torch.testing.assert_close(out["sum_sq"], (xf.double() ** 2).sum(0), rtol=1e-7, atol=0)
+    sample = [0, 1, 63, 64, 2047, 2048, 4031, 4095] + list(np.random.default_rng(5).integers(0, cols, 8))
+    oc = cpu(out)
+    check_channels(oc, x.cpu(), g.cpu(), 1e-4, cols=sample)

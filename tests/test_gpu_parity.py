@@ -105,6 +105,35 @@ def test_fit_with_magnitudes_whose_squares_leave_the_fp32_range(ctx, dtype):
         assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fit_with_magnitudes_whose_squares_fall_below_the_fp32_range(ctx, dtype):
+    """|x| below 1e-19 squares into the fp32 subnormals or to zero; the moments must still be those of the
+    oracle, through the long-segment kernels and through the one-warp-per-segment kernel."""
+    from paper_2506_00486_b200 import Segments
+    rng = np.random.default_rng(18)
+    x = gg_synth.gg_host(rng, 0.9, 1e-26, 3 * TILE + 50, torch.float32).to(dtype)
+    x[::101] = 0
+    out = ctx.gg_fit([dev(x), dev(x[:1000])])
+    torch.cuda.synchronize()
+    for s, xs in enumerate((x, x[:1000])):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(xs))
+        assert out["flags"][s].item() == fl
+        assert_rel(out["sum_abs"][s].item(), s1, 1e-7, "sum_abs")
+        assert_rel(out["sum_sq"][s].item(), s2, 1e-7, "sum_sq")
+        assert_rel(out["beta"][s].item(), b, REL_FIT, "beta")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
+    if dtype == torch.bfloat16:
+        xs = [x[i * 500:(i + 1) * 500] for i in range(70)]
+        out = ctx.gg_fused(Segments([dev(t) for t in xs]), want_penalty=False, want_hist=False)
+        torch.cuda.synchronize()
+        for s, t in enumerate(xs):
+            b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(t))
+            assert out["flags"][s].item() == fl
+            assert_rel(out["sum_sq"][s].item(), s2, 1e-7, "sum_sq")
+            assert_rel(out["beta"][s].item(), b, REL_FIT, "beta")
+            assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
+
+
 def test_fit_over_the_whole_shape_range(ctx):
     """beta from 0.1 to 8 on large samples: the fitted pair matches the oracle's."""
     rng = np.random.default_rng(21)
