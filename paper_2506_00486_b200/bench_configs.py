@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Timings of the secondary workloads (everything but the weight sweep that bench.py reports).
 
-    python -m paper_2506_00486_b200.bench_configs [c1] [c2] [c3] [c4] [codes]
+    python -m paper_2506_00486_b200.bench_configs [c1] [c2] [c3] [c4] [codes] [channels]
 
 Each line gives the CUDA-event time of one call through the C interface on cuda:0, inputs resident
 in device memory, and the algorithmic GB/s (input read once + output written once).  Inputs are the
@@ -74,6 +74,7 @@ def main(which):
         gs = [torch.empty_like(t) for t in xs]
         if "c4" in which:
             run = ctx.make_fused(Segments(xs), grad=Segments(gs), lam=1e-4, step_scale=1 / 16)
+            run()                    # (the first launch of a kernel loads it: keep that out of the sweep timers)
             ctx.timing_enable(True)
             ctx.timing_read()
             ms = timeit(run, 5)
@@ -94,8 +95,26 @@ def main(which):
             rh = ctx.gg_rate_hist(xs, steps)
             ms = timeit(lambda: ctx.gg_eg_rate(rh["hist"]))
             print(f"codes  gg_eg_rate, 8 histograms of 65536 bins: {ms * 1e3:.1f} us")
+    if "channels" in which:
+        for rows, cols in ((16384, 4096), (65536, 4096), (16384, 11008)):
+            a = gg_synth.alpha_for_std(1.0, 0.8)
+            x = gg_synth.gg_device(gen, 0.8, a, rows * cols, torch.bfloat16, dev).view(rows, cols)
+            x.mul_(torch.exp2(torch.arange(cols, device=dev) % 3 - 1.0).to(torch.bfloat16))
+            gg_synth.add_outliers_device(gen, x, 1e-3, 20.0)
+            g = torch.empty((rows, cols), dtype=torch.float32, device=dev)
+            run = ctx.make_fused_channels(x, grad=g, lam=1e-4, step=0.01)
+            run()                    # (the first launch of a kernel loads it: keep that out of the sweep timers)
+            ctx.timing_enable(True)
+            ctx.timing_read()
+            ms = timeit(run, 5)
+            t = ctx.timing_read()
+            ctx.timing_enable(False)
+            print(f"channels  fused, bf16 [{rows}, {cols}], one GG per column, one histogram: {ms * 1e3:.1f} us  "
+                  f"{6 * x.numel() / ms / 1e6:.0f} GB/s  (moments {t[0] / t[1] * 1e3:.1f} us, "
+                  f"gradient + histogram {t[2] / t[3] * 1e3:.1f} us)")
+            del x, g, run
     ctx.close()
 
 
 if __name__ == "__main__":
-    main(set(sys.argv[1:]) or {"c1", "c2", "c3", "c4", "codes"})
+    main(set(sys.argv[1:]) or {"c1", "c2", "c3", "c4", "codes", "channels"})

@@ -6,8 +6,8 @@
 // rows, so every thread accumulates the sums of its own two columns and no transposition happens.
 //   chan_moments_kernel   one CTA per (strip, block of 256 rows): sum |x|, sum x^2, non-finite
 //                         count, min, max per column, written per row block
-//   chan_fit_kernel       one thread per column: adds the row blocks in order, inverts the moment
-//                         ratio from the fit table, derives the constants of the gradient
+//   chan_fit_kernel       16 threads per column: add the row blocks in a fixed order, invert the moment
+//                         ratio from the fit table, derive the constants of the gradient
 //   chan_tail_kernel      one CTA per (strip, slice of rows): builds the per-column gradient tables
 //                         |g| = A_c[e] * B_c[j] (e exponent field, j mantissa bits of the bf16
 //                         pattern; the lane owns its columns, so lane l reads word l of a table
@@ -49,25 +49,58 @@ __device__ __forceinline__ uint32_t load_pair(const uint16_t *row, bool vec, boo
     return w;
 }
 
-// One column's share of a block of rows, in fp64, non-finite entries left out (used when the fp32
-// partials of the block left the fp32 range).
-__device__ __noinline__ void moments_careful(const uint32_t (&w)[kU], int half, double &s1, double &s2)
+// One element in fp64; a non-finite entry is counted and left out (used when the fp32 partials of a
+// block of rows cannot stand for the exact sums).
+__device__ __forceinline__ void moments_careful(uint32_t h, double &s1, double &s2, uint32_t &bad)
 {
+    const uint32_t mag = h & 0x7FFFu;
+    if (mag < 0x7F80u) {
+        const double ax = (double)__uint_as_float(mag << 16);
+        s1 += ax;
+        s2 += ax * ax;
+    } else {
+        bad += 1u;
+    }
+}
+
+// kU rows of the lane's two columns (row u is the 32-bit word word_of(u); rows past the end and missing
+// columns read as zero, which adds nothing to the sums; the caller repairs the extremes) into the
+// running sums.
+template <typename WordOf>
+__device__ __forceinline__ void mom_block(WordOf word_of, double (&s1)[2], double (&s2)[2], uint32_t (&bad)[2],
+                                          __nv_bfloat162 &mn2, __nv_bfloat162 &mx2)
+{
+    float m1[2] = {0.0f, 0.0f}, m2[2] = {0.0f, 0.0f};
+#pragma unroll
     for (int u = 0; u < kU; ++u) {
-        const uint32_t h = (half ? (w[u] >> 16) : w[u]) & 0x7FFFu;
-        if (h < 0x7F80u) {
-            const double ax = (double)__uint_as_float(h << 16);
-            s1 += ax;
-            s2 += ax * ax;
+        const uint32_t w = word_of(u);
+        const float lo = __uint_as_float(w << 16), hi = __uint_as_float(w & 0xFFFF0000u);
+        m1[0] += fabsf(lo);
+        m2[0] = fmaf(lo, lo, m2[0]);
+        m1[1] += fabsf(hi);
+        m2[1] = fmaf(hi, hi, m2[1]);
+        const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w);
+        mn2 = __hmin2(mn2, pr);
+        mx2 = __hmax2(mx2, pr);
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        if (run_sums_exact_enough(m1[k], m2[k])) {
+            s1[k] += (double)m1[k];
+            s2[k] += (double)m2[k];
+        } else {     // an inf or nan (left out of the sums and counted), or squares outside the fp32 range
+#pragma unroll
+            for (int u = 0; u < kU; ++u) moments_careful(k ? (word_of(u) >> 16) : word_of(u), s1[k], s2[k], bad[k]);
         }
     }
 }
 
-__global__ void __launch_bounds__(kMomThreads) chan_moments_kernel(const ChanArgs a)
+__global__ void __launch_bounds__(kMomThreads, 5) chan_moments_kernel(const ChanArgs a)
 {
     __shared__ double red1[kMomWarps][kChanStrip], red2[kMomWarps][kChanStrip];
     __shared__ uint32_t redb[kMomWarps][kChanStrip];
     __shared__ float redmn[kMomWarps][kChanStrip], redmx[kMomWarps][kChanStrip];
+    __shared__ uint32_t ring[2][kU][kMomThreads];     // per-thread slots of the rows in flight
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kChanStrip + 2 * lane;
     const int64_t r_begin = (int64_t)blockIdx.y * kChanMomRows;
@@ -78,40 +111,53 @@ __global__ void __launch_bounds__(kMomThreads) chan_moments_kernel(const ChanArg
 
     double s1[2] = {0.0, 0.0}, s2[2] = {0.0, 0.0};
     uint32_t bad[2] = {0u, 0u};
-    float mn[2] = {INFINITY, INFINITY}, mx[2] = {-INFINITY, -INFINITY};
-    for (int64_t r = r_begin + warp; r < r_end; r += (int64_t)kMomWarps * kU) {
+    // extremes of both columns at once, as packed bf16 (min and max return the non-NaN operand, like fminf)
+    __nv_bfloat162 mn2 = __floats2bfloat162_rn(INFINITY, INFINITY), mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
+    const int64_t stride = (int64_t)kMomWarps * a.ld;
+    const int64_t r0 = r_begin + warp;
+    const uint16_t *p = col + r0 * a.ld;
+    int n_mine = r0 < r_end ? (int)((r_end - r0 + kMomWarps - 1) / kMomWarps) : 0;      // rows of this warp
+    if (vec && ok0) {
+        // Whole blocks of kU rows: the thread stages its words of the next block in its own ring slots with
+        // asynchronous copies while it sums the current one (one commit group per block, so the group that
+        // must have landed is always the one before the last).
+        const uint32_t slot = (uint32_t)__cvta_generic_to_shared(&ring[0][0][threadIdx.x]);
+        constexpr uint32_t kRow = kMomThreads * 4u;
+        const int n_blocks = n_mine / kU;
+        auto stage = [&](const uint16_t *src, uint32_t dst) {
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)u * kRow), "l"(src + u * stride) : "memory");
+        };
+        if (n_blocks > 0) stage(p, slot);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        for (int bk = 0; bk < n_blocks; ++bk) {
+            const uint32_t cur = slot + (uint32_t)(bk & 1) * kU * kRow;
+            if (bk + 1 < n_blocks) stage(p + kU * stride, slot + (uint32_t)((bk + 1) & 1) * kU * kRow);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            mom_block([&](int u) {
+                uint32_t w;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(cur + (uint32_t)u * kRow));
+                return w;
+            }, s1, s2, bad, mn2, mx2);
+            p += kU * stride;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        n_mine -= n_blocks * kU;
+    }
+    for (; n_mine > 0; n_mine -= kU, p += kU * stride) {
         uint32_t w[kU];
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            const int64_t ru = r + (int64_t)u * kMomWarps;
-            w[u] = ru < r_end ? load_pair(col + ru * a.ld, vec, ok0, ok1) : 0u;
-        }
-        float m1[2] = {0.0f, 0.0f}, m2[2] = {0.0f, 0.0f};
-#pragma unroll
-        for (int u = 0; u < kU; ++u) {
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const uint32_t xb = k ? (w[u] & 0xFFFF0000u) : (w[u] << 16);
-                const float ax = __uint_as_float(xb & 0x7FFFFFFFu);
-                m1[k] += ax;
-                m2[k] = fmaf(ax, ax, m2[k]);
-                bad[k] += (xb & 0x7FFFFFFFu) >= 0x7F800000u ? 1u : 0u;
-                mn[k] = fminf(mn[k], __uint_as_float(xb));      // fminf / fmaxf return the non-NaN operand
-                mx[k] = fmaxf(mx[k], __uint_as_float(xb));
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            // (rows past the end and missing columns were read as zero: they add nothing; the extremes are
-            // corrected below)
-            if (run_sums_exact_enough(m1[k], m2[k])) { s1[k] += (double)m1[k]; s2[k] += (double)m2[k]; }
-            else moments_careful(w, k, s1[k], s2[k]);     // inf, nan, or squares outside the fp32 range
-        }
+        for (int u = 0; u < kU; ++u) w[u] = u < n_mine ? load_pair(p + u * stride, vec, ok0, ok1) : 0u;
+        mom_block([&](int u) { return w[u]; }, s1, s2, bad, mn2, mx2);
     }
+    float mn[2] = {__low2float(mn2), __high2float(mn2)}, mx[2] = {__low2float(mx2), __high2float(mx2)};
     // Rows past the end and missing columns entered the extremes as zeros.  Only the last row block and
     // the last strip can have them: there the extremes are taken again over the real entries alone.
     if (r_end - r_begin < kChanMomRows || !ok0 || !ok1) {
-        for (int k = 0; k < 2; ++k) { mn[k] = INFINITY; mx[k] = -INFINITY; }
+        mn[0] = mn[1] = INFINITY;
+        mx[0] = mx[1] = -INFINITY;
         for (int64_t r = r_begin + warp; r < r_end; r += kMomWarps) {
             const uint32_t w = load_pair(col + r * a.ld, vec, ok0, ok1);
             const float v0 = __uint_as_float(w << 16), v1 = __uint_as_float(w & 0xFFFF0000u);
@@ -144,18 +190,34 @@ __global__ void __launch_bounds__(kMomThreads) chan_moments_kernel(const ChanArg
     }
 }
 
-// One thread per column: the row blocks in order, the fit, the clamp flag, the gradient constants.
-__global__ void __launch_bounds__(128) chan_fit_kernel(const ChanArgs a)
+// 32 columns per CTA, 16 threads per column: thread (column, g) adds the row blocks g, g + 16, ... in
+// order, thread (column, 0) adds the 16 partial sums in order and does the fit, the clamp flag and the
+// gradient constants.
+constexpr int kFitCols = 32, kFitGroups = 16;
+__global__ void __launch_bounds__(kFitCols * kFitGroups) chan_fit_kernel(const ChanArgs a)
 {
-    const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= a.cols) return;
+    __shared__ double r1[kFitGroups][kFitCols], r2[kFitGroups][kFitCols];
+    __shared__ uint32_t rb[kFitGroups][kFitCols];
+    __shared__ float rmn[kFitGroups][kFitCols], rmx[kFitGroups][kFitCols];
+    const int cx = threadIdx.x % kFitCols, grp = threadIdx.x / kFitCols;
+    const int64_t c = (int64_t)blockIdx.x * kFitCols + cx;
     double s1 = 0.0, s2 = 0.0;
     uint32_t bad = 0;
     float xmin = INFINITY, xmax = -INFINITY;
-    for (int k = 0; k < a.n_mom_blocks; ++k) {
-        const int64_t o = (int64_t)k * a.cols + c;
-        s1 += a.s1[o]; s2 += a.s2[o]; bad += a.bad[o];
-        xmin = fminf(xmin, a.xmin[o]); xmax = fmaxf(xmax, a.xmax[o]);
+    if (c < a.cols) {
+#pragma unroll 4
+        for (int k = grp; k < a.n_mom_blocks; k += kFitGroups) {
+            const int64_t o = (int64_t)k * a.cols + c;
+            s1 += a.s1[o]; s2 += a.s2[o]; bad += a.bad[o];
+            xmin = fminf(xmin, a.xmin[o]); xmax = fmaxf(xmax, a.xmax[o]);
+        }
+    }
+    r1[grp][cx] = s1; r2[grp][cx] = s2; rb[grp][cx] = bad; rmn[grp][cx] = xmin; rmx[grp][cx] = xmax;
+    __syncthreads();
+    if (grp != 0 || c >= a.cols) return;
+    for (int g = 1; g < kFitGroups; ++g) {
+        s1 += r1[g][cx]; s2 += r2[g][cx]; bad += rb[g][cx];
+        xmin = fminf(xmin, rmn[g][cx]); xmax = fmaxf(xmax, rmx[g][cx]);
     }
     double beta, alpha;
     uint32_t flags = fit_from_sums(s1, s2, a.rows, a.seed, &beta, &alpha) | (bad ? GG_FLAG_NONFINITE : 0u);
@@ -196,7 +258,16 @@ __global__ void __launch_bounds__(128) chan_penalty_kernel(const ChanArgs a)
 
 // ------------------------------------------------------------------------------------ second kernel
 
+// Warp-uniform constants that only the cold paths need.
+struct ChanConst {
+    float inv;
+    int32_t wlo, whi, qmin, qmax;     // count window [wlo, whi), clamp
+    uint32_t flip;                    // sign bit of lambda
+    unsigned long long *hist;
+};
+
 struct TailSmem {
+    uint32_t ring[2][kU][kTailThreads];   // per-thread slots of the rows in flight: two blocks of kU rows
     float a1[2][kAWin + 1][32];       // [k][e - e_lo][lane]: A of column 2 lane + k; row kAWin: the marker
     float bt[2][128][32];             // [k][j][lane]: B of column 2 lane + k
     uint32_t cnt[kSymWin + 2];        // cell 0 and the last: sentinels of the two tails
@@ -205,6 +276,7 @@ struct TailSmem {
     double lg[128];                   // log2(1 + j/128)
     uint32_t clampc[2];
     int e_top;
+    ChanConst cc;
 };
 
 // 2^t for |t| < 1000 within 1e-11 relative: table entries are rounded to fp32 afterwards.
@@ -235,17 +307,12 @@ __device__ __noinline__ float chan_grad_exact(uint32_t mag, double L, double b, 
     return __uint_as_float(__float_as_uint(v) ^ flip);
 }
 
-// fp64 penalty terms |x| |g| of one column over a block of rows.
-__device__ __noinline__ double chan_pen_exact(const uint32_t (&w)[kU], int half, double L, double b)
+// fp64 penalty term |x| |g| of one magnitude pattern.
+__device__ __noinline__ double chan_pen_exact(uint32_t mag, double L, double b)
 {
-    if (!(L == L)) return 0.0;
-    double dp = 0.0;
-    for (int u = 0; u < kU; ++u) {
-        const uint32_t h = (half ? (w[u] >> 16) : w[u]) & 0x7FFFu;
-        const double ax = (double)__uint_as_float(h << 16);
-        if (ax != 0.0) dp += ax * exp2(L + b * log2(ax));
-    }
-    return dp;
+    const double ax = (double)__uint_as_float(mag << 16);
+    if (!(L == L) || ax == 0.0) return 0.0;
+    return ax * exp2(L + b * log2(ax));
 }
 
 // Quantises one value and counts its symbol: the shared window when in reach, else global memory.
@@ -262,29 +329,41 @@ __device__ __noinline__ void chan_count_slow(float x, float inv, int32_t qmin, i
     }
 }
 
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
 __device__ __forceinline__ void red_inc(uint32_t addr)
 {
     asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
 }
 
-// Per-thread constants of the element path.
+// Per-thread constants of the element path (the rest lives in TailSmem::cc).
 struct ChanLane {
-    uint32_t a_addr[2], b_addr[2];   // shared-memory addresses of this lane's word in row 0 of its tables
+    uint32_t a_addr, b_addr;         // shared-memory addresses of this lane's word in row 0 of its first tables
     uint32_t e_lo;                   // exponent field of row 0 of the A tables
     uint32_t cnt_off;                // cell of a value = bits(floor(t) + magic) * 4 + cnt_off (mod 2^32)
     float inv, t_lo, t_hi;           // quantiser scale; t is clamped to [t_lo, t_hi] so that its floor is a cell
+    float near;                      // a smaller |t| lies inside the count window for sure
 };
+constexpr uint32_t kA2 = (kAWin + 1) * 128u;     // byte offset of the second column's A table
+constexpr uint32_t kB2 = 128u * 128u;            // and of its B table
+
+// Row i of the lane's A table / row j of its B table for column HALF.
+template <int HALF>
+__device__ __forceinline__ float lds_a(const ChanLane &ln, uint32_t i)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(ln.a_addr + i * 128u), "n"(HALF ? kA2 : 0u));
+    return v;
+}
+template <int HALF>
+__device__ __forceinline__ float lds_b(const ChanLane &ln, uint32_t j)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(ln.b_addr + j * 128u), "n"(HALF ? kB2 : 0u));
+    return v;
+}
 
 // One element (HALF 0: the low half of w, the lane's even column).  Branch free.
 template <bool GRAD, bool HIST, int HALF>
-__device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanLane &ln, float &mp, uint32_t &anyc)
+__device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanLane &ln, float &mp, float &anyc)
 {
     const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);
     float g = 0.0f;
@@ -292,7 +371,7 @@ __device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanL
         const uint32_t e = HALF ? (w >> 23) & 0xFFu : (w >> 7) & 0xFFu;
         const uint32_t j = HALF ? (w >> 16) & 127u : w & 127u;
         const uint32_t i = min(e - ln.e_lo, (uint32_t)kAWin);       // below the window wraps around to the marker too
-        float ga = lds_f32(ln.a_addr[HALF] + i * 128u) * lds_f32(ln.b_addr[HALF] + j * 128u);
+        float ga = lds_a<HALF>(ln, i) * lds_b<HALF>(ln, j);
         ga = (xb << 1) == 0u ? 0.0f : ga;                            // g(0) = 0 for every shape
         mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), mp);
         g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
@@ -300,7 +379,7 @@ __device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanL
     if constexpr (HIST) {
         if (counted) {
             const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
-            anyc = max(anyc, __float_as_uint(t) & 0x7FFFFFFFu);
+            anyc = fmaxf(anyc, fabsf(t));      // (a nan is ignored here and lands on a sentinel: nan is not counted)
             // outside the window (and nan, which fmaxf replaces by the lower bound) the floor lands on a sentinel
             const float tc = fminf(fmaxf(t, ln.t_lo), ln.t_hi);
             // |tc| < 2^22: the sum lies in [2^23, 2^24) where floats are the integers, so rounding down gives floor
@@ -309,6 +388,13 @@ __device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanL
         }
     }
     return g;
+}
+
+template <typename TG>
+__device__ __forceinline__ void store_one(TG *p, float g)
+{
+    if constexpr (sizeof(TG) == 4) *p = g;
+    else *p = __bfloat16_as_ushort(__float2bfloat16_rn(g));
 }
 
 template <typename TG>
@@ -348,33 +434,152 @@ __device__ __forceinline__ void store_pair(TG *p, float g0, float g1, bool vec, 
     }
 }
 
+// The exact path of one column (HALF) of a block of rows whose fp32 penalty partial is not a usable
+// number (a marker, or a product beyond the fp32 range): fp64 penalty terms of all its rows, and the
+// exact gradient of every element that read a marker, handed to `fix(u, g)`.
+template <int HALF, typename WordOf, typename Fix>
+__device__ __forceinline__ double chan_column_exact(const ChanLane &ln, const TailSmem &sm, int lane, WordOf word_of, Fix fix)
+{
+    const double L = sm.colL[2 * lane + HALF], b = sm.colb[2 * lane + HALF];
+    double dp = 0.0;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const uint32_t w = word_of(u);
+        const uint32_t h = HALF ? (w >> 16) : (w & 0xFFFFu);
+        const uint32_t mag = h & 0x7FFFu;
+        dp += chan_pen_exact(mag, L, b);                       // (rows past the end read as zero: no term)
+        const float av = lds_a<HALF>(ln, min((mag >> 7) - ln.e_lo, (uint32_t)kAWin));
+        if (av != av && mag != 0u)
+            fix(u, __uint_as_float(__float_as_uint(chan_grad_exact(mag, L, b, sm.cc.flip)) ^ ((h & 0x8000u) << 16)));
+    }
+    return dp;
+}
+
+// Elements of a block whose count may have gone to a sentinel: exact test, slow count.
+template <typename WordOf, typename Counted>
+__device__ __forceinline__ void chan_recount(TailSmem &sm, WordOf word_of, Counted counted)
+{
+    const float inv = sm.cc.inv;
+    const int32_t wlo = sm.cc.wlo, whi = sm.cc.whi;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const uint32_t w = word_of(u);
+            const float x = __uint_as_float(k ? (w & 0xFFFF0000u) : (w << 16));
+            const float t = __fmul_rn(x, inv);
+            if (counted(u, k) && !(t >= (float)wlo && t < (float)whi))
+                chan_count_slow(x, inv, sm.cc.qmin, sm.cc.qmax, wlo, whi, sm, sm.cc.hist);
+        }
+    }
+}
+
+// kU whole rows of a whole strip, staged in this thread's ring slots at shared address wbase (row u
+// at wbase + u * kRowBytes).  The gradient pair of a row is written as soon as it is known; an element
+// the tables could not serve is written again, alone, by the exact path.
+constexpr uint32_t kRowBytes = kTailThreads * 4u;
+template <typename TG, bool GRAD, bool HIST>
+__device__ __forceinline__ void chan_block_fast(uint32_t wbase, TG *gp, int64_t sg, int lane, const ChanLane &ln, TailSmem &sm,
+                                                double (&pen)[2])
+{
+    auto word_of = [&](int u) {
+        uint32_t w;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(wbase + (uint32_t)u * kRowBytes));
+        return w;
+    };
+    float mp[2] = {0.0f, 0.0f};
+    float anyc = 0.0f;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const uint32_t w = word_of(u);
+        const float g0 = chan_elem<GRAD, HIST, 0>(w, true, ln, mp[0], anyc);
+        const float g1 = chan_elem<GRAD, HIST, 1>(w, true, ln, mp[1], anyc);
+        if constexpr (GRAD) {
+            if (gp != nullptr) store_pair<TG>(gp + u * sg, g0, g1, true, true, true, false);
+        }
+    }
+    if constexpr (GRAD) {
+        if (mp[0] <= FLT_MAX) pen[0] += (double)mp[0];
+        else pen[0] += chan_column_exact<0>(ln, sm, lane, word_of, [&](int u, float g) { if (gp != nullptr) store_one<TG>(gp + u * sg, g); });
+        if (mp[1] <= FLT_MAX) pen[1] += (double)mp[1];
+        else pen[1] += chan_column_exact<1>(ln, sm, lane, word_of, [&](int u, float g) { if (gp != nullptr) store_one<TG>(gp + u * sg + 1, g); });
+    }
+    if constexpr (HIST) {
+        if (anyc >= ln.near) chan_recount(sm, word_of, [](int, int) { return true; });
+    }
+}
+
+// Up to kU rows with every guard (ragged blocks, the last strip, unaligned rows, accumulation), as a
+// call of its own so that its registers do not weigh on the streaming loop: rows past nvalid and
+// missing columns read as zero and are not counted, and the gradients wait in registers until the
+// exact path has run (they may have to be added to what is stored).  Returns the two penalty
+// contributions.
+template <typename TG, bool GRAD, bool HIST>
+__device__ __noinline__ double2 chan_block_guarded(const uint16_t *p, int64_t sin, TG *gp, int64_t sg, int nvalid, bool ok0,
+                                                   bool ok1, bool vec_in, bool vec_out, bool accumulate, int lane, ChanLane ln,
+                                                   TailSmem *smp)
+{
+    TailSmem &sm = *smp;
+    uint32_t w[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) w[u] = u < nvalid ? load_pair(p + u * sin, vec_in, ok0, ok1) : 0u;
+    auto word_of = [&](int u) { return w[u]; };
+    float g[kU][2];
+    float mp[2] = {0.0f, 0.0f};
+    float anyc = 0.0f;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        g[u][0] = chan_elem<GRAD, HIST, 0>(w[u], ok0 && u < nvalid, ln, mp[0], anyc);
+        g[u][1] = chan_elem<GRAD, HIST, 1>(w[u], ok1 && u < nvalid, ln, mp[1], anyc);
+    }
+    double2 pen = make_double2(0.0, 0.0);
+    if constexpr (GRAD) {
+        if (mp[0] <= FLT_MAX) pen.x = (double)mp[0];
+        else pen.x = chan_column_exact<0>(ln, sm, lane, word_of, [&](int u, float ge) { g[u][0] = ge; });
+        if (mp[1] <= FLT_MAX) pen.y = (double)mp[1];
+        else pen.y = chan_column_exact<1>(ln, sm, lane, word_of, [&](int u, float ge) { g[u][1] = ge; });
+    }
+    if constexpr (HIST) {
+        if (anyc >= ln.near) chan_recount(sm, word_of, [&](int u, int k) { return u < nvalid && (k ? ok1 : ok0); });
+    }
+    if constexpr (GRAD) {
+        if (gp != nullptr) {
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+                if (u < nvalid) store_pair<TG>(gp + u * sg, g[u][0], g[u][1], vec_out, ok0, ok1, accumulate);
+        }
+    }
+    return pen;
+}
+
 template <typename TG, bool GRAD, bool HIST>
 __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(const ChanArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TailSmem &sm = *reinterpret_cast<TailSmem *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t n_strips = (a.cols + kChanStrip - 1) / kChanStrip;
-    const int64_t n_items = n_strips * a.n_slices;
+    const int n_strips = (int)((a.cols + kChanStrip - 1) / kChanStrip);
+    const int n_items = n_strips * a.n_slices;
     const uint32_t flip = a.lambda < 0.0 ? 0x80000000u : 0u;
 
     // count window: the symbols [-kSymWin/2, kSymWin/2) that the clamp leaves alone
     const int32_t wlo = (int32_t)max((int64_t)-kSymWin / 2, (int64_t)a.qmin);
     const int32_t whi = (int32_t)max((int64_t)wlo, min((int64_t)kSymWin / 2, (int64_t)a.qmax + 1));
     const float inv = (float)(1.0 / (double)a.step);
-    // |t| below this is inside the window for sure; one compare per block of rows finds the rest
-    const uint32_t near_bits = (wlo < 0 && whi > 0) ? __float_as_uint((float)min(-wlo, whi)) : 0u;
-    unsigned long long *hist = reinterpret_cast<unsigned long long *>(a.hist);
+    if (tid == 0) {
+        sm.cc.inv = inv; sm.cc.wlo = wlo; sm.cc.whi = whi; sm.cc.qmin = a.qmin; sm.cc.qmax = a.qmax;
+        sm.cc.flip = flip; sm.cc.hist = reinterpret_cast<unsigned long long *>(a.hist);
+    }
 
     ChanLane ln;
-    ln.a_addr[0] = (uint32_t)__cvta_generic_to_shared(&sm.a1[0][0][lane]);
-    ln.a_addr[1] = (uint32_t)__cvta_generic_to_shared(&sm.a1[1][0][lane]);
-    ln.b_addr[0] = (uint32_t)__cvta_generic_to_shared(&sm.bt[0][0][lane]);
-    ln.b_addr[1] = (uint32_t)__cvta_generic_to_shared(&sm.bt[1][0][lane]);
+    ln.a_addr = (uint32_t)__cvta_generic_to_shared(&sm.a1[0][0][lane]);
+    ln.b_addr = (uint32_t)__cvta_generic_to_shared(&sm.bt[0][0][lane]);
     ln.e_lo = 1u;
     ln.inv = inv;
     ln.t_lo = (float)wlo - 0.5f;
     ln.t_hi = (float)whi;
+    // |t| below min(-wlo, whi) is inside the window for sure; one compare per block of rows finds the rest
+    ln.near = (wlo < 0 && whi > 0) ? (float)min(-wlo, whi) : 0.0f;
     // floor(tc) lies in [wlo - 1, whi]; cell = floor(tc) - (wlo - 1)
     ln.cnt_off = (uint32_t)__cvta_generic_to_shared(sm.cnt) - (kMagicBits + (uint32_t)(wlo - 1)) * 4u;
 
@@ -387,13 +592,19 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
     const bool vec_out = ((reinterpret_cast<uintptr_t>(a.grad) & (2 * sizeof(TG) - 1)) == 0) && ((a.grad_ld & 1) == 0) &&
                          ((a.cols & 1) == 0);
     const bool accumulate = a.accumulate != 0;
-    int64_t cur_strip = -1;
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(&sm.ring[0][0][tid]);
+    int cur_strip = -1;
+    __syncthreads();
 
-    for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         // neighbouring CTAs take neighbouring strips of the same rows: their row pieces are adjacent in memory
-        const int64_t strip = item % n_strips, slice = item / n_strips;
-        const int64_t r_begin = a.rows * slice / a.n_slices, r_end = a.rows * (slice + 1) / a.n_slices;
-        const int64_t c0 = strip * kChanStrip + 2 * lane;
+        const int strip = item % n_strips, slice = item / n_strips;
+        // slices are cut at multiples of the rows one pass of the CTA covers, so that only the last one is ragged
+        constexpr int64_t kPass = (int64_t)kTailWarps * kU;
+        const int64_t n_pass = (a.rows + kPass - 1) / kPass;
+        const int64_t r_begin = n_pass * slice / a.n_slices * kPass;
+        const int64_t r_end = min(a.rows, n_pass * (slice + 1) / a.n_slices * kPass);
+        const int64_t c0 = (int64_t)strip * kChanStrip + 2 * lane;
         const bool ok0 = c0 < a.cols, ok1 = c0 + 1 < a.cols;
 
         if (GRAD && strip != cur_strip) {
@@ -403,7 +614,7 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
             if (tid == 0) sm.e_top = 0;
             __syncthreads();
             if (tid < kChanStrip) {
-                const int64_t c = strip * kChanStrip + tid;
+                const int64_t c = (int64_t)strip * kChanStrip + tid;
                 const bool ok = c < a.cols;
                 sm.colL[tid] = ok ? a.L[c] : __longlong_as_double(0x7FF8000000000000ll);
                 sm.colb[tid] = ok ? a.b[c] : 0.0;
@@ -436,67 +647,41 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
         }
 
         // ---- stream the rows of the slice: warp w takes rows r_begin + w, + kTailWarps, ...
-        const uint16_t *col = a.x + c0;
-        TG *gcol = GRAD && a.grad != nullptr ? reinterpret_cast<TG *>(a.grad) + c0 : nullptr;
         double pen[2] = {0.0, 0.0};
-        for (int64_t r = r_begin + warp; r < r_end; r += (int64_t)kTailWarps * kU) {
-            const int nvalid = (int)min((int64_t)kU, (r_end - r + kTailWarps - 1) / kTailWarps);
-            uint32_t w[kU];
+        const int64_t r0 = r_begin + warp;
+        int n_mine = r0 < r_end ? (int)((r_end - r0 + kTailWarps - 1) / kTailWarps) : 0;      // rows of this warp
+        const int64_t sin = (int64_t)kTailWarps * a.ld, sg = (int64_t)kTailWarps * a.grad_ld;
+        const uint16_t *p = a.x + c0 + r0 * a.ld;
+        TG *gp = GRAD && a.grad != nullptr ? reinterpret_cast<TG *>(a.grad) + c0 + r0 * a.grad_ld : nullptr;
+        // Whole blocks of a whole strip with aligned rows: each thread stages its words of the next block
+        // in its own ring slots with asynchronous copies while it works on the current one (one commit
+        // group per block, so the group that must have landed is always the one before the last).
+        if ((int64_t)strip * kChanStrip + kChanStrip <= a.cols && vec_in && (gp == nullptr || vec_out) && !accumulate) {
+            const int n_blocks = n_mine / kU;
+            auto stage = [&](const uint16_t *src, uint32_t dst) {
 #pragma unroll
-            for (int u = 0; u < kU; ++u)
-                w[u] = u < nvalid ? load_pair(col + (r + (int64_t)u * kTailWarps) * a.ld, vec_in, ok0, ok1) : 0u;
-            float g[kU][2];
-            float mp[2] = {0.0f, 0.0f};
-            uint32_t anyc = 0u;
-#pragma unroll
-            for (int u = 0; u < kU; ++u) {
-                g[u][0] = chan_elem<GRAD, HIST, 0>(w[u], ok0 && u < nvalid, ln, mp[0], anyc);
-                g[u][1] = chan_elem<GRAD, HIST, 1>(w[u], ok1 && u < nvalid, ln, mp[1], anyc);
+                for (int u = 0; u < kU; ++u)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)u * kRowBytes), "l"(src + u * sin) : "memory");
+            };
+            if (n_blocks > 0) stage(p, ring);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            for (int bk = 0; bk < n_blocks; ++bk) {
+                const uint32_t cur = ring + (uint32_t)(bk & 1) * kU * kRowBytes;
+                if (bk + 1 < n_blocks) stage(p + kU * sin, ring + (uint32_t)((bk + 1) & 1) * kU * kRowBytes);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+                chan_block_fast<TG, GRAD, HIST>(cur, gp, sg, lane, ln, sm, pen);
+                p += kU * sin;
+                if (gp != nullptr) gp += kU * sg;
             }
-            if constexpr (GRAD) {
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    if (mp[k] <= FLT_MAX) {
-                        pen[k] += (double)mp[k];
-                    } else {
-                        // a marker, or a product beyond the fp32 range: this column's rows again, exactly
-                        const double L = sm.colL[2 * lane + k], b = sm.colb[2 * lane + k];
-                        pen[k] += chan_pen_exact(w, k, L, b);
-#pragma unroll
-                        for (int u = 0; u < kU; ++u) {
-                            const uint32_t h = k ? (w[u] >> 16) : (w[u] & 0xFFFFu);
-                            const uint32_t mag = h & 0x7FFFu;
-                            const uint32_t i = min((mag >> 7) - ln.e_lo, (uint32_t)kAWin);
-                            const float av = lds_f32(ln.a_addr[k] + i * 128u);
-                            if (av != av && mag != 0u)
-                                g[u][k] = __uint_as_float(__float_as_uint(chan_grad_exact(mag, L, b, flip)) ^ ((h & 0x8000u) << 16));
-                        }
-                    }
-                }
-            }
-            if constexpr (HIST) {
-                if (anyc >= near_bits) {
-                    // some element may have missed the window (its count went to a sentinel): exact test, slow count
-                    for (int u = 0; u < nvalid; ++u) {
-                        for (int k = 0; k < 2; ++k) {
-                            if (!(k ? ok1 : ok0)) continue;
-                            const float x = __uint_as_float(k ? (w[u] & 0xFFFF0000u) : (w[u] << 16));
-                            const float t = __fmul_rn(x, inv);
-                            if (!(t >= (float)wlo && t < (float)whi))
-                                chan_count_slow(x, inv, a.qmin, a.qmax, wlo, whi, sm, hist);
-                        }
-                    }
-                }
-            }
-            if constexpr (GRAD) {
-                if (gcol != nullptr) {
-#pragma unroll
-                    for (int u = 0; u < kU; ++u)
-                        if (u < nvalid)
-                            store_pair<TG>(gcol + (r + (int64_t)u * kTailWarps) * a.grad_ld, g[u][0], g[u][1], vec_out, ok0, ok1,
-                                           accumulate);
-                }
-            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            n_mine -= n_blocks * kU;
+        }
+        for (; n_mine > 0; n_mine -= kU, p += kU * sin, gp += gp != nullptr ? kU * sg : 0) {
+            const double2 d = chan_block_guarded<TG, GRAD, HIST>(p, sin, gp, sg, min(n_mine, kU), ok0, ok1, vec_in, vec_out,
+                                                                 accumulate, lane, ln, &sm);
+            pen[0] += d.x;
+            pen[1] += d.y;
         }
 
         if constexpr (GRAD) {
@@ -505,11 +690,11 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
             sm.red[warp][2 * lane + 1] = pen[1];
             __syncthreads();
             if (tid < kChanStrip) {
-                const int64_t c = strip * kChanStrip + tid;
+                const int64_t c = (int64_t)strip * kChanStrip + tid;
                 if (c < a.cols) {
-                    double p = 0.0;
-                    for (int wv = 0; wv < kTailWarps; ++wv) p += sm.red[wv][tid];
-                    a.pen[slice * a.cols + c] = p;
+                    double ps = 0.0;
+                    for (int wv = 0; wv < kTailWarps; ++wv) ps += sm.red[wv][tid];
+                    a.pen[(int64_t)slice * a.cols + c] = ps;
                 }
             }
             __syncthreads();
@@ -518,6 +703,7 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
 
     if constexpr (HIST) {
         __syncthreads();
+        unsigned long long *hist = reinterpret_cast<unsigned long long *>(a.hist);
         const int n_cells = whi - wlo;
         for (int i = tid; i < n_cells; i += kTailThreads) {
             // (every CTA starts at another cell: CTAs that finish together do not walk the bins in step)
@@ -557,7 +743,7 @@ cudaError_t launch_chan_moments(const ChanArgs &a, cudaStream_t st)
 cudaError_t launch_chan_fit(const ChanArgs &a, cudaStream_t st)
 {
     if (a.cols <= 0) return cudaSuccess;
-    chan_fit_kernel<<<(unsigned)((a.cols + 127) / 128), 128, 0, st>>>(a);
+    chan_fit_kernel<<<(unsigned)((a.cols + kFitCols - 1) / kFitCols), kFitCols * kFitGroups, 0, st>>>(a);
     return cudaGetLastError();
 }
 

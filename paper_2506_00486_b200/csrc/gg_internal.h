@@ -124,7 +124,7 @@ cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, c
 // Column segments of a row-major bf16 matrix (gg_fused_channels).  Scratch arrays are indexed
 // [row block][column]; the moments kernel and the second kernel cut the rows differently.
 constexpr int kChanStrip = 64;        // columns per strip: 128 contiguous bytes of a row
-constexpr int kChanMomRows = 256;     // rows per CTA of the moments kernel
+constexpr int kChanMomRows = 512;     // rows per CTA of the moments kernel
 struct ChanArgs {
     const uint16_t *x;
     int64_t rows, cols, ld;
