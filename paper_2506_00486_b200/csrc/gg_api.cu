@@ -690,7 +690,8 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         ka.n_slices = chan_slices(a->rows, a->cols, ctx->sm_count);
         // scratch: doubles first, then the 32-bit arrays
         const size_t nc = (size_t)a->cols, nm = (size_t)n_mom * nc, ns = (size_t)ka.n_slices * nc;
-        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + nc;
+        const size_t n_strips = (nc + kChanStrip - 1) / kChanStrip;
+        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + nc + n_strips * (kChanTabFloats + 1) + 8;
         void *buf = ctx->chan_buf;
         gg_status st = grow(ctx, &buf, &ctx->chan_bytes, (int64_t)(n_dbl * 8 + n_w32 * 4));
         ctx->chan_buf = buf;
@@ -702,6 +703,9 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         ka.xmin = reinterpret_cast<float *>(w + nm);
         ka.xmax = reinterpret_cast<float *>(w + 2 * nm);
         ka.amax = reinterpret_cast<float *>(w + 3 * nm);
+        ka.tab_elo = reinterpret_cast<int32_t *>(w + 3 * nm + nc);
+        // (the tables are copied as 16-byte vectors: n_dbl * 8 is a multiple of 16 only if n_dbl is even)
+        ka.tab = reinterpret_cast<float *>(w + (3 * nm + nc + n_strips + 3) / 4 * 4 + (n_dbl & 1) * 2);
         ka.beta = a->beta; ka.alpha = a->alpha; ka.sum_abs = a->sum_abs; ka.sum_sq = a->sum_sq;
         ka.count = a->count; ka.flags = a->flags; ka.penalty = a->penalty;
         ka.seed = ctx->seed;
@@ -717,7 +721,7 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         if ((want_pg || do_hist) && a->rows > 0) {
             SweepTimer tm(ctx, &ctx->ev_tail, cs);
             GG_CUDA(ctx, launch_chan_tail((gg_dtype)a->grad_dtype, ka, ctx->sm_count, cs));
-            ctx->launches += 1;
+            ctx->launches += 1 + (want_pg ? 1 : 0);
         }
         if (a->penalty) {
             if (a->rows <= 0) GG_CUDA(ctx, cudaMemsetAsync(a->penalty, 0, sizeof(double) * nc, cs));

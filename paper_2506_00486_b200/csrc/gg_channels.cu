@@ -8,7 +8,8 @@
 //                         count, min, max per column, written per row block
 //   chan_fit_kernel       16 threads per column: add the row blocks in a fixed order, invert the moment
 //                         ratio from the fit table, derive the constants of the gradient
-//   chan_tail_kernel      one CTA per (strip, slice of rows): builds the per-column gradient tables
+//   chan_tables_kernel    one CTA per strip: the per-column gradient tables
+//   chan_tail_kernel      one CTA per (strip, slice of rows): loads the strip's gradient tables
 //                         |g| = A_c[e] * B_c[j] (e exponent field, j mantissa bits of the bf16
 //                         pattern; the lane owns its columns, so lane l reads word l of a table
 //                         row and no look-up ever meets a bank conflict), then streams its rows:
@@ -266,6 +267,9 @@ struct ChanConst {
     unsigned long long *hist;
 };
 
+constexpr int kTabFloats = 2 * (kAWin + 1) * 32 + 2 * 128 * 32;     // one strip's A and B tables
+static_assert(kTabFloats == kChanTabFloats && kTabFloats % 4 == 0, "table layout");
+
 struct TailSmem {
     uint32_t ring[2][kU][kTailThreads];   // per-thread slots of the rows in flight: two blocks of kU rows
     float a1[2][kAWin + 1][32];       // [k][e - e_lo][lane]: A of column 2 lane + k; row kAWin: the marker
@@ -273,9 +277,7 @@ struct TailSmem {
     uint32_t cnt[kSymWin + 2];        // cell 0 and the last: sentinels of the two tails
     double red[kTailWarps][kChanStrip];
     double colL[kChanStrip], colb[kChanStrip];
-    double lg[128];                   // log2(1 + j/128)
     uint32_t clampc[2];
-    int e_top;
     ChanConst cc;
 };
 
@@ -332,6 +334,50 @@ __device__ __noinline__ void chan_count_slow(float x, float inv, int32_t qmin, i
 __device__ __forceinline__ void red_inc(uint32_t addr)
 {
     asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+
+// One CTA per strip: the gradient tables of its 64 columns, in the layout of TailSmem::a1 and bt,
+// and the exponent field of the first A row.
+__global__ void __launch_bounds__(kTailThreads) chan_tables_kernel(const ChanArgs a)
+{
+    __shared__ double colL[kChanStrip], colb[kChanStrip], lg[128];
+    __shared__ int e_top;
+    const int tid = threadIdx.x, strip = blockIdx.x;
+    const uint32_t flip = a.lambda < 0.0 ? 0x80000000u : 0u;
+    if (tid == 0) e_top = 0;
+    if (tid < 128) lg[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
+    __syncthreads();
+    if (tid < kChanStrip) {
+        const int64_t c = (int64_t)strip * kChanStrip + tid;
+        const bool ok = c < a.cols;
+        colL[tid] = ok ? a.L[c] : __longlong_as_double(0x7FF8000000000000ll);
+        colb[tid] = ok ? a.b[c] : 0.0;
+        if (ok) atomicMax(&e_top, (int)(__float_as_uint(a.amax[c]) >> 23));
+    }
+    __syncthreads();
+    // the window: 64 exponents up to that of the largest magnitude of the strip
+    const int e_lo = max(1, min(e_top, 254) - (kAWin - 1));
+    if (tid == 0) a.tab_elo[strip] = e_lo;
+    float *ta = a.tab + (int64_t)strip * kTabFloats, *tb = ta + 2 * (kAWin + 1) * 32;
+    for (int idx = tid; idx < 2 * (kAWin + 1) * 32; idx += kTailThreads) {
+        const int l = idx & 31, i = (idx >> 5) % (kAWin + 1), k = idx / (32 * (kAWin + 1));
+        const double L = colL[2 * l + k], b = colb[2 * l + k];
+        float v = 0.0f;                                  // a column without gradient: zero everywhere
+        if (L == L) {
+            // One fp32 factor serves an exponent if the product with B stays in the normal range
+            // (|L + b (e-127)| <= 100); the rest, and the last row, hold the marker.
+            const int e = e_lo + i;
+            const double e0 = L + b * (double)(e - 127);
+            v = __int_as_float(0x7FC00000);
+            if (i < kAWin && e <= 254 && fabs(e0) <= 100.0) v = __uint_as_float(__float_as_uint((float)exp2_short(e0)) ^ flip);
+        }
+        ta[idx] = v;                                     // [k][i][l]
+    }
+    for (int idx = tid; idx < 2 * 128 * 32; idx += kTailThreads) {
+        const int l = idx & 31, j = (idx >> 5) & 127, k = idx >> 12;
+        const double L = colL[2 * l + k], b = colb[2 * l + k];
+        tb[idx] = (L == L) ? (float)exp2_short(b * lg[j]) : 1.0f;      // [k][j][l]
+    }
 }
 
 // Per-thread constants of the element path (the rest lives in TailSmem::cc).
@@ -587,7 +633,6 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
         for (int i = tid; i < kSymWin + 2; i += kTailThreads) sm.cnt[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
-    if (tid < 128) sm.lg[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
     const bool vec_in = ((reinterpret_cast<uintptr_t>(a.x) & 3u) == 0) && ((a.ld & 1) == 0) && ((a.cols & 1) == 0);
     const bool vec_out = ((reinterpret_cast<uintptr_t>(a.grad) & (2 * sizeof(TG) - 1)) == 0) && ((a.grad_ld & 1) == 0) &&
                          ((a.cols & 1) == 0);
@@ -608,41 +653,19 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
         const bool ok0 = c0 < a.cols, ok1 = c0 + 1 < a.cols;
 
         if (GRAD && strip != cur_strip) {
-            // ---- the tables of this strip's 64 columns
+            // ---- the tables of this strip's 64 columns, built once per strip by chan_tables_kernel
             cur_strip = strip;
             __syncthreads();
-            if (tid == 0) sm.e_top = 0;
-            __syncthreads();
+            const uint4 *src = reinterpret_cast<const uint4 *>(a.tab + (int64_t)strip * kTabFloats);
+            uint4 *dst = reinterpret_cast<uint4 *>(&sm.a1[0][0][0]);      // a1 and bt are contiguous
+            for (int i = tid; i < kTabFloats / 4; i += kTailThreads) dst[i] = __ldg(src + i);
             if (tid < kChanStrip) {
                 const int64_t c = (int64_t)strip * kChanStrip + tid;
                 const bool ok = c < a.cols;
                 sm.colL[tid] = ok ? a.L[c] : __longlong_as_double(0x7FF8000000000000ll);
                 sm.colb[tid] = ok ? a.b[c] : 0.0;
-                if (ok) atomicMax(&sm.e_top, (int)(__float_as_uint(a.amax[c]) >> 23));
             }
-            __syncthreads();
-            const int e_lo = max(1, min(sm.e_top, 254) - (kAWin - 1));
-            ln.e_lo = (uint32_t)e_lo;
-            for (int idx = tid; idx < 2 * (kAWin + 1) * 32; idx += kTailThreads) {
-                const int l = idx & 31, i = (idx >> 5) % (kAWin + 1), k = idx / (32 * (kAWin + 1));
-                const double L = sm.colL[2 * l + k], b = sm.colb[2 * l + k];
-                float v = 0.0f;                                  // a column without gradient: zero everywhere
-                if (L == L) {
-                    // One fp32 factor serves an exponent if the product with B stays in the normal range
-                    // (|L + b (e-127)| <= 100); the rest, and the last row, hold the marker.
-                    const int e = e_lo + i;
-                    const double e0 = L + b * (double)(e - 127);
-                    v = __int_as_float(0x7FC00000);
-                    if (i < kAWin && e <= 254 && fabs(e0) <= 100.0)
-                        v = __uint_as_float(__float_as_uint((float)exp2_short(e0)) ^ flip);
-                }
-                sm.a1[k][i][l] = v;
-            }
-            for (int idx = tid; idx < 2 * 128 * 32; idx += kTailThreads) {
-                const int l = idx & 31, j = (idx >> 5) & 127, k = idx >> 12;
-                const double L = sm.colL[2 * l + k], b = sm.colb[2 * l + k];
-                sm.bt[k][j][l] = (L == L) ? (float)exp2_short(b * sm.lg[j]) : 1.0f;
-            }
+            ln.e_lo = (uint32_t)__ldg(a.tab_elo + strip);
             __syncthreads();
         }
 
@@ -771,6 +794,11 @@ cudaError_t launch_chan_tail(gg_dtype grad_dtype, const ChanArgs &a, int sm_coun
     if (a.rows <= 0 || a.cols <= 0 || (!a.do_grad && !a.do_hist)) return cudaSuccess;
     const int64_t n_items = (a.cols + kChanStrip - 1) / kChanStrip * a.n_slices;
     const int grid = (int)min(n_items, (int64_t)sm_count * kCtasPerSm);
+    if (a.do_grad) {
+        chan_tables_kernel<<<(unsigned)((a.cols + kChanStrip - 1) / kChanStrip), kTailThreads, 0, st>>>(a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     if (a.grad != nullptr && grad_dtype == GG_BF16) return launch_tail_typed<uint16_t>(a, grid, st);
     return launch_tail_typed<float>(a, grid, st);
 }

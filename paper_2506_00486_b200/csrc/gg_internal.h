@@ -124,7 +124,8 @@ cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, c
 // Column segments of a row-major bf16 matrix (gg_fused_channels).  Scratch arrays are indexed
 // [row block][column]; the moments kernel and the second kernel cut the rows differently.
 constexpr int kChanStrip = 64;        // columns per strip: 128 contiguous bytes of a row
-constexpr int kChanMomRows = 512;     // rows per CTA of the moments kernel
+constexpr int kChanMomRows = 512;
+constexpr int kChanTabFloats = 2 * 65 * 32 + 2 * 128 * 32;   // A (64 exponents + marker row) and B (128 mantissas), two columns per lane     // rows per CTA of the moments kernel
 struct ChanArgs {
     const uint16_t *x;
     int64_t rows, cols, ld;
@@ -139,6 +140,8 @@ struct ChanArgs {
     double *L, *b;                     // [cols]: |g| = 2^(L + b log2|x|); L is NaN for a column without gradient
     float *amax;                       // [cols] largest finite magnitude
     double *pen;                       // [n_slices * cols] partial sums of |x| |g|
+    float *tab;                        // [strips * kChanTabFloats] gradient tables of every strip
+    int32_t *tab_elo;                  // [strips] exponent field of the first row of a strip's A table
     double *beta, *alpha, *sum_abs, *sum_sq;
     int64_t *count;
     uint32_t *flags;
