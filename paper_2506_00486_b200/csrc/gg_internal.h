@@ -82,6 +82,9 @@ struct FitArgs {
 
 cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
                           const StreamArgs &a, cudaStream_t st);
+// The moments sweep for bf16 input by persistent CTAs (the one-CTA-per-tile kernel of launch_stream gives the
+// same sums tile by tile).  sm_count sizes the grid.
+cudaError_t launch_moments_bf16_sweep(const StreamArgs &a, int sm_count, cudaStream_t st);
 // bf16-input sweeps with a gradient and/or a histogram: persistent CTAs, table look-up gradient,
 // histogram over bf16 bit patterns.  sm_count sizes the grid.
 cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,

@@ -515,6 +515,144 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
     }
 }
 
+// The same sums by persistent CTAs (two of 512 threads per SM), each walking one contiguous range of
+// tiles: inside a segment that range is one run of elements, streamed as 128-bit vectors through a
+// per-thread ring of asynchronous copies (four vectors in flight per thread and no registers held by
+// them), so that the block reduction, the partial-sum stores and the address set-up are paid once per
+// run instead of once per 32 KB tile.  A run's sums go to the slot of its first tile, zeros to the
+// slots of its other tiles.
+constexpr int kSweepThreads = 512, kSweepWarps = kSweepThreads / 32, kSweepCtasPerSm = 2, kSweepDepth = 4;
+
+__device__ __forceinline__ void moments_vec(const uint4 &raw, double &s1, double &s2, uint32_t &bad, __nv_bfloat162 &mn2,
+                                            __nv_bfloat162 &mx2)
+{
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    float m1 = 0.0f, m2 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        m1 += fabsf(lo);
+        m1 += fabsf(hi);
+        m2 = fmaf(lo, lo, m2);
+        m2 = fmaf(hi, hi, m2);
+        const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162 *>(&w[i]);
+        mn2 = __hmin2(mn2, p);      // return the non-NaN operand, like fminf
+        mx2 = __hmax2(mx2, p);
+    }
+    if (run_sums_exact_enough(m1, m2)) {
+        s1 += (double)m1;
+        s2 += (double)m2;
+    } else {
+        // an inf or nan in this vector (to be left out of the sums), or squares outside the fp32 range: the
+        // vector again, element by element in fp64
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            moments_careful(w[i] & 0xFFFFu, s1, s2, bad);
+            moments_careful(w[i] >> 16, s1, s2, bad);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_sweep_kernel(const StreamArgs a)
+{
+    __shared__ uint4 stage[kSweepDepth][kSweepThreads];
+    __shared__ double shRed[2][kSweepWarps];
+    __shared__ uint32_t shBad[kSweepWarps];
+    __shared__ float shMin[kSweepWarps], shMax[kSweepWarps];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t nt = a.map.n_tiles;
+    const int t_begin = (int)(nt * blockIdx.x / gridDim.x);
+    const int t_end = (int)(nt * (blockIdx.x + 1) / gridDim.x);
+    const uint32_t slot0 = (uint32_t)__cvta_generic_to_shared(&stage[0][tid]);
+    constexpr uint32_t kStageBytes = sizeof(uint4) * kSweepThreads;
+
+    for (int t = t_begin; t < t_end;) {
+        // ---- one run: the tiles of this CTA's range that lie in segment s
+        const int s = a.map.tile_seg[t];
+        const int64_t len = a.map.seg_len[s];
+        const int t_first = a.map.tile_prefix[s];
+        const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
+        const int64_t off = (int64_t)(t - t_first) * kTile;
+        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
+        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
+        int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
+        head = min(head, n);
+        const int nv = (int)((n - head) / 8);      // (a CTA's run never exceeds device memory / grid size elements)
+        const int64_t tail0 = head + (int64_t)nv * 8;
+
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t bad = 0;
+        float xmin = INFINITY, xmax = -INFINITY;
+        for (int64_t i = tid; i < head + (n - tail0); i += kSweepThreads) {
+            const int64_t idx = i < head ? i : tail0 + (i - head);
+            const uint32_t h = (uint32_t)__ldg(x + idx);
+            moments_careful(h, s1, s2, bad);
+            xmin = fminf(xmin, __uint_as_float(h << 16));
+            xmax = fmaxf(xmax, __uint_as_float(h << 16));
+        }
+        __nv_bfloat162 mn2 = __floats2bfloat162_rn(INFINITY, INFINITY), mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
+        // Each thread owns slot [d][tid] of every stage d: it fills them with asynchronous 16-byte copies (one
+        // commit group per vector, empty past the end so that the group count stays in step) and reads a slot
+        // back once the group that filled it has landed.
+        const uint4 *xv = reinterpret_cast<const uint4 *>(x + head) + tid;
+#pragma unroll
+        for (int d = 0; d < kSweepDepth - 1; ++d) {
+            if (tid + d * kSweepThreads < nv)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + d * kStageBytes), "l"(xv + d * kSweepThreads) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        for (int v = tid; v < nv; v += kSweepDepth * kSweepThreads) {
+#pragma unroll
+            for (int d = 0; d < kSweepDepth; ++d) {
+                const int vd = v + d * kSweepThreads;
+                if (vd < nv) {
+                    // fill the slot emptied by the previous vector (stage d - 1, cyclically)
+                    if (vd + (kSweepDepth - 1) * kSweepThreads < nv)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + ((d + kSweepDepth - 1) % kSweepDepth) * kStageBytes),
+                                     "l"(xv + (d + kSweepDepth - 1) * kSweepThreads) : "memory");
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                    asm volatile("cp.async.wait_group %0;" ::"n"(kSweepDepth - 1) : "memory");
+                    uint4 r0;
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r0.x), "=r"(r0.y), "=r"(r0.z), "=r"(r0.w) : "r"(slot0 + d * kStageBytes) : "memory");
+                    moments_vec(r0, s1, s2, bad, mn2, mx2);
+                }
+            }
+            xv += kSweepDepth * kSweepThreads;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        xmin = fminf(xmin, fminf(__low2float(mn2), __high2float(mn2)));
+        xmax = fmaxf(xmax, fmaxf(__low2float(mx2), __high2float(mx2)));
+
+        // ---- block reduction in a fixed order: butterfly inside each warp, then the warps in sequence
+        const double w1 = warp_sum(s1), w2 = warp_sum(s2);
+        const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, bad);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            xmin = fminf(xmin, __shfl_xor_sync(0xFFFFFFFFu, xmin, o));
+            xmax = fmaxf(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, o));
+        }
+        if (lane == 0) { shRed[0][warp] = w1; shRed[1][warp] = w2; shBad[warp] = wb; shMin[warp] = xmin; shMax[warp] = xmax; }
+        __syncthreads();
+        for (int tz = t + 1 + tid; tz < t_stop; tz += kSweepThreads) {
+            a.part.s1[tz] = 0.0; a.part.s2[tz] = 0.0; a.part.bad[tz] = 0u;
+            a.part.xmin[tz] = INFINITY; a.part.xmax[tz] = -INFINITY;
+        }
+        if (tid == 0) {
+            double r1 = 0.0, r2 = 0.0;
+            uint32_t rb = 0;
+            float rmin = INFINITY, rmax = -INFINITY;
+            for (int w = 0; w < kSweepWarps; ++w) {
+                r1 += shRed[0][w]; r2 += shRed[1][w]; rb += shBad[w];
+                rmin = fminf(rmin, shMin[w]); rmax = fmaxf(rmax, shMax[w]);
+            }
+            a.part.s1[t] = r1; a.part.s2[t] = r2; a.part.bad[t] = rb;
+            a.part.xmin[t] = rmin; a.part.xmax[t] = rmax;
+        }
+        __syncthreads();
+        t = t_stop;
+    }
+}
+
 template <typename TIn, typename TG>
 cudaError_t launch_typed(int flags, const StreamArgs &a, cudaStream_t st)
 {
@@ -549,6 +687,14 @@ cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, boo
     if (in_dtype == GG_F32)
         return g16 ? launch_typed<float, uint16_t>(flags, a, st) : launch_typed<float, float>(flags, a, st);
     return g16 ? launch_typed<uint16_t, uint16_t>(flags, a, st) : launch_typed<uint16_t, float>(flags, a, st);
+}
+
+cudaError_t launch_moments_bf16_sweep(const StreamArgs &a, int sm_count, cudaStream_t st)
+{
+    if (a.map.n_tiles <= 0) return cudaSuccess;
+    const int grid = (int)min((int64_t)a.map.n_tiles, (int64_t)sm_count * kSweepCtasPerSm);
+    moments_bf16_sweep_kernel<<<grid, kSweepThreads, 0, st>>>(a);
+    return cudaGetLastError();
 }
 
 }  // namespace gg
