@@ -200,7 +200,11 @@ typedef struct {
 /* The whole pass over a list of segments in the fewest sweeps of x: moments -> fit ->
  * penalty + gradient + histogram -> entropy, all enqueued on `stream`.
  * GG_PARAMS_FITTED reads x twice (the gradient needs the fit of the whole segment);
- * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep). */
+ * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep).
+ * The first call with a new layout (segment addresses and lengths) builds and caches its plan with
+ * blocking allocations; later calls with that layout only enqueue kernels and memsets on `stream`
+ * and may be captured in a CUDA graph (the same holds for gg_fused_channels once its scratch is
+ * large enough). */
 gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *args, void *stream);
 
 /* ---- code lengths: the rate the paper defines (Eq. 6-7) and its reporting metrics ------------- */

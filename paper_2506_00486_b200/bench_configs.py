@@ -46,6 +46,11 @@ def main(which):
                              step=torch.full((1,), 1e-3, dtype=torch.float32, device=dev))
         ms = timeit(run)
         print(f"c1  fused, fp32 1024x1024, one segment: {ms * 1e3:.1f} us  {8 * x.numel() / ms / 1e6:.0f} GB/s")
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            run()
+        ms = timeit(graph.replay)
+        print(f"c1  the same call replayed from a CUDA graph: {ms * 1e3:.1f} us")
     if "c2" in which:
         shapes = gg_synth.qwen05b_shapes()
         outs = [torch.empty(r * c, dtype=torch.bfloat16, device=dev) for _, r, c in shapes]

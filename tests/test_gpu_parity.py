@@ -578,3 +578,61 @@ def test_config5_weight_sweep_scaled(ctx):
     out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=w["lam"], step=steps)
     torch.cuda.synchronize()
     check_fused(out, xs, gd, w["lam"], w["hist_id"], w["n_hist"])
+
+
+def test_fused_replays_from_a_cuda_graph(ctx):
+    """After one eager call (plans and scratch exist) the fused pass only enqueues work on the caller's
+    stream, so it can be captured in a CUDA graph; a replay on new data in the same buffers gives the
+    results of a fresh call.  Long segments, many short segments and the channel-wise pass."""
+    from paper_2506_00486_b200 import Segments
+    rng = np.random.default_rng(23)
+    long_x = [gg_synth.gg_host(rng, 0.9, 0.02, 2 * TILE + 77, torch.bfloat16), gg_synth.gg_host(rng, 1.4, 0.5, 5000, torch.bfloat16)]
+    short_x = [gg_synth.gg_host(rng, 1.1, 0.1, 600, torch.bfloat16) for _ in range(70)]
+    mat = torch.stack([gg_synth.gg_host(rng, 0.8, 0.3, 96, torch.bfloat16) for _ in range(300)])      # [300, 96]
+
+    def fresh(xs):
+        return [gg_synth.gg_host(rng, 1.2, 0.05, x.numel(), torch.bfloat16).view(x.shape) for x in xs]
+
+    cases = []
+    for xs in (long_x, short_x):
+        xd = [dev(x) for x in xs]
+        gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+        steps = torch.full((len(xs),), 2.0 ** -8, dtype=torch.float32, device="cuda:0")
+        run = ctx.make_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps)
+        cases.append((run, xd, gd, xs))
+    md = dev(mat)
+    mg = torch.empty(mat.shape, dtype=torch.float32, device="cuda:0")
+    run_c = ctx.make_fused_channels(md, grad=mg, lam=1e-4, step=2.0 ** -8)
+
+    for run, *_ in cases:
+        run()
+    run_c()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for run, *_ in cases:
+            run()
+        run_c()
+    # new data in the captured buffers, then replay
+    new_sets = []
+    for run, xd, gd, xs in cases:
+        xn = fresh(xs)
+        for d, x in zip(xd, xn):
+            d.copy_(x)
+        for g in gd:
+            g.fill_(float("nan"))
+        new_sets.append(xn)
+    mat_n = fresh([mat])[0]
+    md.copy_(mat_n)
+    graph.replay()
+    torch.cuda.synchronize()
+    for (run, xd, gd, xs), xn in zip(cases, new_sets):
+        check_fused(run.outputs, xn, gd, 1e-4, list(range(len(xn))), len(xn))
+    oc = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in run_c.outputs.items()}
+    for c in (0, 31, 64, 95):
+        xo = gg_synth.to_oracle(mat_n[:, c].contiguous())
+        b, a, *_ = o.fit(xo)
+        assert_rel(oc["beta"][c].item(), b, REL_FIT, "beta")
+        _, g = o.penalty_grad(xo, oc["beta"][c].item(), oc["alpha"][c].item(), 1e-4)
+        assert_grad_close(mg[:, c].cpu().numpy(), g)
+    assert oc["hist"].sum().item() == mat.numel()
