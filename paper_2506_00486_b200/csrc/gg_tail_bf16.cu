@@ -212,7 +212,9 @@ __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, 
             // t clamped to just outside the window: the floor of the clamped value lands on a sentinel
             // row for either tail (and for nan, which the maximum replaces by the lower bound)
             const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
-            anyc = max(anyc, __float_as_uint(t) & 0x7FFFFFFFu);
+            // (one float maximum with an absolute-value operand; a nan is ignored here, which is right: it lands on
+            // a sentinel row and is not to be counted)
+            anyc = __float_as_uint(fmaxf(__uint_as_float(anyc), fabsf(t)));
             const float tc = fminf(fmaxf(t, -(float)(kSymCells / 2) - 0.5f), (float)(kSymCells / 2));
             // for |t| < 2^22 the sum lies in [2^23, 2^24) where floats are the integers: rounding down gives floor
             const uint32_t fb = __float_as_uint(__fadd_rd(tc, __uint_as_float(kMagicBits)));
@@ -234,8 +236,8 @@ __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, 
     return 0.0f;
 }
 
-// (symbol mode: some |t| >= kSymCells/2, or a nan, whose bits are larger still; the exact test is
-// redone per element by fix_elem)
+// (symbol mode: some |t| >= kSymCells/2, compared as bit patterns of non-negative floats; the exact
+// test is redone per element by fix_elem)
 template <int MODE>
 __device__ __forceinline__ bool count_miss(uint32_t anyc)
 {
