@@ -281,25 +281,6 @@ struct TailSmem {
     ChanConst cc;
 };
 
-// 2^t for |t| < 1000 within 1e-11 relative: table entries are rounded to fp32 afterwards.
-__device__ __forceinline__ double exp2_short(double t)
-{
-    const double n = rint(t);
-    const double f = (t - n) * 0.69314718055994531;      // |f| <= 0.3466
-    double p = 1.0 / 3628800.0;                           // Taylor series of e^f to degree 10
-    p = fma(p, f, 1.0 / 362880.0);
-    p = fma(p, f, 1.0 / 40320.0);
-    p = fma(p, f, 1.0 / 5040.0);
-    p = fma(p, f, 1.0 / 720.0);
-    p = fma(p, f, 1.0 / 120.0);
-    p = fma(p, f, 1.0 / 24.0);
-    p = fma(p, f, 1.0 / 6.0);
-    p = fma(p, f, 0.5);
-    p = fma(p, f, 1.0);
-    p = fma(p, f, 1.0);
-    return p * __hiloint2double(((int)n + 1023) << 20, 0);
-}
-
 // Exact gradient magnitude (with lambda's sign through `flip`) of a 15-bit magnitude pattern.
 __device__ __noinline__ float chan_grad_exact(uint32_t mag, double L, double b, uint32_t flip)
 {

@@ -1,5 +1,5 @@
-// Moment-ratio inversion from a table (shared by the per-segment fit kernel and the short-segment
-// kernel).
+// Moment-ratio inversion from a table (shared by the per-segment fit kernels and the short-segment
+// kernel), and the short exponential the gradient tables are built with.
 //
 // The table holds, on kSeedCells cells of a uniform grid of u = ln(beta) over
 // [ln GG_BETA_LO, ln GG_BETA_HI], the two smooth functions the fit needs:
@@ -81,6 +81,25 @@ __device__ __forceinline__ uint32_t fit_from_sums(double s1, double s2, int64_t 
     }
     *alpha = sqrt(m2) * exp(lnz);
     return flags;
+}
+
+// 2^t for |t| < 1000 within 1e-11 relative: table entries are rounded to fp32 afterwards.
+__device__ __forceinline__ double exp2_short(double t)
+{
+    const double n = rint(t);
+    const double f = (t - n) * 0.69314718055994531;      // |f| <= 0.3466
+    double p = 1.0 / 3628800.0;                           // Taylor series of e^f to degree 10
+    p = fma(p, f, 1.0 / 362880.0);
+    p = fma(p, f, 1.0 / 40320.0);
+    p = fma(p, f, 1.0 / 5040.0);
+    p = fma(p, f, 1.0 / 720.0);
+    p = fma(p, f, 1.0 / 120.0);
+    p = fma(p, f, 1.0 / 24.0);
+    p = fma(p, f, 1.0 / 6.0);
+    p = fma(p, f, 0.5);
+    p = fma(p, f, 1.0);
+    p = fma(p, f, 1.0);
+    return p * __hiloint2double(((int)n + 1023) << 20, 0);
 }
 
 }  // namespace gg

@@ -504,12 +504,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                     // number; the same bound on L + beta (e-127) keeps the penalty terms |x| |g| normal too
                     const double de = (double)(e - 127);
                     const double e0 = k.L + k.b * de;
-                    if (fabs(e0) <= 100.0 && fabs(e0 + de) <= 100.0) v = (float)(lam < 0.0 ? -exp2(e0) : exp2(e0));
+                    if (fabs(e0) <= 100.0 && fabs(e0 + de) <= 100.0) v = (float)(lam < 0.0 ? -exp2_short(e0) : exp2_short(e0));
                 }
                 tab.a1[e] = v;
             }
 #pragma unroll
-            for (int j = lane; j < 128; j += 32) tab.B[j] = k.active ? (float)exp2(k.b * sm.log2m[j]) : 1.0f;
+            for (int j = lane; j < 128; j += 32) tab.B[j] = k.active ? (float)exp2_short(k.b * sm.log2m[j]) : 1.0f;
             __syncwarp();
         }
         if constexpr (HIST) {
