@@ -692,7 +692,7 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         // scratch: doubles first, then the 32-bit arrays
         const size_t nc = (size_t)a->cols, nm = (size_t)n_mom * nc, ns = (size_t)ka.n_slices * nc;
         const size_t n_strips = (nc + kChanStrip - 1) / kChanStrip;
-        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + nc + n_strips * (kChanTabFloats + 1) + 8;
+        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + 2 * nc + n_strips * (kChanTabFloats + 1) + 8;
         void *buf = ctx->chan_buf;
         gg_status st = grow(ctx, &buf, &ctx->chan_bytes, (int64_t)(n_dbl * 8 + n_w32 * 4));
         ctx->chan_buf = buf;
@@ -704,9 +704,10 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         ka.xmin = reinterpret_cast<float *>(w + nm);
         ka.xmax = reinterpret_cast<float *>(w + 2 * nm);
         ka.amax = reinterpret_cast<float *>(w + 3 * nm);
-        ka.tab_elo = reinterpret_cast<int32_t *>(w + 3 * nm + nc);
+        ka.sd = reinterpret_cast<float *>(w + 3 * nm + nc);
+        ka.tab_elo = reinterpret_cast<int32_t *>(w + 3 * nm + 2 * nc);
         // (the tables are copied as 16-byte vectors: n_dbl * 8 is a multiple of 16 only if n_dbl is even)
-        ka.tab = reinterpret_cast<float *>(w + (3 * nm + nc + n_strips + 3) / 4 * 4 + (n_dbl & 1) * 2);
+        ka.tab = reinterpret_cast<float *>(w + (3 * nm + 2 * nc + n_strips + 3) / 4 * 4 + (n_dbl & 1) * 2);
         ka.beta = a->beta; ka.alpha = a->alpha; ka.sum_abs = a->sum_abs; ka.sum_sq = a->sum_sq;
         ka.count = a->count; ka.flags = a->flags; ka.penalty = a->penalty;
         ka.seed = ctx->seed;

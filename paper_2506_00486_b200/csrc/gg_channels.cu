@@ -23,6 +23,8 @@
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include <type_traits>
+
 #include "gg_fit_table.cuh"
 #include "gg_internal.h"
 
@@ -39,6 +41,13 @@ constexpr int kCtasPerSm = 2;
 constexpr int kAWin = 64;                  // exponents covered by the A table (row kAWin: the marker)
 constexpr int kSymWin = 4096;              // symbols counted in shared memory: [-2048, 2048) cut to [qmin, qmax]
 constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
+// Pattern counting (used when symbols of a strip would miss the symbol window): one cell per bf16
+// magnitude pattern and sign over the 16 binades up to the strip's largest magnitude, one cell for zero.
+constexpr int kSlowWin = 512;
+constexpr uint32_t kPatCells = 16 * 128;       // magnitude patterns in the window: cell pairs 0 .. kPatCells - 1
+constexpr uint32_t kPatZero = kPatCells;       // the cell pair of +-0
+constexpr uint32_t kPatSentinel = kPatCells + 1;
+static_assert((kPatSentinel + 1) * 2 <= kSymWin + 4, "the pattern cells share the symbol cells' array");
 
 // The 32-bit word of columns (2 lane, 2 lane + 1) of one row; missing columns read as zero.
 __device__ __forceinline__ uint32_t load_pair(const uint16_t *row, bool vec, bool ok0, bool ok1)
@@ -244,6 +253,9 @@ __global__ void __launch_bounds__(kFitCols * kFitGroups) chan_fit_kernel(const C
         am = fmaxf(lo <= FLT_MAX ? lo : FLT_MAX, hi <= FLT_MAX ? hi : FLT_MAX);
     }
     a.amax[c] = am;
+    // the standard deviation decides how the second kernel counts this column's strip
+    const double sd = a.rows > 0 ? sqrt(s2 / (double)a.rows) : 0.0;
+    a.sd[c] = sd <= (double)FLT_MAX ? (float)sd : FLT_MAX;
 }
 
 __global__ void __launch_bounds__(128) chan_penalty_kernel(const ChanArgs a)
@@ -274,10 +286,13 @@ struct TailSmem {
     uint32_t ring[2][kU][kTailThreads];   // per-thread slots of the rows in flight: two blocks of kU rows
     float a1[2][kAWin + 1][32];       // [k][e - e_lo][lane]: A of column 2 lane + k; row kAWin: the marker
     float bt[2][128][32];             // [k][j][lane]: B of column 2 lane + k
-    uint32_t cnt[kSymWin + 2];        // cell 0 and the last: sentinels of the two tails
+    uint32_t cnt[kSymWin + 4];        // symbol counting: cell 0 and cell whi - wlo + 1 are the sentinels of the two tails;
+                                      // pattern counting: word (p * 2 + sign), p < kPatCells: the window's patterns, p = kPatZero: zero, p = kPatSentinel: the sentinel
     double red[kTailWarps][kChanStrip];
     double colL[kChanStrip], colb[kChanStrip];
+    uint32_t win[kSlowWin];           // pattern counting: symbols [-kSlowWin/2, kSlowWin/2) of the slow path
     uint32_t clampc[2];
+    int amax_bits, sd_bits;           // largest finite magnitude and largest standard deviation of the current strip's columns (bits of floats)
     ChanConst cc;
 };
 
@@ -307,7 +322,9 @@ __device__ __noinline__ void chan_count_slow(float x, float inv, int32_t qmin, i
         int q = __float2int_rd(t);                 // floor, saturating
         if (q < qmin) { q = qmin; atomicAdd(&sm.clampc[0], 1u); }
         else if (q > qmax) { q = qmax; atomicAdd(&sm.clampc[1], 1u); }
+        // wlo < whi: symbol counting, whose cells the slow path may use; else the small window of its own
         if (q >= wlo && q < whi) atomicAdd(&sm.cnt[q - wlo + 1], 1u);
+        else if (wlo >= whi && (uint32_t)(q + kSlowWin / 2) < (uint32_t)kSlowWin) atomicAdd(&sm.win[q + kSlowWin / 2], 1u);
         else atomicAdd(&hist[q - qmin], 1ull);
     }
 }
@@ -365,7 +382,8 @@ __global__ void __launch_bounds__(kTailThreads) chan_tables_kernel(const ChanArg
 struct ChanLane {
     uint32_t a_addr, b_addr;         // shared-memory addresses of this lane's word in row 0 of its first tables
     uint32_t e_lo;                   // exponent field of row 0 of the A tables
-    uint32_t cnt_off;                // cell of a value = bits(floor(t) + magic) * 4 + cnt_off (mod 2^32)
+    uint32_t cnt_off;                // symbol counting: cell of a value = bits(floor(t) + magic) * 4 + cnt_off (mod 2^32)
+    uint32_t cnt_addr, cbase;        // pattern counting: address of cnt, first magnitude pattern of the window
     float inv, t_lo, t_hi;           // quantiser scale; t is clamped to [t_lo, t_hi] so that its floor is a cell
     float near;                      // a smaller |t| lies inside the count window for sure
 };
@@ -389,7 +407,7 @@ __device__ __forceinline__ float lds_b(const ChanLane &ln, uint32_t j)
 }
 
 // One element (HALF 0: the low half of w, the lane's even column).  Branch free.
-template <bool GRAD, bool HIST, int HALF>
+template <bool GRAD, bool HIST, bool PAT, int HALF>
 __device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanLane &ln, float &mp, float &anyc)
 {
     const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);
@@ -404,7 +422,17 @@ __device__ __forceinline__ float chan_elem(uint32_t w, bool counted, const ChanL
         g = __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
     }
     if constexpr (HIST) {
-        if (counted) {
+        if (counted && PAT) {
+            // by bit pattern: anyc keeps the largest window index (as the bits of a float, whose order they share)
+            const uint32_t mag = HALF ? (w >> 16) & 0x7FFFu : w & 0x7FFFu;
+            // (below the window the difference wraps around to the sentinel too; the window is placed so that no
+            // element has the pattern cbase + kPatCells, which would fall on the zero cell)
+            uint32_t pc = min(mag - ln.cbase, kPatSentinel);
+            pc = mag == 0u ? kPatZero : pc;
+            anyc = __uint_as_float(max(__float_as_uint(anyc), pc));
+            const uint32_t sign4 = HALF ? (w >> 29) & 4u : (w >> 13) & 4u;
+            red_inc(ln.cnt_addr + pc * 8u + sign4);
+        } else if (counted) {
             const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
             anyc = fmaxf(anyc, fabsf(t));      // (a nan is ignored here and lands on a sentinel: nan is not counted)
             // outside the window (and nan, which fmaxf replaces by the lower bound) the floor lands on a sentinel
@@ -483,8 +511,8 @@ __device__ __forceinline__ double chan_column_exact(const ChanLane &ln, const Ta
 }
 
 // Elements of a block whose count may have gone to a sentinel: exact test, slow count.
-template <typename WordOf, typename Counted>
-__device__ __forceinline__ void chan_recount(TailSmem &sm, WordOf word_of, Counted counted)
+template <bool PAT, typename WordOf, typename Counted>
+__device__ __forceinline__ void chan_recount(TailSmem &sm, uint32_t cbase, WordOf word_of, Counted counted)
 {
     const float inv = sm.cc.inv;
     const int32_t wlo = sm.cc.wlo, whi = sm.cc.whi;
@@ -495,8 +523,15 @@ __device__ __forceinline__ void chan_recount(TailSmem &sm, WordOf word_of, Count
             const uint32_t w = word_of(u);
             const float x = __uint_as_float(k ? (w & 0xFFFF0000u) : (w << 16));
             const float t = __fmul_rn(x, inv);
-            if (counted(u, k) && !(t >= (float)wlo && t < (float)whi))
-                chan_count_slow(x, inv, sm.cc.qmin, sm.cc.qmax, wlo, whi, sm, sm.cc.hist);
+            bool miss;
+            if constexpr (PAT) {
+                const uint32_t mag = (k ? (w >> 16) : w) & 0x7FFFu;
+                miss = mag != 0u && mag - cbase >= kPatCells;
+            } else {
+                miss = !(t >= (float)wlo && t < (float)whi);
+            }
+            // (the slow count may only use the shared cells in symbol counting: wlo = whi switches that off)
+            if (counted(u, k) && miss) chan_count_slow(x, inv, sm.cc.qmin, sm.cc.qmax, PAT ? 0 : wlo, PAT ? 0 : whi, sm, sm.cc.hist);
         }
     }
 }
@@ -505,7 +540,7 @@ __device__ __forceinline__ void chan_recount(TailSmem &sm, WordOf word_of, Count
 // at wbase + u * kRowBytes).  The gradient pair of a row is written as soon as it is known; an element
 // the tables could not serve is written again, alone, by the exact path.
 constexpr uint32_t kRowBytes = kTailThreads * 4u;
-template <typename TG, bool GRAD, bool HIST>
+template <typename TG, bool GRAD, bool HIST, bool PAT>
 __device__ __forceinline__ void chan_block_fast(uint32_t wbase, TG *gp, int64_t sg, int lane, const ChanLane &ln, TailSmem &sm,
                                                 double (&pen)[2])
 {
@@ -519,8 +554,8 @@ __device__ __forceinline__ void chan_block_fast(uint32_t wbase, TG *gp, int64_t 
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
         const uint32_t w = word_of(u);
-        const float g0 = chan_elem<GRAD, HIST, 0>(w, true, ln, mp[0], anyc);
-        const float g1 = chan_elem<GRAD, HIST, 1>(w, true, ln, mp[1], anyc);
+        const float g0 = chan_elem<GRAD, HIST, PAT, 0>(w, true, ln, mp[0], anyc);
+        const float g1 = chan_elem<GRAD, HIST, PAT, 1>(w, true, ln, mp[1], anyc);
         if constexpr (GRAD) {
             if (gp != nullptr) store_pair<TG>(gp + u * sg, g0, g1, true, true, true, false);
         }
@@ -532,8 +567,54 @@ __device__ __forceinline__ void chan_block_fast(uint32_t wbase, TG *gp, int64_t 
         else pen[1] += chan_column_exact<1>(ln, sm, lane, word_of, [&](int u, float g) { if (gp != nullptr) store_one<TG>(gp + u * sg + 1, g); });
     }
     if constexpr (HIST) {
-        if (anyc >= ln.near) chan_recount(sm, word_of, [](int, int) { return true; });
+        if (PAT ? __float_as_uint(anyc) >= kPatSentinel : anyc >= ln.near) chan_recount<PAT>(sm, ln.cbase, word_of, [](int, int) { return true; });
     }
+}
+
+// Adds the counted cells to the histogram and empties them (all threads; the caller has synchronised, so
+// all counting under the current layout is complete).  Symbol cells hold symbols wlo .. whi - 1, which the
+// clamp leaves alone; pattern cells are quantised here, one pattern at a time.
+__device__ void chan_flush(TailSmem &sm, bool pat, uint32_t cbase, const ChanArgs &a)
+{
+    unsigned long long *hist = sm.cc.hist;
+    if (pat) {
+        for (uint32_t i = threadIdx.x; i < (kPatSentinel + 1) * 2; i += kTailThreads) {
+            // (every CTA starts at another cell: CTAs that flush together do not walk the bins in step)
+            const uint32_t cw = (i + blockIdx.x * 61u) % ((kPatSentinel + 1) * 2);
+            const uint32_t n = sm.cnt[cw];
+            if (n == 0u) continue;
+            sm.cnt[cw] = 0u;
+            const uint32_t pc = cw >> 1;
+            if (pc == kPatSentinel) continue;          // counted again, one by one, by the slow path
+            const uint32_t h = (pc == kPatZero ? 0u : cbase + pc) | ((cw & 1u) << 15);
+            const float t = __fmul_rn(__uint_as_float(h << 16), sm.cc.inv);
+            if (!(t == t)) continue;                   // (a window that reaches the top binade holds the nan patterns: not counted)
+            int q = __float2int_rd(t);                 // floor, saturating
+            if (q < sm.cc.qmin) { q = sm.cc.qmin; atomicAdd(&sm.clampc[0], n); }
+            else if (q > sm.cc.qmax) { q = sm.cc.qmax; atomicAdd(&sm.clampc[1], n); }
+            // many patterns below the step share the symbols around zero: those meet in the small window first
+            if ((uint32_t)(q + kSlowWin / 2) < (uint32_t)kSlowWin) atomicAdd(&sm.win[q + kSlowWin / 2], n);
+            else atomicAdd(&hist[q - sm.cc.qmin], (unsigned long long)n);
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < kSlowWin; i += kTailThreads) {      // (its symbols are already clamped)
+            const uint32_t n = sm.win[i];
+            if (n != 0u) {
+                sm.win[i] = 0u;
+                atomicAdd(&hist[(i - kSlowWin / 2) - sm.cc.qmin], (unsigned long long)n);
+            }
+        }
+    } else {
+        const int wlo = sm.cc.wlo, n_cells = sm.cc.whi - sm.cc.wlo;
+        for (int i = threadIdx.x; i < n_cells + 2; i += kTailThreads) {
+            const int cidx = (int)(((uint32_t)i + blockIdx.x * 61u) % (uint32_t)(n_cells + 2));
+            const uint32_t n = sm.cnt[cidx];
+            if (n == 0u) continue;
+            sm.cnt[cidx] = 0u;
+            if (cidx >= 1 && cidx <= n_cells) atomicAdd(&hist[(wlo + cidx - 1) - a.qmin], (unsigned long long)n);
+        }
+    }
+    __syncthreads();
 }
 
 // Up to kU rows with every guard (ragged blocks, the last strip, unaligned rows, accumulation), as a
@@ -541,7 +622,7 @@ __device__ __forceinline__ void chan_block_fast(uint32_t wbase, TG *gp, int64_t 
 // missing columns read as zero and are not counted, and the gradients wait in registers until the
 // exact path has run (they may have to be added to what is stored).  Returns the two penalty
 // contributions.
-template <typename TG, bool GRAD, bool HIST>
+template <typename TG, bool GRAD, bool HIST, bool PAT>
 __device__ __noinline__ double2 chan_block_guarded(const uint16_t *p, int64_t sin, TG *gp, int64_t sg, int nvalid, bool ok0,
                                                    bool ok1, bool vec_in, bool vec_out, bool accumulate, int lane, ChanLane ln,
                                                    TailSmem *smp)
@@ -556,8 +637,8 @@ __device__ __noinline__ double2 chan_block_guarded(const uint16_t *p, int64_t si
     float anyc = 0.0f;
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-        g[u][0] = chan_elem<GRAD, HIST, 0>(w[u], ok0 && u < nvalid, ln, mp[0], anyc);
-        g[u][1] = chan_elem<GRAD, HIST, 1>(w[u], ok1 && u < nvalid, ln, mp[1], anyc);
+        g[u][0] = chan_elem<GRAD, HIST, PAT, 0>(w[u], ok0 && u < nvalid, ln, mp[0], anyc);
+        g[u][1] = chan_elem<GRAD, HIST, PAT, 1>(w[u], ok1 && u < nvalid, ln, mp[1], anyc);
     }
     double2 pen = make_double2(0.0, 0.0);
     if constexpr (GRAD) {
@@ -567,7 +648,8 @@ __device__ __noinline__ double2 chan_block_guarded(const uint16_t *p, int64_t si
         else pen.y = chan_column_exact<1>(ln, sm, lane, word_of, [&](int u, float ge) { g[u][1] = ge; });
     }
     if constexpr (HIST) {
-        if (anyc >= ln.near) chan_recount(sm, word_of, [&](int u, int k) { return u < nvalid && (k ? ok1 : ok0); });
+        if (PAT ? __float_as_uint(anyc) >= kPatSentinel : anyc >= ln.near)
+            chan_recount<PAT>(sm, ln.cbase, word_of, [&](int u, int k) { return u < nvalid && (k ? ok1 : ok0); });
     }
     if constexpr (GRAD) {
         if (gp != nullptr) {
@@ -609,9 +691,12 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
     ln.near = (wlo < 0 && whi > 0) ? (float)min(-wlo, whi) : 0.0f;
     // floor(tc) lies in [wlo - 1, whi]; cell = floor(tc) - (wlo - 1)
     ln.cnt_off = (uint32_t)__cvta_generic_to_shared(sm.cnt) - (kMagicBits + (uint32_t)(wlo - 1)) * 4u;
+    ln.cnt_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt);
+    ln.cbase = 0x8000u;
 
     if constexpr (HIST) {
-        for (int i = tid; i < kSymWin + 2; i += kTailThreads) sm.cnt[i] = 0u;
+        for (int i = tid; i < kSymWin + 4; i += kTailThreads) sm.cnt[i] = 0u;
+        for (int i = tid; i < kSlowWin; i += kTailThreads) sm.win[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
     const bool vec_in = ((reinterpret_cast<uintptr_t>(a.x) & 3u) == 0) && ((a.ld & 1) == 0) && ((a.cols & 1) == 0);
@@ -620,6 +705,7 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
     const bool accumulate = a.accumulate != 0;
     const uint32_t ring = (uint32_t)__cvta_generic_to_shared(&sm.ring[0][0][tid]);
     int cur_strip = -1;
+    bool sym_pending = false;      // symbol cells hold counts that are not in the histogram yet
     __syncthreads();
 
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -650,42 +736,80 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
             __syncthreads();
         }
 
+        // ---- how this item counts: by symbol if the symbol window holds the bulk of the strip's symbols, else by
+        // bit pattern over the 16 binades up to the strip's largest magnitude (quantised when flushed)
+        bool pat = false;
+        if constexpr (HIST) {
+            __syncthreads();
+            if (tid == 0) { sm.amax_bits = 0; sm.sd_bits = 0; }
+            __syncthreads();
+            if (tid < kChanStrip && (int64_t)strip * kChanStrip + tid < a.cols) {
+                atomicMax(&sm.amax_bits, (int)__float_as_uint(a.amax[(int64_t)strip * kChanStrip + tid]));
+                atomicMax(&sm.sd_bits, (int)__float_as_uint(a.sd[(int64_t)strip * kChanStrip + tid]));
+            }
+            __syncthreads();
+            // by symbol while the window reaches 6.5 standard deviations of the widest column (the few symbols
+            // beyond are counted one by one)
+            pat = !(6.5f * __int_as_float(sm.sd_bits) * inv < ln.near);
+            if (pat) {
+                if (sym_pending) { chan_flush(sm, false, 0u, a); sym_pending = false; }
+                // 16 binades ending one above that of the largest magnitude (that last one is empty, so no element
+                // has the first pattern after the window), or ending at the top binade of the format
+                const int e_top = sm.amax_bits >> 23;
+                const int e_hi = e_top >= 253 ? 255 : max(16, e_top + 1);
+                ln.cbase = (uint32_t)(e_hi - 15) << 7;
+            } else {
+                sym_pending = true;
+            }
+        }
+
         // ---- stream the rows of the slice: warp w takes rows r_begin + w, + kTailWarps, ...
         double pen[2] = {0.0, 0.0};
-        const int64_t r0 = r_begin + warp;
-        int n_mine = r0 < r_end ? (int)((r_end - r0 + kTailWarps - 1) / kTailWarps) : 0;      // rows of this warp
-        const int64_t sin = (int64_t)kTailWarps * a.ld, sg = (int64_t)kTailWarps * a.grad_ld;
-        const uint16_t *p = a.x + c0 + r0 * a.ld;
-        TG *gp = GRAD && a.grad != nullptr ? reinterpret_cast<TG *>(a.grad) + c0 + r0 * a.grad_ld : nullptr;
-        // Whole blocks of a whole strip with aligned rows: each thread stages its words of the next block
-        // in its own ring slots with asynchronous copies while it works on the current one (one commit
-        // group per block, so the group that must have landed is always the one before the last).
-        if ((int64_t)strip * kChanStrip + kChanStrip <= a.cols && vec_in && (gp == nullptr || vec_out) && !accumulate) {
-            const int n_blocks = n_mine / kU;
-            auto stage = [&](const uint16_t *src, uint32_t dst) {
+        auto stream_item = [&](auto pat_tag) {
+            constexpr bool PAT = decltype(pat_tag)::value;
+            const int64_t r0 = r_begin + warp;
+            int n_mine = r0 < r_end ? (int)((r_end - r0 + kTailWarps - 1) / kTailWarps) : 0;      // rows of this warp
+            const int64_t sin = (int64_t)kTailWarps * a.ld, sg = (int64_t)kTailWarps * a.grad_ld;
+            const uint16_t *p = a.x + c0 + r0 * a.ld;
+            TG *gp = GRAD && a.grad != nullptr ? reinterpret_cast<TG *>(a.grad) + c0 + r0 * a.grad_ld : nullptr;
+            // Whole blocks of a whole strip with aligned rows: each thread stages its words of the next block
+            // in its own ring slots with asynchronous copies while it works on the current one (one commit
+            // group per block, so the group that must have landed is always the one before the last).
+            if ((int64_t)strip * kChanStrip + kChanStrip <= a.cols && vec_in && (gp == nullptr || vec_out) && !accumulate) {
+                const int n_blocks = n_mine / kU;
+                auto stage = [&](const uint16_t *src, uint32_t dst) {
 #pragma unroll
-                for (int u = 0; u < kU; ++u)
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)u * kRowBytes), "l"(src + u * sin) : "memory");
-            };
-            if (n_blocks > 0) stage(p, ring);
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            for (int bk = 0; bk < n_blocks; ++bk) {
-                const uint32_t cur = ring + (uint32_t)(bk & 1) * kU * kRowBytes;
-                if (bk + 1 < n_blocks) stage(p + kU * sin, ring + (uint32_t)((bk + 1) & 1) * kU * kRowBytes);
+                    for (int u = 0; u < kU; ++u)
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)u * kRowBytes), "l"(src + u * sin) : "memory");
+                };
+                if (n_blocks > 0) stage(p, ring);
                 asm volatile("cp.async.commit_group;" ::: "memory");
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
-                chan_block_fast<TG, GRAD, HIST>(cur, gp, sg, lane, ln, sm, pen);
-                p += kU * sin;
-                if (gp != nullptr) gp += kU * sg;
+                for (int bk = 0; bk < n_blocks; ++bk) {
+                    const uint32_t cur = ring + (uint32_t)(bk & 1) * kU * kRowBytes;
+                    if (bk + 1 < n_blocks) stage(p + kU * sin, ring + (uint32_t)((bk + 1) & 1) * kU * kRowBytes);
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                    asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    chan_block_fast<TG, GRAD, HIST, PAT>(cur, gp, sg, lane, ln, sm, pen);
+                    p += kU * sin;
+                    if (gp != nullptr) gp += kU * sg;
+                }
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                n_mine -= n_blocks * kU;
             }
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            n_mine -= n_blocks * kU;
-        }
-        for (; n_mine > 0; n_mine -= kU, p += kU * sin, gp += gp != nullptr ? kU * sg : 0) {
-            const double2 d = chan_block_guarded<TG, GRAD, HIST>(p, sin, gp, sg, min(n_mine, kU), ok0, ok1, vec_in, vec_out,
-                                                                 accumulate, lane, ln, &sm);
-            pen[0] += d.x;
-            pen[1] += d.y;
+            for (; n_mine > 0; n_mine -= kU, p += kU * sin, gp += gp != nullptr ? kU * sg : 0) {
+                const double2 d = chan_block_guarded<TG, GRAD, HIST, PAT>(p, sin, gp, sg, min(n_mine, kU), ok0, ok1, vec_in,
+                                                                          vec_out, accumulate, lane, ln, &sm);
+                pen[0] += d.x;
+                pen[1] += d.y;
+            }
+        };
+        if (HIST && pat) stream_item(std::true_type{});
+        else stream_item(std::false_type{});
+        if constexpr (HIST) {
+            if (pat) {           // the window moves with the strip: empty it now
+                __syncthreads();
+                chan_flush(sm, true, ln.cbase, a);
+            }
         }
 
         if constexpr (GRAD) {
@@ -707,14 +831,7 @@ __global__ void __launch_bounds__(kTailThreads, kCtasPerSm) chan_tail_kernel(con
 
     if constexpr (HIST) {
         __syncthreads();
-        unsigned long long *hist = reinterpret_cast<unsigned long long *>(a.hist);
-        const int n_cells = whi - wlo;
-        for (int i = tid; i < n_cells; i += kTailThreads) {
-            // (every CTA starts at another cell: CTAs that finish together do not walk the bins in step)
-            const int cidx = (int)(((uint32_t)i + blockIdx.x * 61u) % (uint32_t)n_cells);
-            const uint32_t n = sm.cnt[cidx + 1];
-            if (n != 0u) atomicAdd(&hist[(wlo + cidx) - a.qmin], (unsigned long long)n);
-        }
+        if (sym_pending) chan_flush(sm, false, 0u, a);
         if (tid < 2 && a.clamped != nullptr && sm.clampc[tid] != 0u)
             atomicAdd(reinterpret_cast<unsigned long long *>(a.clamped) + tid, (unsigned long long)sm.clampc[tid]);
     }

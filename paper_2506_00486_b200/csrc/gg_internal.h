@@ -142,6 +142,7 @@ struct ChanArgs {
     float *xmin, *xmax;
     double *L, *b;                     // [cols]: |g| = 2^(L + b log2|x|); L is NaN for a column without gradient
     float *amax;                       // [cols] largest finite magnitude
+    float *sd;                         // [cols] standard deviation
     double *pen;                       // [n_slices * cols] partial sums of |x| |g|
     float *tab;                        // [strips * kChanTabFloats] gradient tables of every strip
     int32_t *tab_elo;                  // [strips] exponent field of the first row of a strip's A table
