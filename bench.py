@@ -33,6 +33,8 @@ def parse():
                     help="divide every matrix dimension of the sweep (debugging; 1 = the full workload)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--single-read-steps", type=int, default=20,
+                    help="timed steps of the one-read form of the pass (parameters given), 0 to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"])
     return ap.parse_args()
@@ -287,6 +289,29 @@ def run_ours(args):
                                 "achieved": in_bytes / (first_ms * 1e-3) / 1e9 if first_ms > 0 else None,
                                 "frac": in_bytes / (first_ms * 1e-3) / 1e9 / peak if first_ms > 0 else None}}
 
+    # ---- the one-read form of the same pass (secondary figure): the parameters of the step before (here:
+    # those just fitted) drive penalty and gradient while the new fit is made in the same sweep
+    single = None
+    if args.single_read_steps > 0:
+        from paper_2506_00486_b200 import GG_PARAMS_GIVEN
+        run1 = ctx.make_fused(segs, grad=gsegs, lam=LAM, step=steps_t, param_mode=GG_PARAMS_GIVEN,
+                              beta_in=out["beta"].clone(), alpha_in=out["alpha"].clone(), hist=out["hist"])
+        for _ in range(3):
+            run1()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.single_read_steps):
+            run1()
+        e1.record()
+        barrier()
+        ms1 = max_over_ranks(e0.elapsed_time(e1) / args.single_read_steps, world, dev)
+        v1 = whole_job_gbs(world, alg_bytes, ms1)
+        single = {"value": v1, "unit": UNIT, "ms_per_step": ms1, "steps": args.single_read_steps,
+                  "params": "given (those of the previous step); moments, fit, gradient and histogram in one sweep",
+                  "of_measured_copy_peak": v1 / world / peak}
+        del run1
+
     # ---- end to end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -311,7 +336,8 @@ def run_ours(args):
                        "histograms": n_seg, "bins": 65536, "step": STEP, "lambda": LAM, "params": "fitted in the same call",
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world} (segments are independent)"},
             "fraction_of_hbm_peak": {"of_measured_copy_peak": value / world / peak, "of_nominal_8TBs": value / world / 8000.0},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "single_read": single,
+            "gpu_launches": int(launches),
             "clocks": clocks,
             "check": {"max_abs_beta_error_vs_generating": beta_err, "histogram_total": total_counts,
                       "elements": n_elem},

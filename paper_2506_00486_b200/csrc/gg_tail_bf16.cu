@@ -149,7 +149,9 @@ __device__ __noinline__ void count_rare(uint32_t xb, Smem &sm) { count_symbol(__
 struct Acc {
     double s1 = 0.0, s2 = 0.0, pen = 0.0;
     uint32_t bad = 0;
-    float xmin = INFINITY, xmax = -INFINITY;
+    float xmin = INFINITY, xmax = -INFINITY;     // extremes of the elements taken one by one
+    // extremes of the elements taken as vectors: two bf16 lanes (even and odd elements)
+    __nv_bfloat162 mn2 = __floats2bfloat162_rn(INFINITY, INFINITY), mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
 };
 
 struct Run {   // fp32 partials of one short run of elements
@@ -195,11 +197,11 @@ __device__ __forceinline__ uint32_t symbol_row(uint32_t xb, float inv)
 // the vector's penalty partial NaN, which the caller checks once per vector.  Count: `anyc` keeps
 // the largest |x * inv| (symbol mode) or window index (pattern mode) so that one compare per
 // vector finds elements that missed the window; those count in the sentinel cells.
-template <int FLAGS, int MODE, int HALF>
+template <int FLAGS, int MODE, int HALF, bool MOMENTS_HERE = true>
 __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, Run &r, uint32_t &anyc)
 {
     const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);     // the value as fp32 bits
-    moments_elem<FLAGS>(xb, acc, r);
+    if constexpr (MOMENTS_HERE) moments_elem<FLAGS>(xb, acc, r);
     float ga = 0.0f;
     if constexpr ((FLAGS & kGrad) != 0) {
         const uint32_t e4 = HALF ? ((w >> 21) & 0x3FCu) : ((w >> 5) & 0x3FCu);     // exponent field * 4
@@ -298,6 +300,8 @@ __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &
                     const double ax = (double)__uint_as_float(h << 16);
                     acc.s1 += ax;
                     acc.s2 += ax * ax;
+                } else {
+                    acc.bad += 1u;     // (elements taken one by one never get here with an inf or nan: they count it themselves)
                 }
             }
         }
@@ -429,7 +433,8 @@ __device__ void reduce_partials(const TileScratch &part, int t0, int t1, const A
     if constexpr ((FLAGS & kMoments) != 0) {
         const double w1 = warp_sum(acc.s1), w2 = warp_sum(acc.s2);
         const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, acc.bad);
-        float wmin = acc.xmin, wmax = acc.xmax;
+        float wmin = fminf(acc.xmin, fminf(__low2float(acc.mn2), __high2float(acc.mn2)));
+        float wmax = fmaxf(acc.xmax, fmaxf(__low2float(acc.mx2), __high2float(acc.mx2)));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             wmin = fminf(wmin, __shfl_xor_sync(0xFFFFFFFFu, wmin, o));
@@ -479,8 +484,20 @@ __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool acc
     uint32_t anyc = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        g[2 * i] = one_elem<FLAGS, MODE, 0>(w[i], ln, acc, r, anyc);
-        g[2 * i + 1] = one_elem<FLAGS, MODE, 1>(w[i], ln, acc, r, anyc);
+        if constexpr ((FLAGS & kMoments) != 0) {
+            // both elements of the word at once; an inf or nan makes the run's sums inf or nan, and the run is
+            // then summed again element by element (close_run), where it is counted and left out
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+            r.m1 += fabsf(lo);
+            r.m1 += fabsf(hi);
+            r.m2 = fmaf(lo, lo, r.m2);
+            r.m2 = fmaf(hi, hi, r.m2);
+            const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[i]);
+            acc.mn2 = __hmin2(acc.mn2, pr);      // return the non-NaN operand, like fminf
+            acc.mx2 = __hmax2(acc.mx2, pr);
+        }
+        g[2 * i] = one_elem<FLAGS, MODE, 0, false>(w[i], ln, acc, r, anyc);
+        g[2 * i + 1] = one_elem<FLAGS, MODE, 1, false>(w[i], ln, acc, r, anyc);
     }
     const bool grad_bad = GRAD && !(r.mp <= FLT_MAX);
     if (grad_bad || (HIST && count_miss<MODE>(anyc))) {
