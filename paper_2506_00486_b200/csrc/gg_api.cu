@@ -23,7 +23,11 @@ constexpr int64_t kDefaultChunkBytes = 1ll << 30;
 // A plan is everything that depends only on the layout of a call: segment addresses and lengths,
 // gradient addresses, histogram ids.  It owns the device tables and the per-tile scratch.
 struct Plan {
-    std::string key;
+    // the layout the plan was built for, compared array by array when a call looks for its plan
+    int32_t head[4] = {0, 0, 0, 0};          // n_seg, in_dtype, grad_dtype (-1: none), hist_id given
+    std::vector<gg_seg> segs, grad;
+    std::vector<int32_t> hist_id;
+    int32_t max_hist_id = -1;               // largest entry of hist_id
     int32_t n_seg = 0, n_tiles = 0;
     int64_t max_len = 0;          // longest segment
     void *dev = nullptr;          // one allocation holding all tables and scratch
@@ -109,28 +113,32 @@ gg_status check_segs(const gg_seg *segs, int32_t n_seg, int dtype)
     return GG_OK;
 }
 
+// The cached plan of this layout, or null.  A hit costs three memory compares (the most recently used
+// plan is tried first), and a layout that hits was validated when its plan was built.
+Plan *find_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype, const gg_seg *grad, int grad_dtype,
+                const int32_t *hist_id)
+{
+    const int32_t head[4] = {n_seg, in_dtype, grad ? grad_dtype : -1, hist_id ? 1 : 0};
+    Plan *best = nullptr;
+    for (auto &p : ctx->plans)       // most recently used first
+        if (memcmp(p->head, head, sizeof(head)) == 0 && (best == nullptr || p->last_use > best->last_use)) {
+            if (memcmp(p->segs.data(), segs, sizeof(gg_seg) * (size_t)n_seg) != 0) continue;
+            if (grad && memcmp(p->grad.data(), grad, sizeof(gg_seg) * (size_t)n_seg) != 0) continue;
+            if (hist_id && memcmp(p->hist_id.data(), hist_id, sizeof(int32_t) * (size_t)n_seg) != 0) continue;
+            best = p.get();
+        }
+    if (best) best->last_use = ctx->clock;
+    return best;
+}
+
 // Finds or builds the plan for this layout.  Building allocates and uploads with blocking calls.
 gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype, const gg_seg *grad,
                    int grad_dtype, const int32_t *hist_id, Plan **out)
 {
-    std::string key;
-    key.reserve((size_t)n_seg * 36 + 16);
-    const int32_t head[4] = {n_seg, in_dtype, grad ? grad_dtype : -1, hist_id ? 1 : 0};
-    key.append(reinterpret_cast<const char *>(head), sizeof(head));
-    key.append(reinterpret_cast<const char *>(segs), sizeof(gg_seg) * (size_t)n_seg);
-    if (grad) {
-        for (int32_t s = 0; s < n_seg; ++s)
-            key.append(reinterpret_cast<const char *>(&grad[s].ptr), sizeof(void *));
-    }
-    if (hist_id) key.append(reinterpret_cast<const char *>(hist_id), sizeof(int32_t) * (size_t)n_seg);
-
     ctx->clock++;
-    for (auto &p : ctx->plans) {
-        if (p->key == key) {
-            p->last_use = ctx->clock;
-            *out = p.get();
-            return GG_OK;
-        }
+    if (Plan *hit = find_plan(ctx, segs, n_seg, in_dtype, grad, grad_dtype, hist_id)) {
+        *out = hit;
+        return GG_OK;
     }
     if ((int)ctx->plans.size() >= kMaxPlans) {
         // Evict the least recently used plan.  Work that still uses its tables may be in flight.
@@ -144,7 +152,13 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
 
     std::unique_ptr<Plan> p(new (std::nothrow) Plan);
     if (!p) return GG_ERR_NOMEM;
-    p->key = std::move(key);
+    p->head[0] = n_seg; p->head[1] = in_dtype; p->head[2] = grad ? grad_dtype : -1; p->head[3] = hist_id ? 1 : 0;
+    p->segs.assign(segs, segs + n_seg);
+    if (grad) p->grad.assign(grad, grad + n_seg);
+    if (hist_id) {
+        p->hist_id.assign(hist_id, hist_id + n_seg);
+        for (int32_t s = 0; s < n_seg; ++s) p->max_hist_id = std::max(p->max_hist_id, hist_id[s]);
+    }
     p->n_seg = n_seg;
     std::vector<int32_t> prefix((size_t)n_seg + 1, 0);
     for (int32_t s = 0; s < n_seg; ++s)
@@ -541,13 +555,26 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             (a->param_mode != GG_PARAMS_FITTED || !a->step_out)) return GG_ERR_INVALID_ARG;
         if (a->step_mode == GG_STEP_GIVEN && n_seg > 0 && !a->step) return GG_ERR_INVALID_ARG;
     }
-    gg_status st = check_segs(a->segs, n_seg, a->in_dtype);
-    if (st != GG_OK) return st;
-    st = check_grad(a->segs, a->grad, n_seg, a->grad_dtype);
-    if (st != GG_OK) return st;
-    if (do_hist) {
-        st = check_hist(n_seg, a->hist_id, a->n_hist, a->qmin, a->qmax);
+    // A layout that has a plan was validated when the plan was built: a step that repeats a call pays for
+    // three memory compares, not for a walk over its segments.
+    gg_status st = GG_OK;
+    Plan *p = nullptr;
+    if (n_seg > 0 && a->segs && dtype_ok(a->in_dtype) && (!a->grad || dtype_ok(a->grad_dtype))) {
+        ctx->clock++;
+        p = find_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr);
+    }
+    if (p == nullptr) {
+        st = check_segs(a->segs, n_seg, a->in_dtype);
         if (st != GG_OK) return st;
+        st = check_grad(a->segs, a->grad, n_seg, a->grad_dtype);
+        if (st != GG_OK) return st;
+        if (do_hist) {
+            st = check_hist(n_seg, a->hist_id, a->n_hist, a->qmin, a->qmax);
+            if (st != GG_OK) return st;
+        }
+    } else if (do_hist) {
+        if (a->n_hist < 0 || a->qmax < a->qmin || (int64_t)a->qmax - (int64_t)a->qmin + 1 > (1ll << 24)) return GG_ERR_INVALID_ARG;
+        if (a->hist_id ? p->max_hist_id >= a->n_hist : a->n_hist != n_seg) return GG_ERR_INVALID_ARG;
     }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
@@ -559,9 +586,10 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             GG_CUDA(ctx, cudaMemsetAsync(a->clamped_lo_hi, 0, sizeof(uint64_t) * 2 * (size_t)a->n_hist, cs));
     }
     if (n_seg > 0) {
-        Plan *p = nullptr;
-        st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p);
-        if (st != GG_OK) return st;
+        if (p == nullptr) {
+            st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p);
+            if (st != GG_OK) return st;
+        }
         const gg_dtype in_dt = (gg_dtype)a->in_dtype, g_dt = (gg_dtype)a->grad_dtype;
         const bool want_pg = a->grad != nullptr || a->penalty != nullptr;
         const int tail_flags = (want_pg ? kGrad : 0) | (do_hist ? kHist : 0);

@@ -30,13 +30,26 @@ __device__ __forceinline__ void cubic_basis(double t, double (&w)[4], double (&d
 
 // table: Y[0 .. kSeedCells] followed by Z[0 .. kSeedCells].  log_r must lie strictly between Y[0] and
 // Y[kSeedCells].  Returns beta and writes ln(alpha / sigma).
+// WARP: all 32 lanes of the warp call with the same log_r; the cell is then found in three rounds of 32
+// look-ups side by side instead of eleven one after the other.
+template <bool WARP = false>
 __device__ __forceinline__ double invert_ratio_table(double log_r, const double *table, double *ln_alpha_over_sigma)
 {
     const double *Y = table, *Z = table + (kSeedCells + 1);
-    int i0 = 0, i1 = kSeedCells;            // Y[i0] <= log_r < Y[i1]
-    while (i1 - i0 > 1) {
-        const int m = (i0 + i1) >> 1;
-        if (__ldg(Y + m) <= log_r) i0 = m; else i1 = m;
+    int i0 = 0;                             // Y[i0] <= log_r < Y[i0 + 1]
+    if constexpr (WARP) {
+        static_assert(kSeedCells == 2048, "two rounds of 32 and one of 2");
+        const int lane = threadIdx.x & 31;
+        // nodes 64 l, then 2 l inside the block of 64, then the odd node: each ballot counts the nodes <= log_r
+        i0 = 64 * (__popc(__ballot_sync(0xFFFFFFFFu, __ldg(Y + 64 * lane) <= log_r)) - 1);
+        i0 += 2 * (__popc(__ballot_sync(0xFFFFFFFFu, __ldg(Y + i0 + 2 * lane) <= log_r)) - 1);
+        if (__ldg(Y + i0 + 1) <= log_r) i0 += 1;
+    } else {
+        int i1 = kSeedCells;
+        while (i1 - i0 > 1) {
+            const int m = (i0 + i1) >> 1;
+            if (__ldg(Y + m) <= log_r) i0 = m; else i1 = m;
+        }
     }
     const int j = max(0, min(kSeedCells - 3, i0 - 1));     // first node of the four-point stencil
     const double y0 = __ldg(Y + j), y1 = __ldg(Y + j + 1), y2 = __ldg(Y + j + 2), y3 = __ldg(Y + j + 3);

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
                 lnz = __ldg(a.seed + 2 * kSeedCells + 1);
                 flags |= GG_FLAG_BETA_CLAMPED_HI;
             } else {
-                beta = invert_ratio_table(log_r, a.seed, &lnz);
+                beta = invert_ratio_table<true>(log_r, a.seed, &lnz);      // (every lane is here with the same log_r)
             }
             alpha = sqrt(m2) * exp(lnz);
         } else {

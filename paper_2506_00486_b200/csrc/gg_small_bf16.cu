@@ -388,6 +388,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
             xmin = fminf(xmin, __uint_as_float(xb));
             xmax = fmaxf(xmax, __uint_as_float(xb));
         }
+        // extremes of the vector body as packed bf16 (even and odd elements); the padding of a ragged trip is
+        // guarded below, so no zero enters them
+        __nv_bfloat162 mn2 = __floats2bfloat162_rn(INFINITY, INFINITY), mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
         for (int v0 = lane; v0 < nvec; v0 += 128) {
             // four independent loads per trip
             uint4 r4[4];
@@ -403,16 +406,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
             const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
             float m1 = 0.0f, m2 = 0.0f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16);
-                const uint32_t am = xb & 0x7FFFFFFFu;
-                const bool fin = am < 0x7F800000u;
-                const float af = fin ? __uint_as_float(am) : 0.0f;
-                m1 += af;
-                m2 = fmaf(af, af, m2);
-                bad += fin ? 0u : 1u;
-                xmin = fminf(xmin, __uint_as_float(xb));
-                xmax = fmaxf(xmax, __uint_as_float(xb));
+            for (int i = 0; i < 4; ++i) {
+                // both elements of a word at once; an inf or nan makes the sums inf or nan, and the vector is then
+                // summed again element by element below, where it is counted and left out
+                const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+                m1 += fabsf(lo);
+                m1 += fabsf(hi);
+                m2 = fmaf(lo, lo, m2);
+                m2 = fmaf(hi, hi, m2);
+                const __nv_bfloat162 pr = *reinterpret_cast<const __nv_bfloat162 *>(&w[i]);
+                mn2 = __hmin2(mn2, pr);      // return the non-NaN operand, like fminf
+                mx2 = __hmax2(mx2, pr);
             }
             if (run_sums_exact_enough(m1, m2)) {
                 s1 += (double)m1;
@@ -425,11 +429,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                         const double ax = (double)__uint_as_float(am);
                         s1 += ax;
                         s2 += ax * ax;
+                    } else {
+                        bad += 1u;
                     }
                 }
             }
             }
         }
+        xmin = fminf(xmin, fminf(__low2float(mn2), __high2float(mn2)));
+        xmax = fmaxf(xmax, fmaxf(__low2float(mx2), __high2float(mx2)));
         s1 = warp_sum(s1);
         s2 = warp_sum(s2);
         bad = __reduce_add_sync(kFull, bad);
@@ -457,7 +465,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
                 lnz = __ldg(a.seed + 2 * kSeedCells + 1);
                 flags |= GG_FLAG_BETA_CLAMPED_HI;
             } else {
-                beta = invert_ratio_table(log_r, a.seed, &lnz);
+                beta = invert_ratio_table<true>(log_r, a.seed, &lnz);      // (every lane is here with the same log_r)
             }
             alpha = sqrt(m2) * exp(lnz);       // Eq. 2 with sigma^2 = sum_sq / count
         }
