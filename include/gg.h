@@ -334,7 +334,8 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *args, void *stre
  *             GG_ERR_WORKSPACE and nothing is enqueued
  *   beta, alpha, sum_abs, sum_sq, count, flags   device outputs of ONE element each, as in gg_fit
  *             (sum_abs, sum_sq, count, flags may be NULL)
- * The results are those of gg_fit on the same segment (same kernels, same summation order).
+ * The results are those of gg_fit on the same segment up to the rounding of the fp64 partial sums (this call
+ * sums tile by tile, gg_fit run by run: the sums agree to about 1e-15 relative).
  * The first call on a device looks up the array's device address and the device's architecture; make
  * that first call before any stream capture begins.  Later calls only enqueue three kernels on
  * `stream`.  All calls on a device share the one array, which keeps the previous call's contents; each

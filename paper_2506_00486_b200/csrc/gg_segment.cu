@@ -8,7 +8,7 @@ namespace gg {
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kSegThreads = 128;   // 4 warps = 4 segments per CTA
+constexpr int kSegThreads = 128;   // one CTA of 4 warps per segment
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -24,22 +24,26 @@ __device__ __forceinline__ double log_rho(double beta)
     return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
 }
 
-// One warp per segment.  Lanes sum the tile partials in a fixed order (strided, then a butterfly,
-// so every lane ends with the same bits), then invert the moment ratio: from the context's fit
+// One CTA of four warps per segment.  The threads sum the tile partials in a fixed order (strided over
+// the 128 threads, a butterfly in each warp, the four warps in sequence, so every thread of warp 0 ends
+// with the same bits), then warp 0 inverts the moment ratio: from the context's fit
 // table when there is one, else by 33-section search on
 // ln(beta): each round the 32 lanes evaluate log_rho at the interior points of the bracket and a
 // ballot picks the sub-interval with the sign change; ten rounds shrink [ln .05, ln 20] below
 // 1e-14.  The scale follows Eq. 2 with sigma^2 = sum_sq / count.
 __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
 {
-    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (s >= a.map.n_seg) return;
+    __shared__ double sh1[kSegThreads / 32], sh2[kSegThreads / 32];
+    __shared__ uint32_t shb[kSegThreads / 32];
+    __shared__ float shmn[kSegThreads / 32], shmx[kSegThreads / 32];
+    const int s = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t0 = a.map.tile_prefix[s], t1 = a.map.tile_prefix[s + 1];
     double s1 = 0.0, s2 = 0.0;
     uint32_t bad = 0;
     float xmin = INFINITY, xmax = -INFINITY;
-    for (int t = t0 + lane; t < t1; t += 32) {
+#pragma unroll 4
+    for (int t = t0 + (int)threadIdx.x; t < t1; t += kSegThreads) {
         s1 += a.part.s1[t];
         s2 += a.part.s2[t];
         bad += a.part.bad[t];
@@ -53,6 +57,14 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
     for (int o = 16; o > 0; o >>= 1) {
         xmin = fminf(xmin, __shfl_xor_sync(kFull, xmin, o));
         xmax = fmaxf(xmax, __shfl_xor_sync(kFull, xmax, o));
+    }
+    if (lane == 0) { sh1[warp] = s1; sh2[warp] = s2; shb[warp] = bad; shmn[warp] = xmin; shmx[warp] = xmax; }
+    __syncthreads();
+    if (warp != 0) return;
+    s1 = sh1[0]; s2 = sh2[0]; bad = shb[0]; xmin = shmn[0]; xmax = shmx[0];
+    for (int w = 1; w < kSegThreads / 32; ++w) {
+        s1 += sh1[w]; s2 += sh2[w]; bad += shb[w];
+        xmin = fminf(xmin, shmn[w]); xmax = fmaxf(xmax, shmx[w]);
     }
     const int64_t len = a.map.seg_len[s];
 
@@ -124,13 +136,17 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
 __global__ void __launch_bounds__(kSegThreads)
 penalty_finalize_kernel(const TileMap map, const TileScratch part, const double *beta, double *penalty)
 {
-    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (s >= map.n_seg) return;
+    __shared__ double shp[kSegThreads / 32];
+    const int s = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     double p = 0.0;
-    for (int t = map.tile_prefix[s] + lane; t < map.tile_prefix[s + 1]; t += 32) p += part.pen[t];
+#pragma unroll 4
+    for (int t = map.tile_prefix[s] + (int)threadIdx.x; t < map.tile_prefix[s + 1]; t += kSegThreads) p += part.pen[t];
     p = warp_sum(p);
-    if (lane == 0) {
+    if (lane == 0) shp[warp] = p;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kSegThreads / 32; ++w) p += shp[w];      // fixed order
         const double b = beta[s];
         penalty[s] = b > 0.0 ? p / b : 0.0;
     }
@@ -188,8 +204,7 @@ __global__ void entropy_final_kernel(const double *part, int32_t n_hist, double 
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st)
 {
     if (a.map.n_seg <= 0) return cudaSuccess;
-    const int per = kSegThreads / 32;
-    fit_kernel<<<(a.map.n_seg + per - 1) / per, kSegThreads, 0, st>>>(a);
+    fit_kernel<<<a.map.n_seg, kSegThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -197,8 +212,7 @@ cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part,
                                     double *penalty, cudaStream_t st)
 {
     if (map.n_seg <= 0) return cudaSuccess;
-    const int per = kSegThreads / 32;
-    penalty_finalize_kernel<<<(map.n_seg + per - 1) / per, kSegThreads, 0, st>>>(map, part, beta, penalty);
+    penalty_finalize_kernel<<<map.n_seg, kSegThreads, 0, st>>>(map, part, beta, penalty);
     return cudaGetLastError();
 }
 
