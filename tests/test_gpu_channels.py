@@ -188,3 +188,26 @@ def test_channels_activation_shaped_matrix_sampled_columns(ctx):
     sample = [0, 1, 63, 64, 2047, 2048, 4031, 4095] + list(np.random.default_rng(5).integers(0, cols, 8))
     oc = cpu(out)
     check_channels(oc, x.cpu(), g.cpu(), 1e-4, cols=sample)
+
+
+def test_channels_matrix_with_more_than_2_to_31_elements(ctx):
+    """[2^19, 4100] bf16 (2.15e9 elements: element offsets need 64 bits; the last strip is ragged): sampled columns
+    against the oracle, column sums and the histogram total for the whole matrix."""
+    rows, cols = 1 << 19, 4100
+    gen = torch.Generator(device="cuda:0").manual_seed(45)
+    x = gg_synth.gg_device(gen, 1.1, gg_synth.alpha_for_std(0.5, 1.1), rows * cols, torch.bfloat16, torch.device("cuda:0")).view(rows, cols)
+    g = torch.empty((rows, cols), dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused_channels(x, grad=g, lam=1e-4, step=2.0 ** -6)
+    torch.cuda.synchronize()
+    assert out["hist"].sum().item() == rows * cols
+    assert torch.all(out["count"] == rows)
+    s1 = torch.zeros(cols, dtype=torch.float64, device="cuda:0")
+    for r0 in range(0, rows, 1 << 16):                       # (in slabs: a float64 copy of the matrix would not fit)
+        s1 += x[r0:r0 + (1 << 16)].double().abs().sum(0)
+    torch.testing.assert_close(out["sum_abs"], s1, rtol=1e-7, atol=0)
+    sample = [0, 63, 2050, 4095, 4096, 4099]
+    oc = cpu(out)
+    xs = torch.stack([x[:, c] for c in sample], dim=1).cpu()
+    gs = torch.stack([g[:, c] for c in sample], dim=1).cpu()
+    sub = {k: (v[sample] if isinstance(v, torch.Tensor) and v.numel() == cols else v) for k, v in oc.items()}
+    check_channels(sub, xs, gs, 1e-4, cols=list(range(len(sample))))

@@ -136,3 +136,68 @@ def test_config2_qwen_initialisation_full_size(ctx):
         b, a, *_ = o.fit(gg_synth.to_oracle(outs[s].cpu()))
         assert_rel(fit["beta"][s].item(), b, REL_FIT, "beta")
         assert_rel(fit["alpha"][s].item(), a, REL_FIT, "alpha")
+
+
+def test_one_segment_longer_than_2_to_31_elements(ctx):
+    """A single bf16 segment of 2^31 + 12345 elements (64-bit offsets in both sweeps): 2048 copies of a 2^20-element
+    block and a ragged rest, so that the exact results follow from the oracle's results on the block and the
+    rest: sums and counts add up, the gradient repeats."""
+    from paper_2506_00486_b200 import Segments
+    blk, n = 1 << 20, (1 << 31) + 12345
+    k_full, rest = n // blk, n % blk
+    rng = np.random.default_rng(31)
+    base = gg_synth.gg_host(rng, 0.9, 0.02, blk, torch.bfloat16)
+    base[::1009] = 0
+    x = base.to("cuda:0").repeat(k_full + 1)[:n].contiguous()
+    g = torch.empty(n, dtype=torch.float32, device="cuda:0")
+    step, lam = 2.0 ** -10, 1e-4
+    out = ctx.gg_fused(Segments([x]), grad=Segments([g]), lam=lam, step=torch.full((1,), step, dtype=torch.float32, device="cuda:0"))
+    torch.cuda.synchronize()
+    xb, xr = gg_synth.to_oracle(base), gg_synth.to_oracle(base[:rest])
+    s1b, s2b, _, _ = o.moments(xb)
+    s1r, s2r, _, _ = o.moments(xr)
+    s1, s2 = k_full * s1b + s1r, k_full * s2b + s2r
+    assert out["count"][0].item() == n and out["flags"][0].item() == 0
+    # (every copy of the block rounds its fp32 runs of eight the same way, so these errors do not average out
+    # over the copies: the bound is that of one block, 1e-7)
+    assert_rel(out["sum_abs"][0].item(), s1, 1e-7, "sum_abs")
+    assert_rel(out["sum_sq"][0].item(), s2, 1e-7, "sum_sq")
+    b, a, _ = o.fit_from_moments(s1, s2, n)
+    bg, ag = out["beta"][0].item(), out["alpha"][0].item()
+    assert_rel(bg, b, REL_FIT, "beta")
+    assert_rel(ag, a, REL_FIT, "alpha")
+    # histogram and penalty: 2048 blocks and the rest
+    hb, _ = o.quantise_hist(xb, np.float32(step))
+    hr, _ = o.quantise_hist(xr, np.float32(step))
+    np.testing.assert_array_equal(out["hist"][0].cpu().numpy(), (k_full * hb.astype(np.int64) + hr.astype(np.int64)))
+    pb, gb = o.penalty_grad(xb, bg, ag, lam)
+    pr, _ = o.penalty_grad(xr, bg, ag, lam)
+    assert_rel(out["penalty"][0].item(), k_full * pb + pr, REL_PENALTY, "penalty")
+    # the gradient of the first block, of the block that straddles element 2^31, and of the ragged rest
+    for k in (0, 1023, 2047):
+        assert_grad_close(g[k * blk:(k + 1) * blk].cpu().numpy(), gb)
+    assert_grad_close(g[k_full * blk:].cpu().numpy(), gb[:rest])
+    # every other block repeats the first one bit for bit
+    g2 = g[:k_full * blk].view(k_full, blk)
+    assert bool((g2 == g2[0]).all())
+
+
+def test_sample_elements_past_index_2_to_32(ctx):
+    """gg_sample of one bf16 segment of 2^32 + 4096 elements: the element index is a 64-bit counter (its high
+    word enters the Philox counter).  The oracle regenerates windows of elements around 2^32 and at the end."""
+    n = (1 << 32) + 4096
+    x = torch.empty(n, dtype=torch.bfloat16, device="cuda:0")
+    beta, alpha, seed = 1.3, gg_synth.alpha_for_std(0.02, 1.3), 77
+    att = ctx.gg_sample([x], [beta], [alpha], seed=seed, tensor_id0=5)
+    torch.cuda.synchronize()
+    for i0 in (0, (1 << 32) - 2048, (1 << 32), n - 1000):
+        m = min(3000, n - i0)
+        ref = o.sample(beta, alpha, seed, 5, m, index0=i0)
+        got = x[i0:i0 + m].cpu()
+        refb = o.round_to_bf16_bits(ref).astype(np.int64)
+        gotb = got.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+        assert np.array_equal(refb >> 15, gotb >> 15)                       # signs
+        assert (np.abs((refb & 0x7FFF) - (gotb & 0x7FFF)) <= 1).all()       # one bf16 ulp at most ...
+        assert (refb != gotb).mean() <= 1e-3                                # ... and rarely
+    assert 1 <= att[0].item() <= 64
+    del x
