@@ -125,8 +125,8 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------- CPU oracle arm
 def oracle_sample(divisor):
-    """A bounded sample of the workload for the CPU oracle: the first attention matrix of the sweep
-    (4096 x 4096 at full size), generated on the host with the same recipe."""
+    """A bounded sample of the workload for the CPU oracle: the seven matrices of layer 0 of the sweep,
+    generated on the host with the same recipe."""
     import numpy as np
     import torch
     import gg_synth

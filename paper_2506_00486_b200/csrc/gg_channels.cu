@@ -4,22 +4,28 @@
 // path: a strip of 64 neighbouring columns is 128 contiguous bytes of every row, a warp reads one
 // such row piece per load (lane l holds columns 2l and 2l+1 as one 32-bit word) and walks down the
 // rows, so every thread accumulates the sums of its own two columns and no transposition happens.
-//   chan_moments_kernel   one CTA per (strip, block of 256 rows): sum |x|, sum x^2, non-finite
+//   chan_moments_kernel   one CTA per (strip, block of 512 rows): sum |x|, sum x^2, non-finite
 //                         count, min, max per column, written per row block
 //   chan_fit_kernel       16 threads per column: add the row blocks in a fixed order, invert the moment
 //                         ratio from the fit table, derive the constants of the gradient
-//   chan_tables_kernel    one CTA per strip: the per-column gradient tables
-//   chan_tail_kernel      one CTA per (strip, slice of rows): loads the strip's gradient tables
-//                         |g| = A_c[e] * B_c[j] (e exponent field, j mantissa bits of the bf16
-//                         pattern; the lane owns its columns, so lane l reads word l of a table
-//                         row and no look-up ever meets a bank conflict), then streams its rows:
-//                         gradient, penalty partial per column, symbol counts in shared memory
+//   chan_tables_kernel    one CTA per strip: the per-column gradient tables |g| = A_c[e] * B_c[j]
+//                         (e exponent field, j mantissa bits of the bf16 pattern), laid out so that
+//                         lane l reads word l of a table row: no look-up ever meets a bank conflict
+//   chan_tail_kernel      persistent CTAs over (strip, slice of rows) items: copy the strip's tables
+//                         to shared memory, then stream the rows: gradient, penalty partial per
+//                         column, counts in shared memory
 //   chan_penalty_kernel   one thread per column: adds the slices in order, divides by beta
+// Both sweeps read through per-thread rings of asynchronous 4-byte copies (two blocks of eight rows),
+// so the rows in flight cost no registers.
 // A is kept for a window of 64 exponents below the largest magnitude of the strip; every exponent
 // outside it, zero/subnormal/inf/nan and far binades read a NaN marker, the NaN reaches the
 // column's penalty partial of the current block of rows, and the range check of that partial
 // sends the block's column to an exact fp64 path.  Exact zeros are common in activations and are
 // selected to a zero gradient without the exact path.
+// Counts: by symbol in a 4096-cell window while that reaches 6.5 standard deviations of the strip's
+// widest column, else by bf16 bit pattern over the binades up to the strip's largest magnitude,
+// quantised when the cells are flushed.  An element outside the window in use counts in a sentinel
+// cell and is counted again, one by one, after its block of rows.
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -41,9 +47,8 @@ constexpr int kCtasPerSm = 2;
 constexpr int kAWin = 64;                  // exponents covered by the A table (row kAWin: the marker)
 constexpr int kSymWin = 4096;              // symbols counted in shared memory: [-2048, 2048) cut to [qmin, qmax]
 constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
-// Pattern counting (used when symbols of a strip would miss the symbol window): one cell per bf16
-// magnitude pattern and sign over the 16 binades up to the strip's largest magnitude, one cell for zero.
-constexpr int kSlowWin = 512;
+constexpr int kSlowWin = 512;                  // symbols [-256, 256) of the one-by-one path in pattern counting
+// Pattern counting: one cell per bf16 magnitude pattern and sign over 16 binades, one cell for zero.
 constexpr uint32_t kPatCells = 16 * 128;       // magnitude patterns in the window: cell pairs 0 .. kPatCells - 1
 constexpr uint32_t kPatZero = kPatCells;       // the cell pair of +-0
 constexpr uint32_t kPatSentinel = kPatCells + 1;
