@@ -60,6 +60,12 @@ def main(which):
         print(f"c2  gg_sample, {len(outs)} bf16 matrices, {n:.3e} elements: {ms:.2f} ms  {n / ms / 1e6:.1f} G elements/s")
         ms = timeit(lambda: ctx.gg_fit(outs), 5)
         print(f"c2  gg_fit of them: {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
+        gs = [torch.empty(o_.numel(), dtype=torch.float32, device=dev) for o_ in outs]
+        run = ctx.make_fused(Segments(outs), grad=Segments(gs), lam=1e-4,
+                             step=torch.full((len(outs),), 2.0 ** -10, dtype=torch.float32, device=dev))
+        ms = timeit(run, 5)
+        print(f"c2  fused pass over them (fp32 gradients, one histogram per matrix): {ms:.3f} ms  {6 * n / ms / 1e6:.0f} GB/s")
+        del gs, run
         del outs
     if "c3" in which:
         a = gg_synth.alpha_for_std(1.0, 0.8)
