@@ -567,20 +567,26 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + d * kStageBytes), "l"(xv + d * kThreads) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    uint32_t rd = 0, wr = (kDepth - 1) * kStageBytes;      // byte offsets of the slot to read / to fill next
-    for (int v = tid; v < nv; v += kThreads) {
-        // fill the slot emptied by the previous iteration (its value is in registers since then)
-        if (v + (kDepth - 1) * kThreads < nv)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + wr), "l"(xv + (kDepth - 1) * kThreads) : "memory");
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
-        uint4 r0;
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r0.x), "=r"(r0.y), "=r"(r0.z), "=r"(r0.w) : "r"(slot0 + rd) : "memory");
-        process_vec<TG, FLAGS, MODE>(r0, gv, accumulate, wide, ln, sm, acc);
-        rd = rd + kStageBytes == kDepth * kStageBytes ? 0u : rd + kStageBytes;
-        wr = wr + kStageBytes == kDepth * kStageBytes ? 0u : wr + kStageBytes;
-        xv += kThreads;
-        if (gv != nullptr) gv += kThreads * 8;
+    // (the loop is unrolled over the stages, so that every slot is a compile-time offset)
+    for (int v = tid; v < nv; v += kDepth * kThreads) {
+#pragma unroll
+        for (int d = 0; d < kDepth; ++d) {
+            const int vd = v + d * kThreads;
+            if (vd < nv) {
+                // fill the slot emptied by the previous vector (stage d - 1, cyclically; its value is in registers since then)
+                if (vd + (kDepth - 1) * kThreads < nv)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + ((d + kDepth - 1) % kDepth) * kStageBytes),
+                                 "l"(xv + (d + kDepth - 1) * kThreads) : "memory");
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
+                uint4 r0;
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r0.x), "=r"(r0.y), "=r"(r0.z), "=r"(r0.w) : "r"(slot0 + d * kStageBytes) : "memory");
+                TG *gd = gv != nullptr ? gv + (int64_t)d * kThreads * 8 : nullptr;
+                process_vec<TG, FLAGS, MODE>(r0, gd, accumulate, wide, ln, sm, acc);
+            }
+        }
+        xv += kDepth * kThreads;
+        if (gv != nullptr) gv += kDepth * kThreads * 8;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
