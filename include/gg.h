@@ -286,9 +286,9 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *args, int64_t chunk_by
  * of the same pass and every formula is that of gg_fit, gg_penalty_grad and gg_rate_hist.
  * All columns are quantised with one step into ONE histogram (the rate of the whole tensor). */
 typedef struct {
-    const void *x;               /* device, bf16, element (r, c) at x[r * ld + c]             */
+    const void *x;               /* device, element (r, c) at x[r * ld + c]                   */
     int64_t     rows, cols, ld;  /* ld >= cols, in elements                                   */
-    int32_t     in_dtype;        /* GG_BF16 (GG_F32 is refused with GG_ERR_DTYPE)             */
+    int32_t     in_dtype;        /* GG_BF16 or GG_F32                                         */
     /* fit outputs, device [cols]; beta and alpha are required                                */
     double   *beta, *alpha, *sum_abs, *sum_sq;
     int64_t  *count;
@@ -311,12 +311,12 @@ typedef struct {
 } gg_channel_args;
 
 /* moments -> fit -> penalty + gradient + histogram -> entropy for every column of the matrix, all
- * enqueued on `stream`: the matrix is read twice (row-major, coalesced: a strip of 64 columns is
- * 128 contiguous bytes of every row), the second time from L2 when it fits there.  Results per
+ * enqueued on `stream`: the matrix is read twice (row-major, coalesced: a strip of 64 bf16 or 32 fp32
+ * columns is 128 contiguous bytes of every row), the second time from L2 when it fits there.  Results per
  * column equal those of gg_fused on the gathered column within the same tolerances; sums over a
  * column are reduced in a fixed order.  GG_FLAG_CLAMPED_SYMBOLS is set per column when a histogram
  * is taken.  The first call with a larger matrix than any before allocates scratch (blocking).
- * Errors: GG_ERR_DTYPE for fp32 input, GG_ERR_INVALID_ARG for ld < cols, negative sizes, a missing
+ * Errors: GG_ERR_DTYPE for an unknown dtype, GG_ERR_INVALID_ARG for ld < cols, negative sizes, a missing
  * required pointer or qmin > qmax, GG_ERR_ALIGNMENT for x or grad not element aligned. */
 gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *args, void *stream);
 

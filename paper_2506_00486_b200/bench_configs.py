@@ -107,12 +107,14 @@ def main(which):
             ms = timeit(lambda: ctx.gg_eg_rate(rh["hist"]))
             print(f"codes  gg_eg_rate, 8 histograms of 65536 bins: {ms * 1e3:.1f} us")
     if "channels" in which:
-        for rows, cols, spread in ((16384, 4096, 3), (65536, 4096, 3), (16384, 11008, 3), (16384, 4096, 9)):
+        for rows, cols, spread, dt in ((16384, 4096, 3, torch.bfloat16), (65536, 4096, 3, torch.bfloat16),
+                                       (16384, 11008, 3, torch.bfloat16), (16384, 4096, 9, torch.bfloat16),
+                                       (16384, 4096, 3, torch.float32)):
             # column c scaled by 2^(c mod spread - spread // 2): with 9 the widest columns' symbols leave the
             # shared symbol window and their strips are counted by bit pattern
             a = gg_synth.alpha_for_std(1.0, 0.8)
-            x = gg_synth.gg_device(gen, 0.8, a, rows * cols, torch.bfloat16, dev).view(rows, cols)
-            x.mul_(torch.exp2(torch.arange(cols, device=dev) % spread - float(spread // 2)).to(torch.bfloat16))
+            x = gg_synth.gg_device(gen, 0.8, a, rows * cols, dt, dev).view(rows, cols)
+            x.mul_(torch.exp2(torch.arange(cols, device=dev) % spread - float(spread // 2)).to(dt))
             gg_synth.add_outliers_device(gen, x, 1e-3, 20.0)
             g = torch.empty((rows, cols), dtype=torch.float32, device=dev)
             run = ctx.make_fused_channels(x, grad=g, lam=1e-4, step=0.01)
@@ -122,8 +124,9 @@ def main(which):
             ms = timeit(run, 5)
             t = ctx.timing_read()
             ctx.timing_enable(False)
-            print(f"channels  fused, bf16 [{rows}, {cols}], column scales 2^-{spread // 2}..2^{spread // 2}, one GG per column, one histogram: {ms * 1e3:.1f} us  "
-                  f"{6 * x.numel() / ms / 1e6:.0f} GB/s  (moments {t[0] / t[1] * 1e3:.1f} us, "
+            name = "bf16" if dt == torch.bfloat16 else "fp32"
+            print(f"channels  fused, {name} [{rows}, {cols}], column scales 2^-{spread // 2}..2^{spread // 2}, one GG per column, one histogram: {ms * 1e3:.1f} us  "
+                  f"{(x.element_size() + 4) * x.numel() / ms / 1e6:.0f} GB/s  (moments {t[0] / t[1] * 1e3:.1f} us, "
                   f"gradient + histogram {t[2] / t[3] * 1e3:.1f} us)")
             del x, g, run
     ctx.close()

@@ -683,12 +683,13 @@ static gg_status grow(gg_ctx *ctx, void **buf, int64_t *have, int64_t need)
 gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
 {
     if (!ctx || !a) return GG_ERR_INVALID_ARG;
-    if (a->in_dtype != GG_BF16) return GG_ERR_DTYPE;
+    if (!dtype_ok(a->in_dtype)) return GG_ERR_DTYPE;
+    const bool f32 = a->in_dtype == GG_F32;
     if (a->rows < 0 || a->cols < 0 || a->ld < a->cols) return GG_ERR_INVALID_ARG;
     if (a->cols > 0 && (!a->beta || !a->alpha)) return GG_ERR_INVALID_ARG;
     if (a->rows > 0 && a->cols > 0 && !a->x) return GG_ERR_INVALID_ARG;
     if (a->reduction != GG_SUM && a->reduction != GG_MEAN) return GG_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(a->x) % 2 != 0) return GG_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(a->x) % esize(a->in_dtype) != 0) return GG_ERR_ALIGNMENT;
     if (a->grad) {
         if (!dtype_ok(a->grad_dtype)) return GG_ERR_DTYPE;
         if (a->grad_ld < a->cols) return GG_ERR_INVALID_ARG;
@@ -716,11 +717,12 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         ka.rows = a->rows; ka.cols = a->cols; ka.ld = a->ld;
         ka.grad = a->grad; ka.grad_ld = a->grad_ld; ka.accumulate = a->accumulate_grad;
         ka.n_mom_blocks = (int32_t)n_mom;
-        ka.n_slices = chan_slices(a->rows, a->cols, ctx->sm_count);
+        ka.n_slices = chan_slices(a->rows, a->cols, ctx->sm_count, f32 ? kChanStripF32 : kChanStrip);
         // scratch: doubles first, then the 32-bit arrays
         const size_t nc = (size_t)a->cols, nm = (size_t)n_mom * nc, ns = (size_t)ka.n_slices * nc;
-        const size_t n_strips = (nc + kChanStrip - 1) / kChanStrip;
-        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + 2 * nc + n_strips * (kChanTabFloats + 1) + 8;
+        // table space in units of a narrow (fp32) strip: a wide (bf16) strip takes two
+        const size_t n_strips = 2 * ((nc + kChanStrip - 1) / kChanStrip);
+        const size_t n_dbl = 2 * nm + 2 * nc + ns, n_w32 = 3 * nm + 2 * nc + n_strips * (kChanTabFloats / 2 + 1) + 8;
         void *buf = ctx->chan_buf;
         gg_status st = grow(ctx, &buf, &ctx->chan_bytes, (int64_t)(n_dbl * 8 + n_w32 * 4));
         ctx->chan_buf = buf;
@@ -744,13 +746,14 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         ka.step = a->step; ka.qmin = a->qmin; ka.qmax = a->qmax; ka.hist = a->hist; ka.clamped = a->clamped_lo_hi;
         {
             SweepTimer tm(ctx, &ctx->ev_first, cs);
-            GG_CUDA(ctx, launch_chan_moments(ka, cs));
+            GG_CUDA(ctx, f32 ? launch_chan_moments_f32(ka, cs) : launch_chan_moments(ka, cs));
         }
         GG_CUDA(ctx, launch_chan_fit(ka, cs));
         ctx->launches += 1 + (a->rows > 0);
         if ((want_pg || do_hist) && a->rows > 0) {
             SweepTimer tm(ctx, &ctx->ev_tail, cs);
-            GG_CUDA(ctx, launch_chan_tail((gg_dtype)a->grad_dtype, ka, ctx->sm_count, cs));
+            GG_CUDA(ctx, f32 ? launch_chan_tail_f32((gg_dtype)a->grad_dtype, ka, ctx->sm_count, cs)
+                             : launch_chan_tail((gg_dtype)a->grad_dtype, ka, ctx->sm_count, cs));
             ctx->launches += 1 + (want_pg ? 1 : 0);
         }
         if (a->penalty) {

@@ -876,9 +876,9 @@ cudaError_t launch_chan_fit(const ChanArgs &a, cudaStream_t st)
 // Row slices per strip: enough items to fill two CTAs per SM, in whole rounds of the grid where
 // there are more items than CTAs, and at least 512 rows per item so that the tables (192 entries
 // per column) stay cheap next to the rows they serve.
-int chan_slices(int64_t rows, int64_t cols, int sm_count)
+int chan_slices(int64_t rows, int64_t cols, int sm_count, int strip)
 {
-    const int64_t n_strips = (cols + kChanStrip - 1) / kChanStrip;
+    const int64_t n_strips = (cols + strip - 1) / strip;
     const int64_t slots = (int64_t)sm_count * kCtasPerSm;
     const int64_t most = rows / 512 > 1 ? rows / 512 : 1;
     int64_t best = 1;

@@ -126,11 +126,12 @@ cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, c
                             cudaStream_t st);
 // Column segments of a row-major bf16 matrix (gg_fused_channels).  Scratch arrays are indexed
 // [row block][column]; the moments kernel and the second kernel cut the rows differently.
-constexpr int kChanStrip = 64;        // columns per strip: 128 contiguous bytes of a row
+constexpr int kChanStrip = 64;        // bf16 columns per strip: 128 contiguous bytes of a row
+constexpr int kChanStripF32 = 32;     // fp32 columns per strip: the same 128 bytes
 constexpr int kChanMomRows = 512;
 constexpr int kChanTabFloats = 2 * 65 * 32 + 2 * 128 * 32;   // A (64 exponents + marker row) and B (128 mantissas), two columns per lane     // rows per CTA of the moments kernel
 struct ChanArgs {
-    const uint16_t *x;
+    const uint16_t *x;                 // (fp32 kernels read it as float)
     int64_t rows, cols, ld;
     void *grad;                        // may be null
     int64_t grad_ld;
@@ -160,7 +161,10 @@ struct ChanArgs {
 };
 cudaError_t launch_chan_moments(const ChanArgs &a, cudaStream_t st);
 cudaError_t launch_chan_fit(const ChanArgs &a, cudaStream_t st);
-int chan_slices(int64_t rows, int64_t cols, int sm_count);      // n_slices the second kernel should use
+int chan_slices(int64_t rows, int64_t cols, int sm_count, int strip);      // n_slices the second kernel should use (strip: its columns per strip)
+// fp32 input: one column per lane (gg_channels_f32.cu); fit and penalty kernels are those of the bf16 path
+cudaError_t launch_chan_moments_f32(const ChanArgs &a, cudaStream_t st);
+cudaError_t launch_chan_tail_f32(gg_dtype grad_dtype, const ChanArgs &a, int sm_count, cudaStream_t st);
 cudaError_t launch_chan_tail(gg_dtype grad_dtype, const ChanArgs &a, int sm_count, cudaStream_t st);
 cudaError_t launch_chan_penalty(const ChanArgs &a, cudaStream_t st);
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st);
