@@ -124,21 +124,29 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(divisor):
-    """A bounded sample of the workload for the CPU oracle: the seven matrices of layer 0 of the sweep,
-    generated on the host with the same recipe."""
+def oracle_sample(divisor, max_elements=None):
+    """A bounded sample of the workload for the CPU oracle: the matrices of layer 0 of the sweep (all seven,
+    or as many of them, or as long a piece of the first, as max_elements allows), generated on the host with
+    the same recipe."""
     import numpy as np
     import torch
     import gg_synth
     shapes, betas, alphas = gg_synth.workload_c5_params(
         gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), divisor) if divisor > 1 else None)
     rng = np.random.default_rng(4)
-    xs = []
+    xs, n = [], 0
     for i in range(1, 8):        # layer 0: q, k, v, o, gate, up, down
         _, r, c = shapes[i]
-        xs.append(gg_synth.to_oracle(gg_synth.gg_host(rng, betas[i], alphas[i], r * c, torch.bfloat16)))
-    n = sum(x.size for x in xs)
-    return xs, f"layer 0 of the sweep (7 of 226 bf16 matrices, {n:.3e} of 6.74e9 elements)"
+        m = r * c
+        if max_elements is not None and n + m > max_elements:
+            if not xs:
+                m = max(1024, int(max_elements))
+                xs.append(gg_synth.to_oracle(gg_synth.gg_host(rng, betas[i], alphas[i], m, torch.bfloat16)))
+                n += m
+            break
+        xs.append(gg_synth.to_oracle(gg_synth.gg_host(rng, betas[i], alphas[i], m, torch.bfloat16)))
+        n += m
+    return xs, f"{len(xs)} of the 7 bf16 matrices of layer 0 of the sweep ({n:.3e} of 6.74e9 elements)"
 
 
 def oracle_step(xs):
@@ -175,8 +183,10 @@ def run_reference(args):
         return
     from oracle import gg_oracle as o
     o.build()
-    x, what = oracle_sample(args.divisor)
-    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    # exactly the steps asked for, on a sample sized so that all of them take about two minutes (the oracle
+    # does about 50 M elements per second on 16 cores)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    x, what = oracle_sample(args.divisor, max_elements=120.0 * 50e6 / (steps + warmup))
     gbs, dt = time_oracle(x, steps, warmup)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
