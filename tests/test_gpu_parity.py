@@ -636,3 +636,17 @@ def test_fused_replays_from_a_cuda_graph(ctx):
         _, g = o.penalty_grad(xo, oc["beta"][c].item(), oc["alpha"][c].item(), 1e-4)
         assert_grad_close(mg[:, c].cpu().numpy(), g)
     assert oc["hist"].sum().item() == mat.numel()
+
+
+def test_more_layouts_than_cached_plans(ctx):
+    """The context keeps the plans of the 64 most recently used layouts; more layouts than that evict the
+    oldest ones, which are rebuilt when they come back.  Results do not depend on any of it."""
+    rng = np.random.default_rng(29)
+    xs = [gg_synth.gg_host(rng, 1.0 + 0.01 * i, 0.05, 3000 + 17 * i, torch.bfloat16) for i in range(70)]
+    xd = [dev(x) for x in xs]
+    refs = [o.fit(gg_synth.to_oracle(x)) for x in xs]
+    for rnd in range(2):                               # the second round finds the first layouts evicted
+        for i, t in enumerate(xd):
+            out = ctx.gg_fit([t])
+            assert_rel(out["beta"][0].item(), refs[i][0], REL_FIT, f"beta[{i}] round {rnd}")
+            assert_rel(out["alpha"][0].item(), refs[i][1], REL_FIT, f"alpha[{i}] round {rnd}")
