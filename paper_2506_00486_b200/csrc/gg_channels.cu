@@ -32,6 +32,7 @@
 #include <type_traits>
 
 #include "gg_fit_table.cuh"
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -46,7 +47,6 @@ constexpr int kTailWarps = kTailThreads / 32;
 constexpr int kCtasPerSm = 2;
 constexpr int kAWin = 64;                  // exponents covered by the A table (row kAWin: the marker)
 constexpr int kSymWin = 4096;              // symbols counted in shared memory: [-2048, 2048) cut to [qmin, qmax]
-constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr int kSlowWin = 512;                  // symbols [-256, 256) of the one-by-one path in pattern counting
 // Pattern counting: one cell per bf16 magnitude pattern and sign over 16 binades, one cell for zero.
 constexpr uint32_t kPatCells = 16 * 128;       // magnitude patterns in the window: cell pairs 0 .. kPatCells - 1
@@ -332,11 +332,6 @@ __device__ __noinline__ void chan_count_slow(float x, float inv, int32_t qmin, i
         else if (wlo >= whi && (uint32_t)(q + kSlowWin / 2) < (uint32_t)kSlowWin) atomicAdd(&sm.win[q + kSlowWin / 2], 1u);
         else atomicAdd(&hist[q - qmin], 1ull);
     }
-}
-
-__device__ __forceinline__ void red_inc(uint32_t addr)
-{
-    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
 }
 
 // One CTA per strip: the gradient tables of its 64 columns, in the layout of TailSmem::a1 and bt,

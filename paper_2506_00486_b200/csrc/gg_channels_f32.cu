@@ -14,6 +14,7 @@
 #include <float.h>
 
 #include "gg_fit_table.cuh"
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -25,7 +26,6 @@ constexpr int kU = 8;                      // rows in flight per thread and ring
 constexpr int kTailThreads = 512, kTailWarps = kTailThreads / 32, kCtasPerSm = 2;
 constexpr int kAWin = 64;                  // exponents covered by the A table (row kAWin: the marker)
 constexpr int kSymWin = 4096;              // symbols counted in shared memory: [-2048, 2048) cut to [qmin, qmax]
-constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr int kTabFloats = (kAWin + 1) * 32 + 128 * 32;
 static_assert(2 * kTabFloats == kChanTabFloats, "two fp32 strips take the table space of one bf16 strip");
 
@@ -167,25 +167,6 @@ struct LaneF32 {
     float inv, t_lo, t_hi, near;     // quantiser scale; clamp of t; a smaller |t| is inside the window for sure
     float c1, c2, c3, c4;            // binomial coefficients of (1 + r)^b for the lane's column
 };
-
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void red_inc(uint32_t addr)
-{
-    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
-}
-
-__device__ __forceinline__ float rcp_approx(float v)
-{
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
-    return r;
-}
 
 // Exact gradient magnitude (with lambda's sign through `flip`) of |x| given as fp32 bits.
 __device__ __noinline__ float grad_exact_f32(uint32_t ax, double L, double b, uint32_t flip)

@@ -1,0 +1,41 @@
+// Small device helpers shared by the kernels of the library (not installed).
+#pragma once
+#include <stdint.h>
+
+namespace gg {
+
+// 1.5 * 2^23: for |t| < 2^22 the sum t + magic lies in [2^23, 2^24), where the floats are the integers, so
+// adding with rounding down gives floor(t) = bits(t +rd magic) - bits(magic).
+constexpr uint32_t kMagicBits = 0x4B400000u;
+
+// Shared-memory accesses by 32-bit shared address (one instruction each, no generic-address arithmetic).
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+// (No memory clobber: the counts are read back only after a barrier, and the clobber would keep the compiler
+// from moving the element path's loads across the increment.)
+__device__ __forceinline__ void red_inc(uint32_t addr)
+{
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
+}
+
+__device__ __forceinline__ float rcp_approx(float v)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+
+// Butterfly sum over the warp: every lane ends with the same bits.
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+}  // namespace gg

@@ -2,6 +2,7 @@
 // partials, the moment-ratio inversion (one warp per segment), the penalty sums, and the
 // empirical entropy of a count table.  All arithmetic here is fp64; none of it is bandwidth bound.
 #include "gg_fit_table.cuh"
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -9,13 +10,6 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kSegThreads = 128;   // one CTA of 4 warps per segment
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-    return v;
-}
 
 // ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
 // of the density of Eq. 1; increasing in beta from 0 to 3/4.

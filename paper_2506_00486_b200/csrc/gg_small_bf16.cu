@@ -16,6 +16,7 @@
 #include <float.h>
 
 #include "gg_fit_table.cuh"
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -53,25 +54,6 @@ struct Smem {
     int key_on;
     int below_ok;                      // values below the window quantise to 0 / -1
 };
-
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void red_inc(uint32_t addr)
-{
-    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
-}
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-    return v;
-}
 
 __device__ __forceinline__ double log_rho(double beta)
 {

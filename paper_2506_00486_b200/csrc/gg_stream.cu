@@ -8,6 +8,7 @@
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -88,13 +89,6 @@ __device__ __forceinline__ void store_vec(TG *g, const float (&v)[KV], bool accu
             *reinterpret_cast<uint2 *>(g) = make_uint2(w[0], w[1]);
         }
     }
-}
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
 }
 
 // ---------------------------------------------------------------------------- gradient math

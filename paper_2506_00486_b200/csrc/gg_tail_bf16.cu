@@ -31,6 +31,7 @@
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -44,7 +45,6 @@ constexpr int kCntBinades = 16;                     // pattern-count window
 constexpr uint32_t kCntPat = kCntBinades * 128;     // magnitude patterns in it
 constexpr int kRep = 2;                             // replicas of every pattern-count cell
 constexpr uint32_t kSymCells = 384;                 // symbol-count window: symbols [-192, 192)
-constexpr uint32_t kMagicBits = 0x4B400000u;        // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr uint32_t kSymBase = kMagicBits - kSymCells / 2;
 constexpr int kSymWin = 512;                        // secondary symbol window [-256, 256) of the rare path
 constexpr uint32_t kCntWords = (kSymCells + 2) * 32 > (kCntPat + 1) * 2 * kRep ? (kSymCells + 2) * 32
@@ -87,25 +87,6 @@ struct Smem {
 // A[e] as one factor (with lambda's sign), NaN where that is not possible.  Static shared memory:
 // its address is a compile-time constant, so a look-up is an index and a load.
 __shared__ float s_a1[256];
-
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void red_inc(uint32_t addr)
-{
-    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
-}
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
 
 // |g| (with lambda's sign) for a magnitude pattern the A/B tables do not cover: zero, subnormal,
 // inf, nan.

@@ -22,6 +22,7 @@
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include "gg_device.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -33,7 +34,6 @@ constexpr int kCtasPerSm = 2;
 constexpr int kDepth = 3;                           // pairs of input vectors staged ahead per thread
 constexpr uint32_t kSymCells = 256;                 // row layout: symbols [-128, 128)
 constexpr uint32_t kWinCells = 8192;                // word layout: symbols [-4096, 4096)
-constexpr uint32_t kMagicBits = 0x4B400000u;        // 1.5 * 2^23: floor(t) = bits(t +rd magic) - bits(magic)
 constexpr uint32_t kCntWords = (kSymCells + 2) * 32 > kWinCells + 2 ? (kSymCells + 2) * 32 : kWinCells + 2;
 enum : int { kModeWords = 1, kModeRows = 2 };
 
@@ -63,32 +63,6 @@ struct Smem {
 // A[e] as one factor (with lambda's sign), NaN where that is not possible.  Static shared memory:
 // its address is a compile-time constant, so a look-up is an index and a load.
 __shared__ float s_a1[256];
-
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void red_inc(uint32_t addr)
-{
-    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
-}
-
-__device__ __forceinline__ float rcp_approx(float v)
-{
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
-    return r;
-}
-
-__device__ __forceinline__ double warp_sum(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
 
 // |g| (with lambda's sign) in fp64 for any input: the exact path.
 __device__ __noinline__ float grad_exact(uint32_t xb, double L, double b, int active, uint32_t sign_flip)
