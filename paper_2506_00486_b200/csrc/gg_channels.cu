@@ -530,8 +530,19 @@ __device__ __forceinline__ void chan_recount(TailSmem &sm, uint32_t cbase, WordO
             } else {
                 miss = !(t >= (float)wlo && t < (float)whi);
             }
-            // (the slow count may only use the shared cells in symbol counting: wlo = whi switches that off)
-            if (counted(u, k) && miss) chan_count_slow(x, inv, sm.cc.qmin, sm.cc.qmax, PAT ? 0 : wlo, PAT ? 0 : whi, sm, sm.cc.hist);
+            if (counted(u, k) && miss) {
+                if constexpr (PAT) {
+                    // most misses are small values below the pattern window: their few symbols meet in the small
+                    // window, without a call
+                    const int q = __float2int_rd(t);
+                    if (t == t && (uint32_t)(q + kSlowWin / 2) < (uint32_t)kSlowWin && q >= sm.cc.qmin && q <= sm.cc.qmax) {
+                        atomicAdd(&sm.win[q + kSlowWin / 2], 1u);
+                        continue;
+                    }
+                }
+                // (the slow count may only use the shared cells in symbol counting: wlo = whi switches that off)
+                chan_count_slow(x, inv, sm.cc.qmin, sm.cc.qmax, PAT ? 0 : wlo, PAT ? 0 : whi, sm, sm.cc.hist);
+            }
         }
     }
 }
