@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Timings of the secondary workloads (everything but the weight sweep that bench.py reports).
 
-    python -m paper_2506_00486_b200.bench_configs [c1] [c2] [c3] [c4] [codes] [channels]
+    python -m paper_2506_00486_b200.bench_configs [c1] [c2] [c3] [c4] [codes] [calls] [channels]
 
 Each line gives the CUDA-event time of one call through the C interface on cuda:0, inputs resident
 in device memory, and the algorithmic GB/s (input read once + output written once).  Inputs are the
@@ -106,6 +106,23 @@ def main(which):
             rh = ctx.gg_rate_hist(xs, steps)
             ms = timeit(lambda: ctx.gg_eg_rate(rh["hist"]))
             print(f"codes  gg_eg_rate, 8 histograms of 65536 bins: {ms * 1e3:.1f} us")
+    if "calls" in which:
+        # the single-step entry points on the Llama-7B-shaped sweep with every dimension halved (1.68e9 elements)
+        w = gg_synth.workload_c5_device(dev, torch.bfloat16, shapes=gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), 2), seed=4)
+        flat, offs, lens = w["flat"], w["offsets"], w["lens"]
+        segs = Segments.slices(flat, offs, lens)
+        g = torch.empty(flat.numel(), dtype=torch.float32, device=dev)
+        gsegs = Segments.slices(g, offs, lens)
+        n = flat.numel()
+        steps = torch.full((len(lens),), 2.0 ** -10, dtype=torch.float32, device=dev)
+        fit = ctx.gg_fit(segs)
+        ms = timeit(lambda: ctx.gg_fit(segs))
+        print(f"calls  gg_fit, {len(lens)} bf16 matrices, {n:.3e} elements: {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
+        ms = timeit(lambda: ctx.gg_penalty_grad(segs, fit["beta"], fit["alpha"], 1e-4, grad=gsegs))
+        print(f"calls  gg_penalty_grad (fp32 gradients): {ms:.3f} ms  {6 * n / ms / 1e6:.0f} GB/s")
+        ms = timeit(lambda: ctx.gg_rate_hist(segs, steps))
+        print(f"calls  gg_rate_hist (one histogram per matrix, entropy): {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
+        del w, flat, g, segs, gsegs
     if "channels" in which:
         for rows, cols, spread, dt in ((16384, 4096, 3, torch.bfloat16), (65536, 4096, 3, torch.bfloat16),
                                        (16384, 11008, 3, torch.bfloat16), (16384, 4096, 9, torch.bfloat16),
@@ -133,4 +150,4 @@ def main(which):
 
 
 if __name__ == "__main__":
-    main(set(sys.argv[1:]) or {"c1", "c2", "c3", "c4", "codes", "channels"})
+    main(set(sys.argv[1:]) or {"c1", "c2", "c3", "c4", "codes", "calls", "channels"})

@@ -610,6 +610,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         const int64_t len = a.map.seg_len[s];
         const int t_first = a.map.tile_prefix[s];
         const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
+        const int64_t off = (int64_t)(t - t_first) * kTile;
+        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
+        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
         int mode = kModePattern;
         bool active = false;
 
@@ -663,7 +666,24 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             // the scale of the data is known, else where it is (same key) or from four binades below
             // the step upwards (new key)
             uint32_t want_base = sm.cold.c_base;
-            const double sd = GRAD ? sm.cold.sd : 0.0;
+            double sd = GRAD ? sm.cold.sd : 0.0;
+            if constexpr (!GRAD) {
+                // Without parameters the scale of the data is taken from the first elements of the run (up to
+                // eight per thread): it only decides how the counts are laid out, never what is counted.
+                const int m = (int)min(n, (int64_t)kThreads * 8);
+                float ss = 0.0f;
+                for (int i = tid; i < m; i += kThreads) {
+                    const float v = __uint_as_float((uint32_t)__ldg(x + i) << 16);
+                    if (fabsf(v) <= 1e18f) ss = fmaf(v, v, ss);        // (inf, nan and values whose squares overflow are left out)
+                }
+                const double ws = warp_sum((double)ss);
+                __syncthreads();                                        // (the slots may still be read from the run before)
+                if ((tid & 31) == 0) sm.red[2][tid >> 5] = ws;
+                __syncthreads();
+                double tot = 0.0;
+                for (int w = 0; w < kWarps; ++w) tot += sm.red[2][w];
+                sd = m > 0 ? sqrt(tot / (double)m) : 0.0;
+            }
             if (sd > 0.0) {
                 want_base = (uint32_t)(window_top_exponent(sd, 4) - (kCntBinades - 1)) << 7;
                 // symbol mode: the window's symbols are not clamped and reach 6.5 standard deviations
@@ -697,15 +717,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         __syncthreads();
 
         // ---- stream the run
-        const int64_t off = (int64_t)(t - t_first) * kTile;
-        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
-        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
         TG *gout = nullptr;
         if constexpr (GRAD) {
             if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
         }
         Acc acc;
-        if constexpr (GRAD && HIST) {
+        if constexpr (HIST) {
             if (mode == kModeSymbol) process_range<TG, FLAGS, kModeSymbol>(x, gout, n, accumulate, ln, sm, acc);
             else process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
         } else {

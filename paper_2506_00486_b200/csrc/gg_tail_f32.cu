@@ -401,6 +401,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
         const int64_t len = a.map.seg_len[s];
         const int t_first = a.map.tile_prefix[s];
         const int t_stop = min(t_end, a.map.tile_prefix[s + 1]);
+        const int64_t off = (int64_t)(t - t_first) * kTile;
+        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
+        const float *x = reinterpret_cast<const float *>(a.map.seg_ptr[s]) + off;
         int mode = kModeWords;
 
         if constexpr (GRAD) {
@@ -445,7 +448,24 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
             const float step = a.step[s];
             const float inv = (float)(1.0 / (double)step);
             __syncthreads();                        // (sm.cold.sd of this run is written)
-            const double sd = GRAD ? sm.cold.sd : 0.0;
+            double sd = GRAD ? sm.cold.sd : 0.0;
+            if constexpr (!GRAD) {
+                // Without parameters the scale of the data is taken from the first elements of the run (up to
+                // eight per thread): it only decides how the counts are laid out, never what is counted.
+                const int m = (int)min(n, (int64_t)kThreads * 8);
+                float ss = 0.0f;
+                for (int i = tid; i < m; i += kThreads) {
+                    const float v = __ldg(x + i);
+                    if (fabsf(v) <= 1e18f) ss = fmaf(v, v, ss);        // (inf, nan and values whose squares overflow are left out)
+                }
+                const double ws = warp_sum((double)ss);
+                if ((tid & 31) == 0) sm.red[tid >> 5] = ws;             // (free here: the barrier above follows the run before)
+                __syncthreads();
+                double tot = 0.0;
+                for (int w = 0; w < kWarps; ++w) tot += sm.red[w];
+                sd = m > 0 ? sqrt(tot / (double)m) : 0.0;
+                __syncthreads();
+            }
             // rows when the scale of the data is known and the row window reaches 6.5 standard deviations
             if (sd > 0.0 && step > 0.0f && (double)(kSymCells / 2) * (double)step >= 6.5 * sd && inv < 3.0e38f) mode = kModeRows;
             const bool same_key = have_key && hid == cur_hid && __float_as_uint(inv) == cur_inv_bits && mode == cur_mode;
@@ -473,9 +493,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
         __syncthreads();
 
         // ---- stream the run
-        const int64_t off = (int64_t)(t - t_first) * kTile;
-        const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
-        const float *x = reinterpret_cast<const float *>(a.map.seg_ptr[s]) + off;
         TG *gout = nullptr;
         if constexpr (GRAD) {
             if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
