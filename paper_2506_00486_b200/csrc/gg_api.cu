@@ -34,6 +34,7 @@ struct Plan {
     TileMap map{};
     TileScratch part{};
     double *params = nullptr;     // [2 * n_seg] device staging for host-supplied (beta, alpha)
+    double *sd = nullptr;         // [n_seg] standard deviations, written by the fit of a fused call for its second sweep
     uint64_t last_use = 0;
 };
 
@@ -184,6 +185,7 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     const size_t o_min = take(sizeof(float) * (size_t)n_tiles);
     const size_t o_max = take(sizeof(float) * (size_t)n_tiles);
     const size_t o_par = take(sizeof(double) * 2 * (size_t)n_seg);
+    const size_t o_sd = take(sizeof(double) * (size_t)n_seg);
     const size_t total = off > 0 ? off : 256;
 
     std::vector<char> host(table_bytes > 0 ? table_bytes : 1, 0);
@@ -216,6 +218,7 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     p->part.xmin = reinterpret_cast<float *>(d + o_min);
     p->part.xmax = reinterpret_cast<float *>(d + o_max);
     p->params = reinterpret_cast<double *>(d + o_par);
+    p->sd = reinterpret_cast<double *>(d + o_sd);
     p->last_use = ctx->clock;
     *out = p.get();
     ctx->plans.push_back(std::move(p));
@@ -637,9 +640,10 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
                 GG_CUDA(ctx, launch_sweep(ctx, kMoments, in_dt, g_dt, false, sa, cs));
             }
+            fa.sd_out = p->sd;
             GG_CUDA(ctx, launch_fit(fa, cs));
             ctx->launches += 1 + (p->n_tiles > 0);
-            sa.beta = a->beta; sa.alpha = a->alpha;
+            sa.beta = a->beta; sa.alpha = a->alpha; sa.seg_sd = p->sd;
             sa.step = fa.step_from_alpha ? a->step_out : a->step;
             if (tail_flags) {
                 SweepTimer tm(ctx, &ctx->ev_tail, cs);

@@ -62,6 +62,9 @@ struct StreamArgs {
     int32_t qmin, qmax;
     uint64_t *hist;
     uint64_t *clamped;   // [2 * n_hist] or null
+    // standard deviation of every segment when the caller knows it (the fit of the same call wrote it), else null:
+    // it places the count windows; without it the sweeps take the scale from a sample of each run
+    const double *seg_sd;
 };
 
 struct FitArgs {
@@ -71,6 +74,7 @@ struct FitArgs {
     int64_t *count;
     uint32_t *flags;
     const double *seed;       // the fit table (launch_fit_seed_table), or null: search with lgamma evaluations
+    double *sd_out;           // [n_seg] or null: sqrt(sum_sq / count) of every segment, for the sweep that follows
     int step_from_alpha;
     double step_scale;
     float *step_out;

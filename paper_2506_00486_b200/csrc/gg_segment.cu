@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
                 flags |= GG_FLAG_CLAMPED_SYMBOLS;
         }
         if (a.flags) a.flags[s] = flags;
+        if (a.sd_out) a.sd_out[s] = (len > 0 && s2 > 0.0) ? sqrt(s2 / (double)len) : 0.0;
     }
 }
 

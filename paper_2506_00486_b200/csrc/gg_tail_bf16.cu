@@ -55,7 +55,6 @@ enum : int { kModePattern = 1, kModeSymbol = 2 };
 // memory so that the streaming loop does not carry them in registers.
 struct Cold {
     double L, b;               // g = 2^(L + b log2|x|)
-    double sd;                 // standard deviation of the density the gradient belongs to
     uint32_t sign_flip;        // 0x80000000 if lambda < 0 (the tables then hold -|g|)
     int active;                // 0: the gradient is zero everywhere
     float inv;                 // quantiser: q = floor(x * inv)
@@ -590,7 +589,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         for (int i = tid; i < kSymWin; i += kThreads) sm.win[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
-    if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.symbol_mode = 0; sm.cold.sd = 0.0; }
+    if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.symbol_mode = 0; }
     int cur_hid = -1, cur_mode = kModePattern;
     uint32_t cur_inv_bits = 0;
     bool have_key = false;
@@ -625,8 +624,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                 sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
                 sm.cold.active = active;
                 sm.cold.L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
-                // the standard deviation of the fitted density (Eq. 2-3) places the count windows
-                sm.cold.sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
             }
             __syncthreads();
             const double L = sm.cold.L, b = sm.cold.b;
@@ -666,11 +663,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             // the scale of the data is known, else where it is (same key) or from four binades below
             // the step upwards (new key)
             uint32_t want_base = sm.cold.c_base;
-            double sd = GRAD ? sm.cold.sd : 0.0;
-            if constexpr (!GRAD) {
-                // Without parameters the scale of the data is taken from the first elements of the run (up to
-                // eight per thread): it only decides how the counts are laid out, never what is counted.
-                const int m = (int)min(n, (int64_t)kThreads * 8);
+            double sd = 0.0;
+            if (a.seg_sd != nullptr) {
+                sd = a.seg_sd[s];
+            } else {
+                // Without parameters the scale of the data is taken from the first elements of the run (one
+                // per thread): it only decides how the counts are laid out, never what is counted.
+                const int m = (int)min(n, (int64_t)kThreads);
                 float ss = 0.0f;
                 for (int i = tid; i < m; i += kThreads) {
                     const float v = __uint_as_float((uint32_t)__ldg(x + i) << 16);

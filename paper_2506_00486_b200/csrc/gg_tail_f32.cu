@@ -23,6 +23,7 @@
 #include <float.h>
 
 #include "gg_device.cuh"
+#include "gg_fit_table.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -40,7 +41,6 @@ enum : int { kModeWords = 1, kModeRows = 2 };
 // Constants of the current segment / histogram that only the cold paths need.
 struct Cold {
     double L, b;               // g = 2^(L + b log2|x|)
-    double sd;                 // standard deviation of the density the gradient belongs to
     uint32_t sign_flip;        // 0x80000000 if lambda < 0 (the tables then hold -|g|)
     int active;                // 0: the gradient is zero everywhere
     float inv;                 // quantiser: q = floor(x * inv)
@@ -55,6 +55,8 @@ struct Smem {
     uint32_t cnt[kCntWords];
     uint4 stage[kDepth][2][kThreads];   // per-thread ring: two 16-byte vectors (eight elements) per slot
     float brep[128 * 32];               // row j: B[j] = (1 + j/128)^b in every bank
+    float B[128];
+    double lg[128];                     // log2(1 + j/128)
     double red[kWarps];
     uint32_t clampc[2];
     Cold cold;
@@ -385,7 +387,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
         for (int i = tid; i < (int)kCntWords; i += kThreads) sm.cnt[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
-    if (tid == 0) { sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.rows_mode = 0; sm.cold.sd = 0.0; sm.cold.L = 0.0; sm.cold.b = 0.0; }
+    if (tid == 0) { sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.rows_mode = 0; sm.cold.L = 0.0; sm.cold.b = 0.0; }
+    if (tid < 128) sm.lg[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
     int cur_hid = -1, cur_mode = kModeWords;
     uint32_t cur_inv_bits = 0;
     bool have_key = false;
@@ -417,8 +420,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
                 sm.cold.L = L;
                 sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
                 sm.cold.active = active;
-                // the standard deviation of the fitted density (Eq. 2-3) decides the count layout
-                sm.cold.sd = active ? alpha * exp(0.5 * (lgamma(3.0 / beta) - lgamma(1.0 / beta))) : 0.0;
             }
             if (tid < 256) {
                 // One factor serves exponent k if |L + b (k-127)| <= 100 (its product with B, at most 2^2
@@ -428,15 +429,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
                 if (active) {
                     const double e0 = L + b * (double)(tid - 127);
                     const bool ok = tid >= 1 && tid <= 254 && fabs(e0) <= 100.0 && fabs(b) <= 2.0;
-                    one = ok ? (float)(lam < 0.0 ? -exp2(e0) : exp2(e0)) : __int_as_float(0x7FC00000);
+                    one = ok ? (float)(lam < 0.0 ? -exp2_short(e0) : exp2_short(e0)) : __int_as_float(0x7FC00000);
                 }
                 s_a1[tid] = one;
             } else if (tid < 384) {
                 const int j = tid - 256;
-                // B[j] into every bank of row j
-                const float v = active ? (float)exp2(b * log2(1.0 + (double)j * (1.0 / 128.0))) : 1.0f;
-                for (int q = 0; q < 32; ++q) sm.brep[j * 32 + q] = v;
+                sm.B[j] = active ? (float)exp2_short(b * sm.lg[j]) : 1.0f;
             }
+            __syncthreads();
+            for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];      // B[j] into every bank of row j
             const float bf = (float)b;
             ln.c1 = bf;
             ln.c2 = ln.c1 * (bf - 1.0f) * 0.5f;
@@ -447,12 +448,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
             const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
             const float step = a.step[s];
             const float inv = (float)(1.0 / (double)step);
-            __syncthreads();                        // (sm.cold.sd of this run is written)
-            double sd = GRAD ? sm.cold.sd : 0.0;
-            if constexpr (!GRAD) {
-                // Without parameters the scale of the data is taken from the first elements of the run (up to
-                // eight per thread): it only decides how the counts are laid out, never what is counted.
-                const int m = (int)min(n, (int64_t)kThreads * 8);
+            __syncthreads();
+            double sd = 0.0;
+            if (a.seg_sd != nullptr) {
+                sd = a.seg_sd[s];
+            } else {
+                // The scale of the data is taken from the first elements of the run (one per thread):
+                // it only decides how the counts are laid out, never what is counted.
+                const int m = (int)min(n, (int64_t)kThreads);
                 float ss = 0.0f;
                 for (int i = tid; i < m; i += kThreads) {
                     const float v = __ldg(x + i);
