@@ -200,7 +200,8 @@ typedef struct {
 /* The whole pass over a list of segments in the fewest sweeps of x: moments -> fit ->
  * penalty + gradient + histogram -> entropy, all enqueued on `stream`.
  * GG_PARAMS_FITTED reads x twice (the gradient needs the fit of the whole segment);
- * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep).
+ * GG_PARAMS_GIVEN reads bf16 x once (moments, gradient and histogram in the same sweep; fp32 x takes two
+ * sweeps in either mode).
  * The first call with a new layout (segment addresses and lengths) builds and caches its plan with
  * blocking allocations; later calls with that layout only enqueue kernels and memsets on `stream`
  * and may be captured in a CUDA graph (the same holds for gg_fused_channels once its scratch is

@@ -654,7 +654,17 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         } else {
             // one sweep: moments, gradient (given parameters) and histogram together; then the fit
             sa.beta = a->beta_in; sa.alpha = a->alpha_in; sa.step = a->step;
-            {
+            if (in_dt == GG_F32 && tail_flags != 0) {
+                // fp32 input has no combined persistent sweep: the moments kernel and the gradient + histogram
+                // kernel, both streaming at their own speed, beat the generic kernel that does all three at once
+                {
+                    SweepTimer tm(ctx, &ctx->ev_first, cs);
+                    GG_CUDA(ctx, launch_sweep(ctx, kMoments, in_dt, g_dt, false, sa, cs));
+                }
+                SweepTimer tm(ctx, &ctx->ev_tail, cs);
+                GG_CUDA(ctx, launch_sweep(ctx, tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
+                ctx->launches += p->n_tiles > 0;
+            } else {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
                 GG_CUDA(ctx, launch_sweep(ctx, kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
             }
