@@ -32,6 +32,7 @@
 #include <float.h>
 
 #include "gg_device.cuh"
+#include "gg_fit_table.cuh"
 #include "gg_internal.h"
 
 namespace gg {
@@ -74,6 +75,7 @@ struct Smem {
     float brep[128 * 32];            // row j: B[j] in every bank
     float2 A[256];                   // every exponent: value = A.x * A.y, A.y a power of two
     float B[128];
+    double lg[128];                  // log2(1 + j/128)
     uint32_t win[kSymWin];
     double red[3][kWarps];
     uint32_t bad[kWarps];
@@ -589,6 +591,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         for (int i = tid; i < kSymWin; i += kThreads) sm.win[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
+    if (tid < 128) sm.lg[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
     if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.symbol_mode = 0; }
     int cur_hid = -1, cur_mode = kModePattern;
     uint32_t cur_inv_bits = 0;
@@ -619,21 +622,22 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             const double beta = a.beta[s], alpha = a.alpha[s];
             const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
             active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
+            // (every thread works the two constants out for itself: cheaper than a broadcast and its barrier)
+            const double b = beta - 1.0;
+            const double L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
             if (tid == 0) {
-                sm.cold.b = beta - 1.0;
+                sm.cold.b = b;
                 sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
                 sm.cold.active = active;
-                sm.cold.L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
+                sm.cold.L = L;
             }
-            __syncthreads();
-            const double L = sm.cold.L, b = sm.cold.b;
             if (tid < 256) {
                 const int k = tid;
                 float2 v = make_float2(0.0f, 1.0f);
                 if (active && k >= 1 && k <= 254) {
                     const double e0 = L + b * (double)(k - 127);
                     double ip = rint(e0);
-                    const double f = exp2(e0 - ip);
+                    const double f = exp2_short(e0 - ip);
                     ip = fmin(fmax(ip, -400.0), 400.0);
                     const int ii = (int)ip;
                     const int i1 = max(-100, min(100, ii));
@@ -649,7 +653,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
                 s_a1[k] = one;
             } else if (tid < 384) {
                 const int k = tid - 256;
-                sm.B[k] = active ? (float)exp2(b * log2(1.0 + (double)k * (1.0 / 128.0))) : 1.0f;
+                sm.B[k] = active ? (float)exp2_short(b * sm.lg[k]) : 1.0f;
             }
             __syncthreads();
             for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
