@@ -73,7 +73,7 @@ typedef struct {
 
 #define GG_PARAMS_FITTED 0   /* penalty uses the (beta, alpha) fitted by this call: two reads of x */
 #define GG_PARAMS_GIVEN  1   /* penalty uses caller-supplied (beta, alpha); the fit of this call is
-                                still produced: one read of x                                    */
+                                still produced: one read of bf16 x                               */
 #define GG_STEP_GIVEN      0 /* quantiser step[s] supplied by the caller                        */
 #define GG_STEP_FROM_ALPHA 1 /* step[s] = (float)(fitted alpha[s] * step_scale), also written out */
 
