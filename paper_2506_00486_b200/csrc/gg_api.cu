@@ -251,7 +251,10 @@ struct SweepTimer {
 cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
                          const StreamArgs &sa, cudaStream_t cs)
 {
-    if (in_dtype == GG_BF16 && flags == kMoments) return launch_moments_bf16_sweep(sa, ctx->sm_count, cs);
+    // moments alone: persistent CTAs pay a block reduction per run of tiles instead of one per tile, which wins
+    // for long bf16 segments (fp32 input and short segments stream as fast tile by tile)
+    if (flags == kMoments && in_dtype == GG_BF16 && (int64_t)sa.map.n_tiles >= 16 * (int64_t)sa.map.n_seg)
+        return launch_moments_bf16_sweep(sa, ctx->sm_count, cs);
     if (in_dtype == GG_BF16 && (flags & (kGrad | kHist)) != 0)
         return launch_tail_bf16(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
     if (in_dtype == GG_F32 && (flags & kMoments) == 0 && flags != 0)
