@@ -318,7 +318,8 @@ typedef struct {
  * column are reduced in a fixed order.  GG_FLAG_CLAMPED_SYMBOLS is set per column when a histogram
  * is taken.  The first call with a larger matrix than any before allocates scratch (blocking).
  * Errors: GG_ERR_DTYPE for an unknown dtype, GG_ERR_INVALID_ARG for ld < cols, negative sizes, a missing
- * required pointer or qmin > qmax, GG_ERR_ALIGNMENT for x or grad not element aligned. */
+ * required pointer, qmin > qmax or a step that is not a positive finite number, GG_ERR_ALIGNMENT for x or
+ * grad not element aligned, GG_ERR_WORKSPACE for more than 65535 * 512 rows. */
 gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *args, void *stream);
 
 /* Moments and fit of ONE segment without allocating anything (the paper has no counterpart: this is
