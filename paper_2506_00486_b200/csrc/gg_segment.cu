@@ -162,12 +162,19 @@ entropy_partial_kernel(const uint64_t *hist, int32_t n_bins, double *part)
     const int k0 = slice * per, k1 = min(n_bins, k0 + per);
     double acc = 0.0;
     unsigned long long tot = 0;
-    for (int k = k0 + threadIdx.x; k < k1; k += kEntThreads) {
-        const uint64_t c = row[k];
-        if (c != 0) {
-            const double cd = (double)c;
-            acc += cd * log2(cd);
-            tot += c;
+    // (four independent loads per trip: most bins are empty, so the loop is bound by load latency; the order in
+    // which a thread adds its bins stays fixed)
+    for (int k = k0 + threadIdx.x; k < k1; k += 4 * kEntThreads) {
+        uint64_t c[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) c[u] = k + u * kEntThreads < k1 ? __ldg(row + k + u * kEntThreads) : 0ull;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (c[u] != 0) {
+                const double cd = (double)c[u];
+                acc += cd * log2(cd);
+                tot += c[u];
+            }
         }
     }
     acc = warp_sum(acc);
