@@ -9,7 +9,7 @@ namespace gg {
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kSegThreads = 128;   // one CTA of 4 warps per segment
+constexpr int kSegThreads = 256;   // one CTA of 8 warps per segment
 
 // ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
 // of the density of Eq. 1; increasing in beta from 0 to 3/4.
@@ -18,8 +18,8 @@ __device__ __forceinline__ double log_rho(double beta)
     return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
 }
 
-// One CTA of four warps per segment.  The threads sum the tile partials in a fixed order (strided over
-// the 128 threads, a butterfly in each warp, the four warps in sequence, so every thread of warp 0 ends
+// One CTA of eight warps per segment.  The threads sum the tile partials in a fixed order (strided over
+// the 256 threads, a butterfly in each warp, the eight warps in sequence, so every thread of warp 0 ends
 // with the same bits), then warp 0 inverts the moment ratio: from the context's fit
 // table when there is one, else by 33-section search on
 // ln(beta): each round the 32 lanes evaluate log_rho at the interior points of the bracket and a
