@@ -18,7 +18,7 @@ using namespace gg;
 namespace {
 
 constexpr int kMaxPlans = 64;
-constexpr int64_t kDefaultChunkBytes = 1ll << 30;
+constexpr int64_t kDefaultChunkBytes = 512ll << 20;     // (256 - 512 MiB measured best: the tail of the last chunk is what is not overlapped)
 
 // A plan is everything that depends only on the layout of a call: segment addresses and lengths,
 // gradient addresses, histogram ids.  It owns the device tables and the per-tile scratch.
