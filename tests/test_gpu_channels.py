@@ -212,3 +212,25 @@ def test_channels_matrix_with_more_than_2_to_31_elements(ctx):
     gs = torch.stack([g[:, c] for c in sample], dim=1).cpu()
     sub = {k: (v[sample] if isinstance(v, torch.Tensor) and v.numel() == cols else v) for k, v in oc.items()}
     check_channels(sub, xs, gs, 1e-4, cols=list(range(len(sample))))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_channels_random_shapes_and_alignments(ctx, dtype):
+    """Random small matrices: any row and column count, padded or not, first element at any element offset from a
+    256-byte boundary (aligned and unaligned rows for the vector paths), fp32 and bf16 gradients."""
+    rng = np.random.default_rng(46)
+    for case in range(10):
+        rows, cols = int(rng.integers(1, 700)), int(rng.integers(1, 150))
+        ld = cols + int(rng.integers(0, 4))
+        off = int(rng.integers(0, 8))
+        gdt = torch.bfloat16 if case % 3 == 2 else torch.float32
+        x = channel_matrix(rows, cols, seed=100 + case, wide_scales=(case % 2 == 0), dtype=dtype)
+        flat = torch.zeros(rows * ld + 16, dtype=dtype, device="cuda:0")
+        xd = flat[off:off + rows * ld].view(rows, ld)[:, :cols]
+        xd.copy_(x)
+        gflat = torch.zeros(rows * ld + 16, dtype=gdt, device="cuda:0")
+        gd = gflat[off:off + rows * ld].view(rows, ld)[:, :cols]
+        step = float(2.0 ** rng.integers(-9, -3))
+        out = ctx.gg_fused_channels(xd, grad=gd, lam=3e-4, step=step, qmin=-5000, qmax=4000)
+        torch.cuda.synchronize()
+        check_channels(cpu(out), x, gd.cpu(), 3e-4, step=step, qmin=-5000, qmax=4000)
