@@ -650,3 +650,27 @@ def test_more_layouts_than_cached_plans(ctx):
             out = ctx.gg_fit([t])
             assert_rel(out["beta"][0].item(), refs[i][0], REL_FIT, f"beta[{i}] round {rnd}")
             assert_rel(out["alpha"][0].item(), refs[i][1], REL_FIT, f"alpha[{i}] round {rnd}")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fused_random_layouts(ctx, dtype):
+    """Random segment lists: any number of segments of any length from 0 to a few tiles at any element offset,
+    grouped at random into shared histograms, sum or mean reduction.  Short and long bf16 lists take different
+    kernels; every list must give the oracle's results."""
+    from paper_2506_00486_b200 import Segments, GG_MEAN, GG_SUM
+    rng = np.random.default_rng(47)
+    for case in range(8):
+        n_seg = int(rng.integers(1, 90)) if case % 2 else int(rng.integers(64, 130))
+        cap = 9000 if case % 2 else 3 * TILE
+        lens = [int(np.exp(rng.uniform(0, np.log(cap)))) - 1 for _ in range(n_seg)]
+        xs = [gg_synth.gg_host(rng, float(rng.uniform(0.5, 2.2)), 10.0 ** rng.uniform(-3, 0), n, dtype) for n in lens]
+        xd = misaligned_views(xs, offsets=[int(rng.integers(0, 8)) for _ in xs])
+        gd = [torch.empty(n, dtype=torch.float32, device="cuda:0") for n in lens]
+        n_hist = int(rng.integers(1, 4))
+        hid = [int(rng.integers(0, n_hist)) for _ in xs]
+        steps = torch.full((n_seg,), float(2.0 ** rng.integers(-9, -4)), dtype=torch.float32, device="cuda:0")
+        mean = bool(case & 4)
+        out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=2e-4, step=steps, hist_id=hid, n_hist=n_hist,
+                           reduction=GG_MEAN if mean else GG_SUM, qmin=-3000, qmax=2500)
+        torch.cuda.synchronize()
+        check_fused(out, xs, gd, 2e-4, hid, n_hist, qmin=-3000, qmax=2500, mean=mean)
