@@ -428,36 +428,44 @@ void ggo_eg_rate_grad(const float *x, int64_t n, float step, int32_t qmin, int32
 
 /* ------------------------------------------------ Huffman and fixed-length bits */
 
-static int ggo_cmp_u64(const void *a, const void *b)
-{
-    const uint64_t x = *(const uint64_t *)a, y = *(const uint64_t *)b;
-    return x < y ? -1 : x > y;
-}
-
-/* Average length in bits of a Huffman code for the counts (textbook construction: repeatedly merge
- * the two lightest nodes; the average length is the sum of the merged weights over the total).
- * One occupied bin gives 0 bits.  work: scratch of 2 * n_bins uint64. */
+/* Average length in bits of a Huffman code for the counts, by the textbook construction written out:
+ * every occupied bin is a leaf; while more than one root is left, the two lightest roots (found by a
+ * scan of the whole list) become the children of a new root whose weight is their sum; the code
+ * length of a symbol is the depth of its leaf; the average is sum(count * length) / sum(count).
+ * One occupied bin gives 0 bits.  Quadratic in the number of occupied bins: a checker, not a coder.
+ * work: scratch of 2 * n_bins uint64 (node weights); parent links and root marks are allocated here. */
 double ggo_huffman_bits(const uint64_t *hist, int64_t n_bins, uint64_t *work)
 {
     int64_t n = 0;
-    long double total = 0.0L;
-    for (int64_t b = 0; b < n_bins; ++b) if (hist[b]) { work[n++] = hist[b]; total += (long double)hist[b]; }
+    for (int64_t b = 0; b < n_bins; ++b) if (hist[b]) work[n++] = hist[b];
     if (n <= 1) return 0.0;
-    qsort(work, (size_t)n, sizeof(uint64_t), ggo_cmp_u64);
-    /* two queues: leaves work[0..n) in ascending order, merged nodes in creation order (also ascending) */
-    uint64_t *merged = work + n_bins;
-    int64_t li = 0, mi = 0, mn = 0;
-    long double sum = 0.0L;
-    for (int64_t step = 0; step < n - 1; ++step) {
-        uint64_t pick[2];
-        for (int j = 0; j < 2; ++j) {
-            if (mi >= mn || (li < n && work[li] <= merged[mi])) pick[j] = work[li++];
-            else pick[j] = merged[mi++];
+    int64_t *parent = (int64_t *)malloc(sizeof(int64_t) * (size_t)(2 * n));
+    char *is_root = (char *)malloc((size_t)(2 * n));
+    if (!parent || !is_root) { free(parent); free(is_root); return NAN; }
+    for (int64_t i = 0; i < n; ++i) { parent[i] = -1; is_root[i] = 1; }
+    int64_t nodes = n;
+    for (int64_t roots = n; roots > 1; --roots) {
+        int64_t first = -1, second = -1;       /* the lightest and the next lightest root */
+        for (int64_t i = 0; i < nodes; ++i) {
+            if (!is_root[i]) continue;
+            if (first < 0 || work[i] < work[first]) { second = first; first = i; }
+            else if (second < 0 || work[i] < work[second]) second = i;
         }
-        merged[mn++] = pick[0] + pick[1];
-        sum += (long double)(pick[0] + pick[1]);
+        work[nodes] = work[first] + work[second];
+        parent[nodes] = -1; is_root[nodes] = 1;
+        parent[first] = nodes; parent[second] = nodes;
+        is_root[first] = 0; is_root[second] = 0;
+        ++nodes;
     }
-    return (double)(sum / total);
+    long double bits = 0.0L, total = 0.0L;
+    for (int64_t leaf = 0; leaf < n; ++leaf) {
+        int64_t depth = 0;
+        for (int64_t v = leaf; parent[v] >= 0; v = parent[v]) ++depth;
+        bits += (long double)work[leaf] * (long double)depth;
+        total += (long double)work[leaf];
+    }
+    free(parent); free(is_root);
+    return (double)(bits / total);
 }
 
 /* Bits of a fixed-length code over the occupied symbol range: ceil(log2(max - min + 1)); an empty

@@ -9,6 +9,7 @@
 #include <memory>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "gg_internal.h"
@@ -978,38 +979,52 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
 
 namespace {
 
-// Average Huffman code length of the non-zero counts: sort, then merge the two lightest nodes with
-// two queues (leaves in ascending order, merged nodes in creation order).
-double huffman_bits(const uint64_t *row, int64_t n_bins, std::vector<uint64_t> &leaves, std::vector<uint64_t> &merged)
-{
-    leaves.clear();
-    long double total = 0.0L;
-    for (int64_t b = 0; b < n_bins; ++b)
-        if (row[b]) { leaves.push_back(row[b]); total += (long double)row[b]; }
-    const size_t n = leaves.size();
-    if (n <= 1) return 0.0;
-    std::sort(leaves.begin(), leaves.end());
-    merged.assign(n, 0);
-    size_t li = 0, mi = 0, mn = 0;
-    long double sum = 0.0L;
-    for (size_t it = 0; it + 1 < n; ++it) {
-        uint64_t pick[2];
-        for (int j = 0; j < 2; ++j) {
-            if (mi >= mn || (li < n && leaves[li] <= merged[mi])) pick[j] = leaves[li++];
-            else pick[j] = merged[mi++];
-        }
-        merged[mn++] = pick[0] + pick[1];
-        sum += (long double)(pick[0] + pick[1]);
-    }
-    return (double)(sum / total);
-}
+// Index of the highest set bit of v (v > 0).
+inline int top_bit(uint64_t v) { return 63 - __builtin_clzll(v); }
 
-int eg_length_host(uint64_t m, int k)
+// Average Huffman code length of the occupied bins of one count table.  The tree is grown with a binary
+// min-heap of (weight, node): the two lightest nodes get a common parent until one root is left.  A parent
+// is always created after its children, so one pass from the root down the node numbers gives every depth;
+// the code length of a symbol is the depth of its leaf and the total sum(count * length) stays an integer
+// (128 bits wide: counts go up to 2^63 and depths up to the number of leaves).
+struct HuffmanScratch {
+    std::vector<uint64_t> weight;
+    std::vector<uint32_t> up, depth;
+    std::vector<std::pair<uint64_t, uint32_t>> heap;
+};
+
+double huffman_bits(const uint64_t *row, int64_t n_bins, HuffmanScratch &w)
 {
-    uint64_t v = m + (1ull << k);
-    int fl = -1;
-    while (v) { v >>= 1; ++fl; }
-    return 2 * fl - k + 1;
+    w.weight.clear();
+    for (int64_t b = 0; b < n_bins; ++b)
+        if (row[b] != 0) w.weight.push_back(row[b]);
+    const uint32_t n_leaf = (uint32_t)w.weight.size();
+    if (n_leaf < 2) return 0.0;
+    const uint32_t n_node = 2 * n_leaf - 1;
+    w.weight.resize(n_node);
+    w.up.assign(n_node, n_node);
+    w.heap.clear();
+    for (uint32_t i = 0; i < n_leaf; ++i) w.heap.emplace_back(w.weight[i], i);
+    const auto heavier = [](const std::pair<uint64_t, uint32_t> &x, const std::pair<uint64_t, uint32_t> &y) { return x > y; };
+    std::make_heap(w.heap.begin(), w.heap.end(), heavier);
+    for (uint32_t node = n_leaf; node < n_node; ++node) {
+        uint64_t sum = 0;
+        for (int child = 0; child < 2; ++child) {
+            std::pop_heap(w.heap.begin(), w.heap.end(), heavier);
+            sum += w.heap.back().first;
+            w.up[w.heap.back().second] = node;
+            w.heap.pop_back();
+        }
+        w.weight[node] = sum;
+        w.heap.emplace_back(sum, node);
+        std::push_heap(w.heap.begin(), w.heap.end(), heavier);
+    }
+    w.depth.assign(n_node, 0);
+    for (uint32_t v = n_node - 1; v-- > 0;) w.depth[v] = w.depth[w.up[v]] + 1;
+    unsigned __int128 bits = 0;
+    for (uint32_t i = 0; i < n_leaf; ++i) bits += (unsigned __int128)w.weight[i] * w.depth[i];
+    // the root's weight is the number of symbols
+    return (double)((long double)bits / (long double)w.weight[n_node - 1]);
 }
 
 }  // namespace
@@ -1066,29 +1081,31 @@ gg_status gg_code_stats(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     GG_CUDA(ctx, cudaMemcpyAsync(host.data(), hist, sizeof(uint64_t) * host.size(), cudaMemcpyDeviceToHost, cs));
     GG_CUDA(ctx, cudaStreamSynchronize(cs));
-    std::vector<uint64_t> leaves, merged;
+    HuffmanScratch scratch;
     for (int32_t h = 0; h < n_hist; ++h) {
         const uint64_t *row = host.data() + (size_t)h * (size_t)n_bins;
+        // occupied range of the table (first > last: empty)
+        int64_t first = 0, last = n_bins - 1;
+        while (first <= last && row[first] == 0) ++first;
+        while (last >= first && row[last] == 0) --last;
         if (eg_bits) {
-            long double bits = 0.0L, total = 0.0L;
-            for (int64_t b = 0; b < n_bins; ++b) {
-                if (!row[b]) continue;
+            // a k-th order code spends 2 * top_bit(m + 2^k) - k + 1 bits on the unsigned symbol m; the mapping
+            // of Eq. 6 interleaves the signs, m = 2|q| - [q > 0]
+            unsigned __int128 bits = 0;
+            uint64_t symbols = 0;
+            for (int64_t b = first; b <= last; ++b) {
+                const uint64_t c = row[b];
+                if (c == 0) continue;
                 const int64_t q = (int64_t)qmin + b;
-                const uint64_t m = q < 0 ? (uint64_t)(-2 * q) : (q == 0 ? 0 : (uint64_t)(2 * q - 1));
-                bits += (long double)row[b] * (long double)eg_length_host(m, k);
-                total += (long double)row[b];
+                const uint64_t m = 2 * (uint64_t)(q < 0 ? -q : q) - (q > 0 ? 1u : 0u);
+                bits += (unsigned __int128)c * (uint64_t)(2 * top_bit(m + (1ull << k)) - k + 1);
+                symbols += c;
             }
-            eg_bits[h] = total > 0.0L ? (double)(bits / total) : 0.0;
+            eg_bits[h] = symbols != 0 ? (double)((long double)bits / (long double)symbols) : 0.0;
         }
-        if (hm_bits) hm_bits[h] = huffman_bits(row, n_bins, leaves, merged);
-        if (fl_bits) {
-            int64_t lo = -1, hi = -1;
-            for (int64_t b = 0; b < n_bins; ++b) if (row[b]) { if (lo < 0) lo = b; hi = b; }
-            uint64_t span = lo < 0 ? 0 : (uint64_t)(hi - lo);
-            int bits = 0;
-            while (span) { span >>= 1; ++bits; }
-            fl_bits[h] = (double)bits;
-        }
+        if (hm_bits) hm_bits[h] = huffman_bits(row, n_bins, scratch);
+        // a fixed-length code numbers the last - first + 1 symbols of the occupied range
+        if (fl_bits) fl_bits[h] = last > first ? (double)(top_bit((uint64_t)(last - first)) + 1) : 0.0;
     }
     return GG_OK;
 }

@@ -77,6 +77,47 @@ def test_eg_rate_gradient_is_the_derivative_of_the_relaxed_rate():
     assert fd == pytest.approx(2 / ((m + 2 ** k) * math.log(2.0)), rel=1e-8)
 
 
+@pytest.mark.parametrize("k, qmin, qmax", [(0, -32768, 32767), (3, -32768, 32767), (1, -5, 4)])
+def test_eg_rate_gradient_against_a_numerical_derivative_in_mpmath(k, qmin, qmax):
+    """The relaxed rate (Eq. 6-7 with floor and Map taken as straight-through: slopes 1/step and 2) is
+    R(d) = (1/N) sum_j 2 log2(M_j + 2 (|x_j + d_j| - |x_j|) / step + 2^k) with M_j the mapped symbol of the
+    quantised x_j.  Its partial derivatives at d = 0, taken numerically in 40-digit arithmetic, are what
+    the dR/dG line of the GCT section states.  Symbols are computed here in numpy fp32, not by the oracle."""
+    mpmath = pytest.importorskip("mpmath")
+    mp = mpmath.mp
+    rng = np.random.default_rng(19)
+    n = 72
+    x = gg_synth.gg_host(rng, 0.9, 0.2, n).numpy().astype(np.float32)
+    x[:4] = [0.0, -0.0, 3e-7, -3e-7]                    # zeros: no gradient; a tiny negative value falls in symbol -1
+    x[4:6] = [7.5, -7.5]                                # clamped under the narrow range
+    step, lam = np.float32(2.0 ** -5), 0.81
+    inv = np.float32(1.0 / np.float64(step))
+    q = np.clip(np.floor((x * inv).astype(np.float32)).astype(np.int64), qmin, qmax)
+    M = [(-2 * int(v)) if v < 0 else (0 if v == 0 else 2 * int(v) - 1) for v in q]
+    assert any(v in (qmin, qmax) for v in q) == (qmax < 100)
+    got = o.eg_rate_grad(x, float(step), lam, k, qmin, qmax)
+    old = mp.dps
+    mp.dps = 40
+    try:
+        xs = [mpmath.mpf(float(v)) for v in x]
+        for i in range(n):
+            if x[i] == 0:
+                assert got[i] == 0.0
+                continue
+
+            def rate(d, i=i):
+                tot = mpmath.mpf(0)
+                for j in range(n):
+                    dj = d if j == i else 0
+                    tot += 2 * mpmath.log(M[j] + 2 * (abs(xs[j] + dj) - abs(xs[j])) / mpmath.mpf(float(step)) + 2 ** k, 2)
+                return lam * tot / n
+
+            want = mpmath.diff(rate, 0, h=mpmath.mpf(10) ** -12)
+            assert float(abs(got[i] - want) / abs(want)) < 1e-13, (i, got[i], want)
+    finally:
+        mp.dps = old
+
+
 def _huffman_heap(counts):
     h = [int(c) for c in counts if c]
     if len(h) <= 1:
@@ -149,3 +190,23 @@ def test_gct_step_follows_algorithm_2():
     # a gradient equal to the stored one (and eps = 0) has zero curvature estimate: nothing is added
     gh, _ = o.gct_step(g, g.astype(np.float64), w, step, eta, lam, 0.0, t=5)
     np.testing.assert_allclose(gh, g.astype(np.float64), rtol=0, atol=1e-18)
+
+
+def test_gct_step_hand_computed_case():
+    """Algorithm 2 on three elements, every intermediate written down.
+    step 1/4, k = 0: g = (1/2, -1/4, 1/8) scales to (2, -1, 1/2), symbols (2, -1, 0), Eq. 6 maps them to (3, 2, 0).
+    dR/dg = 4 * 4 / (3 ln 2) * sign / (m + 1) = 7.694373551407805 * (1/4, -1/3, 1).
+    eta = 1/2, eps = 1/4, stored gradients (3/4, -3/4, 1): h = 2 - 2 g / (stored + eps) = (1, 1, 9/5).
+    lambda = 1/8: ghat = g + lambda * dR/dg * h;  w = (1, 2, 3) - eta * ghat."""
+    g = np.array([0.5, -0.25, 0.125], dtype=np.float32)
+    stored = np.array([0.75, -0.75, 1.0])
+    w = np.array([1.0, 2.0, 3.0])
+    dr = o.eg_rate_grad(g, 0.25, 1.0, 0)
+    np.testing.assert_allclose(dr, [1.9235933878519512, -2.5647911838026016, 7.694373551407805], rtol=4e-16)
+    gh, wn = o.gct_step(g, stored, w, 0.25, 0.5, 0.125, 0.25, t=2)
+    np.testing.assert_allclose(gh, [0.7404491734814939, -0.5705988979753252, 1.856234049066756], rtol=4e-16)
+    np.testing.assert_allclose(wn, [0.6297754132592530, 2.2852994489876626, 2.0718829754666220], rtol=4e-16)
+    # the first step of training has no stored gradient: plain descent
+    gh, wn = o.gct_step(g, stored, w, 0.25, 0.5, 0.125, 0.25, t=1)
+    np.testing.assert_array_equal(gh, [0.5, -0.25, 0.125])
+    np.testing.assert_array_equal(wn, [0.75, 2.125, 2.9375])
