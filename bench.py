@@ -37,6 +37,9 @@ def parse():
                     help="timed steps of the one-read form of the pass (parameters given), 0 to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--one-launch", action="store_true",
+                    help="time the one-launch form of the fitted pass (every tensor handed from its moments to its second "
+                         "read through L2; slower on B200, off by default) instead of the two sweeps")
     return ap.parse_args()
 
 
@@ -250,6 +253,8 @@ def run_ours(args):
     gsegs = Segments.slices(gflat, offs, lens)
     steps_t = torch.full((n_seg,), STEP, dtype=torch.float32, device=dev)
     ctx = Context(local)
+    if args.one_launch:
+        ctx.gg_test_hook(0, 1)
     run = ctx.make_fused(segs, grad=gsegs, lam=LAM, step=steps_t)
     in_bytes = n_elem * 2
     g_bytes = n_elem * gflat.element_size()

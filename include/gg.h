@@ -64,6 +64,8 @@ typedef struct {
 #define GG_FLAG_BETA_CLAMPED_HI 4u   /* moment ratio above rho(GG_BETA_HI): beta = GG_BETA_HI */
 #define GG_FLAG_NONFINITE       8u   /* an entry was inf or nan (left out of the moments)     */
 #define GG_FLAG_CLAMPED_SYMBOLS 16u  /* a quantised symbol fell outside [qmin, qmax]          */
+#define GG_FLAG_TIMEOUT         32u  /* a bounded wait inside the one-launch fitted pass ran out: no
+                                        result of this segment is valid (the context stays usable) */
 
 #define GG_BETA_LO 0.05
 #define GG_BETA_HI 20.0
@@ -270,6 +272,24 @@ gg_status gg_gct_step(gg_ctx *ctx, const gg_seg *g, int32_t n_seg, gg_dtype g_dt
  * milliseconds and the number of launches of each kind since the last read, and forgets them. */
 gg_status gg_timing_enable(gg_ctx *ctx, int enable);
 gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double *ms_tail, int64_t *n_tail);
+
+/* The one-launch form of the fitted pass, and its knobs (no counterpart in the paper).  With bf16 input and
+ * GG_PARAMS_FITTED, gg_fused can run moments, fit and gradient + histogram of every tensor in ONE cooperative
+ * launch: all CTAs walk the tensors together (in groups of about 28 MB), a fitting CTA publishes the parameters
+ * of a group once every streaming CTA has delivered its moments, and the second read of the group follows while L2
+ * still holds it, so DRAM sees less than two reads of x.  On B200 this form is SLOWER than the two-launch form
+ * (the per-group hand-over stalls all CTAs at once, while the two-launch sweeps keep DRAM busy), so it is off
+ * unless switched on here.  CTAs of that launch wait for one another (arrival counters and ready words in the
+ * plan); every such wait gives up after a fixed number of polls, marks the segments GG_FLAG_TIMEOUT and lets the
+ * kernel end, so a wait that cannot be satisfied costs a fraction of a second and leaves the context usable.
+ *   GG_HOOK_RESIDENT_MODE   0 (default): two launches; 1: the one-launch form whenever it can run
+ *   GG_HOOK_EXTRA_ARRIVALS  arrivals the fitting CTA waits for beyond the CTAs that exist (default 0); a positive
+ *                           value makes its wait run out: the way to test the time-out path without any fault
+ *   GG_HOOK_WAIT_CAP        polls (about half a microsecond each) after which a wait gives up (default 2^18) */
+#define GG_HOOK_RESIDENT_MODE  0
+#define GG_HOOK_EXTRA_ARRIVALS 1
+#define GG_HOOK_WAIT_CAP       2
+gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value);
 
 /* The same pass for data that lives in HOST memory: every pointer of `args` that gg_fused documents
  * as device memory (segment data, fit outputs, gradient segments, step, histogram, entropy, ...) is

@@ -18,6 +18,8 @@ GG_SUM, GG_MEAN = 0, 1
 GG_PARAMS_FITTED, GG_PARAMS_GIVEN = 0, 1
 GG_STEP_GIVEN, GG_STEP_FROM_ALPHA = 0, 1
 FLAG_DEGENERATE, FLAG_BETA_CLAMPED_LO, FLAG_BETA_CLAMPED_HI, FLAG_NONFINITE, FLAG_CLAMPED_SYMBOLS = 1, 2, 4, 8, 16
+FLAG_TIMEOUT = 32
+HOOK_RESIDENT_MODE, HOOK_EXTRA_ARRIVALS, HOOK_WAIT_CAP = 0, 1, 2
 BETA_LO, BETA_HI = 0.05, 20.0
 
 _SEG_DTYPE = np.dtype([("ptr", np.uint64), ("len", np.int64)])
@@ -98,6 +100,8 @@ def lib():
         L.gg_timing_enable.argtypes = [_P, ctypes.c_int]
         L.gg_timing_read.argtypes = [_P, ctypes.POINTER(d), ctypes.POINTER(i64), ctypes.POINTER(d),
                                      ctypes.POINTER(i64)]
+        L.gg_test_hook.argtypes = [_P, i32, i64]
+        L.gg_test_hook.restype = ctypes.c_int
         L.gg_fit_noalloc.argtypes = [ctypes.c_int, _P, i64, ctypes.c_int, _P, _P, _P, _P, _P, _P, _P]
         L.gg_fit_noalloc.restype = ctypes.c_int
         L.gg_fit_noalloc_max_len.restype = i64
@@ -275,6 +279,10 @@ class Context:
     @property
     def launch_count(self):
         return lib().gg_launch_count(self._h)
+
+    def gg_test_hook(self, what, value):
+        """Knobs of the one-launch fitted pass (HOOK_*), for tests and measurements."""
+        self._check(lib().gg_test_hook(self._h, int(what), int(value)))
 
     def _new(self, n, dtype):
         return torch.empty(n, dtype=dtype, device=self.device)

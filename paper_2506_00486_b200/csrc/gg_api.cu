@@ -19,6 +19,12 @@ using namespace gg;
 namespace {
 
 constexpr int kMaxPlans = 64;
+// The one-launch fitted pass (off unless switched on by gg_test_hook): a group is what L2 keeps from the first
+// read of a tensor to the second while the gradient of the tensor before streams out (measured on B200: about
+// 30 MB of 126), and at most one segment per warp of the fitting CTA.
+constexpr int64_t kGroupBytes = 28ll << 20;
+constexpr int kGroupSegs = 16;
+constexpr uint32_t kWaitCap = 1u << 18;     // polls of about 0.5 us each
 constexpr int64_t kDefaultChunkBytes = 512ll << 20;     // (256 - 512 MiB measured best: the tail of the last chunk is what is not overlapped)
 
 // A plan is everything that depends only on the layout of a call: segment addresses and lengths,
@@ -36,6 +42,10 @@ struct Plan {
     TileScratch part{};
     double *params = nullptr;     // [2 * n_seg] device staging for host-supplied (beta, alpha)
     double *sd = nullptr;         // [n_seg] standard deviations, written by the fit of a fused call for its second sweep
+    // the one-launch fitted pass (bf16 input): groups of consecutive segments and their arrive / ready words
+    int4 *groups = nullptr;
+    int32_t n_groups = 0;
+    uint32_t *sync = nullptr;     // [2 * n_groups]
     uint64_t last_use = 0;
 };
 
@@ -54,6 +64,11 @@ struct gg_ctx {
     void *chan_buf = nullptr;     // scratch of gg_fused_channels (partials per row block and column)
     int64_t chan_bytes = 0;
     double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
+    int resident_grid[2][8];      // CTAs the one-launch pass may use, by gradient type and sweep flags (-1: not asked yet)
+    bool can_cooperate = false;
+    int resident_mode = 0;        // 1: gg_fused takes the one-launch fitted pass whenever it can run
+    int32_t expect_delta = 0;     // test hook: arrivals the fitter waits for beyond the streamers that exist
+    uint32_t wait_cap = kWaitCap;
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
     std::vector<cudaEvent_t> ev_first, ev_tail;   // begin, end, begin, end, ...
@@ -187,6 +202,19 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     const size_t o_max = take(sizeof(float) * (size_t)n_tiles);
     const size_t o_par = take(sizeof(double) * 2 * (size_t)n_seg);
     const size_t o_sd = take(sizeof(double) * (size_t)n_seg);
+    // groups of the one-launch pass: consecutive segments up to kGroupBytes (a longer segment is alone in its group)
+    std::vector<int4> groups;
+    if (in_dtype == GG_BF16) {
+        for (int32_t s = 0; s < n_seg;) {
+            int32_t e = s;
+            int64_t bytes = 0;
+            while (e < n_seg && e - s < kGroupSegs && (e == s || bytes + segs[e].len * 2 <= kGroupBytes)) bytes += segs[e++].len * 2;
+            groups.push_back(make_int4(prefix[(size_t)s], prefix[(size_t)e], s, e));
+            s = e;
+        }
+    }
+    const size_t o_grp = take(sizeof(int4) * groups.size());
+    const size_t o_sync = take(sizeof(uint32_t) * 2 * groups.size());
     const size_t total = off > 0 ? off : 256;
 
     std::vector<char> host(table_bytes > 0 ? table_bytes : 1, 0);
@@ -202,8 +230,14 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
 
     GG_CUDA(ctx, cudaMalloc(&p->dev, total));
     cudaError_t e = cudaMemcpy(p->dev, host.data(), table_bytes, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !groups.empty())
+        e = cudaMemcpy(static_cast<char *>(p->dev) + o_grp, groups.data(), sizeof(int4) * groups.size(), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { cudaFree(p->dev); return cuda_fail(ctx, e); }
     char *d = static_cast<char *>(p->dev);
+    p->groups = reinterpret_cast<int4 *>(d + o_grp);
+    p->sync = reinterpret_cast<uint32_t *>(d + o_sync);
+    p->n_groups = (int32_t)groups.size();
+
     p->map.seg_ptr = reinterpret_cast<const void *const *>(d + o_ptr);
     p->map.grad_ptr = grad ? reinterpret_cast<void *const *>(d + o_gptr) : nullptr;
     p->map.seg_len = reinterpret_cast<const int64_t *>(d + o_len);
@@ -299,6 +333,23 @@ gg_status check_hist(int32_t n_seg, const int32_t *hist_id, int32_t n_hist, int3
     return GG_OK;
 }
 
+// CTAs of the one-launch fitted pass for this kernel variant: all of them must be resident at once, so at most
+// what the occupancy of the variant allows, and two per SM.  0 when the pass is switched off or cannot run.
+int resident_grid(gg_ctx *ctx, int flags, gg_dtype grad_dtype, bool has_grad_out)
+{
+    if (ctx->resident_mode == 0 || !ctx->can_cooperate) return 0;
+    int &slot = ctx->resident_grid[has_grad_out && grad_dtype == GG_BF16 ? 1 : 0][flags & 7];
+    if (slot < 0) {
+        int max_grid = 0;
+        if (resident_bf16_max_grid(flags, grad_dtype, has_grad_out, ctx->sm_count, &max_grid) != cudaSuccess) {
+            cudaGetLastError();
+            max_grid = 0;
+        }
+        slot = std::min(max_grid, 2 * ctx->sm_count);
+    }
+    return slot;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------ C entry points
@@ -352,6 +403,8 @@ gg_status gg_create(gg_ctx **out, int device)
     if (!ctx) return GG_ERR_NOMEM;
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
+    for (auto &row : ctx->resident_grid) for (int &v : row) v = -1;
+    ctx->can_cooperate = prop.cooperativeLaunch != 0;
     {
         DeviceGuard guard(device);
         cudaError_t se = guard.ok ? cudaMalloc(reinterpret_cast<void **>(&ctx->seed), sizeof(double) * 2 * (kSeedCells + 1))
@@ -513,6 +566,26 @@ gg_status gg_sample(gg_ctx *ctx, const gg_seg *out, int32_t n_seg, gg_dtype dtyp
     return GG_OK;
 }
 
+gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value)
+{
+    if (!ctx) return GG_ERR_INVALID_ARG;
+    switch (what) {
+    case GG_HOOK_RESIDENT_MODE:
+        if (value < 0 || value > 1) return GG_ERR_INVALID_ARG;
+        ctx->resident_mode = (int)value;
+        return GG_OK;
+    case GG_HOOK_EXTRA_ARRIVALS:
+        if (value < 0 || value > 1000) return GG_ERR_INVALID_ARG;
+        ctx->expect_delta = (int32_t)value;
+        return GG_OK;
+    case GG_HOOK_WAIT_CAP:
+        if (value < 1 || value > (1ll << 24)) return GG_ERR_INVALID_ARG;
+        ctx->wait_cap = (uint32_t)value;
+        return GG_OK;
+    default: return GG_ERR_INVALID_ARG;
+    }
+}
+
 gg_status gg_timing_enable(gg_ctx *ctx, int enable)
 {
     if (!ctx) return GG_ERR_INVALID_ARG;
@@ -638,6 +711,28 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
                 GG_CUDA(ctx, launch_small_bf16(g_dt, ka, ctx->sm_count, cs));
             }
             ctx->launches += 1 + (do_hist ? 1 : 0);
+        } else if (a->param_mode == GG_PARAMS_FITTED && in_dt == GG_BF16 && tail_flags != 0 &&
+                   ctx->resident_mode == 1 && p->n_groups > 0 &&
+                   resident_grid(ctx, tail_flags, g_dt, a->grad != nullptr) >= 2) {
+            // one launch: every group of segments goes moments -> fit -> gradient + histogram while L2 still holds it
+            const int grid = resident_grid(ctx, tail_flags, g_dt, a->grad != nullptr);
+            GG_CUDA(ctx, cudaMemsetAsync(p->sync, 0, sizeof(uint32_t) * 2 * (size_t)p->n_groups, cs));
+            fa.sd_out = p->sd;
+            sa.beta = a->beta; sa.alpha = a->alpha; sa.seg_sd = p->sd;
+            sa.step = fa.step_from_alpha ? a->step_out : a->step;
+            ResidentArgs ra{};
+            ra.groups = p->groups; ra.n_groups = p->n_groups;
+            ra.arrive = p->sync; ra.ready = p->sync + p->n_groups;
+            ra.expect = (uint32_t)(grid - 1 + ctx->expect_delta);
+            ra.wait_cap = ctx->wait_cap;
+            ra.keep_tiles = (uint32_t)(kGroupBytes / (kTile * 2));
+            ra.fit = fa;
+            {
+                SweepTimer tm(ctx, &ctx->ev_tail, cs);
+                GG_CUDA(ctx, launch_resident_bf16(tail_flags, g_dt, a->grad != nullptr, sa, ra, grid, cs));
+            }
+            ctx->launches += 1;
+            beta_used = a->beta;
         } else if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
             {

@@ -96,6 +96,88 @@ __device__ __forceinline__ uint32_t fit_from_sums(double s1, double s2, int64_t 
     return flags;
 }
 
+// ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
+// of the density of Eq. 1; increasing in beta from 0 to 3/4.
+__device__ __forceinline__ double log_rho(double beta)
+{
+    return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
+}
+
+// The fit of segment s from its reduced sums and extremes, and every per-segment output of the fit step
+// (parameters, sums, count, flags, the quantiser step taken from alpha, the standard deviation for the sweep
+// that follows).  WARP: all 32 lanes of a warp call with the same arguments; lane 0 writes.  Without a fit table
+// (a.seed null) the root is found by 33-section search on ln(beta): each round the 32 lanes evaluate log_rho at
+// the interior points of the bracket and a ballot picks the sub-interval with the sign change.
+__device__ __forceinline__ void fit_finish(const FitArgs &a, int s, int lane, double s1, double s2, uint32_t bad, float xmin,
+                                           float xmax)
+{
+    constexpr unsigned kFull = 0xFFFFFFFFu;
+    const int64_t len = a.map.seg_len[s];
+
+    uint32_t flags = bad ? GG_FLAG_NONFINITE : 0u;
+    double beta = 0.0, alpha = 0.0;
+    if (len <= 0 || !(s2 > 0.0)) {
+        flags |= GG_FLAG_DEGENERATE;
+    } else {
+        const double m1 = s1 / (double)len, m2 = s2 / (double)len;
+        const double log_r = log(m1 * m1 / m2);
+        if (a.seed != nullptr) {
+            // table look-up and cubic interpolation (no lgamma at fit time)
+            double lnz;
+            if (log_r <= __ldg(a.seed)) {
+                beta = GG_BETA_LO;
+                lnz = __ldg(a.seed + kSeedCells + 1);
+                flags |= GG_FLAG_BETA_CLAMPED_LO;
+            } else if (log_r >= __ldg(a.seed + kSeedCells)) {
+                beta = GG_BETA_HI;
+                lnz = __ldg(a.seed + 2 * kSeedCells + 1);
+                flags |= GG_FLAG_BETA_CLAMPED_HI;
+            } else {
+                beta = invert_ratio_table<true>(log_r, a.seed, &lnz);      // (every lane is here with the same log_r)
+            }
+            alpha = sqrt(m2) * exp(lnz);
+        } else {
+        if (log_r <= log_rho(GG_BETA_LO)) {
+            beta = GG_BETA_LO;
+            flags |= GG_FLAG_BETA_CLAMPED_LO;
+        } else if (log_r >= log_rho(GG_BETA_HI)) {
+            beta = GG_BETA_HI;
+            flags |= GG_FLAG_BETA_CLAMPED_HI;
+        } else {
+            double lo = log(GG_BETA_LO), hi = log(GG_BETA_HI);
+            for (int round = 0; round < 12 && hi - lo > 4e-15; ++round) {
+                const double w = (hi - lo) * (1.0 / 33.0);
+                const double ti = lo + w * (double)(lane + 1);
+                const bool below = log_rho(exp(ti)) < log_r;
+                const int k = __popc(__ballot_sync(kFull, below));   // points 1..k lie below the root
+                hi = lo + w * (double)(k + 1);
+                lo = lo + w * (double)k;
+            }
+            beta = exp(0.5 * (lo + hi));
+        }
+        alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+        }
+    }
+    if (lane == 0) {
+        a.beta[s] = beta;
+        a.alpha[s] = alpha;
+        if (a.sum_abs) a.sum_abs[s] = s1;
+        if (a.sum_sq) a.sum_sq[s] = s2;
+        if (a.count) a.count[s] = len;
+        const float step = a.step_from_alpha ? (float)(alpha * a.step_scale) : (a.step ? a.step[s] : 0.0f);
+        if (a.step_from_alpha && a.step_out) a.step_out[s] = step;
+        if (a.hist_on && xmin <= xmax) {
+            // the quantiser is monotone in x, so a symbol clamps iff one of the extremes does
+            const float inv = (float)(1.0 / (double)step);
+            const float tlo = __fmul_rn(xmin, inv), thi = __fmul_rn(xmax, inv);
+            if ((double)floorf(tlo) < (double)a.qmin || (double)floorf(thi) > (double)a.qmax)
+                flags |= GG_FLAG_CLAMPED_SYMBOLS;
+        }
+        if (a.flags) a.flags[s] = flags;
+        if (a.sd_out) a.sd_out[s] = (len > 0 && s2 > 0.0) ? sqrt(s2 / (double)len) : 0.0;
+    }
+}
+
 // 2^t for |t| < 1000 within 1e-11 relative: table entries are rounded to fp32 afterwards.
 __device__ __forceinline__ double exp2_short(double t)
 {

@@ -84,6 +84,22 @@ struct FitArgs {
     int32_t qmin, qmax;
 };
 
+// Arguments of the one-launch fitted pass that keeps tensors in L2 between their two reads (gg_tail_bf16.cu).
+struct ResidentArgs {
+    const int4 *groups;      // [n_groups] {first tile, end tile, first segment, end segment} of consecutive segments
+    int32_t n_groups;
+    uint32_t *arrive;        // [n_groups] streamers that have finished the moments of a group; zero before the launch
+    uint32_t *ready;         // [n_groups] 1 once the group's fit is published; zero before the launch
+    uint32_t expect;         // arrivals that complete a group (the number of streamers)
+    uint32_t wait_cap;       // polls after which a wait gives up
+    uint32_t keep_tiles;     // tiles of a group that are read with the evict-last hint (what L2 can hold through the pass)
+    FitArgs fit;
+};
+// grid: CTAs of the launch (streamers + one fitter), at most what resident_bf16_max_grid reports
+cudaError_t launch_resident_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
+                                 const ResidentArgs &r, int grid, cudaStream_t st);
+cudaError_t resident_bf16_max_grid(int flags, gg_dtype grad_dtype, bool has_grad_out, int sm_count, int *max_grid);
+
 cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
                           const StreamArgs &a, cudaStream_t st);
 // The moments sweep for bf16 input by persistent CTAs (the one-CTA-per-tile kernel of launch_stream gives the

@@ -11,13 +11,6 @@ namespace {
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kSegThreads = 256;   // one CTA of 8 warps per segment
 
-// ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
-// of the density of Eq. 1; increasing in beta from 0 to 3/4.
-__device__ __forceinline__ double log_rho(double beta)
-{
-    return 2.0 * lgamma(2.0 / beta) - lgamma(1.0 / beta) - lgamma(3.0 / beta);
-}
-
 // One CTA of eight warps per segment.  The threads sum the tile partials in a fixed order (strided over
 // the 256 threads, a butterfly in each warp, the eight warps in sequence, so every thread of warp 0 ends
 // with the same bits), then warp 0 inverts the moment ratio: from the context's fit
@@ -60,70 +53,7 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
         s1 += sh1[w]; s2 += sh2[w]; bad += shb[w];
         xmin = fminf(xmin, shmn[w]); xmax = fmaxf(xmax, shmx[w]);
     }
-    const int64_t len = a.map.seg_len[s];
-
-    uint32_t flags = bad ? GG_FLAG_NONFINITE : 0u;
-    double beta = 0.0, alpha = 0.0;
-    if (len <= 0 || !(s2 > 0.0)) {
-        flags |= GG_FLAG_DEGENERATE;
-    } else {
-        const double m1 = s1 / (double)len, m2 = s2 / (double)len;
-        const double log_r = log(m1 * m1 / m2);
-        if (a.seed != nullptr) {
-            // table look-up and cubic interpolation (no lgamma at fit time)
-            double lnz;
-            if (log_r <= __ldg(a.seed)) {
-                beta = GG_BETA_LO;
-                lnz = __ldg(a.seed + kSeedCells + 1);
-                flags |= GG_FLAG_BETA_CLAMPED_LO;
-            } else if (log_r >= __ldg(a.seed + kSeedCells)) {
-                beta = GG_BETA_HI;
-                lnz = __ldg(a.seed + 2 * kSeedCells + 1);
-                flags |= GG_FLAG_BETA_CLAMPED_HI;
-            } else {
-                beta = invert_ratio_table<true>(log_r, a.seed, &lnz);      // (every lane is here with the same log_r)
-            }
-            alpha = sqrt(m2) * exp(lnz);
-        } else {
-        if (log_r <= log_rho(GG_BETA_LO)) {
-            beta = GG_BETA_LO;
-            flags |= GG_FLAG_BETA_CLAMPED_LO;
-        } else if (log_r >= log_rho(GG_BETA_HI)) {
-            beta = GG_BETA_HI;
-            flags |= GG_FLAG_BETA_CLAMPED_HI;
-        } else {
-            double lo = log(GG_BETA_LO), hi = log(GG_BETA_HI);
-            for (int round = 0; round < 12 && hi - lo > 4e-15; ++round) {
-                const double w = (hi - lo) * (1.0 / 33.0);
-                const double ti = lo + w * (double)(lane + 1);
-                const bool below = log_rho(exp(ti)) < log_r;
-                const int k = __popc(__ballot_sync(kFull, below));   // points 1..k lie below the root
-                hi = lo + w * (double)(k + 1);
-                lo = lo + w * (double)k;
-            }
-            beta = exp(0.5 * (lo + hi));
-        }
-        alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
-        }
-    }
-    if (lane == 0) {
-        a.beta[s] = beta;
-        a.alpha[s] = alpha;
-        if (a.sum_abs) a.sum_abs[s] = s1;
-        if (a.sum_sq) a.sum_sq[s] = s2;
-        if (a.count) a.count[s] = len;
-        const float step = a.step_from_alpha ? (float)(alpha * a.step_scale) : (a.step ? a.step[s] : 0.0f);
-        if (a.step_from_alpha && a.step_out) a.step_out[s] = step;
-        if (a.hist_on && xmin <= xmax) {
-            // the quantiser is monotone in x, so a symbol clamps iff one of the extremes does
-            const float inv = (float)(1.0 / (double)step);
-            const float tlo = __fmul_rn(xmin, inv), thi = __fmul_rn(xmax, inv);
-            if ((double)floorf(tlo) < (double)a.qmin || (double)floorf(thi) > (double)a.qmax)
-                flags |= GG_FLAG_CLAMPED_SYMBOLS;
-        }
-        if (a.flags) a.flags[s] = flags;
-        if (a.sd_out) a.sd_out[s] = (len > 0 && s2 > 0.0) ? sqrt(s2 / (double)len) : 0.0;
-    }
+    fit_finish(a, s, lane, s1, s2, bad, xmin, xmax);
 }
 
 // penalty[s] = (1/beta_s) * sum over the segment's tiles of sum |x| |g|

@@ -498,9 +498,24 @@ __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool acc
 // One contiguous run of n elements: scalar head up to the first 16-byte boundary of x, 128-bit
 // vector body fed through the asynchronous-copy ring, scalar tail.  If the gradient's address is
 // not 16-byte aligned at the same element the whole run is scalar.
-template <typename TG, int FLAGS, int MODE>
+// L2 eviction hints of one run: vectors before `split` are copied with policy `first`, the others with `rest`.
+struct Hints {
+    uint64_t first = 0, rest = 0;
+    int split = 0;
+};
+
+template <bool HINT>
+__device__ __forceinline__ void copy16(uint32_t dst, const void *src, uint64_t policy)
+{
+    if constexpr (HINT)
+        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+    else
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+template <typename TG, int FLAGS, int MODE, bool HINT = false>
 __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
-                                              const Lane &ln, Smem &sm, Acc &acc)
+                                              const Lane &ln, Smem &sm, Acc &acc, const Hints hints = Hints())
 {
     constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     const int tid = threadIdx.x;
@@ -546,7 +561,7 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
 #pragma unroll
     for (int d = 0; d < kDepth - 1; ++d) {
         if (tid + d * kThreads < nv)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + d * kStageBytes), "l"(xv + d * kThreads) : "memory");
+            copy16<HINT>(slot0 + d * kStageBytes, xv + d * kThreads, tid + d * kThreads < hints.split ? hints.first : hints.rest);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     // (the loop is unrolled over the stages, so that every slot is a compile-time offset)
@@ -557,8 +572,8 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
             if (vd < nv) {
                 // fill the slot emptied by the previous vector (stage d - 1, cyclically; its value is in registers since then)
                 if (vd + (kDepth - 1) * kThreads < nv)
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + ((d + kDepth - 1) % kDepth) * kStageBytes),
-                                 "l"(xv + (d + kDepth - 1) * kThreads) : "memory");
+                    copy16<HINT>(slot0 + ((d + kDepth - 1) % kDepth) * kStageBytes, xv + (d + kDepth - 1) * kThreads,
+                                 vd + (kDepth - 1) * kThreads < hints.split ? hints.first : hints.rest);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
                 uint4 r0;
@@ -573,39 +588,50 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
-template <typename TG, int FLAGS>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const StreamArgs a)
+// What a CTA carries from one run to the next: the key of the counts in shared memory and the lane constants.
+struct CtaState {
+    int cur_hid = -1, cur_mode = kModePattern;
+    uint32_t cur_inv_bits = 0;
+    bool have_key = false;
+    Lane ln;
+};
+
+// Per-segment parameters: plain loads, or loads that bypass L1 when another CTA of the same launch wrote them.
+template <bool COHERENT, typename T>
+__device__ __forceinline__ T param(const T *p)
 {
-    constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    if constexpr (COHERENT) return __ldcg(p);
+    return *p;
+}
+
+__device__ __forceinline__ void init_cta(Smem &sm, CtaState &cs, bool hist)
+{
     const int tid = threadIdx.x;
-
-    // contiguous range of tiles for this CTA
-    const int64_t nt = a.map.n_tiles;
-    const int t_begin = (int)(nt * blockIdx.x / gridDim.x);
-    const int t_end = (int)(nt * (blockIdx.x + 1) / gridDim.x);
-
-    if constexpr (HIST) {
+    if (hist) {
         for (int i = tid; i < (int)kCntWords; i += kThreads) sm.cnt[i] = 0u;
         for (int i = tid; i < kSymWin; i += kThreads) sm.win[i] = 0u;
         if (tid < 2) sm.clampc[tid] = 0u;
     }
     if (tid < 128) sm.lg[tid] = log2(1.0 + (double)tid * (1.0 / 128.0));
     if (tid == 0) { sm.cold.c_base = 0u; sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.symbol_mode = 0; }
-    int cur_hid = -1, cur_mode = kModePattern;
-    uint32_t cur_inv_bits = 0;
-    bool have_key = false;
-    const bool accumulate = GRAD && a.accumulate != 0;
-    Lane ln;
-    ln.b_addr = (uint32_t)__cvta_generic_to_shared(sm.brep) + (uint32_t)(tid & 31) * 4u;
+    cs.ln.b_addr = (uint32_t)__cvta_generic_to_shared(sm.brep) + (uint32_t)(tid & 31) * 4u;
     // row r of the symbol table is reached as bits(floor(t) + magic) * 128 + s_addr (mod 2^32)
-    ln.s_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + 128u + (uint32_t)(tid & 31) * 4u - kSymBase * 128u;
-    ln.p_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + (uint32_t)(tid & (kRep - 1)) * 4u;
-    ln.cbase = 0x8000u;
-    ln.inv = 0.0f;
+    cs.ln.s_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + 128u + (uint32_t)(tid & 31) * 4u - kSymBase * 128u;
+    cs.ln.p_addr = (uint32_t)__cvta_generic_to_shared(sm.cnt) + (uint32_t)(tid & (kRep - 1)) * 4u;
+    cs.ln.cbase = 0x8000u;
+    cs.ln.inv = 0.0f;
     __syncthreads();
+}
 
+// The tiles [t_begin, t_end) of one CTA, run by run (a run: the tiles of the range that lie in one segment):
+// gradient tables and count layout of the run's segment, then the stream, then the run's partial sums.
+template <typename TG, int FLAGS, bool COHERENT, bool HINT>
+__device__ __forceinline__ void tail_tiles(const StreamArgs &a, Smem &sm, CtaState &cs, int t_begin, int t_end, uint64_t policy)
+{
+    constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    const int tid = threadIdx.x;
+    const bool accumulate = GRAD && a.accumulate != 0;
+    Lane &ln = cs.ln;
     for (int t = t_begin; t < t_end;) {
         // ---- one run: the tiles of this CTA's range that lie in segment s
         const int s = a.map.tile_seg[t];
@@ -619,7 +645,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         bool active = false;
 
         if constexpr (GRAD) {
-            const double beta = a.beta[s], alpha = a.alpha[s];
+            const double beta = param<COHERENT>(a.beta + s), alpha = param<COHERENT>(a.alpha + s);
             const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
             active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
             // (every thread works the two constants out for itself: cheaper than a broadcast and its barrier)
@@ -660,16 +686,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
         }
         if constexpr (HIST) {
             const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
-            const float step = a.step[s];
+            const float step = param<COHERENT>(a.step + s);
             const float inv = (float)(1.0 / (double)step);
-            const bool same_key = have_key && hid == cur_hid && __float_as_uint(inv) == cur_inv_bits;
+            const bool same_key = cs.have_key && hid == cs.cur_hid && __float_as_uint(inv) == cs.cur_inv_bits;
             // where the pattern-count window should sit: 16 binades below 2^5 standard deviations when
             // the scale of the data is known, else where it is (same key) or from four binades below
             // the step upwards (new key)
             uint32_t want_base = sm.cold.c_base;
             double sd = 0.0;
             if (a.seg_sd != nullptr) {
-                sd = a.seg_sd[s];
+                sd = param<COHERENT>(a.seg_sd + s);
             } else {
                 // Without parameters the scale of the data is taken from the first elements of the run (one
                 // per thread): it only decides how the counts are laid out, never what is counted.
@@ -696,14 +722,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             } else if (!same_key) {
                 want_base = (uint32_t)(window_top_exponent((double)step, 11) - (kCntBinades - 1)) << 7;
             }
-            const bool rebase = !same_key || mode != cur_mode || (mode == kModePattern && want_base != sm.cold.c_base);
+            const bool rebase = !same_key || mode != cs.cur_mode || (mode == kModePattern && want_base != sm.cold.c_base);
             __syncthreads();
             if (rebase) {
-                if (have_key) flush_counts(sm, a.clamped, cur_hid);
-                have_key = true;
-                cur_hid = hid;
-                cur_inv_bits = __float_as_uint(inv);
-                cur_mode = mode;
+                if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
+                cs.have_key = true;
+                cs.cur_hid = hid;
+                cs.cur_inv_bits = __float_as_uint(inv);
+                cs.cur_mode = mode;
                 if (tid == 0) {
                     sm.cold.inv = inv;
                     sm.cold.qmin = a.qmin;
@@ -725,19 +751,189 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const S
             if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
         }
         Acc acc;
+        Hints hints;
+        hints.first = policy; hints.rest = policy; hints.split = 0;
         if constexpr (HIST) {
-            if (mode == kModeSymbol) process_range<TG, FLAGS, kModeSymbol>(x, gout, n, accumulate, ln, sm, acc);
-            else process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
+            if (mode == kModeSymbol) process_range<TG, FLAGS, kModeSymbol, HINT>(x, gout, n, accumulate, ln, sm, acc, hints);
+            else process_range<TG, FLAGS, kModePattern, HINT>(x, gout, n, accumulate, ln, sm, acc, hints);
         } else {
-            process_range<TG, FLAGS, kModePattern>(x, gout, n, accumulate, ln, sm, acc);
+            process_range<TG, FLAGS, kModePattern, HINT>(x, gout, n, accumulate, ln, sm, acc, hints);
         }
 
         if constexpr (MOM || GRAD) reduce_partials<FLAGS>(a.part, t, t_stop, acc, sm);
         else __syncthreads();
         t = t_stop;
     }
+}
+
+template <typename TG, int FLAGS>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const StreamArgs a)
+{
+    constexpr bool HIST = (FLAGS & kHist) != 0;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    CtaState cs;
+    init_cta(sm, cs, HIST);
+    // contiguous range of tiles for this CTA
+    const int64_t nt = a.map.n_tiles;
+    const int t_begin = (int)(nt * blockIdx.x / gridDim.x);
+    const int t_end = (int)(nt * (blockIdx.x + 1) / gridDim.x);
+    tail_tiles<TG, FLAGS, false, false>(a, sm, cs, t_begin, t_end, 0);
     if constexpr (HIST) {
-        if (have_key) flush_counts(sm, a.clamped, cur_hid);
+        if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// The whole fitted pass in ONE launch that keeps every tensor in L2 between its two reads.
+//
+// The segments are cut into groups of consecutive segments of about a quarter of L2 (one segment of any length
+// is a group by itself).  All CTAs but the last are streamers and walk the groups together, each on its share
+// of the group's tiles:
+//     moments of group g            (the first `protect` part of the share is read with an evict-last hint)
+//     arrive(g)
+//     last tile of group g - 1      (gradient + counts; this tile was deferred to cover the wait below)
+//     wait until the fit of group g is published
+//     all but the last tile of group g   (gradient + counts; read again, now from L2, with an evict-first hint)
+// The last CTA is the fitter: for every group it waits for all arrivals, adds the run partials of each of the
+// group's segments in a fixed order, inverts the moment ratio and publishes the parameters.  The deferred tile
+// is what hides the fitter's latency: without it every streamer would idle for a barrier and a fit per group.
+// Every wait is bounded: when it runs out the CTA marks the segments GG_FLAG_TIMEOUT (fitter) and returns, and
+// the others run out in turn.  The launch is cooperative, so all CTAs are resident and every wait can end.
+__device__ __forceinline__ bool bounded_wait(const uint32_t *flag, uint32_t want, uint32_t cap, int *sh_ok)
+{
+    if (threadIdx.x == 0) {
+        int ok = 0;
+        for (uint32_t it = 0; it < cap; ++it) {
+            uint32_t v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+            if (v >= want) { ok = 1; break; }
+            __nanosleep(100);
+        }
+        __threadfence();
+        *sh_ok = ok;
+    }
+    __syncthreads();
+    const bool ok = *sh_ok != 0;
+    __syncthreads();      // (the word is written again by the next wait)
+    return ok;
+}
+
+__device__ __forceinline__ void publish(uint32_t *flag, bool add)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (add) atomicAdd(flag, 1u);
+        else asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
+    }
+}
+
+__device__ __forceinline__ uint64_t make_policy(bool keep)
+{
+    uint64_t p;
+    if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// Share of streamer b of the tiles [g0, g0 + n): [first, second).
+__device__ __forceinline__ int2 share_of(int g0, int n, int b, int n_stream)
+{
+    return make_int2(g0 + (int)((int64_t)n * b / n_stream), g0 + (int)((int64_t)n * (b + 1) / n_stream));
+}
+
+__device__ void fitter(const StreamArgs &a, const ResidentArgs &r, int *sh_ok)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_stream = (int)gridDim.x - 1;
+    for (int g = 0; g < r.n_groups; ++g) {
+        if (!bounded_wait(r.arrive + g, r.expect, r.wait_cap, sh_ok)) {
+            // nothing from here on can be trusted: say so per segment and stop (the streamers run out in turn)
+            if (r.fit.flags != nullptr)
+                for (int s = r.groups[g].z + tid; s < a.map.n_seg; s += kThreads) r.fit.flags[s] = GG_FLAG_TIMEOUT;
+            return;
+        }
+        const int4 gr = r.groups[g];
+        const int n = gr.y - gr.x;
+        for (int s = gr.z + warp; s < gr.w; s += kWarps) {
+            const int ts0 = a.map.tile_prefix[s], ts1 = a.map.tile_prefix[s + 1];
+            double s1 = 0.0, s2 = 0.0;
+            uint32_t bad = 0;
+            float xmin = INFINITY, xmax = -INFINITY;
+            // the runs of this segment: one per streamer whose share meets it, at the later of the two starts
+            for (int b = lane; b < n_stream && ts1 > ts0; b += 32) {
+                const int2 sh = share_of(gr.x, n, b, n_stream);
+                const int t0 = max(sh.x, ts0);
+                if (t0 >= min(sh.y, ts1)) continue;
+                s1 += __ldcg(a.part.s1 + t0);
+                s2 += __ldcg(a.part.s2 + t0);
+                bad += __ldcg(a.part.bad + t0);
+                xmin = fminf(xmin, __ldcg(a.part.xmin + t0));
+                xmax = fmaxf(xmax, __ldcg(a.part.xmax + t0));
+            }
+            s1 = warp_sum(s1);
+            s2 = warp_sum(s2);
+            bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                xmin = fminf(xmin, __shfl_xor_sync(0xFFFFFFFFu, xmin, o));
+                xmax = fmaxf(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, o));
+            }
+            fit_finish(r.fit, s, lane, s1, s2, bad, xmin, xmax);
+        }
+        publish(r.ready + g, false);
+    }
+}
+
+template <typename TG, int FLAGS>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) resident_bf16_kernel(const StreamArgs a, const ResidentArgs r)
+{
+    constexpr bool HIST = (FLAGS & kHist) != 0;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    __shared__ int sh_ok;
+    const int n_stream = (int)gridDim.x - 1;
+    if ((int)blockIdx.x == n_stream) { fitter(a, r, &sh_ok); return; }
+
+    CtaState cs;
+    init_cta(sm, cs, HIST);
+    const uint64_t keep = make_policy(true), drop = make_policy(false);
+    int late0 = 0, late1 = 0;      // the deferred last tile of the group before
+    for (int g = 0; g < r.n_groups; ++g) {
+        const int4 gr = r.groups[g];
+        const int n = gr.y - gr.x;
+        const int2 sh = share_of(gr.x, n, (int)blockIdx.x, n_stream);
+        // ---- moments of this CTA's share, run by run
+        // (of a group of more than keep_tiles tiles only the first keep_tiles / n of every share is asked to stay in L2)
+        const int64_t share = sh.y - sh.x;
+        const int t_keep = sh.x + (int)(n <= (int)r.keep_tiles ? share : (share * r.keep_tiles + n - 1) / n);
+        for (int t = sh.x; t < sh.y;) {
+            const int s = a.map.tile_seg[t];
+            const int64_t len = a.map.seg_len[s];
+            const int t_first = a.map.tile_prefix[s];
+            const int t_stop = min(sh.y, a.map.tile_prefix[s + 1]);
+            const int64_t off = (int64_t)(t - t_first) * kTile;
+            const int64_t n_el = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
+            const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
+            Hints hints;
+            hints.first = keep; hints.rest = drop;
+            hints.split = (int)min((int64_t)max(t_keep - t, 0) * (kTile / 8), (int64_t)0x7FFFFFFF);
+            Acc acc;
+            process_range<float, kMoments, kModePattern, true>(x, nullptr, n_el, false, cs.ln, sm, acc, hints);
+            reduce_partials<kMoments>(a.part, t, t_stop, acc, sm);
+            t = t_stop;
+        }
+        publish(r.arrive + g, true);
+        if (late1 > late0) tail_tiles<TG, FLAGS, true, true>(a, sm, cs, late0, late1, drop);
+        if (!bounded_wait(r.ready + g, 1u, 2u * r.wait_cap, &sh_ok)) return;
+        late0 = sh.y - sh.x >= 2 ? sh.y - 1 : sh.y;
+        late1 = sh.y;
+        tail_tiles<TG, FLAGS, true, true>(a, sm, cs, sh.x, late0, drop);
+    }
+    if (late1 > late0) tail_tiles<TG, FLAGS, true, true>(a, sm, cs, late0, late1, drop);
+    if constexpr (HIST) {
+        if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
     }
 }
 
@@ -767,6 +963,35 @@ cudaError_t launch_typed(int flags, const StreamArgs &a, int sm_count, cudaStrea
     }
 }
 
+template <typename TG, int FLAGS>
+cudaError_t resident_one(const StreamArgs &a, const ResidentArgs &r, int grid, int *max_grid, cudaStream_t st)
+{
+    auto kern = resident_bf16_kernel<TG, FLAGS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem));
+    if (e != cudaSuccess) return e;
+    if (max_grid != nullptr) {
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, sizeof(Smem));
+        if (e != cudaSuccess) return e;
+        *max_grid = per_sm * grid;      // (grid: the number of SMs)
+        return cudaSuccess;
+    }
+    void *args[] = {const_cast<StreamArgs *>(&a), const_cast<ResidentArgs *>(&r)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kern), dim3((unsigned)grid), dim3(kThreads), args,
+                                       sizeof(Smem), st);
+}
+
+template <typename TG>
+cudaError_t resident_typed(int flags, const StreamArgs &a, const ResidentArgs &r, int grid, int *max_grid, cudaStream_t st)
+{
+    switch (flags) {
+    case kGrad: return resident_one<TG, kGrad>(a, r, grid, max_grid, st);
+    case kHist: return resident_one<TG, kHist>(a, r, grid, max_grid, st);
+    case kGrad | kHist: return resident_one<TG, kGrad | kHist>(a, r, grid, max_grid, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
@@ -775,6 +1000,22 @@ cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, 
     if (a.map.n_tiles <= 0) return cudaSuccess;
     if (has_grad_out && grad_dtype == GG_BF16) return launch_typed<uint16_t>(flags, a, sm_count, st);
     return launch_typed<float>(flags, a, sm_count, st);
+}
+
+cudaError_t launch_resident_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
+                                 const ResidentArgs &r, int grid, cudaStream_t st)
+{
+    if (r.n_groups <= 0) return cudaSuccess;
+    if (has_grad_out && grad_dtype == GG_BF16) return resident_typed<uint16_t>(flags, a, r, grid, nullptr, st);
+    return resident_typed<float>(flags, a, r, grid, nullptr, st);
+}
+
+cudaError_t resident_bf16_max_grid(int flags, gg_dtype grad_dtype, bool has_grad_out, int sm_count, int *max_grid)
+{
+    StreamArgs a{};
+    ResidentArgs r{};
+    if (has_grad_out && grad_dtype == GG_BF16) return resident_typed<uint16_t>(flags, a, r, sm_count, max_grid, nullptr);
+    return resident_typed<float>(flags, a, r, sm_count, max_grid, nullptr);
 }
 
 }  // namespace gg
