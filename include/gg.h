@@ -349,7 +349,12 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *args, void *stre
  * allocations, a step whose buffer addresses must not move, a plug-in that is given buffers and a
  * stream and nothing more) cannot afford that.  This call needs no context and calls neither
  * cudaMalloc, cudaFree nor any allocating routine: its tables and partials live in a fixed array of
- * about 0.7 MB inside the library image, which every GPU that loads the library holds until exit.
+ * about 0.7 MB inside the library image.  The CUDA runtime places that array, and the code of the three kernels,
+ * on a device when the library's module is first loaded there, which by default happens lazily at the first call
+ * on that device, and the device then holds them until the process exits.  A caller whose allocator is about to
+ * take or freeze all device memory should therefore make one warm-up call per device and element type
+ * beforehand (or run with CUDA_MODULE_LOADING=EAGER); a first call made when no memory is left can fail with
+ * GG_ERR_CUDA.
  *   device    CUDA device that owns `x` and the outputs (compute capability 10.x, index < 64)
  *   x         device data of type `dtype`, `len` elements, element aligned
  *   len       0 <= len <= gg_fit_noalloc_max_len() (2^28 elements); a longer segment is refused with

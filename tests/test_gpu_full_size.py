@@ -132,7 +132,7 @@ def test_config2_qwen_initialisation_full_size(ctx):
         refb = o.round_to_bf16_bits(ref).astype(np.int64)
         got = outs[s].cpu().view(torch.int16).numpy().astype(np.int64) & 0xFFFF
         diff = np.abs(refb - got)
-        assert diff.max() <= 1 and int((diff != 0).sum()) <= max(1, got.size // 100_000)
+        assert diff.max() <= 1 and int((diff != 0).sum()) == 0          # (bf16 storage: see test_sample_parity)
         b, a, *_ = o.fit(gg_synth.to_oracle(outs[s].cpu()))
         assert_rel(fit["beta"][s].item(), b, REL_FIT, "beta")
         assert_rel(fit["alpha"][s].item(), a, REL_FIT, "alpha")
@@ -197,7 +197,6 @@ def test_sample_elements_past_index_2_to_32(ctx):
         refb = o.round_to_bf16_bits(ref).astype(np.int64)
         gotb = got.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
         assert np.array_equal(refb >> 15, gotb >> 15)                       # signs
-        assert (np.abs((refb & 0x7FFF) - (gotb & 0x7FFF)) <= 1).all()       # one bf16 ulp at most ...
-        assert (refb != gotb).mean() <= 1e-3                                # ... and rarely
+        assert np.array_equal(refb, gotb)                                   # bf16 storage: the same patterns
     assert 1 <= att[0].item() <= 64
     del x

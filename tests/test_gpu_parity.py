@@ -326,9 +326,11 @@ def test_sample_parity(ctx, dtype):
         np.testing.assert_array_equal(np.signbit(ref), np.signbit(got.float().numpy()))
         total += n
         mism += int((diff != 0).sum())
-    # libm and device math may differ in the last fp64 bit: a value that sits on a rounding
-    # boundary of the storage type can land on either side, which is rare
-    assert mism <= max(1, total // 100_000)
+    # libm and device math differ in the last bits of the fp64 value (about 1e-15 relative): a value that sits that
+    # close to a rounding boundary of the storage type can land on either side.  Per element that has probability
+    # about 1e-7 in fp32 and 1e-12 in bf16, so at most one element in a million may differ, none in bf16.
+    print(f"sampled values that differ from the oracle by one storage ulp: {mism} of {total} ({dtype})")
+    assert mism <= (0 if dtype == torch.bfloat16 else -(-total // 1_000_000))
 
 
 def test_sample_then_fit_recovers_parameters(ctx):
@@ -349,6 +351,48 @@ def test_sample_then_fit_recovers_parameters(ctx):
         b, a, *_ = o.fit(gg_synth.to_oracle(t))
         assert_rel(bh, b, REL_FIT, "beta")
         assert_rel(ah, a, REL_FIT, "alpha")
+
+
+def test_fused_pass_is_deterministic(ctx):
+    """Every output of the fused pass repeats bit for bit from call to call: partial sums are added in a fixed
+    order and counts are integers.  Long bf16 and fp32 segments (the two-sweep kernels), many short bf16
+    segments (the one-warp-per-segment kernel), and the single-step calls."""
+    from paper_2506_00486_b200 import Segments
+    rng = np.random.default_rng(53)
+    sets = {
+        "long_bf16": [gg_synth.gg_host(rng, 0.9, 0.02, n, torch.bfloat16) for n in (5 * TILE + 77, 3 * TILE, 40001)],
+        "long_f32": [gg_synth.gg_host(rng, 0.6, 1e-3, n, torch.float32) for n in (4 * TILE + 5, 2 * TILE + 1)],
+        "short_bf16": [gg_synth.gg_host(rng, 1.2, 0.3, int(rng.integers(1, 5000)), torch.bfloat16) for _ in range(100)],
+    }
+    for name, xs in sets.items():
+        xd = [dev(x) for x in xs]
+        gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+        n = len(xs)
+        steps = torch.full((n,), 2.0 ** -9, dtype=torch.float32, device="cuda:0")
+        hid = [s % 3 for s in range(n)]
+        run = ctx.make_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps, hist_id=hid, n_hist=3)
+        snaps = []
+        for _ in range(3):
+            for g in gd:
+                g.fill_(float("nan"))
+            out = run()
+            torch.cuda.synchronize()
+            snaps.append(([g.clone() for g in gd], {k: v.clone() for k, v in out.items() if isinstance(v, torch.Tensor)}))
+        for grads, outs in snaps[1:]:
+            for a, b in zip(grads, snaps[0][0]):
+                assert torch.equal(a.view(torch.int32), b.view(torch.int32)), name
+            for k, v in outs.items():
+                assert torch.equal(v.view(torch.uint8), snaps[0][1][k].view(torch.uint8)), (name, k)
+        # the single-step calls on the same data
+        beta, alpha = snaps[0][1]["beta"], snaps[0][1]["alpha"]
+        pens, hists = [], []
+        for _ in range(2):
+            pens.append(ctx.gg_penalty_grad(xd, beta, alpha, 1e-4, grad=gd).clone())
+            h = ctx.gg_rate_hist(xd, steps, hist_id=hid, n_hist=3)
+            hists.append((h["hist"].clone(), h["entropy_bits"].clone()))
+        torch.cuda.synchronize()
+        assert torch.equal(pens[0].view(torch.int64), pens[1].view(torch.int64)), name
+        assert torch.equal(hists[0][0], hists[1][0]) and torch.equal(hists[0][1].view(torch.int64), hists[1][1].view(torch.int64)), name
 
 
 # ------------------------------------------------------------------------------------- gg_fused

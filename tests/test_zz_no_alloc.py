@@ -63,6 +63,61 @@ def test_noalloc_fit_matches_gg_fit_on_two_calls_in_a_row():
     ctx.close()
 
 
+def test_noalloc_fit_against_the_oracle_without_touching_device_memory():
+    """The same entry point against the fp64 oracle (its fit searches the root with lgamma evaluations: no table,
+    because a table would have to be allocated): both element types, a 4-byte aligned fp32 pointer that is not
+    16-byte aligned, a shape clamped at either end, an all-zero and an empty segment.  After the first call the
+    free device memory must not move: that is what the entry point is for."""
+    import numpy as np
+    import __graft_entry__ as entry
+    entry.build()
+    from oracle import gg_oracle as o
+    from paper_2506_00486_b200 import binding
+    L = binding.lib()
+    rng = np.random.default_rng(78)
+    spikes = np.zeros(3_000_000, dtype=np.float32)
+    spikes[1234567] = 3.0                                 # one non-zero entry: ratio 1/n = 3.3e-7 < rho(0.05) = 4.1e-7, clamped low
+    buf = torch.zeros(3 * TILE + 16, dtype=torch.float32, device="cuda:0")
+    host_odd = gg_synth.gg_host(rng, 0.8, 0.05, 3 * TILE + 9, torch.float32)
+    buf[3:3 + host_odd.numel()].copy_(host_odd)
+    cases = [(gg_synth.gg_host(rng, 0.7, 0.02, 9 * TILE + 1234, torch.bfloat16), None),
+             (gg_synth.gg_host(rng, 1.9, 0.3, 2 * TILE + 5, torch.float32), None),
+             (host_odd, buf[3:3 + host_odd.numel()]),
+             (torch.full((4000,), -2.5, dtype=torch.bfloat16), None),          # constant magnitude: ratio 1, clamped high
+             (torch.from_numpy(spikes), None),
+             (torch.zeros(100, dtype=torch.float32), None),
+             (torch.zeros(0, dtype=torch.bfloat16), None)]
+    xs = [(h, d if d is not None else h.to("cuda:0")) for h, d in cases]
+    call_noalloc(L, xs[0][1])                            # first calls on the device (one per element type): they look the
+    call_noalloc(L, xs[1][1])                            # array up and make the runtime load the kernels
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info(0)[0]
+    outs = [torch.empty(1, dtype=dt, device="cuda:0") for dt in (torch.float64,) * 4 + (torch.int64, torch.int32)]
+    torch.cuda.synchronize()
+    free1 = torch.cuda.mem_get_info(0)[0]
+    seen = set()
+    for h, d in xs:
+        p = ctypes.c_void_p
+        st = L.gg_fit_noalloc(0, p(d.data_ptr()) if d.numel() else None, d.numel(), 0 if d.dtype == torch.float32 else 1,
+                              *(p(t.data_ptr()) for t in outs), p(torch.cuda.current_stream().cuda_stream))
+        assert st == 0
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info(0)[0] == free1     # nothing was allocated by the call
+        beta, alpha, s1, s2 = (t.item() for t in outs[:4])
+        b, a, r1, r2, n, fl = o.fit(gg_synth.to_oracle(h))
+        assert outs[4].item() == n == h.numel() and outs[5].item() == fl
+        seen.add(fl)
+        if fl & o.FLAG_DEGENERATE:
+            assert beta == 0.0 and alpha == 0.0
+            continue
+        assert_rel(beta, b, REL_FIT, "beta")
+        assert_rel(alpha, a, REL_FIT, "alpha")
+        assert_rel(s1, r1, 1e-7, "sum_abs")
+        assert_rel(s2, r2, 1e-7, "sum_sq")
+    assert free1 <= free0
+    assert {0, o.FLAG_DEGENERATE, o.FLAG_BETA_CLAMPED_LO, o.FLAG_BETA_CLAMPED_HI} <= seen
+
+
 def test_noalloc_fit_refuses_segments_beyond_its_fixed_capacity():
     import __graft_entry__ as entry
     entry.build()
