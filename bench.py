@@ -32,6 +32,9 @@ def parse():
     ap.add_argument("--divisor", type=int, default=1,
                     help="divide every matrix dimension of the sweep (debugging; 1 = the full workload)")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--sweep-steps", type=int, default=20,
+                    help="steps of the separate loop that times the two sweeps of the pass with the library's event pairs")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the other workloads (the `secondary` object)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--single-read-steps", type=int, default=20,
                     help="timed steps of the one-read form of the pass (parameters given), 0 to skip")
@@ -263,8 +266,6 @@ def run_ours(args):
     for _ in range(args.warmup):
         run()
     barrier()
-    ctx.timing_enable(True)
-    ctx.timing_read()
     sampler = ClockSampler(local) if rank == 0 else None
     launches0 = ctx.launch_count
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -276,6 +277,11 @@ def run_ours(args):
     barrier()
     ms = ev0.elapsed_time(ev1) / max(args.steps, 1)
     launches = ctx.launch_count - launches0
+    # the two sweeps by themselves, in a loop of their own: the library's event pairs stay out of the headline loop
+    ctx.timing_enable(True)
+    ctx.timing_read()
+    for _ in range(args.sweep_steps):
+        run()
     ms_first, n_first, ms_tail, n_tail = ctx.timing_read()
     ctx.timing_enable(False)
     clocks = sampler.stop() if sampler else None
@@ -293,9 +299,11 @@ def run_ours(args):
     tail_ms = ms_tail / max(n_tail, 1)
     first_ms = ms_first / max(n_first, 1)
     achieved = alg_bytes / (tail_ms * 1e-3) / 1e9 if tail_ms > 0 else None
-    tr = traffic_per_element(args.grad_dtype)
+    tr = None if args.one_launch else traffic_per_element(args.grad_dtype)
     traffic = tr * n_elem if tr is not None else None
-    roofline = {"bound": "hbm", "kernel": "tail_bf16_kernel<%s grad, grad|hist> (second sweep)" % args.grad_dtype,
+    kernel = ("resident_bf16_kernel<%s grad, grad|hist> (moments, fit and second read in one launch)" if args.one_launch
+              else "tail_bf16_kernel<%s grad, grad|hist> (second sweep)") % args.grad_dtype
+    roofline = {"bound": "hbm", "kernel": kernel,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                 "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
                 "traffic": traffic, "peak_source": peak_src, "ms_per_launch": tail_ms,
@@ -332,6 +340,16 @@ def run_ours(args):
     if not args.no_e2e:
         e2e = run_e2e(args, ctx, w, world, dev, gdtype, in_bytes, g_bytes, alg_bytes, barrier)
 
+    # ---- the other workloads (rank 0, one GPU): a few timed calls each, as fractions of the same measured peak
+    secondary = None
+    if rank == 0 and world == 1 and not args.no_secondary and args.divisor == 1:
+        from paper_2506_00486_b200 import bench_configs
+        secondary = {}
+        for r in bench_configs.cases(ctx, dev):
+            if "gbs" in r and r.get("bound") != "alu":
+                r["of_measured_copy_peak"] = r["gbs"] / peak
+            secondary[r.pop("name")] = r
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import gg_oracle as o
@@ -352,6 +370,7 @@ def run_ours(args):
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world} (segments are independent)"},
             "fraction_of_hbm_peak": {"of_measured_copy_peak": value / world / peak, "of_nominal_8TBs": value / world / 8000.0},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "single_read": single,
+            "secondary": secondary,
             "gpu_launches": int(launches),
             "clocks": clocks,
             "check": {"max_abs_beta_error_vs_generating": beta_err, "histogram_total": total_counts,

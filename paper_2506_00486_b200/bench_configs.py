@@ -1,11 +1,11 @@
 #!/usr/bin/env python
-"""Timings of the secondary workloads (everything but the weight sweep that bench.py reports).
+"""Timings of the secondary workloads (everything but the weight sweep that bench.py times as its headline).
 
     python -m paper_2506_00486_b200.bench_configs [c1] [c2] [c3] [c4] [codes] [calls] [channels]
 
-Each line gives the CUDA-event time of one call through the C interface on cuda:0, inputs resident
-in device memory, and the algorithmic GB/s (input read once + output written once).  Inputs are the
-seeded synthetic tensors of gg_synth drawn on the device.
+Each record gives the CUDA-event time of one call through the C interface on cuda:0, inputs resident in
+device memory, and the algorithmic GB/s (input read once + output written once).  Inputs are the seeded
+synthetic tensors of gg_synth drawn on the device.  bench.py puts the same records into its JSON line.
 """
 import os
 import sys
@@ -19,6 +19,8 @@ if ROOT not in sys.path:
 
 import gg_synth  # noqa: E402
 from paper_2506_00486_b200 import Context, Segments  # noqa: E402
+
+ALL = ("c1", "c2", "c3", "c4", "codes", "calls", "channels")
 
 
 def timeit(fn, n=10, warmup=3):
@@ -34,9 +36,30 @@ def timeit(fn, n=10, warmup=3):
     return e0.elapsed_time(e1) / n
 
 
-def main(which):
-    dev = torch.device("cuda", 0)
-    ctx = Context(0)
+def rec(name, what, ms, alg_bytes=None, steps=10, **extra):
+    r = {"name": name, "what": what, "ms": ms, "steps": steps}
+    if alg_bytes is not None:
+        r["algorithmic_bytes"] = int(alg_bytes)
+        r["gbs"] = alg_bytes / ms / 1e6
+    r.update(extra)
+    return r
+
+
+def sweeps(ctx, run, n=5):
+    """Time of a fused call and of its two sweeps (the library's own event pairs)."""
+    run()                            # (the first launch of a kernel loads it: keep that out of the sweep timers)
+    ms = timeit(run, n)              # the call as a user sees it: no event pairs inside
+    ctx.timing_enable(True)
+    ctx.timing_read()
+    for _ in range(n):
+        run()
+    t = ctx.timing_read()
+    ctx.timing_enable(False)
+    return ms, (t[0] / t[1] if t[1] else None), (t[2] / t[3] if t[3] else None)
+
+
+def cases(ctx, dev, which=ALL):
+    """Yields one record per secondary measurement."""
     gen = torch.Generator(device=dev)
     gen.manual_seed(2)
     if "c1" in which:
@@ -44,29 +67,27 @@ def main(which):
         g = torch.empty_like(x)
         run = ctx.make_fused(Segments([x]), grad=Segments([g]), lam=1e-4,
                              step=torch.full((1,), 1e-3, dtype=torch.float32, device=dev))
-        ms = timeit(run)
-        print(f"c1  fused, fp32 1024x1024, one segment: {ms * 1e3:.1f} us  {8 * x.numel() / ms / 1e6:.0f} GB/s")
+        yield rec("c1_fused", "fused pass, fp32 1024x1024, one segment (fits in L2: launch latency, not bandwidth)",
+                  timeit(run), 8 * x.numel())
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             run()
-        ms = timeit(graph.replay)
-        print(f"c1  the same call replayed from a CUDA graph: {ms * 1e3:.1f} us")
+        yield rec("c1_fused_graph", "the same call replayed from a CUDA graph", timeit(graph.replay), 8 * x.numel())
+        del graph
     if "c2" in which:
         shapes = gg_synth.qwen05b_shapes()
         outs = [torch.empty(r * c, dtype=torch.bfloat16, device=dev) for _, r, c in shapes]
         beta, al = 1.3, gg_synth.alpha_for_std(0.02, 1.3)
         n = sum(o.numel() for o in outs)
         ms = timeit(lambda: ctx.gg_sample(outs, [beta] * len(outs), [al] * len(outs), seed=1), 3, 1)
-        print(f"c2  gg_sample, {len(outs)} bf16 matrices, {n:.3e} elements: {ms:.2f} ms  {n / ms / 1e6:.1f} G elements/s")
-        ms = timeit(lambda: ctx.gg_fit(outs), 5)
-        print(f"c2  gg_fit of them: {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
+        yield rec("c2_sample", f"gg_sample, {len(outs)} bf16 matrices of a Qwen-0.5B-shaped decoder, {n:.3e} elements",
+                  ms, 2 * n, steps=3, g_elements_per_s=n / ms / 1e6, bound="alu")
+        yield rec("c2_fit", "gg_fit of them", timeit(lambda: ctx.gg_fit(outs), 5), 2 * n, steps=5)
         gs = [torch.empty(o_.numel(), dtype=torch.float32, device=dev) for o_ in outs]
         run = ctx.make_fused(Segments(outs), grad=Segments(gs), lam=1e-4,
                              step=torch.full((len(outs),), 2.0 ** -10, dtype=torch.float32, device=dev))
-        ms = timeit(run, 5)
-        print(f"c2  fused pass over them (fp32 gradients, one histogram per matrix): {ms:.3f} ms  {6 * n / ms / 1e6:.0f} GB/s")
-        del gs, run
-        del outs
+        yield rec("c2_fused", "fused pass over them (fp32 gradients, one histogram per matrix)", timeit(run, 5), 6 * n, steps=5)
+        del gs, run, outs
     if "c3" in which:
         a = gg_synth.alpha_for_std(1.0, 0.8)
         x = gg_synth.gg_device(gen, 0.8, a, 8 * 2048 * 4096, torch.bfloat16, dev).view(8 * 2048, 4096)
@@ -75,37 +96,47 @@ def main(which):
         nseg = x.shape[0]
         run = ctx.make_fused(Segments.rows(x), grad=Segments.rows(g), lam=1e-4,
                              step=torch.full((nseg,), 0.01, dtype=torch.float32, device=dev), hist_id=[0] * nseg, n_hist=1)
-        ms = timeit(run)
-        print(f"c3  fused, bf16 [8, 2048, 4096], per-token segments, one histogram: {ms * 1e3:.1f} us  "
-              f"{6 * x.numel() / ms / 1e6:.0f} GB/s")
-        del x, g, run
+        yield rec("c3_fused", "fused pass, bf16 [8, 2048, 4096] activations with outliers, per-token segments, one histogram",
+                  timeit(run), 6 * x.numel())
+        del g, run
+        xf = x.float()
+        gf = torch.empty_like(xf)
+        run = ctx.make_fused(Segments.rows(xf), grad=Segments.rows(gf), lam=1e-4,
+                             step=torch.full((nseg,), 0.01, dtype=torch.float32, device=dev), hist_id=[0] * nseg, n_hist=1)
+        yield rec("c3_fused_fp32", "the same activations in fp32", timeit(run), 8 * xf.numel())
+        del x, xf, gf, run
     if "c4" in which or "codes" in which:
         n = 25_000_000
         xs = [gg_synth.gg_device(gen, 0.5, 10 ** (-6 + 3 * u), n, torch.float32, dev) for u in np.linspace(0.05, 0.95, 8)]
         gs = [torch.empty_like(t) for t in xs]
         if "c4" in which:
             run = ctx.make_fused(Segments(xs), grad=Segments(gs), lam=1e-4, step_scale=1 / 16)
-            run()                    # (the first launch of a kernel loads it: keep that out of the sweep timers)
-            ctx.timing_enable(True)
-            ctx.timing_read()
-            ms = timeit(run, 5)
-            t = ctx.timing_read()
-            ctx.timing_enable(False)
-            print(f"c4  fused, 8 fp32 buckets of 25 M, step = alpha / 16: {ms:.3f} ms  {8 * 8 * n / ms / 1e6:.0f} GB/s  "
-                  f"(moments {t[0] / t[1]:.3f} ms, gradient + histogram {t[2] / t[3]:.3f} ms)")
+            ms, first, tail = sweeps(ctx, run)
+            yield rec("c4_fused", "fused pass, 8 fp32 gradient buckets of 25 M, step = alpha / 16", ms, 8 * 8 * n, steps=5,
+                      first_sweep_ms=first, second_sweep_ms=tail)
+            fit = run.outputs
+            from paper_2506_00486_b200 import GG_PARAMS_GIVEN
+            steps = run.outputs["step"].clone()
+            run1 = ctx.make_fused(Segments(xs), grad=Segments(gs), lam=1e-4, step=steps, param_mode=GG_PARAMS_GIVEN,
+                                  beta_in=fit["beta"].clone(), alpha_in=fit["alpha"].clone())
+            ms, first, tail = sweeps(ctx, run1)
+            yield rec("c4_fused_given", "the same with the parameters of the step before (penalty lags one step)", ms, 8 * 8 * n,
+                      steps=5, first_sweep_ms=first, second_sweep_ms=tail)
+            del run, run1
         if "codes" in which:
             w = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(8)]
             steps = torch.tensor([10 ** (-6 + 3 * u) / 16 for u in np.linspace(0.05, 0.95, 8)], dtype=torch.float32, device=dev)
             sx, sg, sw = Segments(xs), Segments(gs), Segments(w)
             for t_ in gs:
                 t_.fill_(1e-4)
-            ms = timeit(lambda: ctx.gg_gct_step(sx, sg, sw, steps, 1e-3, 0.05, 1e-8, 2))
-            print(f"codes  gg_gct_step, 8 x 25 M fp32: {ms:.3f} ms  {20 * 8 * n / ms / 1e6:.0f} GB/s (3 reads + 2 writes)")
-            ms = timeit(lambda: ctx.gg_eg_rate_grad(sx, steps, 0.3, sg))
-            print(f"codes  gg_eg_rate_grad, 8 x 25 M fp32: {ms:.3f} ms  {8 * 8 * n / ms / 1e6:.0f} GB/s (1 read + 1 write)")
+            yield rec("gct_step", "gg_gct_step (Algorithm 2), 8 x 25 M fp32: 3 reads + 2 writes",
+                      timeit(lambda: ctx.gg_gct_step(sx, sg, sw, steps, 1e-3, 0.05, 1e-8, 2)), 20 * 8 * n)
+            yield rec("eg_rate_grad", "gg_eg_rate_grad, 8 x 25 M fp32: 1 read + 1 write",
+                      timeit(lambda: ctx.gg_eg_rate_grad(sx, steps, 0.3, sg)), 8 * 8 * n)
             rh = ctx.gg_rate_hist(xs, steps)
-            ms = timeit(lambda: ctx.gg_eg_rate(rh["hist"]))
-            print(f"codes  gg_eg_rate, 8 histograms of 65536 bins: {ms * 1e3:.1f} us")
+            yield rec("eg_rate", "gg_eg_rate, 8 histograms of 65536 bins", timeit(lambda: ctx.gg_eg_rate(rh["hist"])), 8 * 8 * 65536)
+            del w
+        del xs, gs
     if "calls" in which:
         # the single-step entry points on the Llama-7B-shaped sweep with every dimension halved (1.68e9 elements)
         w = gg_synth.workload_c5_device(dev, torch.bfloat16, shapes=gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), 2), seed=4)
@@ -116,12 +147,12 @@ def main(which):
         n = flat.numel()
         steps = torch.full((len(lens),), 2.0 ** -10, dtype=torch.float32, device=dev)
         fit = ctx.gg_fit(segs)
-        ms = timeit(lambda: ctx.gg_fit(segs))
-        print(f"calls  gg_fit, {len(lens)} bf16 matrices, {n:.3e} elements: {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
-        ms = timeit(lambda: ctx.gg_penalty_grad(segs, fit["beta"], fit["alpha"], 1e-4, grad=gsegs))
-        print(f"calls  gg_penalty_grad (fp32 gradients): {ms:.3f} ms  {6 * n / ms / 1e6:.0f} GB/s")
-        ms = timeit(lambda: ctx.gg_rate_hist(segs, steps))
-        print(f"calls  gg_rate_hist (one histogram per matrix, entropy): {ms:.3f} ms  {2 * n / ms / 1e6:.0f} GB/s")
+        yield rec("call_fit", f"gg_fit, {len(lens)} bf16 matrices (Llama-7B shapes with halved dimensions), {n:.3e} elements",
+                  timeit(lambda: ctx.gg_fit(segs)), 2 * n)
+        yield rec("call_penalty_grad", "gg_penalty_grad on them (fp32 gradients)",
+                  timeit(lambda: ctx.gg_penalty_grad(segs, fit["beta"], fit["alpha"], 1e-4, grad=gsegs)), 6 * n)
+        yield rec("call_rate_hist", "gg_rate_hist on them (one histogram per matrix, entropy)",
+                  timeit(lambda: ctx.gg_rate_hist(segs, steps)), 2 * n)
         del w, flat, g, segs, gsegs
     if "channels" in which:
         for rows, cols, spread, dt in ((16384, 4096, 3, torch.bfloat16), (65536, 4096, 3, torch.bfloat16),
@@ -135,19 +166,27 @@ def main(which):
             gg_synth.add_outliers_device(gen, x, 1e-3, 20.0)
             g = torch.empty((rows, cols), dtype=torch.float32, device=dev)
             run = ctx.make_fused_channels(x, grad=g, lam=1e-4, step=0.01)
-            run()                    # (the first launch of a kernel loads it: keep that out of the sweep timers)
-            ctx.timing_enable(True)
-            ctx.timing_read()
-            ms = timeit(run, 5)
-            t = ctx.timing_read()
-            ctx.timing_enable(False)
+            ms, first, tail = sweeps(ctx, run)
             name = "bf16" if dt == torch.bfloat16 else "fp32"
-            print(f"channels  fused, {name} [{rows}, {cols}], column scales 2^-{spread // 2}..2^{spread // 2}, one GG per column, one histogram: {ms * 1e3:.1f} us  "
-                  f"{(x.element_size() + 4) * x.numel() / ms / 1e6:.0f} GB/s  (moments {t[0] / t[1] * 1e3:.1f} us, "
-                  f"gradient + histogram {t[2] / t[3] * 1e3:.1f} us)")
+            yield rec(f"channels_{name}_{rows}x{cols}_spread{spread}",
+                      f"gg_fused_channels, {name} [{rows}, {cols}], column scales 2^-{spread // 2}..2^{spread // 2}, one GG per column, one histogram",
+                      ms, (x.element_size() + 4) * x.numel(), steps=5, first_sweep_ms=first, second_sweep_ms=tail)
             del x, g, run
+
+
+def main(which):
+    dev = torch.device("cuda", 0)
+    ctx = Context(0)
+    for r in cases(ctx, dev, which):
+        line = f"{r['name']:<36s} {r['ms'] * 1e3:10.1f} us"
+        if "gbs" in r:
+            line += f"  {r['gbs']:7.0f} GB/s"
+        for k in ("first_sweep_ms", "second_sweep_ms", "g_elements_per_s"):
+            if r.get(k) is not None:
+                line += f"  {k} {r[k]:.3f}"
+        print(line + "   " + r["what"], flush=True)
     ctx.close()
 
 
 if __name__ == "__main__":
-    main(set(sys.argv[1:]) or {"c1", "c2", "c3", "c4", "codes", "calls", "channels"})
+    main(set(sys.argv[1:]) or set(ALL))
