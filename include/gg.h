@@ -75,7 +75,7 @@ typedef struct {
 
 #define GG_PARAMS_FITTED 0   /* penalty uses the (beta, alpha) fitted by this call: two reads of x */
 #define GG_PARAMS_GIVEN  1   /* penalty uses caller-supplied (beta, alpha); the fit of this call is
-                                still produced: one read of bf16 x                               */
+                                still produced: one read of x                                    */
 #define GG_STEP_GIVEN      0 /* quantiser step[s] supplied by the caller                        */
 #define GG_STEP_FROM_ALPHA 1 /* step[s] = (float)(fitted alpha[s] * step_scale), also written out */
 
@@ -202,8 +202,7 @@ typedef struct {
 /* The whole pass over a list of segments in the fewest sweeps of x: moments -> fit ->
  * penalty + gradient + histogram -> entropy, all enqueued on `stream`.
  * GG_PARAMS_FITTED reads x twice (the gradient needs the fit of the whole segment);
- * GG_PARAMS_GIVEN reads bf16 x once (moments, gradient and histogram in the same sweep; fp32 x takes two
- * sweeps in either mode).
+ * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep).
  * The first call with a new layout (segment addresses and lengths) builds and caches its plan with
  * blocking allocations; later calls with that layout only enqueue kernels and memsets on `stream`
  * and may be captured in a CUDA graph (the same holds for gg_fused_channels once its scratch is

@@ -9,7 +9,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgg_b200.so")
-SOURCES = ["gg_api.cu", "gg_stream.cu", "gg_tail_bf16.cu", "gg_tail_f32.cu", "gg_small_bf16.cu", "gg_segment.cu", "gg_sample.cu", "gg_codes.cu", "gg_channels.cu", "gg_channels_f32.cu", "gg_noalloc.cu"]
+SOURCES = ["gg_api.cu", "gg_stream.cu", "gg_tail_bf16.cu", "gg_tail_f32.cu", "gg_small_bf16.cu", "gg_team.cu", "gg_segment.cu", "gg_sample.cu", "gg_codes.cu", "gg_channels.cu", "gg_channels_f32.cu", "gg_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -292,7 +292,7 @@ cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype gra
         return launch_moments_bf16_sweep(sa, ctx->sm_count, cs);
     if (in_dtype == GG_BF16 && (flags & (kGrad | kHist)) != 0)
         return launch_tail_bf16(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
-    if (in_dtype == GG_F32 && (flags & kMoments) == 0 && flags != 0)
+    if (in_dtype == GG_F32 && (flags & (kGrad | kHist)) != 0)
         return launch_tail_f32(flags, grad_dtype, has_grad_out, sa, ctx->sm_count, cs);
     return launch_stream(flags, in_dtype, grad_dtype, has_grad_out, sa, cs);
 }
@@ -689,8 +689,8 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         const double *beta_used;
         // Many short bf16 segments with fitted parameters: one kernel, one warp per segment, does the
         // whole pass (below a few dozen segments the two-sweep path fills the GPU better).
-        const bool small_path = a->param_mode == GG_PARAMS_FITTED && in_dt == GG_BF16 && p->max_len <= kSmallSegMax &&
-                                n_seg >= 64;
+        // (bf16: one warp per segment; fp32: one team of four warps per segment)
+        const bool small_path = a->param_mode == GG_PARAMS_FITTED && p->max_len <= kSmallSegMax && n_seg >= 64;
         if (small_path) {
             SmallArgs ka{};
             ka.map = p->map;
@@ -708,7 +708,8 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             ka.cta_counts = ctx->small_counts;
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
-                GG_CUDA(ctx, launch_small_bf16(g_dt, ka, ctx->sm_count, cs));
+                if (in_dt == GG_BF16) GG_CUDA(ctx, launch_small_bf16(g_dt, ka, ctx->sm_count, cs));
+                else GG_CUDA(ctx, launch_team_f32(g_dt, ka, ctx->sm_count, cs));
             }
             ctx->launches += 1 + (do_hist ? 1 : 0);
         } else if (a->param_mode == GG_PARAMS_FITTED && in_dt == GG_BF16 && tail_flags != 0 &&
@@ -753,17 +754,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         } else {
             // one sweep: moments, gradient (given parameters) and histogram together; then the fit
             sa.beta = a->beta_in; sa.alpha = a->alpha_in; sa.step = a->step;
-            if (in_dt == GG_F32 && tail_flags != 0) {
-                // fp32 input has no combined persistent sweep: the moments kernel and the gradient + histogram
-                // kernel, both streaming at their own speed, beat the generic kernel that does all three at once
-                {
-                    SweepTimer tm(ctx, &ctx->ev_first, cs);
-                    GG_CUDA(ctx, launch_sweep(ctx, kMoments, in_dt, g_dt, false, sa, cs));
-                }
-                SweepTimer tm(ctx, &ctx->ev_tail, cs);
-                GG_CUDA(ctx, launch_sweep(ctx, tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
-                ctx->launches += p->n_tiles > 0;
-            } else {
+            {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
                 GG_CUDA(ctx, launch_sweep(ctx, kMoments | tail_flags, in_dt, g_dt, a->grad != nullptr, sa, cs));
             }

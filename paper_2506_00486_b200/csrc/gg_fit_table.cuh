@@ -108,8 +108,14 @@ __device__ __forceinline__ double log_rho(double beta)
 // that follows).  WARP: all 32 lanes of a warp call with the same arguments; lane 0 writes.  Without a fit table
 // (a.seed null) the root is found by 33-section search on ln(beta): each round the 32 lanes evaluate log_rho at
 // the interior points of the bracket and a ballot picks the sub-interval with the sign change.
-__device__ __forceinline__ void fit_finish(const FitArgs &a, int s, int lane, double s1, double s2, uint32_t bad, float xmin,
-                                           float xmax)
+// The results every lane holds on return: the parameters and the quantiser step of the segment.
+struct FitResult {
+    double beta, alpha;
+    float step;
+};
+
+__device__ __forceinline__ FitResult fit_finish(const FitArgs &a, int s, int lane, double s1, double s2, uint32_t bad, float xmin,
+                                                float xmax)
 {
     constexpr unsigned kFull = 0xFFFFFFFFu;
     const int64_t len = a.map.seg_len[s];
@@ -158,13 +164,13 @@ __device__ __forceinline__ void fit_finish(const FitArgs &a, int s, int lane, do
         alpha = sqrt(m2) * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
         }
     }
+    const float step = a.step_from_alpha ? (float)(alpha * a.step_scale) : (a.step ? a.step[s] : 0.0f);
     if (lane == 0) {
         a.beta[s] = beta;
         a.alpha[s] = alpha;
         if (a.sum_abs) a.sum_abs[s] = s1;
         if (a.sum_sq) a.sum_sq[s] = s2;
         if (a.count) a.count[s] = len;
-        const float step = a.step_from_alpha ? (float)(alpha * a.step_scale) : (a.step ? a.step[s] : 0.0f);
         if (a.step_from_alpha && a.step_out) a.step_out[s] = step;
         if (a.hist_on && xmin <= xmax) {
             // the quantiser is monotone in x, so a symbol clamps iff one of the extremes does
@@ -176,6 +182,7 @@ __device__ __forceinline__ void fit_finish(const FitArgs &a, int s, int lane, do
         if (a.flags) a.flags[s] = flags;
         if (a.sd_out) a.sd_out[s] = (len > 0 && s2 > 0.0) ? sqrt(s2 / (double)len) : 0.0;
     }
+    return FitResult{beta, alpha, step};
 }
 
 // 2^t for |t| < 1000 within 1e-11 relative: table entries are rounded to fp32 afterwards.

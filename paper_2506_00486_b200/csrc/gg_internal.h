@@ -135,12 +135,19 @@ struct SmallArgs {
 };
 constexpr int kSmallSlotWords = 8200;  // a CTA's count cells and its histogram key
 int small_grid(int32_t n_seg, int sm_count);   // CTAs launch_small_bf16 uses
+// Turns the pattern-count slots of n_slots CTAs (kSmallSlotWords words each, key in the last four) into symbols.
+cudaError_t launch_small_flush(const uint32_t *cta_counts, int n_slots, int32_t qmin, int32_t qmax, uint64_t *hist, uint64_t *clamped,
+                               cudaStream_t st);
 cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st);
+// Whole pass for short fp32 segments: one team of four warps per segment, the segment held in registers between the
+// moments and the gradient (gg_team.cu).  cta_counts as for launch_small_bf16.
+int team_grid(int32_t n_seg, int sm_count);    // CTAs launch_team_f32 uses
+cudaError_t launch_team_f32(gg_dtype grad_dtype, const SmallArgs &a, int sm_count, cudaStream_t st);
 // Fills the fit table, 2 * (kSeedCells + 1) doubles: ln rho(beta_i) and then ln(alpha/sigma)(beta_i), ln beta_i
 // evenly spaced over [ln GG_BETA_LO, ln GG_BETA_HI].
 cudaError_t launch_fit_seed_table(double *table, cudaStream_t st);
 
-// fp32-input sweeps with a gradient and/or a histogram but no moments (flags in kGrad, kHist, kGrad | kHist):
+// fp32-input sweeps with a gradient and/or a histogram, with or without the moments (any flags with kGrad or kHist):
 // persistent CTAs, table + series gradient, symbol counts in shared memory.
 cudaError_t launch_tail_f32(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a, int sm_count,
                             cudaStream_t st);

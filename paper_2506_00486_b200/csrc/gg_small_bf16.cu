@@ -18,6 +18,7 @@
 #include "gg_fit_table.cuh"
 #include "gg_device.cuh"
 #include "gg_internal.h"
+#include "gg_small_common.cuh"
 
 namespace gg {
 namespace {
@@ -26,16 +27,7 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kCtasPerSm = 2;
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kCntBinades = 32;
-constexpr uint32_t kCntPat = kCntBinades * 128;
 constexpr int kTabExp = 64;          // exponents around the segment's scale whose A is evaluated
-// count cells of a CTA: two per pattern of the window (sign), the sentinel pair that swallows the
-// first-pass counts of values outside the window, and the pair for values below the window
-constexpr uint32_t kSentinel = kCntPat * 2, kBelow = kCntPat * 2 + 2;
-constexpr uint32_t kCells = kCntPat * 2 + 4;
-static_assert(kCells + 4 <= (uint32_t)kSmallSlotWords, "scratch slot");
-constexpr int kMaxSlots = 1024;      // CTAs of one launch whose tables the flush kernel can take
-
 struct WarpTab {
     float a1[256];       // A[e] as one factor (with lambda's sign); NaN where that is not possible or not evaluated
     float B[128];
@@ -70,15 +62,6 @@ __global__ void seed_table_kernel(double *table)
     table[kSeedCells + 1 + i] = 0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta));
 }
 
-// The gradient magnitude in fp64 for one magnitude pattern: the exact path.  The caller adds its
-// penalty term |x| |g| before rounding the gradient to fp32 (which may underflow or overflow).
-__device__ __noinline__ double grad_fp64(uint32_t mag, double L, double b, bool active)
-{
-    const float ax = __uint_as_float(mag << 16);
-    if (!active || ax == 0.0f) return 0.0;
-    return exp2(L + b * log2((double)ax));
-}
-
 template <typename TG>
 __device__ __forceinline__ float load_grad(const TG *g)
 {
@@ -107,22 +90,6 @@ struct SegConst {
     uint32_t c_base;
     bool below_ok;
 };
-
-// Quantises one value and counts its symbol in global memory (elements the CTA table does not serve).
-// Returns 1 / 2 if the symbol was clamped at the low / high end, else 0.  (Everything by value: a
-// structure passed by reference to a function that is not inlined would live in local memory.)
-__device__ __noinline__ int count_global(uint32_t xb, float inv, int32_t qmin, int32_t qmax, unsigned long long *row)
-{
-    const float t = __fmul_rn(__uint_as_float(xb), inv);
-    int clamped = 0;
-    if (t == t) {                               // NaN is skipped
-        int q = __float2int_rd(t);              // floor, saturating
-        if (q < qmin) { q = qmin; clamped = 1; }
-        else if (q > qmax) { q = qmax; clamped = 2; }
-        atomicAdd(&row[q - qmin], 1ull);
-    }
-    return clamped;
-}
 
 // One element of a 32-bit word w holding two bf16 values (HALF 0: low half, 1: high half).  Branch
 // free.  Gradient: a NaN entry of the warp's A table makes the vector's penalty partial NaN, which
@@ -188,14 +155,6 @@ __device__ __forceinline__ float small_fix(uint32_t xb, float g, bool grad_bad, 
         }
     }
     return g;
-}
-
-// Exponent field of the top binade of the CTA's pattern-count window: 2^11 steps.
-__device__ __forceinline__ int window_top_exponent(double step)
-{
-    int e = 127 + 11;
-    if (step > 0.0 && step < 1e300) e = ilogb(step) + 127 + 11;
-    return max(kCntBinades, min(254, e));
 }
 
 // Second pass over one segment by one warp.
@@ -629,6 +588,15 @@ cudaError_t launch_small_bf16(gg_dtype grad_dtype, const SmallArgs &a, int sm_co
     if (a.map.n_seg <= 0) return cudaSuccess;
     if (a.do_grad && a.map.grad_ptr != nullptr && grad_dtype == GG_BF16) return launch_typed<uint16_t>(a, sm_count, st);
     return launch_typed<float>(a, sm_count, st);
+}
+
+cudaError_t launch_small_flush(const uint32_t *cta_counts, int n_slots, int32_t qmin, int32_t qmax, uint64_t *hist, uint64_t *clamped,
+                               cudaStream_t st)
+{
+    if (n_slots <= 0) return cudaSuccess;
+    if (n_slots > kMaxSlots) return cudaErrorInvalidValue;
+    small_flush_kernel<<<(kCells + 31) / 32, dim3(32, 8), 0, st>>>(cta_counts, n_slots, qmin, qmax, hist, clamped);
+    return cudaGetLastError();
 }
 
 int small_grid(int32_t n_seg, int sm_count)

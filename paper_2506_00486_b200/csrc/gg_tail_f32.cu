@@ -1,5 +1,6 @@
-// fp32-input sweep with a gradient and/or a histogram: the counterpart of the bf16 pattern kernel for
-// tensors whose elements are full fp32 numbers (gradient buckets and the like).
+// fp32-input sweep with a gradient and/or a histogram (and, when the parameters are given, the moments of the
+// next fit in the same read): the counterpart of the bf16 pattern kernel for tensors whose elements are full
+// fp32 numbers (gradient buckets and the like).
 //
 // Persistent CTAs each walk one contiguous range of tiles; inside a segment that is one contiguous
 // run of elements, streamed as pairs of 128-bit vectors through a per-thread ring of shared-memory
@@ -57,9 +58,18 @@ struct Smem {
     float brep[128 * 32];               // row j: B[j] = (1 + j/128)^b in every bank
     float B[128];
     double lg[128];                     // log2(1 + j/128)
-    double red[kWarps];
+    double red[3][kWarps];             // sum |x|, sum x^2, sum |x| |g| of the warps
+    uint32_t bad[kWarps];
+    float mn[kWarps], mx[kWarps];
     uint32_t clampc[2];
     Cold cold;
+};
+
+// Per-thread sums of one run.
+struct Acc {
+    double s1 = 0.0, s2 = 0.0, pen = 0.0;
+    uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
 };
 
 // A[e] as one factor (with lambda's sign), NaN where that is not possible.  Static shared memory:
@@ -112,10 +122,17 @@ template <> struct Window<kModeWords> {
 // partial NaN, which the caller checks once per vector.  Count: `anyt` keeps the largest |x * inv|
 // so that one compare per vector finds symbols outside the window; those count on a sentinel.
 template <int FLAGS, int MODE>
-__device__ __forceinline__ float one_elem(uint32_t xb, const Lane &ln, float &mp, float &anyt)
+__device__ __forceinline__ float one_elem(uint32_t xb, const Lane &ln, float &mp, float &anyt, float &m1, float &m2, Acc &acc)
 {
     float ga = 0.0f;
     const float x = __uint_as_float(xb);
+    if constexpr ((FLAGS & kMoments) != 0) {
+        // fp32 sums of the vector; an inf or nan makes them inf or nan, and the vector is then summed again in fp64
+        m1 += fabsf(x);
+        m2 = fmaf(x, x, m2);
+        acc.xmin = fminf(acc.xmin, x);          // fminf / fmaxf return the non-NaN operand
+        acc.xmax = fmaxf(acc.xmax, x);
+    }
     if constexpr ((FLAGS & kGrad) != 0) {
         const uint32_t ax = xb & 0x7FFFFFFFu;
         const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(s_a1) + ((ax >> 21) & 0x3FCu));
@@ -271,14 +288,14 @@ __device__ __forceinline__ void store8(TG *g, const float (&v)[8], bool accumula
 // penalty partial.  Returns through g.
 template <int FLAGS, int MODE>
 __device__ __forceinline__ void process8(const uint4 &lo, const uint4 &hi, int n, float (&g)[8], const Lane &ln, Smem &sm,
-                                         double &pen, uint32_t (&clampc)[2])
+                                         Acc &acc, uint32_t (&clampc)[2])
 {
-    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-    float mp = 0.0f, anyt = 0.0f;
+    float mp = 0.0f, anyt = 0.0f, m1 = 0.0f, m2 = 0.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        if (i < n) g[i] = one_elem<FLAGS, MODE>(w[i], ln, mp, anyt);
+        if (i < n) g[i] = one_elem<FLAGS, MODE>(w[i], ln, mp, anyt, m1, m2, acc);
     }
     const bool grad_bad = GRAD && !(mp <= FLT_MAX);
     if (grad_bad || (HIST && count_miss<MODE>(anyt))) {
@@ -287,10 +304,27 @@ __device__ __forceinline__ void process8(const uint4 &lo, const uint4 &hi, int n
             if (i < n) g[i] = fix_elem<FLAGS, MODE>(w[i], g[i], grad_bad, ln, sm, clampc);
         }
     }
+    if constexpr (MOM) {
+        if (run_sums_exact_enough(m1, m2)) {
+            acc.s1 += (double)m1;
+            acc.s2 += (double)m2;
+        } else {     // a square or a sum outside the fp32 range, or an inf or nan entry: these elements again in fp64
+            for (int e = 0; e < n; ++e) {
+                const uint32_t ab = w[e] & 0x7FFFFFFFu;
+                if (ab < 0x7F800000u) {
+                    const double ax = (double)__uint_as_float(ab);
+                    acc.s1 += ax;
+                    acc.s2 += ax * ax;
+                } else {
+                    acc.bad += 1u;
+                }
+            }
+        }
+    }
     if constexpr (GRAD) {
         // a product or a gradient that left the fp32 range, or a NaN marker, sends the vector to fp64
-        if (mp <= FLT_MAX) pen += (double)mp;
-        else pen += pen_exact(lo, hi, n, sm.cold.L, sm.cold.b, sm.cold.active);
+        if (mp <= FLT_MAX) acc.pen += (double)mp;
+        else acc.pen += pen_exact(lo, hi, n, sm.cold.L, sm.cold.b, sm.cold.active);
     }
 }
 
@@ -299,7 +333,7 @@ __device__ __forceinline__ void process8(const uint4 &lo, const uint4 &hi, int n
 // 16-byte aligned at the same element the whole run is scalar.
 template <typename TG, int FLAGS, int MODE>
 __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t n, bool accumulate, const Lane &ln,
-                                              Smem &sm, double &pen, uint32_t (&clampc)[2])
+                                              Smem &sm, Acc &acc, uint32_t (&clampc)[2])
 {
     constexpr bool GRAD = (FLAGS & kGrad) != 0;
     const int tid = threadIdx.x;
@@ -313,7 +347,7 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
         const int64_t idx = i < head ? i : tail0 + (i - head);
         float g[8];
         process8<FLAGS, MODE>(make_uint4(__float_as_uint(__ldg(x + idx)), 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u), 1, g, ln,
-                              sm, pen, clampc);
+                              sm, acc, clampc);
         if constexpr (GRAD) {
             if (gout != nullptr) {
                 float v = g[0];
@@ -358,7 +392,7 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(slot0 + rd) : "memory");
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(slot0 + rd + kHalfBytes) : "memory");
         float g[8];
-        process8<FLAGS, MODE>(lo, hi, 8, g, ln, sm, pen, clampc);
+        process8<FLAGS, MODE>(lo, hi, 8, g, ln, sm, acc, clampc);
         if constexpr (GRAD) {
             if (gv != nullptr) store8<TG>(gv, g, accumulate, wide);
         }
@@ -373,7 +407,7 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
 template <typename TG, int FLAGS>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const StreamArgs a)
 {
-    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -462,10 +496,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
                     if (fabsf(v) <= 1e18f) ss = fmaf(v, v, ss);        // (inf, nan and values whose squares overflow are left out)
                 }
                 const double ws = warp_sum((double)ss);
-                if ((tid & 31) == 0) sm.red[tid >> 5] = ws;             // (free here: the barrier above follows the run before)
+                if ((tid & 31) == 0) sm.red[2][tid >> 5] = ws;          // (free here: the barrier above follows the run before)
                 __syncthreads();
                 double tot = 0.0;
-                for (int w = 0; w < kWarps; ++w) tot += sm.red[w];
+                for (int w = 0; w < kWarps; ++w) tot += sm.red[2][w];
                 sd = m > 0 ? sqrt(tot / (double)m) : 0.0;
                 __syncthreads();
             }
@@ -500,28 +534,58 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
         if constexpr (GRAD) {
             if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
         }
-        double pen = 0.0;
+        Acc acc;
         uint32_t clampc[2] = {0u, 0u};
-        if (HIST && mode == kModeRows) process_range<TG, FLAGS, kModeRows>(x, gout, n, accumulate, ln, sm, pen, clampc);
-        else process_range<TG, FLAGS, kModeWords>(x, gout, n, accumulate, ln, sm, pen, clampc);
+        if (HIST && mode == kModeRows) process_range<TG, FLAGS, kModeRows>(x, gout, n, accumulate, ln, sm, acc, clampc);
+        else process_range<TG, FLAGS, kModeWords>(x, gout, n, accumulate, ln, sm, acc, clampc);
 
-        // ---- per-run results: the penalty partial in a fixed order (butterfly, then the warps in
-        // sequence) to the slot of the run's first tile, zeros to its other tiles; clamp counts
+        // ---- per-run results: the partial sums in a fixed order (butterfly, then the warps in sequence) to the
+        // slot of the run's first tile, zeros to its other tiles; clamp counts
+        if constexpr (MOM) {
+            const double w1 = warp_sum(acc.s1), w2 = warp_sum(acc.s2);
+            const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, acc.bad);
+            float wmin = acc.xmin, wmax = acc.xmax;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                wmin = fminf(wmin, __shfl_xor_sync(0xFFFFFFFFu, wmin, o));
+                wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+            }
+            if (lane == 0) { sm.red[0][warp] = w1; sm.red[1][warp] = w2; sm.bad[warp] = wb; sm.mn[warp] = wmin; sm.mx[warp] = wmax; }
+        }
         if constexpr (GRAD) {
-            const double wp = warp_sum(pen);
-            if (lane == 0) sm.red[warp] = wp;
+            const double wp = warp_sum(acc.pen);
+            if (lane == 0) sm.red[2][warp] = wp;
         }
         if constexpr (HIST) {
             if (clampc[0]) atomicAdd(&sm.clampc[0], clampc[0]);
             if (clampc[1]) atomicAdd(&sm.clampc[1], clampc[1]);
         }
         __syncthreads();
-        if constexpr (GRAD) {
-            for (int tt = t + 1 + tid; tt < t_stop; tt += kThreads) a.part.pen[tt] = 0.0;
+        if constexpr (MOM || GRAD) {
+            for (int tt = t + 1 + tid; tt < t_stop; tt += kThreads) {
+                if constexpr (MOM) {
+                    a.part.s1[tt] = 0.0; a.part.s2[tt] = 0.0; a.part.bad[tt] = 0u;
+                    a.part.xmin[tt] = INFINITY; a.part.xmax[tt] = -INFINITY;
+                }
+                if constexpr (GRAD) a.part.pen[tt] = 0.0;
+            }
             if (tid == 0) {
-                double rp = 0.0;
-                for (int w = 0; w < kWarps; ++w) rp += sm.red[w];
-                a.part.pen[t] = sm.cold.sign_flip ? -rp : rp;     // the penalty carries lambda's sign
+                if constexpr (MOM) {
+                    double r1 = 0.0, r2 = 0.0;
+                    uint32_t rb = 0;
+                    float rmin = INFINITY, rmax = -INFINITY;
+                    for (int w = 0; w < kWarps; ++w) {
+                        r1 += sm.red[0][w]; r2 += sm.red[1][w]; rb += sm.bad[w];
+                        rmin = fminf(rmin, sm.mn[w]); rmax = fmaxf(rmax, sm.mx[w]);
+                    }
+                    a.part.s1[t] = r1; a.part.s2[t] = r2; a.part.bad[t] = rb;
+                    a.part.xmin[t] = rmin; a.part.xmax[t] = rmax;
+                }
+                if constexpr (GRAD) {
+                    double rp = 0.0;
+                    for (int w = 0; w < kWarps; ++w) rp += sm.red[2][w];
+                    a.part.pen[t] = sm.cold.sign_flip ? -rp : rp;     // the penalty carries lambda's sign
+                }
             }
             __syncthreads();
         }
@@ -551,6 +615,9 @@ cudaError_t launch_typed(int flags, const StreamArgs &a, int sm_count, cudaStrea
     case kGrad: return launch_one<TG, kGrad>(a, sm_count, st);
     case kHist: return launch_one<TG, kHist>(a, sm_count, st);
     case kGrad | kHist: return launch_one<TG, kGrad | kHist>(a, sm_count, st);
+    case kMoments | kGrad: return launch_one<TG, kMoments | kGrad>(a, sm_count, st);
+    case kMoments | kHist: return launch_one<TG, kMoments | kHist>(a, sm_count, st);
+    case kMoments | kGrad | kHist: return launch_one<TG, kMoments | kGrad | kHist>(a, sm_count, st);
     default: return cudaErrorInvalidValue;
     }
 }

@@ -456,22 +456,60 @@ def test_fused_step_from_alpha_and_shared_histograms(ctx):
     check_fused(out, xs, gd, 3e-3, hid, 3, step_scale=1 / 16, mean=True)
 
 
-def test_fused_given_parameters_single_sweep(ctx):
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_fused_given_parameters_single_sweep(ctx, dtype):
     """Lagged mode: the gradient uses caller parameters while the same sweep produces the new fit."""
     from paper_2506_00486_b200 import Segments, GG_PARAMS_GIVEN
-    xs = make_segments(torch.bfloat16, seed=10)
-    xd = [dev(x) for x in xs]
+    xs = make_segments(dtype, seed=10)
+    xd = misaligned_views(xs) if dtype == torch.float32 else [dev(x) for x in xs]
     gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
     n = len(xs)
     given = [(0.5 + 0.2 * s, 0.01 * (s + 1)) for s in range(n)]
     bi = torch.tensor([g[0] for g in given], dtype=torch.float64, device="cuda:0")
     ai = torch.tensor([g[1] for g in given], dtype=torch.float64, device="cuda:0")
     steps = torch.full((n,), 0.01, dtype=torch.float32, device="cuda:0")
+    launches0 = ctx.launch_count
     out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps, param_mode=GG_PARAMS_GIVEN,
                        beta_in=bi, alpha_in=ai, qmin=-64, qmax=63)
     torch.cuda.synchronize()
     check_fused(out, xs, gd, 1e-4, list(range(n)), n, given=given, qmin=-64, qmax=63)
     assert (out["flags"].cpu().numpy() & 16).any()       # the narrow clamp was reported
+    assert ctx.launch_count - launches0 == 5             # ONE sweep, then the fit, the penalty sums and two entropy kernels
+
+
+def test_fused_given_parameters_fp32_moments_of_special_values(ctx):
+    """The one-read fp32 sweep takes its moments in fp32 runs of eight and falls back to fp64 where a square leaves
+    the fp32 range or an entry is not finite: the sums, the counts of left-out entries and the extremes (through
+    the clamp flag) must be those of the oracle."""
+    from paper_2506_00486_b200 import Segments, GG_PARAMS_GIVEN
+    rng = np.random.default_rng(12)
+    big = gg_synth.gg_host(rng, 1.0, 1e25, 3 * TILE + 11, torch.float32)            # squares overflow fp32
+    tiny = gg_synth.gg_host(rng, 1.2, 1e-28, 2 * TILE + 3, torch.float32)           # squares underflow
+    mixed = gg_synth.gg_host(rng, 0.8, 0.05, 5 * TILE + 1, torch.float32)
+    mixed[::997] = float("inf")
+    mixed[5::1013] = float("nan")
+    mixed[7::991] = -float("inf")
+    mixed[3] = 3e38
+    mixed[4] = 1e-44                                                                  # subnormal
+    xs = [big, tiny, mixed]
+    xd = [dev(x) for x in xs]
+    gd = [torch.empty(x.numel(), dtype=torch.float32, device="cuda:0") for x in xs]
+    bi = torch.tensor([1.0, 1.2, 0.8], dtype=torch.float64, device="cuda:0")
+    ai = torch.tensor([1e25, 1e-28, 0.05], dtype=torch.float64, device="cuda:0")
+    steps = torch.tensor([1e23, 1e-30, 0.01], dtype=torch.float32, device="cuda:0")
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps, param_mode=GG_PARAMS_GIVEN, beta_in=bi, alpha_in=ai)
+    torch.cuda.synchronize()
+    for s, x in enumerate(xs):
+        xo = gg_synth.to_oracle(x)
+        b, a, s1, s2, n, fl = o.fit(xo)
+        assert (out["flags"][s].item() & 15) == fl
+        assert_rel(out["sum_abs"][s].item(), s1, 1e-6, "sum_abs")
+        assert_rel(out["sum_sq"][s].item(), s2, 1e-6, "sum_sq")
+        assert_rel(out["beta"][s].item(), b, REL_FIT, "beta")
+        assert_rel(out["alpha"][s].item(), a, REL_FIT, "alpha")
+        hist, cl = o.quantise_hist(xo, steps[s].item())
+        np.testing.assert_array_equal(out["hist"][s].cpu().numpy(), hist.astype(np.int64))
+        assert bool(out["flags"][s].item() & 16) == bool(cl.sum() > 0)
 
 
 def test_config1_single_fp32_tensor(ctx):
@@ -521,25 +559,36 @@ def test_config3_activation_rows_scaled(ctx):
     check_fused(out, list(x), list(gd), w["lam"], w["hist_id"], 1)
 
 
-def short_segments(seed, n_seg=150):
-    """Many short bf16 segments of ragged lengths (1 .. 9000), a few of them empty, zero or tiny."""
+# Which kernel a list of short segments takes: bf16, one warp per segment; fp32, one team of four warps per
+# segment, which holds up to 4096 elements in registers and reads longer segments twice.
+SHORT_KINDS = {"warp_bf16": (torch.bfloat16, 9000), "team_f32": (torch.float32, 4000), "team_f32_reread": (torch.float32, 12000)}
+
+
+def short_segments(seed, n_seg=150, kind="warp_bf16"):
+    """Many short segments of ragged lengths, a few of them empty, zero or tiny."""
+    dtype, max_len = SHORT_KINDS[kind]
     rng = np.random.default_rng(seed)
     xs = []
     for s in range(n_seg):
-        n = int(rng.integers(1, 9000))
+        n = int(rng.integers(1, max_len))
         beta = float(rng.uniform(0.5, 2.5))
-        xs.append(gg_synth.gg_host(rng, beta, 10.0 ** rng.uniform(-3, 0.5), n, torch.bfloat16))
-    xs[3] = torch.zeros(0, dtype=torch.bfloat16)
-    xs[4] = torch.zeros(77, dtype=torch.bfloat16)
-    xs[5] = torch.tensor([1.0, -1.0], dtype=torch.bfloat16)
-    xs[6][:8] = torch.tensor([0.0, -0.0, 1e-40, -1e-39, 3e38, -3e38, 1e-30, 1e20]).to(torch.bfloat16)
+        xs.append(gg_synth.gg_host(rng, beta, 10.0 ** rng.uniform(-3, 0.5), n, dtype))
+    xs[3] = torch.zeros(0, dtype=dtype)
+    xs[4] = torch.zeros(77, dtype=dtype)
+    xs[5] = torch.tensor([1.0, -1.0], dtype=dtype)
+    xs[6] = torch.cat([xs[6], xs[6][:8]])
+    xs[6][:8] = torch.tensor([0.0, -0.0, 1e-40, -1e-39, 3e38, -3e38, 1e-30, 1e20]).to(dtype)
+    xs[8] = gg_synth.gg_host(rng, 3.4, 0.2, max_len, dtype)            # shape - 1 beyond the fp32 series: the fp64 path
+    xs[9] = gg_synth.gg_host(rng, 1.0, 1e-30, max_len // 2, dtype)     # far from every other scale
     return xs
 
 
-def test_fused_many_short_segments_fit_only_with_nonfinite_entries(ctx):
+@pytest.mark.parametrize("kind", list(SHORT_KINDS))
+def test_fused_many_short_segments_fit_only_with_nonfinite_entries(ctx, kind):
     from paper_2506_00486_b200 import Segments
-    xs = short_segments(32, n_seg=80)
-    xs[7][:3] = torch.tensor([float("inf"), float("nan"), float("-inf")]).to(torch.bfloat16)
+    xs = short_segments(32, n_seg=80, kind=kind)
+    xs[7] = torch.cat([xs[7], xs[7][:3]])
+    xs[7][:3] = torch.tensor([float("inf"), float("nan"), float("-inf")]).to(xs[7].dtype)
     out = ctx.gg_fused(Segments([dev(x) for x in xs]), want_penalty=False, want_hist=False)
     torch.cuda.synchronize()
     for s, x in enumerate(xs):
@@ -554,12 +603,13 @@ def test_fused_many_short_segments_fit_only_with_nonfinite_entries(ctx):
         assert_rel(out["alpha"][s].item(), a, REL_FIT, f"alpha[{s}]")
 
 
+@pytest.mark.parametrize("kind", list(SHORT_KINDS))
 @pytest.mark.parametrize("variant", ["shared_hist", "own_hist_step_from_alpha", "misaligned_bf16_grad_mean"])
-def test_fused_many_short_segments(ctx, variant):
-    """The one-warp-per-segment path: shared histogram (CTA count table), per-segment histograms with
-    steps taken from the fit (element-wise global counts), misaligned data with bf16 gradients."""
+def test_fused_many_short_segments(ctx, variant, kind):
+    """The one-warp-per-segment and one-team-per-segment paths: shared histogram (CTA count table), per-segment
+    histograms with steps taken from the fit (element-wise global counts), misaligned data with bf16 gradients."""
     from paper_2506_00486_b200 import Segments, GG_MEAN
-    xs = short_segments(31)
+    xs = short_segments(31, kind=kind)
     n = len(xs)
     if variant == "misaligned_bf16_grad_mean":
         xd = misaligned_views(xs, offsets=[(3 * s) % 8 for s in range(n)])
