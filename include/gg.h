@@ -283,11 +283,20 @@ gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double
  * kernel end, so a wait that cannot be satisfied costs a fraction of a second and leaves the context usable.
  *   GG_HOOK_RESIDENT_MODE   0 (default): two launches; 1: the one-launch form whenever it can run
  *   GG_HOOK_EXTRA_ARRIVALS  arrivals the fitting CTA waits for beyond the CTAs that exist (default 0); a positive
- *                           value makes its wait run out: the way to test the time-out path without any fault
+ *                           value makes its wait run out: the way to test the time-out path without any fault (the
+ *                           one-cluster-per-segment form then expects 16 bytes per unit more than it copies, with
+ *                           the same effect on its wait)
  *   GG_HOOK_WAIT_CAP        polls (about half a microsecond each) after which a wait gives up (default 2^18) */
 #define GG_HOOK_RESIDENT_MODE  0
 #define GG_HOOK_EXTRA_ARRIVALS 1
 #define GG_HOOK_WAIT_CAP       2
+#define GG_HOOK_CLUSTER_MODE   3   /* the fitted pass with bf16 segments of 32 KB .. 2 MB staged in the shared memory of a
+                                      thread-block cluster, so that DRAM sees x once (6 bytes per element instead of 8):
+                                      0 (default) never; 1 when the layout suits (segments of similar length, enough of
+                                      them); 2 whenever every segment fits a cluster of 16 and starts on a 16-byte
+                                      boundary.  It moves fewer bytes but takes longer than the two sweeps on an idle
+                                      B200 (a cluster works through load, fit and tables one after the other), which is
+                                      why it is off unless asked for. */
 gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value);
 
 /* The same pass for data that lives in HOST memory: every pointer of `args` that gg_fused documents

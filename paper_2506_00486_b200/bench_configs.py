@@ -20,7 +20,7 @@ if ROOT not in sys.path:
 import gg_synth  # noqa: E402
 from paper_2506_00486_b200 import Context, Segments  # noqa: E402
 
-ALL = ("c1", "c2", "c3", "c4", "codes", "calls", "channels")
+ALL = ("c1", "c2", "c3", "c4", "medium", "codes", "calls", "channels")
 
 
 def timeit(fn, n=10, warmup=3):
@@ -137,6 +137,26 @@ def cases(ctx, dev, which=ALL):
             yield rec("eg_rate", "gg_eg_rate, 8 histograms of 65536 bins", timeit(lambda: ctx.gg_eg_rate(rh["hist"])), 8 * 8 * 65536)
             del w
         del xs, gs
+    if "medium" in which:
+        # bf16 segments between the short-segment kernels and the long sweeps: one thread-block cluster per segment
+        # (the segment staged in shared memory, one DRAM read) against the two sweeps
+        from paper_2506_00486_b200.binding import HOOK_CLUSTER_MODE
+        for n_seg, seg_len, label in ((4096, 32768, "64 KB"), (1024, 131072, "256 KB"), (256, 524288, "1 MB")):
+            x = gg_synth.gg_device(gen, 1.1, gg_synth.alpha_for_std(0.02, 1.1), n_seg * seg_len, torch.bfloat16, dev)
+            g = torch.empty(x.numel(), dtype=torch.float32, device=dev)
+            offs, lens = [s * seg_len for s in range(n_seg)], [seg_len] * n_seg
+            steps = torch.full((n_seg,), 2.0 ** -10, dtype=torch.float32, device=dev)
+            for mode, name in ((2, "cluster"), (0, "sweeps")):
+                ctx.gg_test_hook(HOOK_CLUSTER_MODE, mode)
+                run = ctx.make_fused(Segments.slices(x, offs, lens), grad=Segments.slices(g, offs, lens), lam=1e-4, step=steps,
+                                     hist_id=[0] * n_seg, n_hist=1)
+                yield rec(f"medium_{n_seg}x{seg_len}_{name}",
+                          f"fused pass, {n_seg} bf16 segments of {label}, one histogram; " +
+                          ("one cluster per segment, staged in shared memory" if mode else "moments sweep, then gradient + histogram sweep"),
+                          timeit(run, 5), 6 * x.numel(), steps=5)
+                del run
+            ctx.gg_test_hook(HOOK_CLUSTER_MODE, 0)
+            del x, g
     if "calls" in which:
         # the single-step entry points on the Llama-7B-shaped sweep with every dimension halved (1.68e9 elements)
         w = gg_synth.workload_c5_device(dev, torch.bfloat16, shapes=gg_synth.scaled_shapes(gg_synth.llama7b_shapes(), 2), seed=4)

@@ -19,7 +19,7 @@ GG_PARAMS_FITTED, GG_PARAMS_GIVEN = 0, 1
 GG_STEP_GIVEN, GG_STEP_FROM_ALPHA = 0, 1
 FLAG_DEGENERATE, FLAG_BETA_CLAMPED_LO, FLAG_BETA_CLAMPED_HI, FLAG_NONFINITE, FLAG_CLAMPED_SYMBOLS = 1, 2, 4, 8, 16
 FLAG_TIMEOUT = 32
-HOOK_RESIDENT_MODE, HOOK_EXTRA_ARRIVALS, HOOK_WAIT_CAP = 0, 1, 2
+HOOK_RESIDENT_MODE, HOOK_EXTRA_ARRIVALS, HOOK_WAIT_CAP, HOOK_CLUSTER_MODE = 0, 1, 2, 3
 BETA_LO, BETA_HI = 0.05, 20.0
 
 _SEG_DTYPE = np.dtype([("ptr", np.uint64), ("len", np.int64)])

@@ -37,6 +37,8 @@ struct Plan {
     int32_t max_hist_id = -1;               // largest entry of hist_id
     int32_t n_seg = 0, n_tiles = 0;
     int64_t max_len = 0;          // longest segment
+    int64_t total_len = 0;
+    bool aligned16 = true;        // every segment (and gradient segment) starts on a 16-byte boundary
     void *dev = nullptr;          // one allocation holding all tables and scratch
     TileMap map{};
     TileScratch part{};
@@ -65,7 +67,9 @@ struct gg_ctx {
     int64_t chan_bytes = 0;
     double *seed = nullptr;       // device table that seeds the moment-ratio inversion of the short-segment kernel
     int resident_grid[2][8];      // CTAs the one-launch pass may use, by gradient type and sweep flags (-1: not asked yet)
-    bool can_cooperate = false;
+    bool can_cooperate = false, can_cluster = false;
+    int cluster_mode = 0;         // one cluster per segment for medium bf16 segments: 0 never, 1 when the layout suits, 2 whenever it can run
+    int cluster_max[5];           // resident clusters of size 1, 2, 4, 8, 16 (-1: not asked yet)
     int resident_mode = 0;        // 1: gg_fused takes the one-launch fitted pass whenever it can run
     int32_t expect_delta = 0;     // test hook: arrivals the fitter waits for beyond the streamers that exist
     uint32_t wait_cap = kWaitCap;
@@ -182,7 +186,12 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
         prefix[(size_t)s + 1] = prefix[(size_t)s] + (int32_t)((segs[s].len + kTile - 1) / kTile);
     const int32_t n_tiles = prefix[(size_t)n_seg];
     p->n_tiles = n_tiles;
-    for (int32_t s = 0; s < n_seg; ++s) p->max_len = segs[s].len > p->max_len ? segs[s].len : p->max_len;
+    for (int32_t s = 0; s < n_seg; ++s) {
+        p->max_len = segs[s].len > p->max_len ? segs[s].len : p->max_len;
+        p->total_len += segs[s].len;
+        if (reinterpret_cast<uintptr_t>(segs[s].ptr) % 16 != 0 || (grad && reinterpret_cast<uintptr_t>(grad[s].ptr) % 16 != 0))
+            p->aligned16 = false;
+    }
 
     // layout of the single device block
     size_t off = 0;
@@ -350,6 +359,33 @@ int resident_grid(gg_ctx *ctx, int flags, gg_dtype grad_dtype, bool has_grad_out
     return slot;
 }
 
+// The cluster size (a power of two up to 16) that stages the longest segment of the plan, or 0 when the
+// one-cluster-per-segment kernel does not suit the layout; *n_clusters: clusters to launch.
+int cluster_choice(gg_ctx *ctx, const Plan *p, int flags, gg_dtype grad_dtype, bool has_grad_out, int *n_clusters)
+{
+    if (ctx->cluster_mode == 0 || !ctx->can_cluster || !p->aligned16 || p->n_tiles <= 0) return 0;
+    const int64_t per_cta = cluster_tiles_per_cta();
+    const int64_t max_tiles = (p->max_len + kTile - 1) / kTile;
+    if (max_tiles > 16 * per_cta) return 0;
+    int size = 1, slot = 0;
+    while ((int64_t)size * per_cta < max_tiles) { size *= 2; ++slot; }
+    if (ctx->cluster_mode == 1) {
+        // worth it when segments are too long for the short-segment kernels, most of them need the cluster they get
+        // (the longest decides its size), and there are clusters enough to fill the GPU
+        const int64_t mean_tiles = p->n_tiles / std::max(p->n_seg, 1);
+        if (p->max_len <= kSmallSegMax || 2 * mean_tiles < max_tiles || (int64_t)p->n_seg * size < ctx->sm_count) return 0;
+    }
+    int &cached = ctx->cluster_max[slot];
+    if (cached < 0) {
+        int n = 0;
+        if (cluster_bf16_max_clusters(flags, grad_dtype, has_grad_out, size, &n) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        cached = n;
+    }
+    if (cached <= 0) return 0;
+    *n_clusters = std::min(cached, (int)p->n_seg);
+    return size;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------ C entry points
@@ -404,6 +440,8 @@ gg_status gg_create(gg_ctx **out, int device)
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
     for (auto &row : ctx->resident_grid) for (int &v : row) v = -1;
+    for (int &v : ctx->cluster_max) v = -1;
+    ctx->can_cluster = prop.clusterLaunch != 0;
     ctx->can_cooperate = prop.cooperativeLaunch != 0;
     {
         DeviceGuard guard(device);
@@ -578,6 +616,10 @@ gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value)
         if (value < 0 || value > 1000) return GG_ERR_INVALID_ARG;
         ctx->expect_delta = (int32_t)value;
         return GG_OK;
+    case GG_HOOK_CLUSTER_MODE:
+        if (value < 0 || value > 2) return GG_ERR_INVALID_ARG;
+        ctx->cluster_mode = (int)value;
+        return GG_OK;
     case GG_HOOK_WAIT_CAP:
         if (value < 1 || value > (1ll << 24)) return GG_ERR_INVALID_ARG;
         ctx->wait_cap = (uint32_t)value;
@@ -660,16 +702,31 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
     if (!guard.ok) return GG_ERR_CUDA;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int32_t n_bins = do_hist ? a->qmax - a->qmin + 1 : 0;
+    if (n_seg > 0 && p == nullptr) {
+        st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p);
+        if (st != GG_OK) return st;
+    }
+    // The histograms start from zero.  When the call begins with the persistent bf16 moments sweep, that sweep
+    // clears them on its way (no memset between two launches); otherwise a memset does.
+    const size_t hist_bytes = do_hist ? sizeof(uint64_t) * (size_t)a->n_hist * (size_t)n_bins : 0;
+    int n_clusters = 0;
+    const int csize = (n_seg > 0 && a->param_mode == GG_PARAMS_FITTED && a->in_dtype == GG_BF16 &&
+                       (a->grad != nullptr || a->penalty != nullptr || do_hist) && !(p->max_len <= kSmallSegMax && n_seg >= 64))
+                          ? cluster_choice(ctx, p, ((a->grad != nullptr || a->penalty != nullptr) ? kGrad : 0) | (do_hist ? kHist : 0),
+                                           (gg_dtype)a->grad_dtype, a->grad != nullptr, &n_clusters)
+                          : 0;
+    const bool sweep_first = n_seg > 0 && a->param_mode == GG_PARAMS_FITTED && a->in_dtype == GG_BF16 && ctx->resident_mode == 0 &&
+                             csize == 0 &&
+                             (int64_t)p->n_tiles >= 16 * (int64_t)n_seg &&
+                             !(p->max_len <= kSmallSegMax && n_seg >= 64);
+    const bool clear_in_sweep = do_hist && !a->accumulate_hist && sweep_first && hist_bytes >= (1u << 20) &&
+                                reinterpret_cast<uintptr_t>(a->hist) % 16 == 0 && hist_bytes % 16 == 0;
     if (do_hist && !a->accumulate_hist) {
-        GG_CUDA(ctx, cudaMemsetAsync(a->hist, 0, sizeof(uint64_t) * (size_t)a->n_hist * (size_t)n_bins, cs));
+        if (!clear_in_sweep) GG_CUDA(ctx, cudaMemsetAsync(a->hist, 0, hist_bytes, cs));
         if (a->clamped_lo_hi)
             GG_CUDA(ctx, cudaMemsetAsync(a->clamped_lo_hi, 0, sizeof(uint64_t) * 2 * (size_t)a->n_hist, cs));
     }
     if (n_seg > 0) {
-        if (p == nullptr) {
-            st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p);
-            if (st != GG_OK) return st;
-        }
         const gg_dtype in_dt = (gg_dtype)a->in_dtype, g_dt = (gg_dtype)a->grad_dtype;
         const bool want_pg = a->grad != nullptr || a->penalty != nullptr;
         const int tail_flags = (want_pg ? kGrad : 0) | (do_hist ? kHist : 0);
@@ -734,11 +791,28 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             }
             ctx->launches += 1;
             beta_used = a->beta;
+        } else if (csize > 0) {
+            // one thread-block cluster per segment: the segment is staged in the cluster's shared memory and read from DRAM once
+            fa.sd_out = p->sd;
+            sa.beta = a->beta; sa.alpha = a->alpha; sa.seg_sd = p->sd;
+            sa.step = fa.step_from_alpha ? a->step_out : a->step;
+            ClusterArgs ca{};
+            ca.fit = fa;
+            ca.wait_cap = ctx->wait_cap;
+            ca.extra_tx = 16u * (uint32_t)ctx->expect_delta;
+            {
+                SweepTimer tm(ctx, &ctx->ev_tail, cs);
+                GG_CUDA(ctx, launch_cluster_bf16(tail_flags, g_dt, a->grad != nullptr, sa, ca, csize, n_clusters, cs));
+            }
+            ctx->launches += 1;
+            beta_used = a->beta;
         } else if (a->param_mode == GG_PARAMS_FITTED) {
             // sweep 1: moments; fit; sweep 2: gradient + histogram with the fresh parameters
             {
                 SweepTimer tm(ctx, &ctx->ev_first, cs);
+                if (clear_in_sweep) { sa.zero_ptr = reinterpret_cast<uint4 *>(a->hist); sa.zero_vecs = (int64_t)(hist_bytes / 16); }
                 GG_CUDA(ctx, launch_sweep(ctx, kMoments, in_dt, g_dt, false, sa, cs));
+                sa.zero_ptr = nullptr; sa.zero_vecs = 0;
             }
             fa.sd_out = p->sd;
             GG_CUDA(ctx, launch_fit(fa, cs));

@@ -65,6 +65,10 @@ struct StreamArgs {
     // standard deviation of every segment when the caller knows it (the fit of the same call wrote it), else null:
     // it places the count windows; without it the sweeps take the scale from a sample of each run
     const double *seg_sd;
+    // memory the moments sweep of a fused call clears on its way (the histograms of the sweep that follows), so
+    // that no separate memset sits between two launches: 16-byte vectors, or null
+    uint4 *zero_ptr;
+    int64_t zero_vecs;
 };
 
 struct FitArgs {
@@ -99,6 +103,19 @@ struct ResidentArgs {
 cudaError_t launch_resident_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
                                  const ResidentArgs &r, int grid, cudaStream_t st);
 cudaError_t resident_bf16_max_grid(int flags, gg_dtype grad_dtype, bool has_grad_out, int sm_count, int *max_grid);
+
+// The fitted pass with one thread-block cluster per segment, the segment staged in the cluster's shared memory
+// (bf16 input, segments up to cluster_size * cluster_tiles_per_cta() tiles, 16-byte aligned; gg_tail_bf16.cu).
+struct ClusterArgs {
+    FitArgs fit;
+    uint32_t wait_cap;       // polls after which the wait for the bulk copies gives up
+    uint32_t extra_tx;       // test hook: bytes the barrier expects beyond what is copied (the wait then runs out)
+};
+int cluster_tiles_per_cta();
+cudaError_t launch_cluster_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a, const ClusterArgs &c,
+                                int cluster_size, int n_clusters, cudaStream_t st);
+// clusters of this size that can be resident at once
+cudaError_t cluster_bf16_max_clusters(int flags, gg_dtype grad_dtype, bool has_grad_out, int cluster_size, int *max_clusters);
 
 cudaError_t launch_stream(int flags, gg_dtype in_dtype, gg_dtype grad_dtype, bool has_grad_out,
                           const StreamArgs &a, cudaStream_t st);

@@ -92,19 +92,32 @@ entropy_partial_kernel(const uint64_t *hist, int32_t n_bins, double *part)
     const int k0 = slice * per, k1 = min(n_bins, k0 + per);
     double acc = 0.0;
     unsigned long long tot = 0;
-    // (four independent loads per trip: most bins are empty, so the loop is bound by load latency; the order in
-    // which a thread adds its bins stays fixed)
-    for (int k = k0 + threadIdx.x; k < k1; k += 4 * kEntThreads) {
-        uint64_t c[4];
+    auto add = [&](uint64_t c) {
+        if (c != 0) {
+            const double cd = (double)c;
+            acc += cd * log2(cd);
+            tot += c;
+        }
+    };
+    // (most bins are empty, so the loop is bound by load latency: four independent 16-byte loads, two bins each,
+    // per trip when the slice allows; the order in which a thread adds its bins stays fixed)
+    if ((reinterpret_cast<uintptr_t>(row + k0) & 15u) == 0 && ((k1 - k0) & 1) == 0) {
+        const ulonglong2 *row2 = reinterpret_cast<const ulonglong2 *>(row + k0);
+        const int n2 = (k1 - k0) / 2;
+        for (int k = threadIdx.x; k < n2; k += 4 * kEntThreads) {
+            ulonglong2 c[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) c[u] = k + u * kEntThreads < k1 ? __ldg(row + k + u * kEntThreads) : 0ull;
+            for (int u = 0; u < 4; ++u) c[u] = k + u * kEntThreads < n2 ? __ldg(row2 + k + u * kEntThreads) : make_ulonglong2(0ull, 0ull);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (c[u] != 0) {
-                const double cd = (double)c[u];
-                acc += cd * log2(cd);
-                tot += c[u];
-            }
+            for (int u = 0; u < 4; ++u) { add(c[u].x); add(c[u].y); }
+        }
+    } else {
+        for (int k = k0 + threadIdx.x; k < k1; k += 4 * kEntThreads) {
+            uint64_t c[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) c[u] = k + u * kEntThreads < k1 ? __ldg(row + k + u * kEntThreads) : 0ull;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) add(c[u]);
         }
     }
     acc = warp_sum(acc);

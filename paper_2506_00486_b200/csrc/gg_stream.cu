@@ -560,6 +560,12 @@ __global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_s
     const uint32_t slot0 = (uint32_t)__cvta_generic_to_shared(&stage[0][tid]);
     constexpr uint32_t kStageBytes = sizeof(uint4) * kSweepThreads;
 
+    // this CTA's share of the memory to clear for the sweep that follows (plain stores, a few per thread)
+    if (a.zero_ptr != nullptr) {
+        const int64_t z0 = a.zero_vecs * blockIdx.x / gridDim.x, z1 = a.zero_vecs * (blockIdx.x + 1) / gridDim.x;
+        for (int64_t z = z0 + tid; z < z1; z += kSweepThreads) a.zero_ptr[z] = make_uint4(0u, 0u, 0u, 0u);
+    }
+
     for (int t = t_begin; t < t_end;) {
         // ---- one run: the tiles of this CTA's range that lie in segment s
         const int s = a.map.tile_seg[t];

@@ -28,6 +28,7 @@
 //     counts in a sentinel cell and is redone after its vector.
 // Input vectors reach each thread through a private ring of shared-memory slots filled by
 // asynchronous copies issued kDepth iterations ahead: bytes in flight cost no registers.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -65,13 +66,18 @@ struct Cold {
     int symbol_mode;           // layout of cnt: 1 = rows of symbols, 0 = cells of patterns
 };
 
+struct ClusterPart {
+    double s1, s2;
+    uint32_t bad;
+    float mn, mx;
+};
+
 struct Smem {
     // pattern mode: cell ((p * 2 + sign) * kRep + r) = magnitude pattern c_base + p, replica r; slot
     // p = kCntPat is the sentinel that swallows the counts of out-of-window elements.
     // symbol mode: word ((s + 1) * 32 + lane) = symbol s - kSymCells/2 counted by that lane; the rows
     // before and after the window (s = -1 and s = kSymCells) are the sentinels of the two tails.
     uint32_t cnt[kCntWords];
-    uint4 stage[kDepth][kThreads];   // per-thread ring of input vectors in flight
     float brep[128 * 32];            // row j: B[j] in every bank
     float2 A[256];                   // every exponent: value = A.x * A.y, A.y a power of two
     float B[128];
@@ -83,6 +89,13 @@ struct Smem {
     uint32_t clampc[2];
     Cold cold;
     int e_top;
+    // one-cluster-per-segment kernel: this CTA's moments of the current segment (two slots, used in turn: the other
+    // CTAs of the cluster read them) and the barrier its bulk copies complete on
+    ClusterPart cpart[2];
+    alignas(8) unsigned long long mbar;
+    // per-thread ring of input vectors in flight; the one-cluster-per-segment kernel keeps its share of the segment
+    // here and in the dynamic shared memory that follows the structure
+    alignas(128) uint4 stage[kDepth][kThreads];
 };
 
 // A[e] as one factor (with lambda's sign), NaN where that is not possible.  Static shared memory:
@@ -498,6 +511,32 @@ __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool acc
 // One contiguous run of n elements: scalar head up to the first 16-byte boundary of x, 128-bit
 // vector body fed through the asynchronous-copy ring, scalar tail.  If the gradient's address is
 // not 16-byte aligned at the same element the whole run is scalar.
+// One element taken by itself (the head and the tail of a run that do not fill a 16-byte vector).
+template <typename TG, int FLAGS, int MODE>
+__device__ __forceinline__ void scalar_elem(const uint16_t *x, TG *gout, int64_t idx, bool accumulate, const Lane &ln, Smem &sm, Acc &acc)
+{
+    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    const uint32_t h = (uint32_t)__ldg(x + idx);
+    Run r;
+    uint32_t anyc = 0;
+    float g = one_elem<FLAGS, MODE, 0>(h, ln, acc, r, anyc);
+    const bool grad_bad = GRAD && !(r.mp <= FLT_MAX);
+    if (grad_bad || (HIST && count_miss<MODE>(anyc))) g = fix_elem<FLAGS, MODE>(h << 16, g, grad_bad, ln, sm);
+    close_run<FLAGS>(make_uint4(h, 0u, 0u, 0u), 1, r, acc, sm);
+    if constexpr (GRAD) {
+        if (gout != nullptr) {
+            float v = g;
+            if constexpr (sizeof(TG) == 4) {
+                if (accumulate) v += gout[idx];
+                gout[idx] = v;
+            } else {
+                if (accumulate) v += __uint_as_float((uint32_t)gout[idx] << 16);
+                gout[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+            }
+        }
+    }
+}
+
 // L2 eviction hints of one run: vectors before `split` are copied with policy `first`, the others with `rest`.
 struct Hints {
     uint64_t first = 0, rest = 0;
@@ -517,7 +556,6 @@ template <typename TG, int FLAGS, int MODE, bool HINT = false>
 __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64_t n, bool accumulate,
                                               const Lane &ln, Smem &sm, Acc &acc, const Hints hints = Hints())
 {
-    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
     const int tid = threadIdx.x;
     int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
     head = min(head, n);
@@ -525,28 +563,8 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     const int64_t nvec = (n - head) / 8;
     const int64_t tail0 = head + nvec * 8;
 
-    for (int64_t i = tid; i < head + (n - tail0); i += kThreads) {
-        const int64_t idx = i < head ? i : tail0 + (i - head);
-        const uint32_t h = (uint32_t)__ldg(x + idx);
-        Run r;
-        uint32_t anyc = 0;
-        float g = one_elem<FLAGS, MODE, 0>(h, ln, acc, r, anyc);
-        const bool grad_bad = GRAD && !(r.mp <= FLT_MAX);
-        if (grad_bad || (HIST && count_miss<MODE>(anyc))) g = fix_elem<FLAGS, MODE>(h << 16, g, grad_bad, ln, sm);
-        close_run<FLAGS>(make_uint4(h, 0u, 0u, 0u), 1, r, acc, sm);
-        if constexpr (GRAD) {
-            if (gout != nullptr) {
-                float v = g;
-                if constexpr (sizeof(TG) == 4) {
-                    if (accumulate) v += gout[idx];
-                    gout[idx] = v;
-                } else {
-                    if (accumulate) v += __uint_as_float((uint32_t)gout[idx] << 16);
-                    gout[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-                }
-            }
-        }
-    }
+    for (int64_t i = tid; i < head + (n - tail0); i += kThreads)
+        scalar_elem<TG, FLAGS, MODE>(x, gout, i < head ? i : tail0 + (i - head), accumulate, ln, sm, acc);
 
     // (a CTA's run never exceeds device memory / grid size elements: 32-bit vector indices suffice)
     // Each thread owns slot [d][tid] of every stage d: it fills them with asynchronous 16-byte
@@ -623,13 +641,126 @@ __device__ __forceinline__ void init_cta(Smem &sm, CtaState &cs, bool hist)
     __syncthreads();
 }
 
+// Gradient tables and count layout of the segment a run lies in; returns the count mode of the run.  x, n: the
+// run (its first elements give the scale of the data when the caller does not know it).
+template <int FLAGS, bool COHERENT>
+__device__ __forceinline__ int setup_run(const StreamArgs &a, Smem &sm, CtaState &cs, int s, int64_t len, const uint16_t *x, int64_t n)
+{
+    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    const int tid = threadIdx.x;
+    Lane &ln = cs.ln;
+    int mode = kModePattern;
+    bool active = false;
+
+    if constexpr (GRAD) {
+        const double beta = param<COHERENT>(a.beta + s), alpha = param<COHERENT>(a.alpha + s);
+        const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
+        active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
+        // (every thread works the two constants out for itself: cheaper than a broadcast and its barrier)
+        const double b = beta - 1.0;
+        const double L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
+        if (tid == 0) {
+            sm.cold.b = b;
+            sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
+            sm.cold.active = active;
+            sm.cold.L = L;
+        }
+        if (tid < 256) {
+            const int k = tid;
+            float2 v = make_float2(0.0f, 1.0f);
+            if (active && k >= 1 && k <= 254) {
+                const double e0 = L + b * (double)(k - 127);
+                double ip = rint(e0);
+                const double f = exp2_short(e0 - ip);
+                ip = fmin(fmax(ip, -400.0), 400.0);
+                const int ii = (int)ip;
+                const int i1 = max(-100, min(100, ii));
+                const int i2 = max(-126, min(126, ii - i1));
+                v = make_float2((float)ldexp(lam < 0.0 ? -f : f, i1), __int_as_float((i2 + 127) << 23));
+            }
+            sm.A[k] = v;
+            // One factor serves an exponent if its power-of-two part is 1 (|L + b (e-127)| <= 100:
+            // the product with B then stays in the normal fp32 range).  Zero/subnormal (e = 0),
+            // inf/nan (e = 255) and the far exponents get the marker.  Without a gradient all is zero.
+            float one = 0.0f;
+            if (active) one = (k >= 1 && k <= 254 && v.y == 1.0f) ? v.x : __int_as_float(0x7FC00000);
+            s_a1[k] = one;
+        } else if (tid < 384) {
+            const int k = tid - 256;
+            sm.B[k] = active ? (float)exp2_short(b * sm.lg[k]) : 1.0f;
+        }
+        __syncthreads();
+        for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
+    }
+    if constexpr (HIST) {
+        const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
+        const float step = param<COHERENT>(a.step + s);
+        const float inv = (float)(1.0 / (double)step);
+        const bool same_key = cs.have_key && hid == cs.cur_hid && __float_as_uint(inv) == cs.cur_inv_bits;
+        // where the pattern-count window should sit: 16 binades below 2^5 standard deviations when
+        // the scale of the data is known, else where it is (same key) or from four binades below
+        // the step upwards (new key)
+        uint32_t want_base = sm.cold.c_base;
+        double sd = 0.0;
+        if (a.seg_sd != nullptr) {
+            sd = param<COHERENT>(a.seg_sd + s);
+        } else {
+            // Without parameters the scale of the data is taken from the first elements of the run (one
+            // per thread): it only decides how the counts are laid out, never what is counted.
+            const int m = (int)min(n, (int64_t)kThreads);
+            float ss = 0.0f;
+            for (int i = tid; i < m; i += kThreads) {
+                const float v = __uint_as_float((uint32_t)__ldg(x + i) << 16);
+                if (fabsf(v) <= 1e18f) ss = fmaf(v, v, ss);        // (inf, nan and values whose squares overflow are left out)
+            }
+            const double ws = warp_sum((double)ss);
+            __syncthreads();                                        // (the slots may still be read from the run before)
+            if ((tid & 31) == 0) sm.red[2][tid >> 5] = ws;
+            __syncthreads();
+            double tot = 0.0;
+            for (int w = 0; w < kWarps; ++w) tot += sm.red[2][w];
+            sd = m > 0 ? sqrt(tot / (double)m) : 0.0;
+        }
+        if (sd > 0.0) {
+            want_base = (uint32_t)(window_top_exponent(sd, 4) - (kCntBinades - 1)) << 7;
+            // symbol mode: the window's symbols are not clamped and reach 6.5 standard deviations
+            if (a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 && step > 0.0f &&
+                (double)(kSymCells / 2) * (double)step >= 6.5 * sd && inv < 3.0e38f)
+                mode = kModeSymbol;
+        } else if (!same_key) {
+            want_base = (uint32_t)(window_top_exponent((double)step, 11) - (kCntBinades - 1)) << 7;
+        }
+        const bool rebase = !same_key || mode != cs.cur_mode || (mode == kModePattern && want_base != sm.cold.c_base);
+        __syncthreads();
+        if (rebase) {
+            if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
+            cs.have_key = true;
+            cs.cur_hid = hid;
+            cs.cur_inv_bits = __float_as_uint(inv);
+            cs.cur_mode = mode;
+            if (tid == 0) {
+                sm.cold.inv = inv;
+                sm.cold.qmin = a.qmin;
+                sm.cold.qmax = a.qmax;
+                sm.cold.row = reinterpret_cast<unsigned long long *>(a.hist) +
+                              (int64_t)hid * ((int64_t)a.qmax - (int64_t)a.qmin + 1);
+                sm.cold.c_base = want_base;
+                sm.cold.symbol_mode = mode == kModeSymbol;
+            }
+        }
+        ln.cbase = want_base;
+        ln.inv = inv;
+    }
+    __syncthreads();
+    return mode;
+}
+
 // The tiles [t_begin, t_end) of one CTA, run by run (a run: the tiles of the range that lie in one segment):
 // gradient tables and count layout of the run's segment, then the stream, then the run's partial sums.
 template <typename TG, int FLAGS, bool COHERENT, bool HINT>
 __device__ __forceinline__ void tail_tiles(const StreamArgs &a, Smem &sm, CtaState &cs, int t_begin, int t_end, uint64_t policy)
 {
     constexpr bool MOM = (FLAGS & kMoments) != 0, GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
-    const int tid = threadIdx.x;
     const bool accumulate = GRAD && a.accumulate != 0;
     Lane &ln = cs.ln;
     for (int t = t_begin; t < t_end;) {
@@ -641,109 +772,7 @@ __device__ __forceinline__ void tail_tiles(const StreamArgs &a, Smem &sm, CtaSta
         const int64_t off = (int64_t)(t - t_first) * kTile;
         const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
         const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
-        int mode = kModePattern;
-        bool active = false;
-
-        if constexpr (GRAD) {
-            const double beta = param<COHERENT>(a.beta + s), alpha = param<COHERENT>(a.alpha + s);
-            const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
-            active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
-            // (every thread works the two constants out for itself: cheaper than a broadcast and its barrier)
-            const double b = beta - 1.0;
-            const double L = active ? log2(fabs(lam) * beta) - beta * log2(alpha) : 0.0;
-            if (tid == 0) {
-                sm.cold.b = b;
-                sm.cold.sign_flip = lam < 0.0 ? 0x80000000u : 0u;
-                sm.cold.active = active;
-                sm.cold.L = L;
-            }
-            if (tid < 256) {
-                const int k = tid;
-                float2 v = make_float2(0.0f, 1.0f);
-                if (active && k >= 1 && k <= 254) {
-                    const double e0 = L + b * (double)(k - 127);
-                    double ip = rint(e0);
-                    const double f = exp2_short(e0 - ip);
-                    ip = fmin(fmax(ip, -400.0), 400.0);
-                    const int ii = (int)ip;
-                    const int i1 = max(-100, min(100, ii));
-                    const int i2 = max(-126, min(126, ii - i1));
-                    v = make_float2((float)ldexp(lam < 0.0 ? -f : f, i1), __int_as_float((i2 + 127) << 23));
-                }
-                sm.A[k] = v;
-                // One factor serves an exponent if its power-of-two part is 1 (|L + b (e-127)| <= 100:
-                // the product with B then stays in the normal fp32 range).  Zero/subnormal (e = 0),
-                // inf/nan (e = 255) and the far exponents get the marker.  Without a gradient all is zero.
-                float one = 0.0f;
-                if (active) one = (k >= 1 && k <= 254 && v.y == 1.0f) ? v.x : __int_as_float(0x7FC00000);
-                s_a1[k] = one;
-            } else if (tid < 384) {
-                const int k = tid - 256;
-                sm.B[k] = active ? (float)exp2_short(b * sm.lg[k]) : 1.0f;
-            }
-            __syncthreads();
-            for (int i = tid; i < 128 * 32; i += kThreads) sm.brep[i] = sm.B[i >> 5];
-        }
-        if constexpr (HIST) {
-            const int hid = a.map.hist_id ? a.map.hist_id[s] : s;
-            const float step = param<COHERENT>(a.step + s);
-            const float inv = (float)(1.0 / (double)step);
-            const bool same_key = cs.have_key && hid == cs.cur_hid && __float_as_uint(inv) == cs.cur_inv_bits;
-            // where the pattern-count window should sit: 16 binades below 2^5 standard deviations when
-            // the scale of the data is known, else where it is (same key) or from four binades below
-            // the step upwards (new key)
-            uint32_t want_base = sm.cold.c_base;
-            double sd = 0.0;
-            if (a.seg_sd != nullptr) {
-                sd = param<COHERENT>(a.seg_sd + s);
-            } else {
-                // Without parameters the scale of the data is taken from the first elements of the run (one
-                // per thread): it only decides how the counts are laid out, never what is counted.
-                const int m = (int)min(n, (int64_t)kThreads);
-                float ss = 0.0f;
-                for (int i = tid; i < m; i += kThreads) {
-                    const float v = __uint_as_float((uint32_t)__ldg(x + i) << 16);
-                    if (fabsf(v) <= 1e18f) ss = fmaf(v, v, ss);        // (inf, nan and values whose squares overflow are left out)
-                }
-                const double ws = warp_sum((double)ss);
-                __syncthreads();                                        // (the slots may still be read from the run before)
-                if ((tid & 31) == 0) sm.red[2][tid >> 5] = ws;
-                __syncthreads();
-                double tot = 0.0;
-                for (int w = 0; w < kWarps; ++w) tot += sm.red[2][w];
-                sd = m > 0 ? sqrt(tot / (double)m) : 0.0;
-            }
-            if (sd > 0.0) {
-                want_base = (uint32_t)(window_top_exponent(sd, 4) - (kCntBinades - 1)) << 7;
-                // symbol mode: the window's symbols are not clamped and reach 6.5 standard deviations
-                if (a.qmin <= -(int)(kSymCells / 2) && a.qmax >= (int)(kSymCells / 2) - 1 && step > 0.0f &&
-                    (double)(kSymCells / 2) * (double)step >= 6.5 * sd && inv < 3.0e38f)
-                    mode = kModeSymbol;
-            } else if (!same_key) {
-                want_base = (uint32_t)(window_top_exponent((double)step, 11) - (kCntBinades - 1)) << 7;
-            }
-            const bool rebase = !same_key || mode != cs.cur_mode || (mode == kModePattern && want_base != sm.cold.c_base);
-            __syncthreads();
-            if (rebase) {
-                if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
-                cs.have_key = true;
-                cs.cur_hid = hid;
-                cs.cur_inv_bits = __float_as_uint(inv);
-                cs.cur_mode = mode;
-                if (tid == 0) {
-                    sm.cold.inv = inv;
-                    sm.cold.qmin = a.qmin;
-                    sm.cold.qmax = a.qmax;
-                    sm.cold.row = reinterpret_cast<unsigned long long *>(a.hist) +
-                                  (int64_t)hid * ((int64_t)a.qmax - (int64_t)a.qmin + 1);
-                    sm.cold.c_base = want_base;
-                    sm.cold.symbol_mode = mode == kModeSymbol;
-                }
-            }
-            ln.cbase = want_base;
-            ln.inv = inv;
-        }
-        __syncthreads();
+        const int mode = setup_run<FLAGS, COHERENT>(a, sm, cs, s, len, x, n);
 
         // ---- stream the run
         TG *gout = nullptr;
@@ -770,7 +799,7 @@ template <typename TG, int FLAGS>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_bf16_kernel(const StreamArgs a)
 {
     constexpr bool HIST = (FLAGS & kHist) != 0;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
     CtaState cs;
     init_cta(sm, cs, HIST);
@@ -890,7 +919,7 @@ template <typename TG, int FLAGS>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) resident_bf16_kernel(const StreamArgs a, const ResidentArgs r)
 {
     constexpr bool HIST = (FLAGS & kHist) != 0;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
     __shared__ int sh_ok;
     const int n_stream = (int)gridDim.x - 1;
@@ -934,6 +963,171 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) resident_bf16_kernel(con
     if (late1 > late0) tail_tiles<TG, FLAGS, true, true>(a, sm, cs, late0, late1, drop);
     if constexpr (HIST) {
         if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// The fitted pass for segments of tens of kilobytes to two megabytes with ONE read of x from DRAM: a thread-block
+// cluster per segment, the segment staged in the shared memory of the cluster's CTAs.
+//
+// CTA r of a cluster of C takes the r-th share of the segment's tiles (at most kClusterTiles tiles) and copies it
+// into its shared memory with bulk asynchronous copies that complete on an mbarrier.  Moments come from shared
+// memory; every CTA leaves its sums in a slot of its own shared memory, the cluster synchronises (the hardware
+// barrier of the cluster: its CTAs are scheduled together), and the first warp of every CTA adds the C slots in
+// rank order through distributed shared memory and inverts the moment ratio: every CTA ends with the same bits and
+// nothing else is exchanged.  Gradient tables, gradient, penalty partial and counts then come from the staged copy.
+// Clusters are independent of one another, so while one waits for its barrier or works on a fit the others keep
+// DRAM busy.  The wait for the bulk copies is bounded; if it runs out the CTA stops touching data, keeps taking part
+// in the cluster barriers and marks its segments GG_FLAG_TIMEOUT at the end.
+constexpr int kClusterTiles = 4;                                     // tiles of a segment one CTA can stage (128 KB)
+constexpr size_t kClusterSmem = sizeof(Smem) - sizeof(uint4) * kDepth * kThreads + (size_t)kClusterTiles * kTile * 2;
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t cap)
+{
+    for (uint32_t it = 0; it < cap; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+template <typename TG, int FLAGS>
+__global__ void __launch_bounds__(kThreads, 1) cluster_bf16_kernel(const StreamArgs a, const ClusterArgs c)
+{
+    namespace cg = cooperative_groups;
+    constexpr bool GRAD = (FLAGS & kGrad) != 0, HIST = (FLAGS & kHist) != 0;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int cid = (int)blockIdx.x / C, n_clusters = (int)gridDim.x / C;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    CtaState cs;
+    init_cta(sm, cs, HIST);
+    const uint4 *data = &sm.stage[0][0];
+    const uint32_t data_addr = (uint32_t)__cvta_generic_to_shared(data), bar = (uint32_t)__cvta_generic_to_shared(&sm.mbar);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool accumulate = GRAD && a.accumulate != 0;
+    uint32_t parity = 0;
+    int s_fail = -1;                // first segment whose copies did not arrive in time
+    uint32_t fail_parity = 0;
+    int it = 0;
+    for (int s = cid; s < a.map.n_seg; s += n_clusters, ++it) {
+        // ---- this CTA's share of the segment
+        const int64_t len = a.map.seg_len[s];
+        const int t0 = a.map.tile_prefix[s], T = a.map.tile_prefix[s + 1] - t0;
+        const int t_lo = t0 + (int)((int64_t)T * rank / C), t_hi = t0 + (int)((int64_t)T * (rank + 1) / C);
+        const int64_t off = (int64_t)(t_lo - t0) * kTile;
+        const int n = t_hi > t_lo && s_fail < 0 ? (int)(min(len, (int64_t)(t_hi - t0) * kTile) - off) : 0;
+        const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
+        const int nvec = n / 8;
+
+        // ---- stage it: bulk copies of up to one tile each, all completing on the one barrier
+        bool ok = true;
+        if (nvec > 0) {
+            if (tid == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the reads of the segment before are done
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)nvec * 16u + c.extra_tx) : "memory");
+                for (int v0 = 0; v0 < nvec; v0 += kTile / 8) {
+                    const uint32_t bytes = (uint32_t)min(nvec - v0, kTile / 8) * 16u;
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                                     data_addr + (uint32_t)v0 * 16u),
+                                 "l"(reinterpret_cast<const uint4 *>(x) + v0), "r"(bytes), "r"(bar)
+                                 : "memory");
+                }
+            }
+            ok = mbar_wait(bar, parity, c.wait_cap);
+            if (!ok) ok = mbar_wait(bar, parity, c.wait_cap);      // once more before giving up
+            if (ok) parity ^= 1u;
+        }
+        if (__syncthreads_or(!ok)) {
+            // (no further copy is issued by this CTA; the one in flight is waited for again before the CTA leaves)
+            if (s_fail < 0) { s_fail = s; fail_parity = parity; }
+            ok = false;
+        }
+
+        // ---- moments of the share, from shared memory
+        Acc acc;
+        if (ok) {
+            for (int v = tid; v < nvec; v += kThreads) process_vec<float, kMoments, kModePattern>(data[v], nullptr, false, false, cs.ln, sm, acc);
+            for (int i = nvec * 8 + tid; i < n; i += kThreads) scalar_elem<float, kMoments, kModePattern>(x, nullptr, i, false, cs.ln, sm, acc);
+        }
+        {
+            const double w1 = warp_sum(acc.s1), w2 = warp_sum(acc.s2);
+            const uint32_t wb = __reduce_add_sync(0xFFFFFFFFu, acc.bad);
+            float wmin = fminf(acc.xmin, fminf(__low2float(acc.mn2), __high2float(acc.mn2)));
+            float wmax = fmaxf(acc.xmax, fmaxf(__low2float(acc.mx2), __high2float(acc.mx2)));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                wmin = fminf(wmin, __shfl_xor_sync(0xFFFFFFFFu, wmin, o));
+                wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+            }
+            if (lane == 0) { sm.red[0][warp] = w1; sm.red[1][warp] = w2; sm.bad[warp] = wb; sm.mn[warp] = wmin; sm.mx[warp] = wmax; }
+            __syncthreads();
+            if (tid == 0) {
+                ClusterPart p{0.0, 0.0, 0u, INFINITY, -INFINITY};
+                for (int w = 0; w < kWarps; ++w) {
+                    p.s1 += sm.red[0][w]; p.s2 += sm.red[1][w]; p.bad += sm.bad[w];
+                    p.mn = fminf(p.mn, sm.mn[w]); p.mx = fmaxf(p.mx, sm.mx[w]);
+                }
+                sm.cpart[it & 1] = p;
+            }
+        }
+        cluster.sync();
+
+        // ---- the fit, by the first warp of every CTA: the C slots in rank order, the same bits everywhere
+        if (warp == 0) {
+            double s1 = 0.0, s2 = 0.0;
+            uint32_t bad = 0;
+            float xmin = INFINITY, xmax = -INFINITY;
+            for (int r = 0; r < C; ++r) {
+                const ClusterPart *p = cluster.map_shared_rank(&sm.cpart[it & 1], r);
+                s1 += p->s1; s2 += p->s2; bad += p->bad;
+                xmin = fminf(xmin, p->mn); xmax = fmaxf(xmax, p->mx);
+            }
+            fit_finish(c.fit, s, lane, s1, s2, bad, xmin, xmax);      // (every CTA writes the same values to the outputs)
+        }
+        __syncthreads();
+
+        // ---- gradient tables, then gradient, penalty partial and counts from the staged copy
+        if (ok && n > 0) {
+            const int mode = setup_run<FLAGS, false>(a, sm, cs, s, len, x, n);
+            TG *gout = nullptr;
+            if constexpr (GRAD) {
+                if (a.map.grad_ptr != nullptr) gout = reinterpret_cast<TG *>(a.map.grad_ptr[s]) + off;
+            }
+            TG *gv = gout != nullptr ? gout + (int64_t)tid * 8 : nullptr;
+            const bool wide = (reinterpret_cast<uintptr_t>(gv) & 31u) == 0;
+            Acc acc2;
+            auto second = [&](auto mode_tag) {
+                constexpr int MODE = decltype(mode_tag)::value;
+                for (int v = tid; v < nvec; v += kThreads)
+                    process_vec<TG, FLAGS, MODE>(data[v], gout != nullptr ? gout + (int64_t)v * 8 : nullptr, accumulate, wide, cs.ln, sm, acc2);
+                for (int i = nvec * 8 + tid; i < n; i += kThreads) scalar_elem<TG, FLAGS, MODE>(x, gout, i, accumulate, cs.ln, sm, acc2);
+            };
+            if (HIST && mode == kModeSymbol) second(std::integral_constant<int, kModeSymbol>());
+            else second(std::integral_constant<int, kModePattern>());
+            if constexpr (GRAD) reduce_partials<FLAGS>(a.part, t_lo, t_hi, acc2, sm);
+            else __syncthreads();
+        } else if (GRAD && t_hi > t_lo) {
+            for (int t = t_lo + tid; t < t_hi; t += kThreads) a.part.pen[t] = 0.0;
+        }
+    }
+    if constexpr (HIST) {
+        if (cs.have_key) flush_counts(sm, a.clamped, cs.cur_hid);
+    }
+    cluster.sync();       // nobody leaves while another CTA may still read its slots
+    if (s_fail >= 0) {
+        // (the copies that were late must not land in memory this CTA has given up)
+        mbar_wait(bar, fail_parity, c.wait_cap < (1u << 16) ? c.wait_cap * 64u : (1u << 22));
+        if (c.fit.flags != nullptr && tid == 0)
+            for (int s = s_fail; s < a.map.n_seg; s += n_clusters) atomicOr(c.fit.flags + s, GG_FLAG_TIMEOUT);
     }
 }
 
@@ -992,6 +1186,47 @@ cudaError_t resident_typed(int flags, const StreamArgs &a, const ResidentArgs &r
     }
 }
 
+template <typename TG, int FLAGS>
+cudaError_t cluster_one(const StreamArgs &a, const ClusterArgs &c, int cluster_size, int n_clusters, int *max_clusters, cudaStream_t st)
+{
+    auto kern = cluster_bf16_kernel<TG, FLAGS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterSmem);
+    if (e != cudaSuccess) return e;
+    if (cluster_size > 8) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kClusterSmem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_clusters != nullptr) {
+        cfg.gridDim = dim3((unsigned)cluster_size);
+        return cudaOccupancyMaxActiveClusters(max_clusters, kern, &cfg);
+    }
+    cfg.gridDim = dim3((unsigned)(cluster_size * n_clusters));
+    return cudaLaunchKernelEx(&cfg, kern, a, c);
+}
+
+template <typename TG>
+cudaError_t cluster_typed(int flags, const StreamArgs &a, const ClusterArgs &c, int cluster_size, int n_clusters, int *max_clusters,
+                          cudaStream_t st)
+{
+    switch (flags) {
+    case kGrad: return cluster_one<TG, kGrad>(a, c, cluster_size, n_clusters, max_clusters, st);
+    case kHist: return cluster_one<TG, kHist>(a, c, cluster_size, n_clusters, max_clusters, st);
+    case kGrad | kHist: return cluster_one<TG, kGrad | kHist>(a, c, cluster_size, n_clusters, max_clusters, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_tail_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a,
@@ -1017,5 +1252,23 @@ cudaError_t resident_bf16_max_grid(int flags, gg_dtype grad_dtype, bool has_grad
     if (has_grad_out && grad_dtype == GG_BF16) return resident_typed<uint16_t>(flags, a, r, sm_count, max_grid, nullptr);
     return resident_typed<float>(flags, a, r, sm_count, max_grid, nullptr);
 }
+
+cudaError_t launch_cluster_bf16(int flags, gg_dtype grad_dtype, bool has_grad_out, const StreamArgs &a, const ClusterArgs &c,
+                                int cluster_size, int n_clusters, cudaStream_t st)
+{
+    if (n_clusters <= 0) return cudaSuccess;
+    if (has_grad_out && grad_dtype == GG_BF16) return cluster_typed<uint16_t>(flags, a, c, cluster_size, n_clusters, nullptr, st);
+    return cluster_typed<float>(flags, a, c, cluster_size, n_clusters, nullptr, st);
+}
+
+cudaError_t cluster_bf16_max_clusters(int flags, gg_dtype grad_dtype, bool has_grad_out, int cluster_size, int *max_clusters)
+{
+    StreamArgs a{};
+    ClusterArgs c{};
+    if (has_grad_out && grad_dtype == GG_BF16) return cluster_typed<uint16_t>(flags, a, c, cluster_size, 0, max_clusters, nullptr);
+    return cluster_typed<float>(flags, a, c, cluster_size, 0, max_clusters, nullptr);
+}
+
+int cluster_tiles_per_cta() { return kClusterTiles; }
 
 }  // namespace gg
