@@ -41,6 +41,13 @@ __device__ __forceinline__ Block4 philox4x32_10(uint32_t c0, uint32_t c1, uint32
 
 __device__ __forceinline__ double u01(uint32_t r) { return ((double)r + 0.5) * (1.0 / 4294967296.0); }
 
+__device__ __forceinline__ float rcp_approx_f(float v)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+
 // Per-segment constants of the sampler.
 struct GammaConst {
     double beta, alpha;
@@ -97,6 +104,92 @@ __device__ __forceinline__ double gg_from_gamma(const GammaConst &k, uint32_t k0
     return (r.w0 & 0x80000000u) ? -x : x;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// bf16 output: attempt 0 in fp32 with running error bounds.
+//
+// A bf16 value keeps 8 significant bits, so the variate is needed to about 1e-3 relative: almost always an fp32
+// evaluation of the same formulas lands in the same bf16 cell and on the same side of the acceptance test as the
+// fp64 one.  The fp32 path therefore carries a bound on its own error (the documented bounds of logf, expf, cospif,
+// with a factor of two to spare, and the roundings of the uniforms to 24 bits) and gives a result only when
+//   * the acceptance test is decided with that bound to spare on either side, and
+//   * the fp32 variate is further from the midpoint between two bf16 values than the bound (and is a normal number).
+// Otherwise (about one element in a hundred) the element goes to the fp64 path from attempt 0, which is the
+// definition.  What the fp32 path returns is therefore bit for bit what the fp64 path would.
+enum : int { kFastAccept = 0, kFastReject = 1, kFastUnsure = 2 };
+
+struct FastConst {
+    float c, d, ln_d, a, beta, alpha;
+    bool boost;        // a < 1: the variate is multiplied by u'^(1/a)
+    bool usable;       // the constants are in a range where the bounds below hold
+};
+
+__device__ __forceinline__ FastConst fast_const(const GammaConst &k)
+{
+    FastConst f;
+    f.c = (float)k.c; f.d = (float)k.d; f.ln_d = (float)k.ln_d; f.a = (float)k.a; f.beta = (float)k.beta; f.alpha = (float)k.alpha;
+    f.boost = k.a < 1.0;
+    // shapes between 0.1 and 8 and scales that are normal fp32 numbers: d <= 10, a <= 10, the exponent below stays
+    // within the range where expf keeps its relative accuracy
+    f.usable = k.beta >= 0.1 && k.beta <= 8.0 && k.alpha >= 1e-30 && k.alpha <= 1e30;
+    return f;
+}
+
+// uniform (r + 1/2) 2^-32 to fp32: relative error below 1.2e-7 (the conversion of r and the addition)
+__device__ __forceinline__ float u01f(uint32_t r) { return fmaf((float)r, 2.3283064365386963e-10f, 1.1641532182693481e-10f); }
+
+// Attempt 0 of element (i1, i0) in fp32.  kFastAccept: *bits holds the bf16 pattern of the variate.
+__device__ __forceinline__ int fast_attempt0(const FastConst &f, const Block4 &r, const Block4 &aux, uint16_t *bits)
+{
+    // ---- Box-Muller normal z with its error bound ez
+    const float l0 = logf(u01f(r.w0));                       // <= 0; error 1.2e-7 (1 + |l0|)
+    if (!(l0 < -1e-3f)) return kFastUnsure;                  // radius near zero: its relative error is unbounded here
+    const float R = sqrtf(-2.0f * l0);
+    // cos(2 pi u1) from the angle folded into the first quadrant in integers, so that the fp32 angle is exact to 1e-7 of pi/2
+    const uint32_t quad = r.w1 >> 30;
+    uint32_t frac = r.w1 & 0x3FFFFFFFu;
+    if (quad & 1u) frac = 0x3FFFFFFFu - frac;
+    float cs = cospif(fmaf((float)frac, 4.656612873077393e-10f, 2.3283064365386963e-10f));      // cos(pi/2 * (frac + 1/2) 2^-30)
+    if ((quad + 1u) & 2u) cs = -cs;
+    const float z = R * cs;
+    const float ez = R * fmaf(6e-8f, rcp_approx_f(-l0), 5e-7f);
+    // ---- Marsaglia-Tsang: w = 1 + c z, v = w^3, test ln u < z^2/2 + d (1 - v + ln v)
+    const float w = fmaf(f.c, z, 1.0f);
+    const float ew = fmaf(f.c, ez, 4e-7f);
+    if (!(w > 8.0f * ew)) return kFastUnsure;                // w <= 0 rejects, but only the fp64 path may say so this close
+    const float rw = rcp_approx_f(w);
+    const float lw = logf(w);
+    const float elw = fmaf(ew * 1.1f, rw, 1e-6f);            // (ew / w <= 1/8: the second-order term is within the 1.1)
+    const float v = w * w * w;
+    const float ev = v * fmaf(3.5f * ew, rw, 2e-7f);
+    const float rhs = fmaf(0.5f * z, z, f.d * (1.0f - v + 3.0f * lw));
+    // errors of z^2/2, of d (1 - v + 3 ln w), of the roundings of the sum (by its magnitude) and of ln u (3e-6)
+    const float mag = fmaf(0.5f * z, z, f.d * (1.0f + v + 3.0f * fabsf(lw)));
+    const float erhs = fmaf(fabsf(z), ez, fmaf(f.d, fmaf(3.0f, elw, ev), fmaf(2.4e-7f, mag, 5e-6f)));
+    const float lu = logf(u01f(r.w2));
+    if (lu - erhs > rhs) return kFastReject;
+    if (!(lu + erhs < rhs)) return kFastUnsure;
+    // ---- the variate alpha G^(1/beta), G = d v (times u'^(1/a) for a < 1), in the log domain
+    float lg = fmaf(3.0f, lw, f.ln_d);
+    float elg = fmaf(3.0f, elw, 3e-7f);
+    if (f.boost) {
+        const float lb = logf(u01f(aux.w1));
+        lg = fmaf(f.beta, lb, lg);
+        elg += f.beta * fmaf(2.5e-7f, -lb, 2.5e-7f);
+    }
+    elg = fmaf(1.2e-7f, fabsf(lg), elg);
+    const float arg = lg * f.a;
+    const float x = f.alpha * expf(arg);
+    const float E = fmaf(f.a, elg, fmaf(1.2e-7f, fabsf(arg), 4e-7f));      // relative error bound of x
+    const uint32_t xb = __float_as_uint(x);
+    const uint32_t ex = xb >> 23;
+    if (ex < 16u || ex > 250u) return kFastUnsure;                          // subnormal, zero, huge: the fp64 path rounds those
+    const int low = (int)(xb & 0xFFFFu) - 0x8000;
+    const float reach = fmaf(E, 33554432.0f, 2.0f);                         // the bound in fp32 ulps, twice over
+    if (fabsf((float)low) <= reach) return kFastUnsure;
+    *bits = (uint16_t)(((xb + 0x8000u) >> 16) | ((aux.w0 >> 16) & 0x8000u));
+    return kFastAccept;
+}
+
 // fp64 -> bf16, round to nearest even in one step: truncate to fp32, fold everything that was
 // dropped into the last fp32 bit (round to odd), then round the 16 spare bits away.
 __device__ __forceinline__ uint16_t double_to_bf16(double x)
@@ -131,6 +224,7 @@ sample_kernel(const TileMap map, const double *beta, const double *alpha, uint32
     const int n = (int)min((int64_t)kTile, len - off);
     T *out = reinterpret_cast<T *>(const_cast<void *>(map.seg_ptr[s])) + off;
     const GammaConst gk = gamma_const(beta[s], alpha[s]);
+    const FastConst fk = fast_const(gk);
     const uint32_t tensor = tensor_id0 + (uint32_t)s;
     if (threadIdx.x == 0) n_queued = 0;
     __syncthreads();
@@ -148,22 +242,41 @@ sample_kernel(const TileMap map, const double *beta, const double *alpha, uint32
         worst = max(worst, accepted ? tt + 1u : kMaxAttempts + 1u);
         store_variate<T>(out + i, accepted ? gg_from_gamma(gk, k0, k1, tensor, i0, i1, ln_g) : 0.0);
     };
+    // (queue entries: the element in the low 16 bits, the attempt to start from above them)
+    auto later = [&](int i, uint32_t t0) {
+        const int q = atomicAdd(&n_queued, 1);
+        if (q < kQueue) queue[q] = i | (int)(t0 << 16);
+        else finish(i, t0);                            // (queue full: finish it here)
+    };
     for (int i = threadIdx.x; i < n; i += kThreads) {
         const uint64_t index = (uint64_t)(off + i);
         const uint32_t i0 = (uint32_t)index, i1 = (uint32_t)(index >> 32);
+        if constexpr (sizeof(T) == 2) {
+            if (fk.usable) {
+                const Block4 r = philox4x32_10(i0, i1, 0u, tensor, k0, k1);
+                const Block4 aux = philox4x32_10(i0, i1, 0xFFFFFFFFu, tensor, k0, k1);
+                uint16_t bits;
+                const int verdict = fast_attempt0(fk, r, aux, &bits);
+                if (verdict == kFastAccept) {
+                    worst = max(worst, 1u);
+                    out[i] = bits;
+                } else {
+                    later(i, verdict == kFastReject ? 1u : 0u);
+                }
+                continue;
+            }
+        }
         double ln_g;
         if (gamma_attempt(gk, k0, k1, tensor, i0, i1, 0u, ln_g)) {
             worst = max(worst, 1u);
             store_variate<T>(out + i, gg_from_gamma(gk, k0, k1, tensor, i0, i1, ln_g));
         } else {
-            const int q = atomicAdd(&n_queued, 1);
-            if (q < kQueue) queue[q] = i;
-            else finish(i, 1u);                        // (queue full: finish it here)
+            later(i, 1u);
         }
     }
     __syncthreads();
     const int nq = min(n_queued, kQueue);
-    for (int q = threadIdx.x; q < nq; q += kThreads) finish(queue[q], 1u);
+    for (int q = threadIdx.x; q < nq; q += kThreads) finish(queue[q] & 0xFFFF, (uint32_t)queue[q] >> 16);
     if (max_attempts != nullptr) {
         worst = __reduce_max_sync(0xFFFFFFFFu, worst);
         if ((threadIdx.x & 31) == 0 && worst != 0) atomicMax(&max_attempts[s], worst);

@@ -138,6 +138,23 @@ def test_config2_qwen_initialisation_full_size(ctx):
         assert_rel(fit["alpha"][s].item(), a, REL_FIT, "alpha")
 
 
+def test_sampled_bf16_values_equal_the_oracle_over_millions_of_elements(ctx):
+    """bf16 output takes attempt 0 in fp32 with error bounds and hands every doubtful element to the fp64 path, so
+    its values must be the oracle's bit for bit: four shapes (gamma shape above and below 1), 3 M elements each."""
+    n = 3_000_000
+    betas = [0.3, 0.8, 1.0, 2.5]
+    alphas = [gg_synth.alpha_for_std(0.02, b) for b in betas]
+    outs = [torch.empty(n, dtype=torch.bfloat16, device="cuda:0") for _ in betas]
+    att = ctx.gg_sample(outs, betas, alphas, seed=0xABCDEF0123, tensor_id0=7)
+    torch.cuda.synchronize()
+    for s, (b, a) in enumerate(zip(betas, alphas)):
+        ref, ratt = o.sample(b, a, 0xABCDEF0123, 7 + s, n, want_attempts=True)
+        assert att[s].item() == int(ratt.max())
+        refb = o.round_to_bf16_bits(ref).astype(np.int64)
+        got = outs[s].cpu().view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+        assert np.array_equal(refb, got), (b, int((refb != got).sum()))
+
+
 def test_one_segment_longer_than_2_to_31_elements(ctx):
     """A single bf16 segment of 2^31 + 12345 elements (64-bit offsets in both sweeps): 2048 copies of a 2^20-element
     block and a ragged rest, so that the exact results follow from the oracle's results on the block and the
