@@ -20,8 +20,12 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
  *    enqueue work; they do not wait for the device.  Exception: the first call that sees a new
  *    segment layout (addresses, lengths, dtype, histogram ids) allocates and uploads a small
- *    plan with blocking calls; make that first call outside stream capture.  A context serves
- *    one stream at a time.
+ *    plan with blocking calls; make that first call outside stream capture.  A context keeps the
+ *    plans of the 64 layouts used last: a call that brings in a 65th frees the oldest plan after
+ *    waiting for the work last enqueued with it (an event; the whole device if that work was
+ *    captured in a graph), and a call that needs more histogram or channel scratch than any
+ *    before it reallocates that scratch after waiting for the device.  All of these belong outside
+ *    stream capture too.  A context serves one stream at a time.
  *  - A segment is a contiguous run of `len` elements.  Pointers need only element alignment;
  *    16-byte aligned segments take the vectorised path.
  *  - Per-segment conditions are reported in `flags` (GG_FLAG_*), never as an error status.
@@ -298,6 +302,13 @@ gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double
                                       B200 (a cluster works through load, fit and tables one after the other), which is
                                       why it is off unless asked for. */
 gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value);
+
+/* Bounds-checking build (no counterpart in the paper: a debugging aid that stands in for a memory checker).  A
+ * library built with -DGG_BOUNDS (paper_2506_00486_b200/build.py --bounds) tests the index of every checked global
+ * load and store of its streaming kernels against the extent of the segment or buffer it belongs to, counts the
+ * ones that would have left it and skips them; nothing traps.  Returns the number of such accesses since the library
+ * was loaded (after waiting for the device), or -1 from a normal build, which has no checks. */
+int64_t gg_debug_bounds_violations(void);
 
 /* The same pass for data that lives in HOST memory: every pointer of `args` that gg_fused documents
  * as device memory (segment data, fit outputs, gradient segments, step, histogram, entropy, ...) is

@@ -11,7 +11,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libgg_b200.so")
+# GG_B200_LIB selects another build of the same library (the bounds-checking one of build.py --bounds)
+_LIB_PATH = os.environ.get("GG_B200_LIB") or os.path.join(_HERE, "libgg_b200.so")
 
 GG_F32, GG_BF16 = 0, 1
 GG_SUM, GG_MEAN = 0, 1
@@ -100,6 +101,7 @@ def lib():
         L.gg_timing_enable.argtypes = [_P, ctypes.c_int]
         L.gg_timing_read.argtypes = [_P, ctypes.POINTER(d), ctypes.POINTER(i64), ctypes.POINTER(d),
                                      ctypes.POINTER(i64)]
+        L.gg_debug_bounds_violations.restype = i64
         L.gg_test_hook.argtypes = [_P, i32, i64]
         L.gg_test_hook.restype = ctypes.c_int
         L.gg_fit_noalloc.argtypes = [ctypes.c_int, _P, i64, ctypes.c_int, _P, _P, _P, _P, _P, _P, _P]
@@ -245,7 +247,14 @@ def _stream_ptr(device):
 class Context:
     """One gg_ctx on one CUDA device.  Use from one stream at a time."""
 
-    def __init__(self, device=0):
+    GUARD_BYTES, GUARD_FILL = 256, 0xA5
+
+    def __init__(self, device=0, guard=False):
+        """guard=True puts 256 bytes of a fill pattern before and after every output tensor this object allocates
+        (fit results, penalties, histograms, entropies, counters); check_guards() then tells whether a kernel
+        wrote outside an output."""
+        self._guard = bool(guard)
+        self._guarded = []
         self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
         if self.device.type != "cuda":
             raise RuntimeError("the GG library runs on CUDA devices only")
@@ -284,8 +293,33 @@ class Context:
         """Knobs of the one-launch fitted pass (HOOK_*), for tests and measurements."""
         self._check(lib().gg_test_hook(self._h, int(what), int(value)))
 
-    def _new(self, n, dtype):
-        return torch.empty(n, dtype=dtype, device=self.device)
+    def _new(self, n, dtype, zero=False):
+        shape = (n,) if isinstance(n, int) else tuple(n)
+        if not self._guard:
+            return (torch.zeros if zero else torch.empty)(shape, dtype=dtype, device=self.device)
+        import weakref
+        nbytes = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        pad = self.GUARD_BYTES
+        raw = torch.full((nbytes + 2 * pad,), self.GUARD_FILL, dtype=torch.uint8, device=self.device)
+        body = raw[pad:pad + nbytes]
+        if zero:
+            body.zero_()
+        out = body.view(dtype).view(shape)
+        self._guarded.append((weakref.ref(out), raw, nbytes))
+        return out
+
+    def check_guards(self):
+        """Raises if any byte around a live guarded output has changed (after waiting for the device)."""
+        torch.cuda.synchronize(self.device)
+        pad, keep = self.GUARD_BYTES, []
+        for ref, raw, nbytes in self._guarded:
+            if ref() is None:
+                continue
+            keep.append((ref, raw, nbytes))
+            ok = bool((raw[:pad] == self.GUARD_FILL).all()) and bool((raw[pad + nbytes:] == self.GUARD_FILL).all())
+            if not ok:
+                raise AssertionError(f"a kernel wrote outside an output of {nbytes} bytes")
+        self._guarded = keep
 
     # ------------------------------------------------------------------ gg_fit
     def gg_fit(self, segs):
@@ -323,11 +357,11 @@ class Context:
         n_hist = n if n_hist is None else int(n_hist)
         nb = qmax - qmin + 1
         if hist is None:
-            hist = torch.empty((n_hist, nb), dtype=torch.int64, device=self.device)
+            hist = self._new((n_hist, nb), torch.int64)
             if accumulate:
                 hist.zero_()
         ent = self._new(n_hist, torch.float64)
-        clamped = torch.zeros((n_hist, 2), dtype=torch.int64, device=self.device)
+        clamped = self._new((n_hist, 2), torch.int64, zero=True)
         hid = None if hist_id is None else np.ascontiguousarray(hist_id, dtype=np.int32)
         self._check(lib().gg_rate_hist(
             self._h, segs.ptr, n, segs.code, _ptr(step), None if hid is None else hid.ctypes.data,
@@ -380,10 +414,10 @@ class Context:
             n_hist = n if n_hist is None else int(n_hist)
             nb = qmax - qmin + 1
             if hist is None:
-                hist = torch.zeros((n_hist, nb), dtype=torch.int64, device=self.device)
+                hist = self._new((n_hist, nb), torch.int64, zero=True)
             out["hist"] = hist
             out["entropy_bits"] = self._new(n_hist, torch.float64)
-            out["clamped"] = torch.zeros((n_hist, 2), dtype=torch.int64, device=self.device)
+            out["clamped"] = self._new((n_hist, 2), torch.int64, zero=True)
             if step is not None:
                 a.step_mode, a.step = GG_STEP_GIVEN, _ptr(step)
                 out["step"] = step
@@ -438,10 +472,10 @@ class Context:
         if step is not None:
             nb = qmax - qmin + 1
             if hist is None:
-                hist = torch.zeros(nb, dtype=torch.int64, device=self.device)
+                hist = self._new(nb, torch.int64, zero=True)
             out["hist"] = hist
             out["entropy_bits"] = self._new(1, torch.float64)
-            out["clamped"] = torch.zeros(2, dtype=torch.int64, device=self.device)
+            out["clamped"] = self._new(2, torch.int64, zero=True)
             a.step, a.qmin, a.qmax = float(step), int(qmin), int(qmax)
             a.hist, a.accumulate_hist = _ptr(hist), int(bool(accumulate_hist))
             a.entropy_bits, a.clamped_lo_hi = _ptr(out["entropy_bits"]), _ptr(out["clamped"])

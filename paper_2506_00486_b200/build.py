@@ -27,16 +27,22 @@ def _stale(target, sources):
     return any(os.path.getmtime(s) > t for s in sources)
 
 
-def build(force=False, verbose=False, ptxas_info=False):
-    os.makedirs(BUILD, exist_ok=True)
+def build(force=False, verbose=False, ptxas_info=False, bounds=False):
+    """Builds the library.  bounds=True builds libgg_b200_bounds.so instead: the same sources with -DGG_BOUNDS, whose
+    streaming kernels count (and skip) every checked global access that would leave its buffer; run the GPU tests
+    on it with GG_B200_LIB pointing at it."""
+    build_dir = BUILD + ("_bounds" if bounds else "")
+    lib = LIB.replace(".so", "_bounds.so") if bounds else LIB
+    os.makedirs(build_dir, exist_ok=True)
     hdrs = _deps()
     objs, jobs = [], []
     for src in SOURCES:
         path = os.path.join(CSRC, src)
-        obj = os.path.join(BUILD, src.replace(".cu", ".o"))
+        obj = os.path.join(build_dir, src.replace(".cu", ".o"))
         objs.append(obj)
         if force or _stale(obj, [path] + hdrs):
-            cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if ptxas_info else []) + ["-c", path, "-o", obj]
+            cmd = (["nvcc"] + NVCC_FLAGS + (["-DGG_BOUNDS"] if bounds else []) + (["-Xptxas", "-v"] if ptxas_info else []) +
+                   ["-c", path, "-o", obj])
             jobs.append(cmd)
 
     def run(cmd):
@@ -50,10 +56,10 @@ def build(force=False, verbose=False, ptxas_info=False):
             for log in ex.map(run, jobs):
                 if verbose or ptxas_info:
                     sys.stderr.write(log)
-    if jobs or _stale(LIB, objs):
-        run(["nvcc", "-shared", "-o", LIB] + objs + ["-lcudart"])
-    return LIB
+    if jobs or _stale(lib, objs):
+        run(["nvcc", "-shared", "-o", lib] + objs + ["-lcudart"])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv, bounds="--bounds" in sys.argv))

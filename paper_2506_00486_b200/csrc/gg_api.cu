@@ -12,9 +12,21 @@
 #include <utility>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "gg_internal.h"
 
 using namespace gg;
+
+// Readers of the per-unit violation counters of a bounds-checking build (empty in a normal build).
+static std::vector<unsigned long long (*)()> &bounds_readers()
+{
+    static std::vector<unsigned long long (*)()> readers;
+    return readers;
+}
+namespace gg {
+void gg_register_bounds_reader(unsigned long long (*reader)()) { bounds_readers().push_back(reader); }
+}  // namespace gg
 
 namespace {
 
@@ -49,6 +61,7 @@ struct Plan {
     int32_t n_groups = 0;
     uint32_t *sync = nullptr;     // [2 * n_groups]
     uint64_t last_use = 0;
+    cudaEvent_t used = nullptr;   // recorded after the last work enqueued with this plan: what an eviction waits for
 };
 
 }  // namespace
@@ -83,6 +96,7 @@ struct gg_ctx {
         void *in = nullptr, *grad = nullptr;
         int64_t in_bytes = 0, grad_bytes = 0;
     } slot[2];
+    cudaEvent_t host_ready = nullptr, host_done = nullptr;   // join points of the two staging streams
     void *host_dev = nullptr;     // device block for per-segment outputs and histograms
     int64_t host_dev_bytes = 0;
 };
@@ -162,12 +176,19 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
         return GG_OK;
     }
     if ((int)ctx->plans.size() >= kMaxPlans) {
-        // Evict the least recently used plan.  Work that still uses its tables may be in flight.
-        GG_CUDA(ctx, cudaDeviceSynchronize());
+        // Evict the least recently used plan.  Work that still uses its tables may be in flight: wait for the event
+        // recorded after its last use (not for the whole device; an event recorded inside a stream capture cannot
+        // be waited for, and then the device is).
         size_t victim = 0;
         for (size_t i = 1; i < ctx->plans.size(); ++i)
             if (ctx->plans[i]->last_use < ctx->plans[victim]->last_use) victim = i;
-        cudaFree(ctx->plans[victim]->dev);
+        Plan *v = ctx->plans[victim].get();
+        if (v->used == nullptr || cudaEventSynchronize(v->used) != cudaSuccess) {
+            cudaGetLastError();
+            GG_CUDA(ctx, cudaDeviceSynchronize());
+        }
+        if (v->used) cudaEventDestroy(v->used);
+        cudaFree(v->dev);
         ctx->plans.erase(ctx->plans.begin() + (long)victim);
     }
 
@@ -264,16 +285,25 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
     p->params = reinterpret_cast<double *>(d + o_par);
     p->sd = reinterpret_cast<double *>(d + o_sd);
     p->last_use = ctx->clock;
+    if (cudaEventCreateWithFlags(&p->used, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); p->used = nullptr; }
     *out = p.get();
     ctx->plans.push_back(std::move(p));
     return GG_OK;
 }
 
-// Brackets one launch with events when timing is on.
+// After the last launch that uses the plan's tables.
+void mark_used(Plan *p, cudaStream_t cs)
+{
+    if (p != nullptr && p->used != nullptr && cudaEventRecord(p->used, cs) != cudaSuccess) cudaGetLastError();
+}
+
+// Brackets one sweep of a fused call: an NVTX range (visible to a profiler that is attached, free otherwise) and,
+// when timing is on, a pair of events.
 struct SweepTimer {
     gg_ctx *ctx; std::vector<cudaEvent_t> *list; cudaStream_t st; bool on;
     SweepTimer(gg_ctx *c, std::vector<cudaEvent_t> *l, cudaStream_t s) : ctx(c), list(l), st(s), on(c->timing)
     {
+        nvtxRangePushA(l == &c->ev_first ? "gg: first sweep (moments, or the whole pass)" : "gg: second sweep (gradient + histogram)");
         if (!on) return;
         cudaEvent_t e = nullptr;
         if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
@@ -282,6 +312,7 @@ struct SweepTimer {
     }
     ~SweepTimer()
     {
+        nvtxRangePop();
         if (!on) return;
         cudaEvent_t e = nullptr;
         if (cudaEventCreate(&e) != cudaSuccess) { cudaEventDestroy(list->back()); list->pop_back(); return; }
@@ -465,7 +496,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     if (!ctx) return GG_OK;
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
-    for (auto &p : ctx->plans) cudaFree(p->dev);
+    for (auto &p : ctx->plans) { if (p->used) cudaEventDestroy(p->used); cudaFree(p->dev); }
     for (cudaEvent_t e : ctx->ev_first) cudaEventDestroy(e);
     for (cudaEvent_t e : ctx->ev_tail) cudaEventDestroy(e);
     for (auto &sl : ctx->slot) {
@@ -474,6 +505,8 @@ gg_status gg_destroy(gg_ctx *ctx)
         if (sl.in) cudaFree(sl.in);
         if (sl.grad) cudaFree(sl.grad);
     }
+    if (ctx->host_ready) cudaEventDestroy(ctx->host_ready);
+    if (ctx->host_done) cudaEventDestroy(ctx->host_done);
     if (ctx->host_dev) cudaFree(ctx->host_dev);
     if (ctx->seed) cudaFree(ctx->seed);
     if (ctx->small_counts) cudaFree(ctx->small_counts);
@@ -508,6 +541,7 @@ gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
     fa.count = count; fa.flags = flags; fa.seed = ctx->seed;
     GG_CUDA(ctx, launch_fit(fa, cs));
     ctx->launches += 1;
+    mark_used(p, cs);
     return GG_OK;
 }
 
@@ -539,6 +573,7 @@ gg_status gg_penalty_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dty
         GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta, penalty, cs));
         ctx->launches += 1;
     }
+    mark_used(p, cs);
     return GG_OK;
 }
 
@@ -569,6 +604,7 @@ gg_status gg_rate_hist(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype 
         sa.step = step; sa.qmin = qmin; sa.qmax = qmax; sa.hist = hist; sa.clamped = clamped_lo_hi;
         GG_CUDA(ctx, launch_sweep(ctx, kHist, dtype, GG_F32, false, sa, cs));
         ctx->launches += p->n_tiles > 0;
+        mark_used(p, cs);
     }
     if (entropy_bits && n_hist > 0) {
         st = run_entropy(ctx, hist, n_hist, n_bins, entropy_bits, cs);
@@ -601,7 +637,19 @@ gg_status gg_sample(gg_ctx *ctx, const gg_seg *out, int32_t n_seg, gg_dtype dtyp
     if (max_attempts) GG_CUDA(ctx, cudaMemsetAsync(max_attempts, 0, sizeof(uint32_t) * (size_t)n_seg, cs));
     GG_CUDA(ctx, launch_sample(p->map, dtype, p->params, p->params + n_seg, seed, tensor_id0, max_attempts, cs));
     ctx->launches += p->n_tiles > 0;
+    mark_used(p, cs);
     return GG_OK;
+}
+
+int64_t gg_debug_bounds_violations(void)
+{
+#ifdef GG_BOUNDS
+    unsigned long long total = 0;
+    for (auto reader : bounds_readers()) total += reader();
+    return (int64_t)total;
+#else
+    return -1;
+#endif
 }
 
 gg_status gg_test_hook(gg_ctx *ctx, int32_t what, int64_t value)
@@ -840,6 +888,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta_used, a->penalty, cs));
             ctx->launches += 1;
         }
+        mark_used(p, cs);
     }
     if (do_hist && a->entropy_bits && a->n_hist > 0) {
         gg_status es = run_entropy(ctx, a->hist, a->n_hist, n_bins, a->entropy_bits, cs);
@@ -1036,9 +1085,9 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
             GG_CUDA(ctx, cudaMemsetAsync(d + o_cl, 0, 16 * (size_t)n_hist, s0));
         }
     }
-    cudaEvent_t ready = nullptr, done1 = nullptr;
-    GG_CUDA(ctx, cudaEventCreateWithFlags(&ready, cudaEventDisableTiming));
-    GG_CUDA(ctx, cudaEventCreateWithFlags(&done1, cudaEventDisableTiming));
+    if (ctx->host_ready == nullptr) GG_CUDA(ctx, cudaEventCreateWithFlags(&ctx->host_ready, cudaEventDisableTiming));
+    if (ctx->host_done == nullptr) GG_CUDA(ctx, cudaEventCreateWithFlags(&ctx->host_done, cudaEventDisableTiming));
+    cudaEvent_t ready = ctx->host_ready, done1 = ctx->host_done;
     gg_status result = GG_OK;
     cudaError_t ce = cudaEventRecord(ready, s0);
     if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s1, ready, 0);
@@ -1126,8 +1175,6 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
     }
     // always drain both streams before returning: host buffers are the caller's again
     cudaError_t e0 = cudaStreamSynchronize(s0), e1 = cudaStreamSynchronize(s1);
-    cudaEventDestroy(ready);
-    cudaEventDestroy(done1);
     if (result == GG_OK && e0 != cudaSuccess) result = cuda_fail(ctx, e0);
     if (result == GG_OK && e1 != cudaSuccess) result = cuda_fail(ctx, e1);
     return result;
@@ -1224,6 +1271,7 @@ gg_status gg_eg_rate_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dty
     GG_CUDA(ctx, launch_eg_grad(p->map, dtype, grad_dtype, step, qmin, qmax, k, lambda, accumulate,
                                 static_cast<cudaStream_t>(stream)));
     ctx->launches += p->n_tiles > 0;
+    mark_used(p, static_cast<cudaStream_t>(stream));
     return GG_OK;
 }
 
@@ -1293,6 +1341,8 @@ gg_status gg_gct_step(gg_ctx *ctx, const gg_seg *g, int32_t n_seg, gg_dtype g_dt
                                  g_dtype, step, qmin, qmax, k, eta, lambda, eps, t >= 2 ? 1 : 0,
                                  static_cast<cudaStream_t>(stream)));
     ctx->launches += pg->n_tiles > 0;
+    mark_used(pg, static_cast<cudaStream_t>(stream));
+    mark_used(pw, static_cast<cudaStream_t>(stream));
     return GG_OK;
 }
 

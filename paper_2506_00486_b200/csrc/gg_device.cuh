@@ -1,5 +1,6 @@
 // Small device helpers shared by the kernels of the library (not installed).
 #pragma once
+#include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace gg {
@@ -29,6 +30,35 @@ __device__ __forceinline__ float rcp_approx(float v)
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
     return r;
 }
+
+// ---- bounds-checking build (-DGG_BOUNDS): every checked global access tests its index against the extent it must
+// stay in; a violation is counted (never trapped on) and the access is skipped, so a run of the test suite on such a
+// build ends normally and reports how many accesses would have left their buffers.  A normal build compiles the
+// checks away.  Each translation unit has its own counter; gg_debug_bounds_violations adds them up.
+#ifdef GG_BOUNDS
+static __device__ unsigned long long gg_bounds_count;
+void gg_register_bounds_reader(unsigned long long (*reader)());
+namespace {
+unsigned long long gg_bounds_read_this_unit()
+{
+    unsigned long long v = 0;
+    cudaDeviceSynchronize();
+    if (cudaMemcpyFromSymbol(&v, gg_bounds_count, sizeof(v)) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return v;
+}
+const int gg_bounds_registered = (gg_register_bounds_reader(&gg_bounds_read_this_unit), 0);
+}  // namespace
+// true if index i lies in [0, n); else counts the violation
+__device__ __forceinline__ bool gg_in_bounds(long long i, long long n)
+{
+    if (i >= 0 && i < n) return true;
+    atomicAdd(&gg_bounds_count, 1ull);
+    return false;
+}
+#define GG_IN_BOUNDS(i, n) gg_in_bounds((long long)(i), (long long)(n))
+#else
+#define GG_IN_BOUNDS(i, n) true
+#endif
 
 // Butterfly sum over the warp: every lane ends with the same bits.
 __device__ __forceinline__ double warp_sum(double v)

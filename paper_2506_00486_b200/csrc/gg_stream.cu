@@ -585,6 +585,7 @@ __global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_s
         float xmin = INFINITY, xmax = -INFINITY;
         for (int64_t i = tid; i < head + (n - tail0); i += kSweepThreads) {
             const int64_t idx = i < head ? i : tail0 + (i - head);
+            if (!GG_IN_BOUNDS(idx, n)) continue;
             const uint32_t h = (uint32_t)__ldg(x + idx);
             moments_careful(h, s1, s2, bad);
             xmin = fminf(xmin, __uint_as_float(h << 16));
@@ -597,7 +598,7 @@ __global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_s
         const uint4 *xv = reinterpret_cast<const uint4 *>(x + head) + tid;
 #pragma unroll
         for (int d = 0; d < kSweepDepth - 1; ++d) {
-            if (tid + d * kSweepThreads < nv)
+            if (tid + d * kSweepThreads < nv && GG_IN_BOUNDS(head + (int64_t)(tid + d * kSweepThreads) * 8 + 7, n))
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + d * kStageBytes), "l"(xv + d * kSweepThreads) : "memory");
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
@@ -607,7 +608,7 @@ __global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_s
                 const int vd = v + d * kSweepThreads;
                 if (vd < nv) {
                     // fill the slot emptied by the previous vector (stage d - 1, cyclically)
-                    if (vd + (kSweepDepth - 1) * kSweepThreads < nv)
+                    if (vd + (kSweepDepth - 1) * kSweepThreads < nv && GG_IN_BOUNDS(head + (int64_t)(vd + (kSweepDepth - 1) * kSweepThreads) * 8 + 7, n))
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot0 + ((d + kSweepDepth - 1) % kSweepDepth) * kStageBytes),
                                      "l"(xv + (d + kSweepDepth - 1) * kSweepThreads) : "memory");
                     asm volatile("cp.async.commit_group;" ::: "memory");

@@ -563,8 +563,10 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     const int64_t nvec = (n - head) / 8;
     const int64_t tail0 = head + nvec * 8;
 
-    for (int64_t i = tid; i < head + (n - tail0); i += kThreads)
-        scalar_elem<TG, FLAGS, MODE>(x, gout, i < head ? i : tail0 + (i - head), accumulate, ln, sm, acc);
+    for (int64_t i = tid; i < head + (n - tail0); i += kThreads) {
+        const int64_t idx = i < head ? i : tail0 + (i - head);
+        if (GG_IN_BOUNDS(idx, n)) scalar_elem<TG, FLAGS, MODE>(x, gout, idx, accumulate, ln, sm, acc);
+    }
 
     // (a CTA's run never exceeds device memory / grid size elements: 32-bit vector indices suffice)
     // Each thread owns slot [d][tid] of every stage d: it fills them with asynchronous 16-byte
@@ -578,7 +580,7 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     constexpr uint32_t kStageBytes = sizeof(uint4) * kThreads;
 #pragma unroll
     for (int d = 0; d < kDepth - 1; ++d) {
-        if (tid + d * kThreads < nv)
+        if (tid + d * kThreads < nv && GG_IN_BOUNDS(head + (int64_t)(tid + d * kThreads) * 8 + 7, n))
             copy16<HINT>(slot0 + d * kStageBytes, xv + d * kThreads, tid + d * kThreads < hints.split ? hints.first : hints.rest);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
@@ -589,14 +591,14 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
             const int vd = v + d * kThreads;
             if (vd < nv) {
                 // fill the slot emptied by the previous vector (stage d - 1, cyclically; its value is in registers since then)
-                if (vd + (kDepth - 1) * kThreads < nv)
+                if (vd + (kDepth - 1) * kThreads < nv && GG_IN_BOUNDS(head + (int64_t)(vd + (kDepth - 1) * kThreads) * 8 + 7, n))
                     copy16<HINT>(slot0 + ((d + kDepth - 1) % kDepth) * kStageBytes, xv + (d + kDepth - 1) * kThreads,
                                  vd + (kDepth - 1) * kThreads < hints.split ? hints.first : hints.rest);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
                 uint4 r0;
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r0.x), "=r"(r0.y), "=r"(r0.z), "=r"(r0.w) : "r"(slot0 + d * kStageBytes) : "memory");
-                TG *gd = gv != nullptr ? gv + (int64_t)d * kThreads * 8 : nullptr;
+                TG *gd = gv != nullptr && GG_IN_BOUNDS(head + (int64_t)vd * 8 + 7, n) ? gv + (int64_t)d * kThreads * 8 : nullptr;
                 process_vec<TG, FLAGS, MODE>(r0, gd, accumulate, wide, ln, sm, acc);
             }
         }
@@ -1031,7 +1033,7 @@ __global__ void __launch_bounds__(kThreads, 1) cluster_bf16_kernel(const StreamA
         // ---- stage it: bulk copies of up to one tile each, all completing on the one barrier
         bool ok = true;
         if (nvec > 0) {
-            if (tid == 0) {
+            if (tid == 0 && GG_IN_BOUNDS(off + (int64_t)nvec * 8 - 1, len) && GG_IN_BOUNDS(nvec - 1, kClusterTiles * kTile / 8)) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the reads of the segment before are done
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)nvec * 16u + c.extra_tx) : "memory");
                 for (int v0 = 0; v0 < nvec; v0 += kTile / 8) {

@@ -345,6 +345,7 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
 
     for (int64_t i = tid; i < head + (n - tail0); i += kThreads) {
         const int64_t idx = i < head ? i : tail0 + (i - head);
+        if (!GG_IN_BOUNDS(idx, n)) continue;
         float g[8];
         process8<FLAGS, MODE>(make_uint4(__float_as_uint(__ldg(x + idx)), 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u), 1, g, ln,
                               sm, acc, clampc);
@@ -379,13 +380,14 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
     };
 #pragma unroll
     for (int d = 0; d < kDepth - 1; ++d) {
-        if (tid + d * kThreads < nv) fill(slot0 + d * kStageBytes, xv + 2 * d * kThreads);
+        if (tid + d * kThreads < nv && GG_IN_BOUNDS(head + (int64_t)(tid + d * kThreads) * 8 + 7, n)) fill(slot0 + d * kStageBytes, xv + 2 * d * kThreads);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     uint32_t rd = 0, wr = (kDepth - 1) * kStageBytes;      // byte offsets of the slot to read / to fill next
     for (int v = tid; v < nv; v += kThreads) {
         // fill the slot emptied by the previous iteration (its values are in registers since then)
-        if (v + (kDepth - 1) * kThreads < nv) fill(slot0 + wr, xv + 2 * (kDepth - 1) * kThreads);
+        if (v + (kDepth - 1) * kThreads < nv && GG_IN_BOUNDS(head + (int64_t)(v + (kDepth - 1) * kThreads) * 8 + 7, n))
+            fill(slot0 + wr, xv + 2 * (kDepth - 1) * kThreads);
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
         uint4 lo, hi;
@@ -394,7 +396,7 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
         float g[8];
         process8<FLAGS, MODE>(lo, hi, 8, g, ln, sm, acc, clampc);
         if constexpr (GRAD) {
-            if (gv != nullptr) store8<TG>(gv, g, accumulate, wide);
+            if (gv != nullptr && GG_IN_BOUNDS(head + (int64_t)v * 8 + 7, n)) store8<TG>(gv, g, accumulate, wide);
         }
         rd = rd + kStageBytes == kDepth * kStageBytes ? 0u : rd + kStageBytes;
         wr = wr + kStageBytes == kDepth * kStageBytes ? 0u : wr + kStageBytes;

@@ -282,7 +282,9 @@ __device__ __forceinline__ void second_pass(const float *x, const uint4 *xv, TG 
 #pragma unroll
         for (int u = 0; u < RV; ++u) {
             const int v = tt + u * kTeam;
-            if (v < nvec) second_vec<TG, GRAD, HIST>(reg[u], gout != nullptr ? gout + head + v * EPV : nullptr, accumulate, k, ad, tm, sm, pen, clampc);
+            if (v < nvec)
+                second_vec<TG, GRAD, HIST>(reg[u], gout != nullptr && GG_IN_BOUNDS(head + v * EPV + EPV - 1, head + nvec * EPV) ? gout + head + v * EPV : nullptr,
+                                           accumulate, k, ad, tm, sm, pen, clampc);
         }
     } else {
         // (loads run three vectors ahead of their use)
@@ -368,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) team_kernel(const SmallA
 #pragma unroll
             for (int u = 0; u < RV; ++u) {
                 reg[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (tt + u * kTeam < nvec) reg[u] = __ldg(xv + tt + u * kTeam);
+                if (tt + u * kTeam < nvec && GG_IN_BOUNDS(head + (tt + u * kTeam) * EPV + EPV - 1, len)) reg[u] = __ldg(xv + tt + u * kTeam);
             }
         }
         double s1 = 0.0, s2 = 0.0;

@@ -24,3 +24,17 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """With a bounds-checking build of the library (GG_B200_LIB=...libgg_b200_bounds.so) the run must end with no
+    checked access outside its buffer."""
+    if not os.environ.get("GG_B200_LIB"):
+        return
+    from paper_2506_00486_b200 import binding
+    if binding._lib is None:
+        return
+    n = binding.lib().gg_debug_bounds_violations()
+    print(f"\nbounds-checking build: {n} checked accesses outside their buffers")
+    if n > 0:
+        session.exitstatus = 1

@@ -23,9 +23,16 @@ def ctx():
     import __graft_entry__ as entry
     entry.build()
     from paper_2506_00486_b200 import Context
-    c = Context(0)
+    c = Context(0, guard=True)        # fill patterns around every output the binding allocates
     yield c
     c.close()
+
+
+@pytest.fixture(autouse=True)
+def outputs_stay_inside_their_buffers(ctx):
+    """After every test: no kernel wrote before or after a fit result, penalty, histogram, entropy or counter."""
+    yield
+    ctx.check_guards()
 
 
 def dev(t):
