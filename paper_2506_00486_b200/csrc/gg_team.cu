@@ -32,7 +32,7 @@ constexpr int kThreads = kTeam * kTeams;
 constexpr int kCtasPerSm = 2;
 constexpr int kTabExp = 64;                    // exponents around the segment's scale whose A is evaluated
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr uint32_t kWinCells = 8192;           // fp32 input: symbols [-4096, 4096) of the CTA's table
+constexpr uint32_t kWinCells = kSymWin;        // symbols [-4096, 4096) of the CTA's table
 constexpr uint32_t kSymCells = kWinCells + 2;  // with the two sentinels of the tails
 constexpr uint32_t kCntWords = kSymCells;
 static_assert(kSymCells + 4 <= (uint32_t)kSmallSlotWords, "scratch slot");
@@ -533,39 +533,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) team_kernel(const SmallA
             slot[kSymCells + 0] = (uint32_t)sm.key_on;
             slot[kSymCells + 1] = (uint32_t)sm.key_hid;
             slot[kSymCells + 2] = sm.key_inv_bits;
+            slot[kSymCells + 3] = 0u;
         }
     }
-}
-
-// fp32 input: one thread per symbol cell adds up the runs of CTA slots that share a key (histogram, step); each run
-// is one 64-bit addition.  The sentinel cells (first and last) are not counted.
-__global__ void team_flush_symbols_kernel(const uint32_t *__restrict__ cta_counts, int n_slots, int32_t qmin, int32_t qmax, uint64_t *hist,
-                                          uint64_t *clamped)
-{
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x + 1;
-    if (c > kWinCells) return;
-    const int64_t n_bins = (int64_t)qmax - (int64_t)qmin + 1;
-    unsigned long long run = 0;
-    uint32_t k_hid = 0, k_inv = 0;
-    bool have = false;
-    auto emit = [&]() {
-        if (run == 0) return;
-        int q = (int)c - 1 - (int)(kWinCells / 2);
-        unsigned long long *cl = reinterpret_cast<unsigned long long *>(clamped);
-        if (q < qmin) { q = qmin; if (cl) atomicAdd(cl + 2 * k_hid, run); }
-        else if (q > qmax) { q = qmax; if (cl) atomicAdd(cl + 2 * k_hid + 1, run); }
-        atomicAdd(reinterpret_cast<unsigned long long *>(hist) + (int64_t)k_hid * n_bins + (q - qmin), run);
-        run = 0;
-    };
-    for (int b = 0; b < n_slots; ++b) {
-        const uint32_t *slot = cta_counts + (size_t)b * kSmallSlotWords;
-        if (__ldg(slot + kSymCells) == 0u) continue;            // this CTA had no table
-        const uint32_t hid = __ldg(slot + kSymCells + 1), inv = __ldg(slot + kSymCells + 2);
-        if (have && (hid != k_hid || inv != k_inv)) emit();
-        k_hid = hid; k_inv = inv; have = true;
-        run += __ldg(slot + c);
-    }
-    emit();
 }
 
 template <typename TG>
@@ -581,7 +551,7 @@ cudaError_t launch_typed(const SmallArgs &a, int sm_count, cudaStream_t st)
     if (!a.do_hist) return a.do_grad ? go(team_kernel<TG, true, false>) : go(team_kernel<TG, false, false>);
     cudaError_t e = a.do_grad ? go(team_kernel<TG, true, true>) : go(team_kernel<TG, false, true>);
     if (e != cudaSuccess) return e;
-    team_flush_symbols_kernel<<<(kWinCells + 255) / 256, 256, 0, st>>>(a.cta_counts, grid, a.qmin, a.qmax, a.hist, a.clamped);
+    flush_slots_kernel<true><<<(kSymCells + 31) / 32, dim3(32, 8), 0, st>>>(a.cta_counts, grid, a.qmin, a.qmax, a.hist, a.clamped);
     return cudaGetLastError();
 }
 
