@@ -89,6 +89,7 @@ struct gg_ctx {
     // optional device timing of the two sweeps of gg_fused (event pairs, summed on read)
     bool timing = false;
     std::vector<cudaEvent_t> ev_first, ev_tail;   // begin, end, begin, end, ...
+    std::vector<cudaEvent_t> ev_pool;             // events handed back by gg_timing_read, for the next sweeps
     // gg_fused_host staging (created on first use)
     struct HostSlot {
         gg_ctx *ctx = nullptr;
@@ -305,17 +306,24 @@ struct SweepTimer {
     {
         nvtxRangePushA(l == &c->ev_first ? "gg: first sweep (moments, or the whole pass)" : "gg: second sweep (gradient + histogram)");
         if (!on) return;
-        cudaEvent_t e = nullptr;
-        if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+        cudaEvent_t e = take_event(c);
+        if (e == nullptr) { on = false; return; }
         cudaEventRecord(e, st);
         list->push_back(e);
+    }
+    static cudaEvent_t take_event(gg_ctx *c)
+    {
+        cudaEvent_t e = nullptr;
+        if (!c->ev_pool.empty()) { e = c->ev_pool.back(); c->ev_pool.pop_back(); return e; }
+        if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return e;
     }
     ~SweepTimer()
     {
         nvtxRangePop();
         if (!on) return;
-        cudaEvent_t e = nullptr;
-        if (cudaEventCreate(&e) != cudaSuccess) { cudaEventDestroy(list->back()); list->pop_back(); return; }
+        cudaEvent_t e = take_event(ctx);
+        if (e == nullptr) { ctx->ev_pool.push_back(list->back()); list->pop_back(); return; }
         cudaEventRecord(e, st);
         list->push_back(e);
     }
@@ -499,6 +507,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     for (auto &p : ctx->plans) { if (p->used) cudaEventDestroy(p->used); cudaFree(p->dev); }
     for (cudaEvent_t e : ctx->ev_first) cudaEventDestroy(e);
     for (cudaEvent_t e : ctx->ev_tail) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
     for (auto &sl : ctx->slot) {
         if (sl.ctx) gg_destroy(sl.ctx);
         if (sl.stream) cudaStreamDestroy(sl.stream);
@@ -700,7 +709,7 @@ gg_status gg_timing_read(gg_ctx *ctx, double *ms_first, int64_t *n_first, double
             if (e != cudaSuccess) result = cuda_fail(ctx, e);
             else { ms[k] += (double)t; cnt[k] += 1; }
         }
-        for (cudaEvent_t e : l) cudaEventDestroy(e);
+        for (cudaEvent_t e : l) ctx->ev_pool.push_back(e);      // (kept for the next sweeps: no event is created per call)
         l.clear();
     }
     if (ms_first) *ms_first = ms[0];
