@@ -1,0 +1,106 @@
+"""Randomised parity of gg_fused over everything that decides which kernels run: element type, segment lengths from
+empty to 70 tiles (short-segment kernels, the two sweeps, the optional one-launch and cluster forms), alignment,
+gradient type, shared histograms, sum or mean, fitted or given parameters, steps given or taken from the fit, the sign
+of lambda, the clamp range.  Every case is compared with the fp64 oracle: fit, flags, gradient element by element,
+penalty, histogram, clamp counters, entropy; and no output may be written outside its buffer."""
+import numpy as np
+import pytest
+import torch
+
+import gg_synth
+from oracle import gg_oracle as o
+from parity_util import ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+TILE = 16384
+
+
+@pytest.mark.parametrize("seed0", [11, 12])
+def test_fused_random_cases_over_every_option(seed0):
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2506_00486_b200 import GG_MEAN, GG_PARAMS_GIVEN, GG_SUM, Context, Segments
+    ctx = Context(0, guard=True)
+    n_cases = 40
+    failures = []
+    for case in range(n_cases):
+        rng = np.random.default_rng(seed0 * 100000 + case)
+        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        kind = rng.choice(["short", "medium", "long", "mixed"])
+        if kind == "short":
+            n_seg, cap = int(rng.integers(64, 200)), int(rng.choice([600, 5000, 16000]))
+        elif kind == "medium":
+            n_seg, cap = int(rng.integers(2, 40)), int(rng.choice([3 * TILE, 20 * TILE]))
+        elif kind == "long":
+            n_seg, cap = int(rng.integers(1, 5)), 70 * TILE
+        else:
+            n_seg, cap = int(rng.integers(1, 100)), 10 * TILE
+        lens = [max(0, int(np.exp(rng.uniform(0, np.log(cap)))) - 1) for _ in range(n_seg)]
+        xs = [gg_synth.gg_host(rng, float(rng.uniform(0.3, 2.6)), 10.0 ** rng.uniform(-4, 1), n, dtype) for n in lens]
+        if rng.random() < 0.3 and lens[0] > 10:
+            xs[0][:4] = torch.tensor([0.0, -0.0, 3e38, 1e-39]).to(dtype)
+        misalign = rng.random() < 0.4
+        offs = [int(rng.integers(0, 8)) if misalign else 0 for _ in xs]
+        xd = []
+        for t, off in zip(xs, offs):
+            buf = torch.zeros(t.numel() + 16, dtype=t.dtype, device="cuda:0"); buf[off:off + t.numel()].copy_(t); xd.append(buf[off:off + t.numel()])
+        gdt = torch.float32 if rng.random() < 0.7 else torch.bfloat16
+        gd = [torch.full((n,), 0.5, dtype=gdt, device="cuda:0") for n in lens]
+        n_hist = int(rng.integers(1, 4)); hid = [int(rng.integers(0, n_hist)) for _ in xs]
+        mean = rng.random() < 0.3
+        given = rng.random() < 0.3
+        step_alpha = (not given) and rng.random() < 0.3
+        lam = float(rng.choice([1e-4, -3e-3, 2.0]))
+        resident = int(rng.random() < 0.3 and dtype == torch.bfloat16); cluster = int(rng.choice([0, 0, 1, 2]))
+        ctx.gg_test_hook(0, resident)      # the one-launch form on or off
+        ctx.gg_test_hook(3, cluster)       # the cluster form: never / when the layout suits / whenever it can run
+        qmin, qmax = (-32768, 32767) if rng.random() < 0.5 else (-300, 250)
+        kw = dict(grad=Segments(gd), lam=lam, hist_id=hid, n_hist=n_hist, reduction=GG_MEAN if mean else GG_SUM, qmin=qmin, qmax=qmax)
+        step_val = float(2.0 ** rng.integers(-10, -3))
+        if step_alpha: kw["step_scale"] = 1 / 8
+        else: kw["step"] = torch.full((n_seg,), step_val, dtype=torch.float32, device="cuda:0")
+        giv = None
+        if given:
+            giv = [(float(rng.uniform(0.4, 2.4)), 10.0 ** rng.uniform(-3, 0)) for _ in xs]
+            kw.update(param_mode=GG_PARAMS_GIVEN, beta_in=torch.tensor([g[0] for g in giv], dtype=torch.float64, device="cuda:0"),
+                      alpha_in=torch.tensor([g[1] for g in giv], dtype=torch.float64, device="cuda:0"))
+        desc = f"case {case} dtype={dtype} kind={kind} n_seg={n_seg} cap={cap} mis={misalign} gdt={gdt} given={given} step_alpha={step_alpha} lam={lam} res={resident} clu={cluster} q=({qmin},{qmax}) mean={mean}"
+        try:
+            out = ctx.gg_fused(Segments(xd), **kw)
+            torch.cuda.synchronize(); ctx.check_guards()
+            nb = qmax - qmin + 1
+            ref_hist = np.zeros((n_hist, nb), dtype=np.uint64); ref_cl = np.zeros((n_hist, 2), dtype=np.uint64)
+            steps_used = out["step"].cpu().numpy()
+            for s, x in enumerate(xs):
+                xo = gg_synth.to_oracle(x)
+                b, a, s1, s2, n, fl = o.fit(xo)
+                assert (out["flags"][s].item() & 15) == fl, ("flags", s)
+                bg, ag = out["beta"][s].item(), out["alpha"][s].item()
+                if fl & 1: assert bg == 0 and ag == 0
+                else: assert abs(bg - b) <= 1e-5 * b and abs(ag - a) <= 1e-5 * a, ("fit", s, bg, b)
+                bu, au = (bg, ag) if giv is None else giv[s]
+                lam_s = lam / max(n, 1) if mean else lam
+                pen, g = o.penalty_grad(xo, bu, au, lam_s)
+                got = gd[s].float().cpu().numpy().astype(np.float64) - 0.5 if False else None
+                # gradient written (not accumulated): compare
+                gg = gd[s].cpu()
+                if gdt == torch.float32:
+                    fin = np.isfinite(g.astype(np.float32))
+                    d = ulp_distance(gg.numpy()[fin], g[fin]); assert d.size == 0 or d.max() <= 4, ("grad", s, int(d.max()))
+                else:
+                    ref = o.round_to_bf16_bits(g).astype(np.int64); gb = gg.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
+                    fin = np.isfinite(g) & (np.abs(g) < 3e38)
+                    assert np.abs((ref & 0x7FFF) - (gb & 0x7FFF))[fin].max(initial=0) <= 1, ("grad16", s)
+                if np.isfinite(pen) and abs(pen) > 0: assert abs(out["penalty"][s].item() - pen) <= 1e-6 * abs(pen), ("pen", s, out["penalty"][s].item(), pen)
+                if step_alpha: assert steps_used[s] == np.float32(ag / 8), ("step", s)
+                if steps_used[s] > 0 and np.isfinite(steps_used[s]):
+                    o.quantise_hist(xo, steps_used[s], qmin, qmax, hist=ref_hist[hid[s]], clamped=ref_cl[hid[s]])
+            if not (step_alpha and any((out["flags"][s].item() & 1) for s in range(n_seg))):
+                assert np.array_equal(out["hist"].cpu().numpy(), ref_hist.astype(np.int64)), "hist"
+                assert np.array_equal(out["clamped"].cpu().numpy(), ref_cl.astype(np.int64)), "clamped"
+                for h in range(n_hist): assert abs(out["entropy_bits"][h].item() - o.entropy_bits(ref_hist[h])) <= 1e-9, "entropy"
+        except AssertionError as e:
+            failures.append((desc, str(e)))
+    ctx.close()
+    assert not failures, failures
