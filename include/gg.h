@@ -19,13 +19,18 @@
  *    caller pointer beyond the work it has enqueued.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
  *    enqueue work; they do not wait for the device.  Exception: the first call that sees a new
- *    segment layout (addresses, lengths, dtype, histogram ids) allocates and uploads a small
- *    plan with blocking calls; make that first call outside stream capture.  A context keeps the
- *    plans of the 64 layouts used last: a call that brings in a 65th frees the oldest plan after
- *    waiting for the work last enqueued with it (an event; the whole device if that work was
- *    captured in a graph), and a call that needs more histogram or channel scratch than any
- *    before it reallocates that scratch after waiting for the device.  All of these belong outside
- *    stream capture too.  A context serves one stream at a time.
+ *    segment layout (lengths, dtype, histogram ids, and the addresses) allocates and uploads a
+ *    small plan with blocking calls; make that first call outside stream capture.  A context
+ *    keeps up to 64 plans, up to 16 of them for one layout at different addresses.  When the
+ *    same layout comes with addresses no plan has (buffers that an allocator moved, the same
+ *    shapes in another layer) and the layout has its 16 plans or the context its 64, the least
+ *    recently used plan of that layout is pointed at the new addresses: two small uploads from
+ *    pinned memory, ordered on `stream`, no allocation and no wait for the device (also outside
+ *    stream capture: a replayed upload would carry the addresses of capture time).  Only a new
+ *    layout in a full context frees the oldest plan, after waiting for the work last enqueued
+ *    with it (an event; the whole device if that work was captured in a graph); and a call that
+ *    needs more histogram or channel scratch than any before it reallocates that scratch after
+ *    waiting for the device.  A context serves one stream at a time.
  *  - A segment is a contiguous run of `len` elements.  Pointers need only element alignment;
  *    16-byte aligned segments take the vectorised path.
  *  - Per-segment conditions are reported in `flags` (GG_FLAG_*), never as an error status.
@@ -96,6 +101,9 @@ int gg_version(void);
 const char *gg_last_cuda_error(const gg_ctx *ctx);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t gg_launch_count(const gg_ctx *ctx);
+/* Plans this context has built (what = 0: each one an allocation and a blocking upload) and plans it has pointed
+ * at other addresses (what = 1) since creation; -1 for any other `what`. */
+int64_t gg_plan_stats(const gg_ctx *ctx, int32_t what);
 
 /* ---- host helpers (no device work) --------------------------------------------------------- */
 

@@ -84,6 +84,8 @@ def lib():
         L.gg_last_cuda_error.restype = ctypes.c_char_p
         L.gg_launch_count.argtypes = [_P]
         L.gg_launch_count.restype = i64
+        L.gg_plan_stats.argtypes = [_P, i32]
+        L.gg_plan_stats.restype = i64
         for name, args in (("gg_alpha_from_std", [d, d]), ("gg_init_alpha", [i64, d, d]),
                            ("gg_diff_entropy_bits", [d, d])):
             getattr(L, name).argtypes = args
@@ -288,6 +290,11 @@ class Context:
     @property
     def launch_count(self):
         return lib().gg_launch_count(self._h)
+
+    @property
+    def plan_stats(self):
+        """(plans built, plans pointed at other addresses) since the context was created."""
+        return lib().gg_plan_stats(self._h, 0), lib().gg_plan_stats(self._h, 1)
 
     def gg_test_hook(self, what, value):
         """Knobs of the one-launch fitted pass (HOOK_*), for tests and measurements."""

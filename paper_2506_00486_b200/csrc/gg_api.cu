@@ -31,6 +31,7 @@ void gg_register_bounds_reader(unsigned long long (*reader)()) { bounds_readers(
 namespace {
 
 constexpr int kMaxPlans = 64;
+constexpr int kMaxPlansPerLayout = 16;   // plans of one layout (same lengths, types and histogram ids) that differ in their addresses
 // The one-launch fitted pass (off unless switched on by gg_test_hook): a group is what L2 keeps from the first
 // read of a tensor to the second while the gradient of the tensor before streams out (measured on B200: about
 // 30 MB of 126), and at most one segment per warp of the fitting CTA.
@@ -62,6 +63,11 @@ struct Plan {
     uint32_t *sync = nullptr;     // [2 * n_groups]
     uint64_t last_use = 0;
     cudaEvent_t used = nullptr;   // recorded after the last work enqueued with this plan: what an eviction waits for
+    // a plan whose layout fits a call with other addresses is pointed at them: the two address tables are uploaded
+    // again from this pinned staging block, in stream order
+    size_t o_ptr = 0, o_gptr = 0;
+    void *pin = nullptr;
+    cudaEvent_t repointed = nullptr;   // recorded after the upload: the staging block may be filled again
 };
 
 }  // namespace
@@ -72,6 +78,7 @@ struct gg_ctx {
     std::vector<std::unique_ptr<Plan>> plans;
     uint64_t clock = 0;
     int64_t launches = 0;
+    int64_t plan_builds = 0, plan_repoints = 0;
     std::string cuda_error;
     double *ent_part = nullptr;   // scratch of the entropy kernels: 2 * kEntSplit doubles per histogram
     int64_t ent_hists = 0;
@@ -167,14 +174,80 @@ Plan *find_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype, co
     return best;
 }
 
-// Finds or builds the plan for this layout.  Building allocates and uploads with blocking calls.
+void free_plan(Plan *v)
+{
+    if (v->used) cudaEventDestroy(v->used);
+    if (v->repointed) cudaEventDestroy(v->repointed);
+    if (v->pin) cudaFreeHost(v->pin);
+    cudaFree(v->dev);
+}
+
+// Same lengths, types and histogram ids; the addresses may differ.
+bool same_layout(const Plan &p, const int32_t (&head)[4], const gg_seg *segs, int32_t n_seg, const int32_t *hist_id)
+{
+    if (memcmp(p.head, head, sizeof(head)) != 0) return false;
+    for (int32_t s = 0; s < n_seg; ++s)
+        if (p.segs[(size_t)s].len != segs[s].len) return false;
+    return !hist_id || memcmp(p.hist_id.data(), hist_id, sizeof(int32_t) * (size_t)n_seg) == 0;
+}
+
+// Points a plan at other addresses: no allocation on the device and no wait for the device; the upload of the two
+// address tables is ordered on `cs` behind the work that still reads the old ones.
+gg_status repoint(gg_ctx *ctx, Plan *p, const gg_seg *segs, const gg_seg *grad, cudaStream_t cs)
+{
+    const size_t n = (size_t)p->n_seg;
+    if (p->pin == nullptr) {
+        GG_CUDA(ctx, cudaHostAlloc(&p->pin, sizeof(void *) * 2 * n, cudaHostAllocDefault));
+        cudaError_t e = cudaEventCreateWithFlags(&p->repointed, cudaEventDisableTiming);
+        if (e != cudaSuccess) { cudaFreeHost(p->pin); p->pin = nullptr; p->repointed = nullptr; return cuda_fail(ctx, e); }
+    } else {
+        GG_CUDA(ctx, cudaEventSynchronize(p->repointed));      // the upload before this one has read the block
+    }
+    void **tab = static_cast<void **>(p->pin);
+    p->aligned16 = true;
+    for (size_t s = 0; s < n; ++s) {
+        tab[s] = segs[s].ptr;
+        tab[n + s] = grad ? grad[s].ptr : nullptr;
+        if (reinterpret_cast<uintptr_t>(segs[s].ptr) % 16 != 0 || (grad && reinterpret_cast<uintptr_t>(grad[s].ptr) % 16 != 0))
+            p->aligned16 = false;
+    }
+    char *d = static_cast<char *>(p->dev);
+    GG_CUDA(ctx, cudaMemcpyAsync(d + p->o_ptr, tab, sizeof(void *) * n, cudaMemcpyHostToDevice, cs));
+    if (grad) GG_CUDA(ctx, cudaMemcpyAsync(d + p->o_gptr, tab + n, sizeof(void *) * n, cudaMemcpyHostToDevice, cs));
+    GG_CUDA(ctx, cudaEventRecord(p->repointed, cs));
+    p->segs.assign(segs, segs + n);
+    if (grad) p->grad.assign(grad, grad + n);
+    p->last_use = ctx->clock;
+    ctx->plan_repoints++;
+    return GG_OK;
+}
+
+// Finds or builds the plan for this layout.  Building allocates and uploads with blocking calls; a layout that
+// already has kMaxPlansPerLayout plans (or any plan, once the cache is full) gets its least recently used plan
+// pointed at the new addresses instead, which neither allocates nor blocks.
 gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype, const gg_seg *grad,
-                   int grad_dtype, const int32_t *hist_id, Plan **out)
+                   int grad_dtype, const int32_t *hist_id, Plan **out, void *stream)
 {
     ctx->clock++;
     if (Plan *hit = find_plan(ctx, segs, n_seg, in_dtype, grad, grad_dtype, hist_id)) {
         *out = hit;
         return GG_OK;
+    }
+    {
+        const int32_t head[4] = {n_seg, in_dtype, grad ? grad_dtype : -1, hist_id ? 1 : 0};
+        Plan *lru = nullptr;
+        int same = 0;
+        for (auto &q : ctx->plans)
+            if (same_layout(*q, head, segs, n_seg, hist_id)) {
+                ++same;
+                if (lru == nullptr || q->last_use < lru->last_use) lru = q.get();
+            }
+        if (lru != nullptr && (same >= kMaxPlansPerLayout || (int)ctx->plans.size() >= kMaxPlans)) {
+            gg_status st = repoint(ctx, lru, segs, grad, static_cast<cudaStream_t>(stream));
+            if (st != GG_OK) return st;
+            *out = lru;
+            return GG_OK;
+        }
     }
     if ((int)ctx->plans.size() >= kMaxPlans) {
         // Evict the least recently used plan.  Work that still uses its tables may be in flight: wait for the event
@@ -188,8 +261,7 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
             cudaGetLastError();
             GG_CUDA(ctx, cudaDeviceSynchronize());
         }
-        if (v->used) cudaEventDestroy(v->used);
-        cudaFree(v->dev);
+        free_plan(v);
         ctx->plans.erase(ctx->plans.begin() + (long)victim);
     }
 
@@ -265,6 +337,8 @@ gg_status get_plan(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, int in_dtype,
         e = cudaMemcpy(static_cast<char *>(p->dev) + o_grp, groups.data(), sizeof(int4) * groups.size(), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { cudaFree(p->dev); return cuda_fail(ctx, e); }
     char *d = static_cast<char *>(p->dev);
+    p->o_ptr = o_ptr; p->o_gptr = o_gptr;
+    ctx->plan_builds++;
     p->groups = reinterpret_cast<int4 *>(d + o_grp);
     p->sync = reinterpret_cast<uint32_t *>(d + o_sync);
     p->n_groups = (int32_t)groups.size();
@@ -451,6 +525,12 @@ const char *gg_status_str(gg_status s)
 const char *gg_last_cuda_error(const gg_ctx *ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
 int64_t gg_launch_count(const gg_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+int64_t gg_plan_stats(const gg_ctx *ctx, int32_t what)
+{
+    if (!ctx) return 0;
+    return what == 0 ? ctx->plan_builds : what == 1 ? ctx->plan_repoints : -1;
+}
+
 double gg_alpha_from_std(double sigma, double beta)
 {
     return sigma * exp(0.5 * (lgamma(1.0 / beta) - lgamma(3.0 / beta)));
@@ -504,7 +584,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     if (!ctx) return GG_OK;
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
-    for (auto &p : ctx->plans) { if (p->used) cudaEventDestroy(p->used); cudaFree(p->dev); }
+    for (auto &p : ctx->plans) free_plan(p.get());
     for (cudaEvent_t e : ctx->ev_first) cudaEventDestroy(e);
     for (cudaEvent_t e : ctx->ev_tail) cudaEventDestroy(e);
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
@@ -536,7 +616,7 @@ gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
     Plan *p = nullptr;
-    st = get_plan(ctx, segs, n_seg, dtype, nullptr, 0, nullptr, &p);
+    st = get_plan(ctx, segs, n_seg, dtype, nullptr, 0, nullptr, &p, stream);
     if (st != GG_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     StreamArgs sa{};
@@ -569,7 +649,7 @@ gg_status gg_penalty_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dty
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
     Plan *p = nullptr;
-    st = get_plan(ctx, segs, n_seg, in_dtype, grad, grad_dtype, nullptr, &p);
+    st = get_plan(ctx, segs, n_seg, in_dtype, grad, grad_dtype, nullptr, &p, stream);
     if (st != GG_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     StreamArgs sa{};
@@ -606,7 +686,7 @@ gg_status gg_rate_hist(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype 
     }
     if (n_seg > 0) {
         Plan *p = nullptr;
-        st = get_plan(ctx, segs, n_seg, dtype, nullptr, 0, hist_id, &p);
+        st = get_plan(ctx, segs, n_seg, dtype, nullptr, 0, hist_id, &p, stream);
         if (st != GG_OK) return st;
         StreamArgs sa{};
         sa.map = p->map; sa.part = p->part;
@@ -636,7 +716,7 @@ gg_status gg_sample(gg_ctx *ctx, const gg_seg *out, int32_t n_seg, gg_dtype dtyp
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
     Plan *p = nullptr;
-    st = get_plan(ctx, out, n_seg, dtype, nullptr, 0, nullptr, &p);
+    st = get_plan(ctx, out, n_seg, dtype, nullptr, 0, nullptr, &p, stream);
     if (st != GG_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     // (beta, alpha) come from pageable host memory: the copy is staged before the call returns
@@ -760,7 +840,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int32_t n_bins = do_hist ? a->qmax - a->qmin + 1 : 0;
     if (n_seg > 0 && p == nullptr) {
-        st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p);
+        st = get_plan(ctx, a->segs, n_seg, a->in_dtype, a->grad, a->grad_dtype, do_hist ? a->hist_id : nullptr, &p, stream);
         if (st != GG_OK) return st;
     }
     // The histograms start from zero.  When the call begins with the persistent bf16 moments sweep, that sweep
@@ -1275,7 +1355,7 @@ gg_status gg_eg_rate_grad(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dty
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
     Plan *p = nullptr;
-    st = get_plan(ctx, segs, n_seg, dtype, grad, grad_dtype, nullptr, &p);
+    st = get_plan(ctx, segs, n_seg, dtype, grad, grad_dtype, nullptr, &p, stream);
     if (st != GG_OK) return st;
     GG_CUDA(ctx, launch_eg_grad(p->map, dtype, grad_dtype, step, qmin, qmax, k, lambda, accumulate,
                                 static_cast<cudaStream_t>(stream)));
@@ -1342,9 +1422,9 @@ gg_status gg_gct_step(gg_ctx *ctx, const gg_seg *g, int32_t n_seg, gg_dtype g_dt
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return GG_ERR_CUDA;
     Plan *pg = nullptr, *pw = nullptr;
-    st = get_plan(ctx, g, n_seg, g_dtype, ghat, GG_F32, nullptr, &pg);
+    st = get_plan(ctx, g, n_seg, g_dtype, ghat, GG_F32, nullptr, &pg, stream);
     if (st != GG_OK) return st;
-    st = get_plan(ctx, w, n_seg, GG_F32, nullptr, 0, nullptr, &pw);      // (for its device table of the weight addresses)
+    st = get_plan(ctx, w, n_seg, GG_F32, nullptr, 0, nullptr, &pw, stream);      // (for its device table of the weight addresses)
     if (st != GG_OK) return st;
     GG_CUDA(ctx, launch_gct_step(pg->map, const_cast<void *const *>(reinterpret_cast<const void *const *>(pw->map.seg_ptr)),
                                  g_dtype, step, qmin, qmax, k, eta, lambda, eps, t >= 2 ? 1 : 0,

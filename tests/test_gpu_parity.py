@@ -775,3 +775,41 @@ def test_fused_random_layouts(ctx, dtype):
                            reduction=GG_MEAN if mean else GG_SUM, qmin=-3000, qmax=2500)
         torch.cuda.synchronize()
         check_fused(out, xs, gd, 2e-4, hid, n_hist, qmin=-3000, qmax=2500, mean=mean)
+
+
+def test_one_layout_at_many_addresses_reuses_its_plans(ctx):
+    """The same segment lengths at addresses that keep changing (buffers an allocator moves, the same shapes in
+    another layer): after the layout's 16 plans exist, a call with new addresses points the least recently used
+    of them at the new buffers instead of building a plan.  Every call must still read and write the buffers it
+    was given: checked against the oracle at several of the 100 positions, the misaligned ones among them."""
+    from paper_2506_00486_b200 import Context, Segments
+    c = Context(0)
+    rng = np.random.default_rng(31)
+    lens = [40000, 7, 20000]
+    stride, n_pos = 1000, 100
+    pool = gg_synth.gg_host(rng, 0.9, 0.03, sum(lens) + stride * n_pos + 8, torch.bfloat16)
+    pool_d = dev(pool)
+    gpool = torch.full((pool.numel(),), 7.0, dtype=torch.float32, device="cuda:0")
+    steps = torch.full((3,), 2.0 ** -9, dtype=torch.float32, device="cuda:0")
+
+    def windows(k, buf):
+        o0 = k * stride + (k % 3)                 # (every third position starts on a 16-byte boundary)
+        return [buf[o0:o0 + lens[0]], buf[o0 + lens[0]:o0 + lens[0] + lens[1]],
+                buf[o0 + lens[0] + lens[1]:o0 + sum(lens)]]
+
+    other = [dev(gg_synth.gg_host(rng, 1.2, 0.1, 5000, torch.bfloat16))]
+    for rnd in range(2):
+        for k in range(n_pos):
+            xd, gd = windows(k, pool_d), windows(k, gpool)
+            out = c.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps)
+            if k % 10 == 3:
+                c.gg_fit(other)                   # (another layout in between changes nothing)
+            if k in (0, 1, 17, 50, 64, 65, 99):
+                torch.cuda.synchronize()
+                check_fused(out, windows(k, pool), gd, 1e-4, [0, 1, 2], 3)
+                gpool[k * stride:(k + 1) * stride + sum(lens) + 8] = 7.0
+    torch.cuda.synchronize()
+    built, repointed = c.plan_stats
+    assert built == 16 + 1                        # the layout's plans and the other layout's one
+    assert repointed == 2 * n_pos - 16            # every other call found its layout but not its addresses
+    c.close()
