@@ -85,6 +85,13 @@ typedef struct {
 #define GG_PARAMS_FITTED 0   /* penalty uses the (beta, alpha) fitted by this call: two reads of x */
 #define GG_PARAMS_GIVEN  1   /* penalty uses caller-supplied (beta, alpha); the fit of this call is
                                 still produced: one read of x                                    */
+#define GG_RATE_EG       2   /* no GG penalty: `grad` gets the gradient of lambda * R, R the mean
+                                Exponential-Golomb code length of order eg_k of the quantised symbols
+                                (Eq. 6-7, in the relaxed form of the gradient constrained training
+                                section, as gg_eg_rate_grad computes it), and penalty[s] = lambda * R of
+                                the histogram segment s counts into; the fit of this call is still
+                                produced: one read of x for moments, gradient and histogram.  Needs a
+                                histogram (hist != NULL) with GG_STEP_GIVEN.  gg_fused only           */
 #define GG_STEP_GIVEN      0 /* quantiser step[s] supplied by the caller                        */
 #define GG_STEP_FROM_ALPHA 1 /* step[s] = (float)(fitted alpha[s] * step_scale), also written out */
 
@@ -190,7 +197,7 @@ typedef struct {
     int64_t  *count;
     uint32_t *flags;
     /* penalty and gradient                                                                   */
-    int32_t       param_mode;    /* GG_PARAMS_FITTED or GG_PARAMS_GIVEN                       */
+    int32_t       param_mode;    /* GG_PARAMS_FITTED, GG_PARAMS_GIVEN or GG_RATE_EG           */
     const double *beta_in, *alpha_in;   /* device [n_seg], GG_PARAMS_GIVEN only               */
     double        lambda;
     int32_t       reduction;     /* GG_SUM or GG_MEAN                                         */
@@ -209,12 +216,15 @@ typedef struct {
     int32_t       accumulate_hist;
     double       *entropy_bits;  /* device [n_hist] or NULL                                   */
     uint64_t     *clamped_lo_hi; /* device [2*n_hist] or NULL                                 */
+    /* GG_RATE_EG only                                                                        */
+    int32_t       eg_k;          /* order of the Exponential-Golomb code, 0 .. 30             */
+    double       *eg_bits;       /* device [n_hist] or NULL: mean code length per histogram   */
 } gg_fused_args;
 
 /* The whole pass over a list of segments in the fewest sweeps of x: moments -> fit ->
  * penalty + gradient + histogram -> entropy, all enqueued on `stream`.
  * GG_PARAMS_FITTED reads x twice (the gradient needs the fit of the whole segment);
- * GG_PARAMS_GIVEN reads x once (moments, gradient and histogram in the same sweep).
+ * GG_PARAMS_GIVEN and GG_RATE_EG read x once (moments, gradient and histogram in the same sweep).
  * The first call with a new layout (segment addresses and lengths) builds and caches its plan with
  * blocking allocations; later calls with that layout only enqueue kernels and memsets on `stream`
  * and may be captured in a CUDA graph (the same holds for gg_fused_channels once its scratch is

@@ -173,7 +173,22 @@ def cases(ctx, dev, which=ALL):
                   timeit(lambda: ctx.gg_penalty_grad(segs, fit["beta"], fit["alpha"], 1e-4, grad=gsegs)), 6 * n)
         yield rec("call_rate_hist", "gg_rate_hist on them (one histogram per matrix, entropy)",
                   timeit(lambda: ctx.gg_rate_hist(segs, steps)), 2 * n)
-        del w, flat, g, segs, gsegs
+        # the training step of the paper's rate-constrained objective (loss + lambda * R, R the Exponential-Golomb
+        # code length of Eq. 6-7): gradient of the rate, histogram and rate of every matrix
+        from paper_2506_00486_b200 import GG_RATE_EG
+        run = ctx.make_fused(segs, grad=gsegs, lam=1e-4, step=steps, param_mode=GG_RATE_EG, eg_k=0)
+        yield rec("rate_step_fused", "gg_fused with GG_RATE_EG on them: fit, gradient of lambda * R, histogram, entropy and code length "
+                  "of every matrix from one read (fp32 gradients)", timeit(run), 6 * n)
+
+        hist = run.outputs["hist"]
+
+        def separate():
+            ctx.gg_eg_rate_grad(segs, steps, 1e-4, gsegs, k=0)
+            ctx.gg_rate_hist(segs, steps, hist=hist)
+            ctx.gg_eg_rate(hist, k=0)
+        yield rec("rate_step_separate", "the same from the single-step calls (gg_eg_rate_grad, gg_rate_hist, gg_eg_rate: two reads, no fit)",
+                  timeit(separate), 6 * n)
+        del w, flat, g, segs, gsegs, run
     if "channels" in which:
         for rows, cols, spread, dt in ((16384, 4096, 3, torch.bfloat16), (65536, 4096, 3, torch.bfloat16),
                                        (16384, 11008, 3, torch.bfloat16), (16384, 4096, 9, torch.bfloat16),

@@ -16,7 +16,7 @@ _LIB_PATH = os.environ.get("GG_B200_LIB") or os.path.join(_HERE, "libgg_b200.so"
 
 GG_F32, GG_BF16 = 0, 1
 GG_SUM, GG_MEAN = 0, 1
-GG_PARAMS_FITTED, GG_PARAMS_GIVEN = 0, 1
+GG_PARAMS_FITTED, GG_PARAMS_GIVEN, GG_RATE_EG = 0, 1, 2
 GG_STEP_GIVEN, GG_STEP_FROM_ALPHA = 0, 1
 FLAG_DEGENERATE, FLAG_BETA_CLAMPED_LO, FLAG_BETA_CLAMPED_HI, FLAG_NONFINITE, FLAG_CLAMPED_SYMBOLS = 1, 2, 4, 8, 16
 FLAG_TIMEOUT = 32
@@ -39,6 +39,7 @@ class FusedArgs(ctypes.Structure):
         ("step_mode", ctypes.c_int32), ("step", _P), ("step_scale", ctypes.c_double), ("step_out", _P),
         ("hist_id", _P), ("n_hist", ctypes.c_int32), ("qmin", ctypes.c_int32), ("qmax", ctypes.c_int32),
         ("hist", _P), ("accumulate_hist", ctypes.c_int32), ("entropy_bits", _P), ("clamped_lo_hi", _P),
+        ("eg_k", ctypes.c_int32), ("eg_bits", _P),
     ]
 
 
@@ -395,10 +396,12 @@ class Context:
     def make_fused(self, segs, grad=None, lam=1e-4, reduction=GG_SUM, accumulate_grad=False,
                    param_mode=GG_PARAMS_FITTED, beta_in=None, alpha_in=None, want_penalty=True,
                    step=None, step_scale=None, hist_id=None, n_hist=None, qmin=-32768, qmax=32767,
-                   want_hist=True, accumulate_hist=False, hist=None):
+                   want_hist=True, accumulate_hist=False, hist=None, eg_k=0):
         """Allocates the outputs of the fused pass once and returns a callable that enqueues it.
 
-        step: device float32 tensor [n_seg] (GG_STEP_GIVEN); or step_scale: float, step = alpha * scale."""
+        step: device float32 tensor [n_seg] (GG_STEP_GIVEN); or step_scale: float, step = alpha * scale.
+        param_mode=GG_RATE_EG: the gradient and penalty of the Exponential-Golomb rate of order eg_k (Eq. 6-7)
+        instead of the GG penalty; out["eg_bits"] holds the mean code length per histogram."""
         segs = _as_segments(segs)
         n = len(segs)
         gsegs = None if grad is None else _as_segments(grad)
@@ -437,6 +440,9 @@ class Context:
             a.n_hist, a.qmin, a.qmax = n_hist, int(qmin), int(qmax)
             a.hist, a.accumulate_hist = _ptr(hist), int(bool(accumulate_hist))
             a.entropy_bits, a.clamped_lo_hi = _ptr(out["entropy_bits"]), _ptr(out["clamped"])
+            if int(param_mode) == GG_RATE_EG:
+                out["eg_bits"] = self._new(n_hist, torch.float64)
+                a.eg_k, a.eg_bits = int(eg_k), _ptr(out["eg_bits"])
 
         def run():
             self._check(lib().gg_fused(self._h, ctypes.byref(a), _stream_ptr(self.device)))

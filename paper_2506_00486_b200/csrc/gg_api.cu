@@ -420,14 +420,21 @@ cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype gra
 }
 
 // Entropy of n_hist count tables; grows the context's scratch (blocking) the first time a call needs more.
-gg_status run_entropy(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
-                      cudaStream_t cs)
+gg_status ensure_entropy_scratch(gg_ctx *ctx, int32_t n_hist)
 {
     if (n_hist > ctx->ent_hists) {
         if (ctx->ent_part) { GG_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(ctx->ent_part); ctx->ent_part = nullptr; ctx->ent_hists = 0; }
         GG_CUDA(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->ent_part), sizeof(double) * 2 * kEntSplit * (size_t)n_hist));
         ctx->ent_hists = n_hist;
     }
+    return GG_OK;
+}
+
+gg_status run_entropy(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
+                      cudaStream_t cs)
+{
+    gg_status es = ensure_entropy_scratch(ctx, n_hist);
+    if (es != GG_OK) return es;
     GG_CUDA(ctx, launch_entropy(hist, n_hist, n_bins, entropy_bits, ctx->ent_part, cs));
     ctx->launches += 2;
     return GG_OK;
@@ -804,7 +811,8 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
     if (!ctx || !a) return GG_ERR_INVALID_ARG;
     const int32_t n_seg = a->n_seg;
     if (n_seg > 0 && (!a->beta || !a->alpha)) return GG_ERR_INVALID_ARG;
-    if (a->param_mode != GG_PARAMS_FITTED && a->param_mode != GG_PARAMS_GIVEN) return GG_ERR_INVALID_ARG;
+    if (a->param_mode != GG_PARAMS_FITTED && a->param_mode != GG_PARAMS_GIVEN && a->param_mode != GG_RATE_EG) return GG_ERR_INVALID_ARG;
+    const bool eg = a->param_mode == GG_RATE_EG;
     if (a->param_mode == GG_PARAMS_GIVEN && n_seg > 0 && (!a->beta_in || !a->alpha_in)) return GG_ERR_INVALID_ARG;
     if (a->reduction != GG_SUM && a->reduction != GG_MEAN) return GG_ERR_INVALID_ARG;
     if (a->step_mode != GG_STEP_GIVEN && a->step_mode != GG_STEP_FROM_ALPHA) return GG_ERR_INVALID_ARG;
@@ -814,6 +822,8 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             (a->param_mode != GG_PARAMS_FITTED || !a->step_out)) return GG_ERR_INVALID_ARG;
         if (a->step_mode == GG_STEP_GIVEN && n_seg > 0 && !a->step) return GG_ERR_INVALID_ARG;
     }
+    // the code-length rate is a function of the symbols: it needs the quantiser of the histogram step
+    if (eg && (!do_hist || a->step_mode != GG_STEP_GIVEN || a->eg_k < 0 || a->eg_k > 30)) return GG_ERR_INVALID_ARG;
     // A layout that has a plan was validated when the plan was built: a step that repeats a call pays for
     // three memory compares, not for a walk over its segments.
     gg_status st = GG_OK;
@@ -962,6 +972,17 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
                 ctx->launches += p->n_tiles > 0;
             }
             beta_used = a->beta;
+        } else if (eg) {
+            // one sweep: moments, the gradient of lambda * R (Eq. 7) and the histogram together; then the fit.  The
+            // rate itself comes from the histogram afterwards.
+            sa.step = a->step; sa.eg_k = a->eg_k;
+            {
+                SweepTimer tm(ctx, &ctx->ev_first, cs);
+                GG_CUDA(ctx, launch_sweep(ctx, kMoments | kHist | (a->grad ? kGrad | kEg : 0), in_dt, g_dt, a->grad != nullptr, sa, cs));
+            }
+            GG_CUDA(ctx, launch_fit(fa, cs));
+            ctx->launches += 1 + (p->n_tiles > 0);
+            beta_used = nullptr;
         } else {
             // one sweep: moments, gradient (given parameters) and histogram together; then the fit
             sa.beta = a->beta_in; sa.alpha = a->alpha_in; sa.step = a->step;
@@ -973,7 +994,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             ctx->launches += 1 + (p->n_tiles > 0);
             beta_used = a->beta_in;
         }
-        if (a->penalty && !small_path) {
+        if (a->penalty && !small_path && !eg) {
             GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta_used, a->penalty, cs));
             ctx->launches += 1;
         }
@@ -982,6 +1003,21 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
     if (do_hist && a->entropy_bits && a->n_hist > 0) {
         gg_status es = run_entropy(ctx, a->hist, a->n_hist, n_bins, a->entropy_bits, cs);
         if (es != GG_OK) return es;
+    }
+    if (eg && a->n_hist > 0 && (a->eg_bits || (a->penalty && n_seg > 0))) {
+        // mean code length of every histogram; the penalty of a segment is lambda times that of its histogram
+        double *bits = a->eg_bits;
+        if (bits == nullptr) {
+            gg_status es = ensure_entropy_scratch(ctx, a->n_hist);      // (free again once the entropy kernels above are done)
+            if (es != GG_OK) return es;
+            bits = ctx->ent_part;
+        }
+        GG_CUDA(ctx, launch_eg_rate(a->hist, a->n_hist, n_bins, a->qmin, a->eg_k, bits, cs));
+        ctx->launches += 1;
+        if (a->penalty && n_seg > 0) {
+            GG_CUDA(ctx, launch_eg_penalty(bits, p->map.hist_id, a->lambda, a->penalty, n_seg, cs));
+            ctx->launches += 1;
+        }
     }
     return GG_OK;
 }
@@ -1089,7 +1125,7 @@ gg_status gg_fused_host(gg_ctx *ctx, const gg_fused_args *a, int64_t chunk_bytes
     if (!ctx || !a) return GG_ERR_INVALID_ARG;
     const int32_t n_seg = a->n_seg;
     if (n_seg > 0 && (!a->beta || !a->alpha)) return GG_ERR_INVALID_ARG;
-    if (a->param_mode != GG_PARAMS_FITTED && a->param_mode != GG_PARAMS_GIVEN) return GG_ERR_INVALID_ARG;
+    if (a->param_mode != GG_PARAMS_FITTED && a->param_mode != GG_PARAMS_GIVEN) return GG_ERR_INVALID_ARG;      // (GG_RATE_EG: device buffers only)
     if (a->param_mode == GG_PARAMS_GIVEN && n_seg > 0 && (!a->beta_in || !a->alpha_in)) return GG_ERR_INVALID_ARG;
     if (a->step_mode != GG_STEP_GIVEN && a->step_mode != GG_STEP_FROM_ALPHA) return GG_ERR_INVALID_ARG;
     const bool do_hist = a->hist != nullptr;

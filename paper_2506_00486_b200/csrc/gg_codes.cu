@@ -194,6 +194,22 @@ __global__ void __launch_bounds__(kThreads) gct_step_kernel(const TileMap map, v
 
 }  // namespace
 
+namespace {
+__global__ void eg_penalty_kernel(const double *eg_bits, const int32_t *hist_id, double lambda, double *penalty, int32_t n_seg)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < n_seg) penalty[s] = lambda * eg_bits[hist_id[s]];
+}
+}  // namespace
+
+cudaError_t launch_eg_penalty(const double *eg_bits, const int32_t *hist_id, double lambda, double *penalty, int32_t n_seg,
+                              cudaStream_t st)
+{
+    if (n_seg <= 0) return cudaSuccess;
+    eg_penalty_kernel<<<(n_seg + 255) / 256, 256, 0, st>>>(eg_bits, hist_id, lambda, penalty, n_seg);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_eg_rate(const uint64_t *hist, int32_t n_hist, int32_t n_bins, int32_t qmin, int32_t k, double *eg_bits,
                            cudaStream_t st)
 {

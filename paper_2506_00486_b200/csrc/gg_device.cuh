@@ -60,6 +60,33 @@ __device__ __forceinline__ bool gg_in_bounds(long long i, long long n)
 #define GG_IN_BOUNDS(i, n) true
 #endif
 
+// ---- gradient of lambda * R, R the mean k-th order Exponential-Golomb code length of the quantised symbols (Eq. 6-7),
+// in the relaxed form of the gradient constrained training section: for an element x of a segment of N elements
+//     g = c * sign(x) / (Map(q) + 2^k),   c = lambda * 4 inv / (N ln 2),   q the (clamped) symbol of x,
+// and g = 0 where x is zero or nan.  Map is Eq. 6: 0, 1, -1, 2, -2, ... -> 0, 1, 2, 3, 4, ...
+// From the symbol: the reciprocal unit plus one Newton step (half an ulp), then the product with c.
+__device__ __forceinline__ float eg_grad_of_symbol(int q, float c, uint32_t two_k)
+{
+    const int n = -q;
+    const uint32_t m = ((uint32_t)n << 1) ^ (uint32_t)(n >> 31);      // q > 0: 2q - 1; q < 0: -2q; 0: 0
+    const float den = (float)(m + two_k);                              // exact below 2^24
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(den));
+    r = fmaf(r, fmaf(-den, r, 1.0f), r);
+    return c * r;
+}
+
+// The same for any fp32 bit pattern, with the quantiser written out (fp32 product, floor, clamp): the careful path.
+__device__ __forceinline__ float eg_grad_exact(uint32_t xb, float inv, int32_t qmin, int32_t qmax, float c, uint32_t two_k)
+{
+    const float x = __uint_as_float(xb);
+    const float t = __fmul_rn(x, inv);
+    if (!(t == t) || x == 0.0f) return 0.0f;
+    const int q = max(qmin, min(qmax, __float2int_rd(t)));             // floor, saturating, then the clamp
+    const float g = eg_grad_of_symbol(q, c, two_k);
+    return __uint_as_float(__float_as_uint(g) ^ (xb & 0x80000000u));
+}
+
 // Butterfly sum over the warp: every lane ends with the same bits.
 __device__ __forceinline__ double warp_sum(double v)
 {

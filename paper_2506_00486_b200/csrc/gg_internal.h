@@ -15,7 +15,9 @@ constexpr int kStreamThreads = 256;
 // (rare) rest goes straight to global memory.
 constexpr int kWindow = 4096;
 
-enum StreamFlags : int { kMoments = 1, kGrad = 2, kHist = 4 };
+// kEg (with kGrad and kHist): the gradient is that of lambda * R, R the mean Exponential-Golomb code length of the
+// quantised symbols (Eq. 6-7), instead of that of the GG penalty
+enum StreamFlags : int { kMoments = 1, kGrad = 2, kHist = 4, kEg = 8 };
 
 // Moments are summed in fp32 over a short run of elements and then added in fp64.  The fp32 sums m1 = sum |x|
 // and m2 = sum x^2 of a run can stand for the exact ones unless a square left the fp32 range: upwards
@@ -69,6 +71,7 @@ struct StreamArgs {
     // that no separate memset sits between two launches: 16-byte vectors, or null
     uint4 *zero_ptr;
     int64_t zero_vecs;
+    int32_t eg_k;        // order of the Exponential-Golomb code (kEg)
 };
 
 struct FitArgs {
@@ -218,6 +221,9 @@ cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part,
 constexpr int kEntSplit = 16;
 cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
                            double *scratch, cudaStream_t st);
+// penalty[s] = lambda * eg_bits[hist_id[s]] (hist_id: device array)
+cudaError_t launch_eg_penalty(const double *eg_bits, const int32_t *hist_id, double lambda, double *penalty, int32_t n_seg,
+                              cudaStream_t st);
 cudaError_t launch_eg_rate(const uint64_t *hist, int32_t n_hist, int32_t n_bins, int32_t qmin, int32_t k, double *eg_bits,
                            cudaStream_t st);
 cudaError_t launch_eg_grad(const TileMap &map, gg_dtype in_dtype, gg_dtype grad_dtype, const float *step, int32_t qmin,

@@ -64,6 +64,8 @@ struct Cold {
     unsigned long long *row;   // the current histogram, bin 0 = symbol qmin
     uint32_t c_base;           // first magnitude pattern of the pattern-count window
     int symbol_mode;           // layout of cnt: 1 = rows of symbols, 0 = cells of patterns
+    float eg_c;                // code-length gradient (kEg): the factor c of the segment
+    uint32_t eg_two_k;
 };
 
 struct ClusterPart {
@@ -199,6 +201,9 @@ struct Lane {
     uint32_t p_addr;   // pattern mode: cnt + (lane mod kRep) * 4
     float inv;         // quantiser scale (symbol mode)
     uint64_t inv2;     // the same twice, for the pair arithmetic
+    float eg_c;        // code-length gradient (kEg): c of the segment, 2^k, the clamp of the symbols
+    uint32_t eg_two_k;
+    int32_t qmin, qmax;
 };
 
 template <int FLAGS>
@@ -236,11 +241,18 @@ __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, 
     const uint32_t xb = HALF ? (w & 0xFFFF0000u) : (w << 16);     // the value as fp32 bits
     if constexpr (MOMENTS_HERE) moments_elem<FLAGS>(xb, acc, r);
     float ga = 0.0f;
-    if constexpr ((FLAGS & kGrad) != 0) {
+    constexpr bool EG = (FLAGS & kEg) != 0;
+    if constexpr ((FLAGS & kGrad) != 0 && !EG) {
         const uint32_t e4 = HALF ? ((w >> 21) & 0x3FCu) : ((w >> 5) & 0x3FCu);     // exponent field * 4
         const uint32_t j = HALF ? ((w >> 16) & 127u) : (w & 127u);
         const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(s_a1) + e4);
         ga = a * lds_f32(j * 128u + ln.b_addr);
+    }
+    if constexpr (EG && MODE != kModeSymbol) {
+        // (pattern counting does not form the symbol: the quantiser here; a nan gives no gradient)
+        const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
+        const int q = max(ln.qmin, min(ln.qmax, __float2int_rd(t)));
+        ga = (t == t) ? eg_grad_of_symbol(q, ln.eg_c, ln.eg_two_k) : 0.0f;
     }
     if constexpr ((FLAGS & kHist) != 0) {
         if constexpr (MODE == kModeSymbol) {
@@ -249,11 +261,16 @@ __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, 
             const float t = __fmul_rn(__uint_as_float(xb), ln.inv);
             // (one float maximum with an absolute-value operand; a nan is ignored here, which is right: it lands on
             // a sentinel row and is not to be counted)
-            anyc = __float_as_uint(fmaxf(__uint_as_float(anyc), fabsf(t)));
+            // (with the code-length gradient a nan must be found too, since its gradient is zero and not the sentinel
+            // row's: the maximum is then taken on the bit patterns, where a nan is the largest)
+            if constexpr (EG) anyc = max(anyc, __float_as_uint(fabsf(t)));
+            else anyc = __float_as_uint(fmaxf(__uint_as_float(anyc), fabsf(t)));
             const float tc = fminf(fmaxf(t, -(float)(kSymCells / 2) - 0.5f), (float)(kSymCells / 2));
             // for |t| < 2^22 the sum lies in [2^23, 2^24) where floats are the integers: rounding down gives floor
             const uint32_t fb = __float_as_uint(__fadd_rd(tc, __uint_as_float(kMagicBits)));
             red_inc(fb * 128u + ln.s_addr);     // (s_addr already holds minus 128 times the bits of symbol -kSymCells/2)
+            // (the symbols of the window are not clamped in this mode; an element outside it is redone by fix_elem)
+            if constexpr (EG) ga = eg_grad_of_symbol((int)(fb - kMagicBits), ln.eg_c, ln.eg_two_k);
         } else {
             static_assert(kRep == 2, "cell stride");
             const uint32_t mag = HALF ? ((w >> 16) & 0x7FFFu) : (w & 0x7FFFu);
@@ -264,7 +281,11 @@ __device__ __forceinline__ float one_elem(uint32_t w, const Lane &ln, Acc &acc, 
             red_inc(p * 16u + sign8 + ln.p_addr);
         }
     }
-    if constexpr ((FLAGS & kGrad) != 0) {
+    if constexpr (EG) {
+        // (no penalty partial: the rate comes from the histogram; zero has no gradient)
+        ga = (xb << 1) != 0u ? ga : 0.0f;
+        return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));
+    } else if constexpr ((FLAGS & kGrad) != 0) {
         r.mp = fmaf(fabsf(__uint_as_float(xb)), fabsf(ga), r.mp);
         return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
     }
@@ -329,7 +350,7 @@ template <int FLAGS, int MODE>
 __device__ __forceinline__ float fix_elem(uint32_t xb, float g, bool grad_bad, const Lane &ln, Smem &sm)
 {
     const uint32_t mag = (xb & 0x7FFFFFFFu) >> 16;
-    if constexpr ((FLAGS & kGrad) != 0) {
+    if constexpr ((FLAGS & kGrad) != 0 && (FLAGS & kEg) == 0) {
         if (grad_bad) {
             const float a = s_a1[mag >> 7];
             if (a != a) {     // this element read a NaN marker: zero needs no table, the rest the exact path
@@ -343,6 +364,10 @@ __device__ __forceinline__ float fix_elem(uint32_t xb, float g, bool grad_bad, c
         if constexpr (MODE == kModeSymbol) miss = symbol_row(xb, ln.inv) >= kSymCells;
         else miss = mag - ln.cbase >= kCntPat;
         if (miss) count_rare(xb, sm);
+        if constexpr ((FLAGS & kEg) != 0) {
+            // (symbol mode: the element missed the window, so its symbol was a sentinel's)
+            if (miss && MODE == kModeSymbol) g = eg_grad_exact(xb, ln.inv, ln.qmin, ln.qmax, ln.eg_c, ln.eg_two_k);
+        }
     }
     return g;
 }
@@ -382,7 +407,7 @@ __device__ __forceinline__ void close_run(const uint4 &raw, int n, Run &r, Acc &
             }
         }
     }
-    if constexpr ((FLAGS & kGrad) != 0) {
+    if constexpr ((FLAGS & kGrad) != 0 && (FLAGS & kEg) == 0) {
         // a product or a gradient that left the fp32 range, or a NaN marker, sends the run to fp64
         if (run_penalty(r) <= FLT_MAX) acc.pen += (double)run_penalty(r);
         else acc.pen += pen_rare(raw, n, sm);
@@ -575,7 +600,7 @@ __device__ __forceinline__ void process_vec(const uint4 &raw, TG *gdst, bool acc
         // (the pair arithmetic saves a tenth of the instructions: a gain where instruction issue binds, which is the
         // bf16-gradient variant; with fp32 gradients the sweep is bound by DRAM and the board's power limit, and
         // measured 0.4 % slower with it)
-        if constexpr (sizeof(TG) == 2) {
+        if constexpr (sizeof(TG) == 2 && (FLAGS & kEg) == 0) {
             two_elems<FLAGS, MODE>(w[i], ln, r, anyc, g[2 * i], g[2 * i + 1]);
         } else {
             g[2 * i] = one_elem<FLAGS, MODE, 0, false>(w[i], ln, acc, r, anyc);
@@ -743,7 +768,15 @@ __device__ __forceinline__ int setup_run(const StreamArgs &a, Smem &sm, CtaState
     int mode = kModePattern;
     bool active = false;
 
-    if constexpr (GRAD) {
+    if constexpr (GRAD && (FLAGS & kEg) != 0) {
+        // code-length gradient: one factor per segment (Eq. 7 relaxed), no tables
+        const float inv_s = (float)(1.0 / (double)param<COHERENT>(a.step + s));
+        ln.eg_c = (float)(a.lambda * 4.0 * (double)inv_s / ((double)len * 0.6931471805599453094));
+        ln.eg_two_k = 1u << a.eg_k;
+        ln.qmin = a.qmin;
+        ln.qmax = a.qmax;
+        if (tid == 0) { sm.cold.active = 0; sm.cold.sign_flip = 0u; sm.cold.L = 0.0; sm.cold.b = 0.0; }
+    } else if constexpr (GRAD) {
         const double beta = param<COHERENT>(a.beta + s), alpha = param<COHERENT>(a.alpha + s);
         const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
         active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
@@ -1245,6 +1278,7 @@ cudaError_t launch_typed(int flags, const StreamArgs &a, int sm_count, cudaStrea
     case kMoments | kGrad: return launch_one<TG, kMoments | kGrad>(a, sm_count, st);
     case kMoments | kHist: return launch_one<TG, kMoments | kHist>(a, sm_count, st);
     case kMoments | kGrad | kHist: return launch_one<TG, kMoments | kGrad | kHist>(a, sm_count, st);
+    case kMoments | kGrad | kHist | kEg: return launch_one<TG, kMoments | kGrad | kHist | kEg>(a, sm_count, st);
     default: return cudaErrorInvalidValue;
     }
 }

@@ -106,6 +106,9 @@ struct Lane {
     uint32_t c_addr;   // count address base: see one_elem
     float inv;         // quantiser scale
     float c1, c2, c3, c4;   // binomial coefficients of (1 + r)^b
+    float eg_c;        // code-length gradient (kEg): the factor c of the segment, 2^k, the clamp of the symbols
+    uint32_t eg_two_k;
+    int32_t qmin, qmax;
 };
 
 template <int MODE> struct Window;
@@ -133,7 +136,8 @@ __device__ __forceinline__ float one_elem(uint32_t xb, const Lane &ln, float &mp
         acc.xmin = fminf(acc.xmin, x);          // fminf / fmaxf return the non-NaN operand
         acc.xmax = fmaxf(acc.xmax, x);
     }
-    if constexpr ((FLAGS & kGrad) != 0) {
+    constexpr bool EG = (FLAGS & kEg) != 0;
+    if constexpr ((FLAGS & kGrad) != 0 && !EG) {
         const uint32_t ax = xb & 0x7FFFFFFFu;
         const float a = *reinterpret_cast<const float *>(reinterpret_cast<const char *>(s_a1) + ((ax >> 21) & 0x3FCu));
         const float bj = lds_f32(((ax >> 16) & 127u) * 128u + ln.b_addr);
@@ -146,13 +150,21 @@ __device__ __forceinline__ float one_elem(uint32_t xb, const Lane &ln, float &mp
     }
     if constexpr ((FLAGS & kHist) != 0) {
         const float t = __fmul_rn(x, ln.inv);
-        anyt = fmaxf(anyt, fabsf(t));           // (a nan leaves anyt alone; see count_miss)
+        // (a nan leaves anyt alone, see count_miss; with the code-length gradient it must be found, since its gradient
+        // is zero and not the sentinel's: the maximum is then taken on the bit patterns, where a nan is the largest)
+        if constexpr (EG) anyt = __uint_as_float(max(__float_as_uint(anyt), __float_as_uint(fabsf(t))));
+        else anyt = fmaxf(anyt, fabsf(t));
         // t clamped to just outside the window: the floor of the clamped value lands on a sentinel for
         // either tail (and for nan, which the maximum replaces by the lower bound)
         const float tc = fminf(fmaxf(t, -Window<MODE>::kHalf - 0.5f), Window<MODE>::kHalf);
         // for |t| < 2^22 the sum lies in [2^23, 2^24) where floats are the integers: rounding down gives floor
         const uint32_t fb = __float_as_uint(__fadd_rd(tc, __uint_as_float(kMagicBits)));
         red_inc((fb << Window<MODE>::kShift) + ln.c_addr);   // (c_addr holds minus the shifted bits of the first symbol)
+        if constexpr (EG) {
+            // the symbol of an element inside the window (one outside is redone by fix_elem); zero has no gradient
+            const int q = max(ln.qmin, min(ln.qmax, (int)(fb - kMagicBits)));
+            ga = (xb << 1) != 0u ? eg_grad_of_symbol(q, ln.eg_c, ln.eg_two_k) : 0.0f;
+        }
     }
     if constexpr ((FLAGS & kGrad) != 0)
         return __uint_as_float(__float_as_uint(ga) ^ (xb & 0x80000000u));   // the table carries lambda's sign
@@ -163,14 +175,14 @@ __device__ __forceinline__ float one_elem(uint32_t xb, const Lane &ln, float &mp
 // sentinel and, being skipped by the quantiser, needs no second count.  With a gradient it is
 // found through the penalty partial.)
 template <int MODE>
-__device__ __forceinline__ bool count_miss(float anyt) { return anyt >= Window<MODE>::kHalf; }
+__device__ __forceinline__ bool count_miss(float anyt) { return !(anyt < Window<MODE>::kHalf); }      // (a nan counts as a miss)
 
 // Redo of whatever part of an element the branch-free path could not do; g is the gradient from the
 // first pass.  grad_bad: the vector's penalty partial left the fp32 range.
 template <int FLAGS, int MODE>
 __device__ __forceinline__ float fix_elem(uint32_t xb, float g, bool grad_bad, const Lane &ln, Smem &sm, uint32_t (&clampc)[2])
 {
-    if constexpr ((FLAGS & kGrad) != 0) {
+    if constexpr ((FLAGS & kGrad) != 0 && (FLAGS & kEg) == 0) {
         if (grad_bad) {
             const float a = s_a1[(xb >> 23) & 0xFFu];
             if (a != a) {     // this element read a NaN marker
@@ -185,6 +197,9 @@ __device__ __forceinline__ float fix_elem(uint32_t xb, float g, bool grad_bad, c
         if (t >= Window<MODE>::kHalf || t < -Window<MODE>::kHalf) {
             const int c = count_global(xb, ln.inv, sm.cold.qmin, sm.cold.qmax, sm.cold.row);
             if (c) clampc[c - 1] += 1u;
+        }
+        if constexpr ((FLAGS & kEg) != 0) {
+            if (!(t < Window<MODE>::kHalf && t >= -Window<MODE>::kHalf)) g = eg_grad_exact(xb, ln.inv, ln.qmin, ln.qmax, ln.eg_c, ln.eg_two_k);
         }
     }
     return g;
@@ -321,7 +336,7 @@ __device__ __forceinline__ void process8(const uint4 &lo, const uint4 &hi, int n
             }
         }
     }
-    if constexpr (GRAD) {
+    if constexpr (GRAD && (FLAGS & kEg) == 0) {
         // a product or a gradient that left the fp32 range, or a NaN marker, sends the vector to fp64
         if (mp <= FLT_MAX) acc.pen += (double)mp;
         else acc.pen += pen_exact(lo, hi, n, sm.cold.L, sm.cold.b, sm.cold.active);
@@ -445,7 +460,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) tail_f32_kernel(const St
         const float *x = reinterpret_cast<const float *>(a.map.seg_ptr[s]) + off;
         int mode = kModeWords;
 
-        if constexpr (GRAD) {
+        if constexpr (GRAD && (FLAGS & kEg) != 0) {
+            // code-length gradient: one factor per segment (Eq. 7 relaxed), no tables
+            const float inv_s = (float)(1.0 / (double)a.step[s]);
+            ln.eg_c = (float)(a.lambda * 4.0 * (double)inv_s / ((double)len * 0.6931471805599453094));
+            ln.eg_two_k = 1u << a.eg_k;
+            ln.qmin = a.qmin;
+            ln.qmax = a.qmax;
+        } else if constexpr (GRAD) {
             const double beta = a.beta[s], alpha = a.alpha[s];
             const double lam = a.mean_reduction ? a.lambda / (double)len : a.lambda;
             const bool active = (beta > 0.0) && (alpha > 0.0) && (lam != 0.0) && (lam == lam);
@@ -620,6 +642,7 @@ cudaError_t launch_typed(int flags, const StreamArgs &a, int sm_count, cudaStrea
     case kMoments | kGrad: return launch_one<TG, kMoments | kGrad>(a, sm_count, st);
     case kMoments | kHist: return launch_one<TG, kMoments | kHist>(a, sm_count, st);
     case kMoments | kGrad | kHist: return launch_one<TG, kMoments | kGrad | kHist>(a, sm_count, st);
+    case kMoments | kGrad | kHist | kEg: return launch_one<TG, kMoments | kGrad | kHist | kEg>(a, sm_count, st);
     default: return cudaErrorInvalidValue;
     }
 }

@@ -103,3 +103,75 @@ def test_gct_step_parity_over_three_steps(ctx, g_dtype):
             assert ulp_distance(got_h, gh).max() <= 1
             assert ulp_distance(got_w, wn).max() <= 1
             h64[s], w64[s] = got_h.astype(np.float64), got_w.astype(np.float64)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("variant", ["coarse", "fine", "clamped"])
+def test_fused_pass_with_the_code_length_rate(ctx, dtype, variant):
+    """GG_RATE_EG: moments and fit, the gradient of lambda * R (Eq. 6-7), the histogram, its entropy and its mean code
+    length from ONE read of x.  Every output against the oracle's separate functions.  coarse: 192 (bf16) or 128
+    (fp32) steps reach 6.5 standard deviations, so the kernels count by symbol in lane-private rows; fine: they do
+    not; clamped: the symbols are cut to a narrow range inside the count window."""
+    from paper_2506_00486_b200 import GG_RATE_EG, Segments
+    rng = np.random.default_rng({"coarse": 51, "fine": 52, "clamped": 53}[variant])
+    spec = [(0.7, 0.02, 3 * TILE + 77), (1.0, 0.02, 5), (2.0, 0.02, 0), (1.3, 0.02, 2 * TILE), (0.9, 0.02, 40000)]
+    xs = [gg_synth.gg_host(rng, b, gg_synth_alpha(0.02, b), n, dtype) for b, a, n in spec]
+    xs[0][:6] = torch.tensor([0.0, -0.0, float("nan"), 1e-30, float("inf"), -7.5]).to(dtype)     # specials and a far outlier
+    xs[3][100] = float("-inf")
+    # the first segment starts two elements into its buffer (not on a 16-byte boundary)
+    buf = torch.zeros(xs[0].numel() + 8, dtype=dtype, device="cuda:0")
+    buf[2:2 + xs[0].numel()].copy_(xs[0])
+    xd = [buf[2:2 + xs[0].numel()]] + [x.to("cuda:0") for x in xs[1:]]
+    gd = [torch.full((x.numel() + 4,), 3.0, dtype=torch.float32, device="cuda:0")[2:2 + x.numel()] for x in xs]
+    step_val = {"coarse": 0.02 / 16, "fine": 0.02 / 3000, "clamped": 0.02 / 16}[variant]
+    qmin, qmax = (-50, 40) if variant == "clamped" else (-32768, 32767)
+    k, lam = (2, -0.3) if variant == "fine" else (0, 0.3)
+    steps = torch.full((len(xs),), step_val, dtype=torch.float32, device="cuda:0")
+    hid = [0, 1, 1, 2, 0]
+    out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=lam, step=steps, hist_id=hid, n_hist=3, qmin=qmin, qmax=qmax,
+                       param_mode=GG_RATE_EG, eg_k=k)
+    torch.cuda.synchronize()
+    nb = qmax - qmin + 1
+    ref_hist = np.zeros((3, nb), dtype=np.uint64)
+    ref_cl = np.zeros((3, 2), dtype=np.uint64)
+    step32 = steps[0].item()
+    for s, x in enumerate(xs):
+        xo = gg_synth.to_oracle(x)
+        b, a, s1, s2, n, fl = o.fit(xo)
+        assert (out["flags"][s].item() & 15) == fl
+        if not (fl & o.FLAG_DEGENERATE):
+            assert abs(out["beta"][s].item() / b - 1) <= 1e-5 and abs(out["alpha"][s].item() / a - 1) <= 1e-5
+        if x.numel():
+            ref = o.eg_rate_grad(xo, step32, lam, k, qmin, qmax)
+            assert_grad_close(gd[s].cpu().numpy(), ref, max_ulp=2)
+        o.quantise_hist(xo, step32, qmin, qmax, hist=ref_hist[hid[s]], clamped=ref_cl[hid[s]])
+    np.testing.assert_array_equal(out["hist"].cpu().numpy(), ref_hist.astype(np.int64))
+    np.testing.assert_array_equal(out["clamped"].cpu().numpy(), ref_cl.astype(np.int64))
+    for h in range(3):
+        assert abs(out["entropy_bits"][h].item() - o.entropy_bits(ref_hist[h])) <= 1e-9
+        bits = o.eg_rate_hist(ref_hist[h], k, qmin)
+        assert abs(out["eg_bits"][h].item() - bits) <= 1e-12 * max(1.0, bits)
+    for s in range(len(xs)):
+        want = lam * out["eg_bits"][hid[s]].item()
+        assert out["penalty"][s].item() == pytest.approx(want, rel=1e-15, abs=0.0)
+
+
+def gg_synth_alpha(sigma, beta):
+    from paper_2506_00486_b200 import gg_alpha_from_std
+    return gg_alpha_from_std(sigma, beta)
+
+
+def test_code_length_rate_mode_needs_a_histogram_with_a_given_step(ctx):
+    from paper_2506_00486_b200 import GG_RATE_EG, GGError
+    x = [torch.ones(4096, dtype=torch.bfloat16, device="cuda:0")]
+    before = ctx.launch_count
+    with pytest.raises(GGError) as e:
+        ctx.gg_fused(x, lam=0.1, want_hist=False, param_mode=GG_RATE_EG)
+    assert e.value.status == 1
+    with pytest.raises(GGError) as e:
+        ctx.gg_fused(x, lam=0.1, step_scale=0.1, param_mode=GG_RATE_EG)
+    assert e.value.status == 1
+    with pytest.raises(GGError) as e:
+        ctx.gg_fused(x, lam=0.1, step=torch.ones(1, device="cuda:0"), param_mode=GG_RATE_EG, eg_k=31)
+    assert e.value.status == 1
+    assert ctx.launch_count == before
