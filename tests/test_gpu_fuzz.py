@@ -1,8 +1,9 @@
 """Randomised parity of gg_fused over everything that decides which kernels run: element type, segment lengths from
 empty to 70 tiles (short-segment kernels, the two sweeps, the optional one-launch and cluster forms), alignment,
 gradient type, shared histograms, sum or mean, fitted or given parameters, steps given or taken from the fit, the sign
-of lambda, the clamp range.  Every case is compared with the fp64 oracle: fit, flags, gradient element by element,
-penalty, histogram, clamp counters, entropy; and no output may be written outside its buffer."""
+of lambda, the clamp range, the GG penalty or the code-length rate of Eq. 6-7.  Every case is compared with the fp64
+oracle: fit, flags, gradient element by element, penalty, histogram, clamp counters, entropy (and code length); and no
+output may be written outside its buffer."""
 import numpy as np
 import pytest
 import torch
@@ -20,7 +21,7 @@ TILE = 16384
 def test_fused_random_cases_over_every_option(seed0):
     import __graft_entry__ as entry
     entry.build()
-    from paper_2506_00486_b200 import GG_MEAN, GG_PARAMS_GIVEN, GG_SUM, Context, Segments
+    from paper_2506_00486_b200 import GG_MEAN, GG_PARAMS_GIVEN, GG_RATE_EG, GG_SUM, Context, Segments
     ctx = Context(0, guard=True)
     n_cases = 40
     failures = []
@@ -65,7 +66,12 @@ def test_fused_random_cases_over_every_option(seed0):
             giv = [(float(rng.uniform(0.4, 2.4)), 10.0 ** rng.uniform(-3, 0)) for _ in xs]
             kw.update(param_mode=GG_PARAMS_GIVEN, beta_in=torch.tensor([g[0] for g in giv], dtype=torch.float64, device="cuda:0"),
                       alpha_in=torch.tensor([g[1] for g in giv], dtype=torch.float64, device="cuda:0"))
-        desc = f"case {case} dtype={dtype} kind={kind} n_seg={n_seg} cap={cap} mis={misalign} gdt={gdt} given={given} step_alpha={step_alpha} lam={lam} res={resident} clu={cluster} q=({qmin},{qmax}) mean={mean}"
+        # (drawn from a generator of its own, so that the cases of the other options stay what they were)
+        rng_eg = np.random.default_rng(seed0 * 100000 + 50000 + case)
+        eg = (not given) and (not step_alpha) and rng_eg.random() < 0.3
+        eg_k = int(rng_eg.choice([0, 1, 4]))
+        if eg: kw.update(param_mode=GG_RATE_EG, eg_k=eg_k)
+        desc = f"case {case} eg={eg} dtype={dtype} kind={kind} n_seg={n_seg} cap={cap} mis={misalign} gdt={gdt} given={given} step_alpha={step_alpha} lam={lam} res={resident} clu={cluster} q=({qmin},{qmax}) mean={mean}"
         try:
             out = ctx.gg_fused(Segments(xd), **kw)
             torch.cuda.synchronize(); ctx.check_guards()
@@ -82,12 +88,15 @@ def test_fused_random_cases_over_every_option(seed0):
                 bu, au = (bg, ag) if giv is None else giv[s]
                 lam_s = lam / max(n, 1) if mean else lam
                 pen, g = o.penalty_grad(xo, bu, au, lam_s)
+                if eg:
+                    g = o.eg_rate_grad(xo, steps_used[s], lam, eg_k, qmin, qmax) if n else g
+                    pen = float("nan")       # (checked against the histogram's code length below)
                 got = gd[s].float().cpu().numpy().astype(np.float64) - 0.5 if False else None
                 # gradient written (not accumulated): compare
                 gg = gd[s].cpu()
                 if gdt == torch.float32:
                     fin = np.isfinite(g.astype(np.float32))
-                    d = ulp_distance(gg.numpy()[fin], g[fin]); assert d.size == 0 or d.max() <= 4, ("grad", s, int(d.max()))
+                    d = ulp_distance(gg.numpy()[fin], g[fin]); assert d.size == 0 or d.max() <= (2 if eg else 4), ("grad", s, int(d.max()))
                 else:
                     ref = o.round_to_bf16_bits(g).astype(np.int64); gb = gg.view(torch.int16).numpy().astype(np.int64) & 0xFFFF
                     fin = np.isfinite(g) & (np.abs(g) < 3e38)
@@ -100,6 +109,11 @@ def test_fused_random_cases_over_every_option(seed0):
                 assert np.array_equal(out["hist"].cpu().numpy(), ref_hist.astype(np.int64)), "hist"
                 assert np.array_equal(out["clamped"].cpu().numpy(), ref_cl.astype(np.int64)), "clamped"
                 for h in range(n_hist): assert abs(out["entropy_bits"][h].item() - o.entropy_bits(ref_hist[h])) <= 1e-9, "entropy"
+                if eg:
+                    for h in range(n_hist):
+                        bits = o.eg_rate_hist(ref_hist[h], eg_k, qmin)
+                        assert abs(out["eg_bits"][h].item() - bits) <= 1e-12 * max(1.0, bits), "eg_bits"
+                    for s in range(n_seg): assert out["penalty"][s].item() == lam * out["eg_bits"][hid[s]].item(), ("eg penalty", s)
         except AssertionError as e:
             failures.append((desc, str(e)))
     ctx.close()
