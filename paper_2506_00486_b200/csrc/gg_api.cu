@@ -80,7 +80,8 @@ struct gg_ctx {
     int64_t launches = 0;
     int64_t plan_builds = 0, plan_repoints = 0;
     std::string cuda_error;
-    double *ent_part = nullptr;   // scratch of the entropy kernels: 2 * kEntSplit doubles per histogram
+    double *ent_part = nullptr;   // scratch of the entropy step: 2 * kEntSplit doubles per histogram
+    uint32_t *ent_done = nullptr; // and one counter per histogram (zero between calls)
     int64_t ent_hists = 0;
     uint32_t *small_counts = nullptr;   // scratch of the short-segment kernel: one slot of count cells per CTA
     void *chan_buf = nullptr;     // scratch of gg_fused_channels (partials per row block and column)
@@ -423,8 +424,14 @@ cudaError_t launch_sweep(gg_ctx *ctx, int flags, gg_dtype in_dtype, gg_dtype gra
 gg_status ensure_entropy_scratch(gg_ctx *ctx, int32_t n_hist)
 {
     if (n_hist > ctx->ent_hists) {
-        if (ctx->ent_part) { GG_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(ctx->ent_part); ctx->ent_part = nullptr; ctx->ent_hists = 0; }
+        if (ctx->ent_part) {
+            GG_CUDA(ctx, cudaDeviceSynchronize());
+            cudaFree(ctx->ent_part); cudaFree(ctx->ent_done);
+            ctx->ent_part = nullptr; ctx->ent_done = nullptr; ctx->ent_hists = 0;
+        }
         GG_CUDA(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->ent_part), sizeof(double) * 2 * kEntSplit * (size_t)n_hist));
+        GG_CUDA(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->ent_done), sizeof(uint32_t) * (size_t)n_hist));
+        GG_CUDA(ctx, cudaMemset(ctx->ent_done, 0, sizeof(uint32_t) * (size_t)n_hist));
         ctx->ent_hists = n_hist;
     }
     return GG_OK;
@@ -435,8 +442,8 @@ gg_status run_entropy(gg_ctx *ctx, const uint64_t *hist, int32_t n_hist, int32_t
 {
     gg_status es = ensure_entropy_scratch(ctx, n_hist);
     if (es != GG_OK) return es;
-    GG_CUDA(ctx, launch_entropy(hist, n_hist, n_bins, entropy_bits, ctx->ent_part, cs));
-    ctx->launches += 2;
+    GG_CUDA(ctx, launch_entropy(hist, n_hist, n_bins, entropy_bits, ctx->ent_part, ctx->ent_done, cs));
+    ctx->launches += 1;
     return GG_OK;
 }
 
@@ -608,6 +615,7 @@ gg_status gg_destroy(gg_ctx *ctx)
     if (ctx->small_counts) cudaFree(ctx->small_counts);
     if (ctx->chan_buf) cudaFree(ctx->chan_buf);
     if (ctx->ent_part) cudaFree(ctx->ent_part);
+    if (ctx->ent_done) cudaFree(ctx->ent_done);
     delete ctx;
     return GG_OK;
 }
@@ -873,6 +881,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         if (a->clamped_lo_hi)
             GG_CUDA(ctx, cudaMemsetAsync(a->clamped_lo_hi, 0, sizeof(uint64_t) * 2 * (size_t)a->n_hist, cs));
     }
+    bool entropy_done = false;
     if (n_seg > 0) {
         const gg_dtype in_dt = (gg_dtype)a->in_dtype, g_dt = (gg_dtype)a->grad_dtype;
         const bool want_pg = a->grad != nullptr || a->penalty != nullptr;
@@ -994,13 +1003,22 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
             ctx->launches += 1 + (p->n_tiles > 0);
             beta_used = a->beta_in;
         }
-        if (a->penalty && !small_path && !eg) {
+        // the penalty sums of the segments and the entropy of the histograms: one launch for both
+        const bool pen_here = a->penalty && !small_path && !eg;
+        if (pen_here && do_hist && a->entropy_bits && a->n_hist > 0) {
+            gg_status es = ensure_entropy_scratch(ctx, a->n_hist);
+            if (es != GG_OK) return es;
+            GG_CUDA(ctx, launch_finish(p->map, p->part, beta_used, a->penalty, n_seg, a->hist, a->n_hist, n_bins, a->entropy_bits,
+                                       ctx->ent_part, ctx->ent_done, cs));
+            ctx->launches += 1;
+            entropy_done = true;
+        } else if (pen_here) {
             GG_CUDA(ctx, launch_penalty_finalize(p->map, p->part, beta_used, a->penalty, cs));
             ctx->launches += 1;
         }
         mark_used(p, cs);
     }
-    if (do_hist && a->entropy_bits && a->n_hist > 0) {
+    if (do_hist && a->entropy_bits && a->n_hist > 0 && !entropy_done) {
         gg_status es = run_entropy(ctx, a->hist, a->n_hist, n_bins, a->entropy_bits, cs);
         if (es != GG_OK) return es;
     }

@@ -219,8 +219,13 @@ cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part,
                                     double *penalty, cudaStream_t st);
 // scratch: 2 * kEntSplit * n_hist doubles
 constexpr int kEntSplit = 16;
+// The entropy of n_hist count tables and / or the penalty sums of n_pen segments in one launch.  scratch: 2 * kEntSplit
+// doubles per histogram; done: one counter per histogram, zero between calls (the kernel leaves them so).
+cudaError_t launch_finish(const TileMap &map, const TileScratch &part, const double *beta, double *penalty, int32_t n_pen,
+                          const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits, double *scratch,
+                          uint32_t *done, cudaStream_t st);
 cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
-                           double *scratch, cudaStream_t st);
+                           double *scratch, uint32_t *done, cudaStream_t st);
 // penalty[s] = lambda * eg_bits[hist_id[s]] (hist_id: device array)
 cudaError_t launch_eg_penalty(const double *eg_bits, const int32_t *hist_id, double lambda, double *penalty, int32_t n_seg,
                               cudaStream_t st);

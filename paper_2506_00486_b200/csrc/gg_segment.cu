@@ -58,11 +58,9 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
 
 // penalty[s] = (1/beta_s) * sum over the segment's tiles of sum |x| |g|
 //            = lambda_s * sum (|x|/alpha_s)^beta_s   since |x| |g| = lambda beta (|x|/alpha)^beta.
-__global__ void __launch_bounds__(kSegThreads)
-penalty_finalize_kernel(const TileMap map, const TileScratch part, const double *beta, double *penalty)
+__device__ __forceinline__ void penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta, double *penalty, int s)
 {
     __shared__ double shp[kSegThreads / 32];
-    const int s = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     double p = 0.0;
 #pragma unroll 4
@@ -80,13 +78,16 @@ penalty_finalize_kernel(const TileMap map, const TileScratch part, const double 
 // Entropy of a count table, H = log2 N - (1/N) sum_{c>0} c log2 c, in two steps so that one large
 // table keeps many SMs busy: kEntSplit CTAs per histogram each reduce a slice of the bins to
 // (sum c log2 c, sum c) in a fixed order, then one thread per histogram adds the slices in order.
+// The slices of a histogram need no second launch: the CTA that finishes a histogram's last slice (a ticket from an
+// atomic counter; nobody waits) adds all slices in their fixed order and writes the entropy, then puts the counter
+// back to zero for the next call.
 constexpr int kEntThreads = 256;
-__global__ void __launch_bounds__(kEntThreads)
-entropy_partial_kernel(const uint64_t *hist, int32_t n_bins, double *part)
+static_assert(kEntThreads == kSegThreads, "one launch serves both");
+__device__ __forceinline__ void entropy_slice(const uint64_t *hist, int32_t n_bins, double *part, uint32_t *done, double *entropy_bits, int block)
 {
     __shared__ double shAcc[kEntThreads / 32];
     __shared__ unsigned long long shTot[kEntThreads / 32];
-    const int h = blockIdx.x / kEntSplit, slice = blockIdx.x % kEntSplit;
+    const int h = block / kEntSplit, slice = block % kEntSplit;
     const uint64_t *row = hist + (int64_t)h * n_bins;
     const int per = (n_bins + kEntSplit - 1) / kEntSplit;
     const int k0 = slice * per, k1 = min(n_bins, k0 + per);
@@ -130,18 +131,27 @@ entropy_partial_kernel(const uint64_t *hist, int32_t n_bins, double *part)
         double ra = 0.0;
         unsigned long long rt = 0;
         for (int w = 0; w < kEntThreads / 32; ++w) { ra += shAcc[w]; rt += shTot[w]; }
-        part[2 * blockIdx.x] = ra;
-        part[2 * blockIdx.x + 1] = (double)rt;      // (exact below 2^53 symbols)
+        part[2 * block] = ra;
+        part[2 * block + 1] = (double)rt;      // (exact below 2^53 symbols)
+        __threadfence();
+        if (atomicAdd(done + h, 1u) == (uint32_t)(kEntSplit - 1)) {
+            __threadfence();
+            double sa = 0.0, st = 0.0;
+            for (int k = 0; k < kEntSplit; ++k) { sa += __ldcg(part + 2 * (h * kEntSplit + k)); st += __ldcg(part + 2 * (h * kEntSplit + k) + 1); }
+            entropy_bits[h] = st == 0.0 ? 0.0 : log2(st) - sa / st;
+            done[h] = 0u;
+        }
     }
 }
 
-__global__ void entropy_final_kernel(const double *part, int32_t n_hist, double *entropy_bits)
+// What follows the sweeps of a call, in one launch: the first n_ent CTAs take the entropy slices, the others one
+// segment's penalty sum each.
+__global__ void __launch_bounds__(kSegThreads)
+finish_kernel(const TileMap map, const TileScratch part, const double *beta, double *penalty, const uint64_t *hist, int32_t n_bins,
+              double *ent_part, uint32_t *ent_done, double *entropy_bits, int n_ent)
 {
-    const int h = blockIdx.x * blockDim.x + threadIdx.x;
-    if (h >= n_hist) return;
-    double ra = 0.0, rt = 0.0;
-    for (int s = 0; s < kEntSplit; ++s) { ra += part[2 * (h * kEntSplit + s)]; rt += part[2 * (h * kEntSplit + s) + 1]; }
-    entropy_bits[h] = rt == 0.0 ? 0.0 : log2(rt) - ra / rt;
+    if ((int)blockIdx.x < n_ent) entropy_slice(hist, n_bins, ent_part, ent_done, entropy_bits, (int)blockIdx.x);
+    else penalty_finalize(map, part, beta, penalty, (int)blockIdx.x - n_ent);
 }
 
 }  // namespace
@@ -153,23 +163,26 @@ cudaError_t launch_fit(const FitArgs &a, cudaStream_t st)
     return cudaGetLastError();
 }
 
-cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
-                                    double *penalty, cudaStream_t st)
+cudaError_t launch_finish(const TileMap &map, const TileScratch &part, const double *beta, double *penalty, int32_t n_pen,
+                          const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits, double *scratch,
+                          uint32_t *done, cudaStream_t st)
 {
-    if (map.n_seg <= 0) return cudaSuccess;
-    penalty_finalize_kernel<<<map.n_seg, kSegThreads, 0, st>>>(map, part, beta, penalty);
+    const int n_ent = n_hist > 0 ? n_hist * kEntSplit : 0;
+    if (n_ent + n_pen <= 0) return cudaSuccess;
+    finish_kernel<<<n_ent + n_pen, kSegThreads, 0, st>>>(map, part, beta, penalty, hist, n_bins, scratch, done, entropy_bits, n_ent);
     return cudaGetLastError();
 }
 
-cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
-                           double *scratch, cudaStream_t st)
+cudaError_t launch_penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta,
+                                    double *penalty, cudaStream_t st)
 {
-    if (n_hist <= 0) return cudaSuccess;
-    entropy_partial_kernel<<<n_hist * kEntSplit, kEntThreads, 0, st>>>(hist, n_bins, scratch);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    entropy_final_kernel<<<(n_hist + 127) / 128, 128, 0, st>>>(scratch, n_hist, entropy_bits);
-    return cudaGetLastError();
+    return launch_finish(map, part, beta, penalty, map.n_seg, nullptr, 0, 0, nullptr, nullptr, nullptr, st);
+}
+
+cudaError_t launch_entropy(const uint64_t *hist, int32_t n_hist, int32_t n_bins, double *entropy_bits,
+                           double *scratch, uint32_t *done, cudaStream_t st)
+{
+    return launch_finish(TileMap{}, TileScratch{}, nullptr, nullptr, 0, hist, n_hist, n_bins, entropy_bits, scratch, done, st);
 }
 
 }  // namespace gg

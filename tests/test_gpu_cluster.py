@@ -12,8 +12,8 @@ from test_gpu_parity import TILE, check_fused, dev, misaligned_views
 
 pytestmark = pytest.mark.gpu
 
-CLUSTER_LAUNCHES = 4      # the pass, the penalty sums, two entropy kernels
-SWEEP_LAUNCHES = 6        # moments, fit, second sweep, the penalty sums, two entropy kernels
+CLUSTER_LAUNCHES = 2      # the pass; the penalty sums and the entropy together
+SWEEP_LAUNCHES = 4        # moments, fit, second sweep; the penalty sums and the entropy together
 
 
 @pytest.fixture()

@@ -481,7 +481,7 @@ def test_fused_given_parameters_single_sweep(ctx, dtype):
     torch.cuda.synchronize()
     check_fused(out, xs, gd, 1e-4, list(range(n)), n, given=given, qmin=-64, qmax=63)
     assert (out["flags"].cpu().numpy() & 16).any()       # the narrow clamp was reported
-    assert ctx.launch_count - launches0 == 5             # ONE sweep, then the fit, the penalty sums and two entropy kernels
+    assert ctx.launch_count - launches0 == 3             # ONE sweep, then the fit, then the penalty sums and the entropy together
 
 
 def test_fused_given_parameters_fp32_moments_of_special_values(ctx):
