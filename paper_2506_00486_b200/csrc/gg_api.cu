@@ -642,7 +642,7 @@ gg_status gg_fit(gg_ctx *ctx, const gg_seg *segs, int32_t n_seg, gg_dtype dtype,
     FitArgs fa{};
     fa.map = p->map; fa.part = p->part;
     fa.beta = beta; fa.alpha = alpha; fa.sum_abs = sum_abs; fa.sum_sq = sum_sq;
-    fa.count = count; fa.flags = flags; fa.seed = ctx->seed;
+    fa.count = count; fa.flags = flags; fa.seed = ctx->seed; fa.in_dtype_plus1 = (int)dtype + 1;
     GG_CUDA(ctx, launch_fit(fa, cs));
     ctx->launches += 1;
     mark_used(p, cs);
@@ -894,7 +894,7 @@ gg_status gg_fused(gg_ctx *ctx, const gg_fused_args *a, void *stream)
         FitArgs fa{};
         fa.map = p->map; fa.part = p->part;
         fa.beta = a->beta; fa.alpha = a->alpha; fa.sum_abs = a->sum_abs; fa.sum_sq = a->sum_sq;
-        fa.count = a->count; fa.flags = a->flags; fa.seed = ctx->seed;
+        fa.count = a->count; fa.flags = a->flags; fa.seed = ctx->seed; fa.in_dtype_plus1 = a->in_dtype + 1;
         fa.step_from_alpha = do_hist && a->step_mode == GG_STEP_FROM_ALPHA;
         fa.step_scale = a->step_scale; fa.step_out = a->step_out;
         fa.hist_on = do_hist; fa.step = a->step; fa.qmin = a->qmin; fa.qmax = a->qmax;

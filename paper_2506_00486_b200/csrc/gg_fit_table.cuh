@@ -97,6 +97,40 @@ __device__ __forceinline__ uint32_t fit_from_sums(double s1, double s2, int64_t 
     return flags;
 }
 
+// Flat-topped data make the fit ill-conditioned: d ln(beta) / d ln(rho) grows from 4 at beta = 2 to 150 at beta = 20, so
+// above rho(4) = 1/sqrt(2) the last bits of the fp32 run sums that the sweeps feed into their fp64 partials (about 1e-7
+// relative for a segment of a single run) would show in the fifth digit of beta.  In a long segment those roundings
+// average out; for a short one the warp that fits takes the two sums again in fp64 straight from the elements (at most
+// kCarefulLen of them: a microsecond or two, and rare), in a fixed order, non-finite entries left out as everywhere.
+constexpr int64_t kCarefulLen = 8192;
+constexpr double kCarefulLogRatio = -0.34657359027997264;      // ln rho(4) = -ln(2) / 2
+
+// WARP: all 32 lanes call with the same arguments and end with the same sums.
+__device__ __forceinline__ void careful_sums(const void *ptr, int in_dtype, int64_t len, int lane, double &s1, double &s2)
+{
+    double t1 = 0.0, t2 = 0.0;
+    if (in_dtype == GG_F32) {
+        const float *x = static_cast<const float *>(ptr);
+        for (int64_t i = lane; i < len; i += 32) {
+            const uint32_t ab = __float_as_uint(__ldg(x + i)) & 0x7FFFFFFFu;
+            if (ab < 0x7F800000u) { const double ax = (double)__uint_as_float(ab); t1 += ax; t2 = fma(ax, ax, t2); }
+        }
+    } else {
+        const uint16_t *x = static_cast<const uint16_t *>(ptr);
+        for (int64_t i = lane; i < len; i += 32) {
+            const uint32_t h = (uint32_t)__ldg(x + i) & 0x7FFFu;
+            if (h < 0x7F80u) { const double ax = (double)__uint_as_float(h << 16); t1 += ax; t2 = fma(ax, ax, t2); }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, o);
+        t2 += __shfl_xor_sync(0xFFFFFFFFu, t2, o);
+    }
+    s1 = t1;
+    s2 = t2;
+}
+
 // ln of rho(beta) = Gamma(2/beta)^2 / (Gamma(1/beta) Gamma(3/beta)), the ratio (E|x|)^2 / E[x^2]
 // of the density of Eq. 1; increasing in beta from 0 to 3/4.
 __device__ __forceinline__ double log_rho(double beta)
@@ -126,8 +160,14 @@ __device__ __forceinline__ FitResult fit_finish(const FitArgs &a, int s, int lan
     if (len <= 0 || !(s2 > 0.0)) {
         flags |= GG_FLAG_DEGENERATE;
     } else {
-        const double m1 = s1 / (double)len, m2 = s2 / (double)len;
-        const double log_r = log(m1 * m1 / m2);
+        double m1 = s1 / (double)len, m2 = s2 / (double)len;
+        double log_r = log(m1 * m1 / m2);
+        if (log_r > kCarefulLogRatio && len <= kCarefulLen && a.in_dtype_plus1 != 0) {
+            careful_sums(a.map.seg_ptr[s], a.in_dtype_plus1 - 1, len, lane, s1, s2);
+            m1 = s1 / (double)len;
+            m2 = s2 / (double)len;
+            log_r = log(m1 * m1 / m2);
+        }
         if (a.seed != nullptr) {
             // table look-up and cubic interpolation (no lgamma at fit time)
             double lnz;

@@ -85,6 +85,7 @@ struct FitArgs {
     int step_from_alpha;
     double step_scale;
     float *step_out;
+    int in_dtype_plus1;       // element type of the segments + 1 (gg_dtype), or 0 when the fit cannot read them again
     // when a histogram is part of the call: GG_FLAG_CLAMPED_SYMBOLS from the segment's extremes
     int hist_on;
     const float *step;

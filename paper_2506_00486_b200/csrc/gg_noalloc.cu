@@ -153,7 +153,7 @@ gg_status gg_fit_noalloc(int device, const void *x, int64_t len, gg_dtype dtype,
     fa.map = map;
     fa.part = part;
     fa.beta = beta; fa.alpha = alpha; fa.sum_abs = sum_abs; fa.sum_sq = sum_sq;
-    fa.count = count; fa.flags = flags;
+    fa.count = count; fa.flags = flags; fa.in_dtype_plus1 = (int)dtype + 1;
     e = launch_fit(fa, cs);
     if (e != cudaSuccess) { cudaGetLastError(); return GG_ERR_CUDA; }
     return GG_OK;

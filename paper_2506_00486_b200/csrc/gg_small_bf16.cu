@@ -394,8 +394,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) small_bf16_kernel(const 
         if (len <= 0 || !(s2 > 0.0)) {
             flags |= GG_FLAG_DEGENERATE;
         } else {
-            const double m1 = s1 / (double)len, m2 = s2 / (double)len;
-            const double log_r = log(m1 * m1 / m2);
+            double m1 = s1 / (double)len, m2 = s2 / (double)len;
+            double log_r = log(m1 * m1 / m2);
+            if (log_r > kCarefulLogRatio && len <= kCarefulLen) {      // (an ill-conditioned fit: the sums again in fp64)
+                careful_sums(a.map.seg_ptr[s], (int)GG_BF16, len, lane, s1, s2);
+                m1 = s1 / (double)len;
+                m2 = s2 / (double)len;
+                log_r = log(m1 * m1 / m2);
+            }
             double lnz;
             if (log_r <= __ldg(a.seed)) {
                 beta = GG_BETA_LO;

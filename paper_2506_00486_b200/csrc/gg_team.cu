@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) team_kernel(const SmallA
     FitArgs fa{};
     fa.map = a.map;
     fa.beta = a.beta; fa.alpha = a.alpha; fa.sum_abs = a.sum_abs; fa.sum_sq = a.sum_sq; fa.count = a.count; fa.flags = a.flags;
-    fa.seed = a.seed;
+    fa.seed = a.seed; fa.in_dtype_plus1 = (int)GG_F32 + 1;
     fa.step_from_alpha = HISTK && a.do_hist && a.step_from_alpha; fa.step_scale = a.step_scale; fa.step_out = a.step_out;
     fa.hist_on = HISTK && a.do_hist; fa.step = (HISTK && a.do_hist && !a.step_from_alpha) ? a.step : nullptr;
     fa.qmin = a.qmin; fa.qmax = a.qmax;

@@ -813,3 +813,35 @@ def test_one_layout_at_many_addresses_reuses_its_plans(ctx):
     assert built == 16 + 1                        # the layout's plans and the other layout's one
     assert repointed == 2 * n_pos - 16            # every other call found its layout but not its addresses
     c.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("path", ["sweeps", "short"])
+def test_fit_of_short_flat_topped_segments(ctx, dtype, path):
+    """Few elements of similar magnitude: the moment ratio lies just below 3/4, where beta is 10 .. 20 and moves by
+    up to 150 times the relative change of the ratio, so the sums have to be right to the last bits of fp64, not of
+    the fp32 run sums that suffice elsewhere.  Thousands of such segments, so that the unlucky roundings occur; with
+    one long segment in the list they take the sweeps and the fit kernel, without it the short-segment kernels."""
+    rng = np.random.default_rng(61 + (path == "short"))
+    n_seg = 3000
+    lens = [int(rng.integers(6, 48)) for _ in range(n_seg)]
+    if path == "sweeps":
+        lens[7] = 20000
+    xs = [gg_synth.gg_host(rng, float(rng.uniform(9.0, 19.0)), 10.0 ** rng.uniform(-3, 2), n, dtype) for n in lens]
+    flat = torch.cat(xs).to("cuda:0")
+    offs = np.concatenate([[0], np.cumsum(lens)])
+    xd = [flat[offs[s]:offs[s + 1]] for s in range(n_seg)]
+    fit = ctx.gg_fit(xd)
+    out = ctx.gg_fused(xd, lam=1e-4, step=torch.full((n_seg,), 2.0 ** -6, dtype=torch.float32, device="cuda:0"),
+                       hist_id=[0] * n_seg, n_hist=1)
+    torch.cuda.synchronize()
+    res = {k: (fit[k].cpu().numpy(), out[k].cpu().numpy()) for k in ("beta", "alpha", "flags")}
+    large = 0
+    for s, x in enumerate(xs):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(x))
+        large += 8.0 < b < 20.0
+        for which in (0, 1):
+            assert (int(res["flags"][which][s]) & 15) == fl, (s, which)
+            assert_rel(float(res["beta"][which][s]), b, REL_FIT, f"beta[{s}] of call {which}")
+            assert_rel(float(res["alpha"][which][s]), a, REL_FIT, f"alpha[{s}] of call {which}")
+    assert large >= 150                 # (the case is what it says; most of the others clamp at 20)
