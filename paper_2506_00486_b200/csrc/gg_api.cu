@@ -1084,7 +1084,7 @@ gg_status gg_fused_channels(gg_ctx *ctx, const gg_channel_args *a, void *stream)
         const bool want_pg = a->grad != nullptr || a->penalty != nullptr;
         ChanArgs ka{};
         ka.x = static_cast<const uint16_t *>(a->x);
-        ka.rows = a->rows; ka.cols = a->cols; ka.ld = a->ld;
+        ka.rows = a->rows; ka.cols = a->cols; ka.ld = a->ld; ka.in_f32 = f32 ? 1 : 0;
         ka.grad = a->grad; ka.grad_ld = a->grad_ld; ka.accumulate = a->accumulate_grad;
         ka.n_mom_blocks = (int32_t)n_mom;
         ka.n_slices = chan_slices(a->rows, a->cols, ctx->sm_count, f32 ? kChanStripF32 : kChanStrip);

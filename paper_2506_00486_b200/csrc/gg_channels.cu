@@ -214,6 +214,7 @@ __global__ void __launch_bounds__(kFitCols * kFitGroups) chan_fit_kernel(const C
     __shared__ double r1[kFitGroups][kFitCols], r2[kFitGroups][kFitCols];
     __shared__ uint32_t rb[kFitGroups][kFitCols];
     __shared__ float rmn[kFitGroups][kFitCols], rmx[kFitGroups][kFitCols];
+    __shared__ int need[kFitCols];
     const int cx = threadIdx.x % kFitCols, grp = threadIdx.x / kFitCols;
     const int64_t c = (int64_t)blockIdx.x * kFitCols + cx;
     double s1 = 0.0, s2 = 0.0;
@@ -229,10 +230,44 @@ __global__ void __launch_bounds__(kFitCols * kFitGroups) chan_fit_kernel(const C
     }
     r1[grp][cx] = s1; r2[grp][cx] = s2; rb[grp][cx] = bad; rmn[grp][cx] = xmin; rmx[grp][cx] = xmax;
     __syncthreads();
-    if (grp != 0 || c >= a.cols) return;
-    for (int g = 1; g < kFitGroups; ++g) {
-        s1 += r1[g][cx]; s2 += r2[g][cx]; bad += rb[g][cx];
-        xmin = fminf(xmin, rmn[g][cx]); xmax = fmaxf(xmax, rmx[g][cx]);
+    const bool lead = grp == 0 && c < a.cols;
+    if (grp == 0) need[cx] = 0;
+    if (lead) {
+        for (int g = 1; g < kFitGroups; ++g) {
+            s1 += r1[g][cx]; s2 += r2[g][cx]; bad += rb[g][cx];
+            xmin = fminf(xmin, rmn[g][cx]); xmax = fmaxf(xmax, rmx[g][cx]);
+        }
+        // an ill-conditioned fit of a short column (see careful_sums): its sums again in fp64, by the column's 16 threads
+        if (a.rows > 0 && a.rows <= kCarefulLen && s2 > 0.0) {
+            const double m1 = s1 / (double)a.rows, m2 = s2 / (double)a.rows;
+            need[cx] = log(m1 * m1 / m2) > kCarefulLogRatio;
+        }
+    }
+    __syncthreads();
+    if (c < a.cols && need[cx]) {
+        double t1 = 0.0, t2 = 0.0;
+        for (int64_t r = grp; r < a.rows; r += kFitGroups) {
+            double ax;
+            bool fin;
+            if (a.in_f32) {
+                const uint32_t ab = __float_as_uint(__ldg(reinterpret_cast<const float *>(a.x) + r * a.ld + c)) & 0x7FFFFFFFu;
+                fin = ab < 0x7F800000u;
+                ax = (double)__uint_as_float(ab);
+            } else {
+                const uint32_t h = (uint32_t)__ldg(a.x + r * a.ld + c) & 0x7FFFu;
+                fin = h < 0x7F80u;
+                ax = (double)__uint_as_float(h << 16);
+            }
+            if (fin) { t1 += ax; t2 = fma(ax, ax, t2); }
+        }
+        r1[grp][cx] = t1;
+        r2[grp][cx] = t2;
+    }
+    __syncthreads();
+    if (!lead) return;
+    if (need[cx]) {
+        s1 = r1[0][cx]; s2 = r2[0][cx];
+        for (int g = 1; g < kFitGroups; ++g) { s1 += r1[g][cx]; s2 += r2[g][cx]; }
     }
     double beta, alpha;
     uint32_t flags = fit_from_sums(s1, s2, a.rows, a.seed, &beta, &alpha) | (bad ? GG_FLAG_NONFINITE : 0u);

@@ -180,6 +180,7 @@ constexpr int kChanMomRows = 512;
 constexpr int kChanTabFloats = 2 * 65 * 32 + 2 * 128 * 32;   // A (64 exponents + marker row) and B (128 mantissas), two columns per lane     // rows per CTA of the moments kernel
 struct ChanArgs {
     const uint16_t *x;                 // (fp32 kernels read it as float)
+    int in_f32;                        // the elements are fp32 (ld counts elements of that type)
     int64_t rows, cols, ld;
     void *grad;                        // may be null
     int64_t grad_ld;

@@ -234,3 +234,25 @@ def test_channels_random_shapes_and_alignments(ctx, dtype):
         out = ctx.gg_fused_channels(xd, grad=gd, lam=3e-4, step=step, qmin=-5000, qmax=4000)
         torch.cuda.synchronize()
         check_channels(cpu(out), x, gd.cpu(), 3e-4, step=step, qmin=-5000, qmax=4000)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_channels_short_flat_topped_columns(ctx, dtype):
+    """Columns of a few dozen rows with flat-topped data: beta between 10 and 20, where it moves by up to 150 times the
+    relative change of the moment ratio.  The fit then needs the column sums to the last bits of fp64 (the fit kernel
+    takes them again from the elements); checked on 3000 columns, so that the unlucky roundings occur."""
+    rng = np.random.default_rng(71)
+    rows, cols = 40, 3000
+    x = torch.empty((rows, cols), dtype=dtype)
+    for c in range(cols):
+        x[:, c] = gg_synth.gg_host(rng, float(rng.uniform(9.0, 19.0)), 10.0 ** rng.uniform(-3, 2), rows, dtype)
+    out = cpu(ctx.gg_fused_channels(x.to("cuda:0"), lam=1e-4, step=2.0 ** -6))
+    torch.cuda.synchronize()
+    large = 0
+    for c in range(cols):
+        b, a, s1, s2, n, fl = o.fit(gg_synth.to_oracle(x[:, c].contiguous()))
+        large += 8.0 < b < 20.0
+        assert (out["flags"][c].item() & 15) == fl, f"flags[{c}]"
+        assert_rel(out["beta"][c].item(), b, REL_FIT, f"beta[{c}]")
+        assert_rel(out["alpha"][c].item(), a, REL_FIT, f"alpha[{c}]")
+    assert large >= 150
