@@ -32,9 +32,10 @@
  *    needs more histogram or channel scratch than any before it reallocates that scratch after
  *    waiting for the device.  A context serves one stream at a time.
  *  - A segment is a contiguous run of `len` elements.  Pointers need only element alignment;
- *    16-byte aligned segments take the vectorised path.  Long segments stream fastest when the
- *    gradient starts on a 1 KB boundary (a warp then writes whole 1 KB blocks): a gradient buffer
- *    that is only 256-byte aligned measured 5 % slower on the 7B-sized sweep.
+ *    16-byte aligned segments take the vectorised path.  Long segments stream fastest when input
+ *    and gradient sit at the same element offset from a 1 KB boundary (slices of aligned buffers
+ *    do): the kernels then start their vector body where both begin a block.  Unrelated offsets
+ *    of the two measured up to 6 % slower on the 7B-sized sweep.
  *  - Per-segment conditions are reported in `flags` (GG_FLAG_*), never as an error status.
  */
 #ifndef GG_B200_H

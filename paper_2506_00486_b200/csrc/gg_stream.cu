@@ -308,6 +308,9 @@ __global__ void __launch_bounds__(kThreads) stream_kernel(const StreamArgs a)
     int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / sizeof(TIn));
     head = min(head, n);
     if (gout != nullptr && (reinterpret_cast<uintptr_t>(gout + head) & 15u) != 0) head = n;
+    // (the body starts a 512-byte block of the gradient, or of x when there is none)
+    else head = (int)aligned_head(head, n, reinterpret_cast<uintptr_t>(x), reinterpret_cast<uintptr_t>(gout), (unsigned)sizeof(TIn),
+                                  (unsigned)sizeof(TG), 512u);
     const int nvec = (n - head) / KV;
     const int tail0 = head + nvec * KV;
     const bool accumulate = GRAD && a.accumulate != 0;
@@ -429,7 +432,7 @@ __global__ void __launch_bounds__(kThreads) moments_bf16_kernel(const StreamArgs
     const int n = (int)min((int64_t)kTile, len - off);
     const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
     int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
-    head = min(head, n);
+    head = (int)aligned_head(head, n, reinterpret_cast<uintptr_t>(x), 0ull, 2u, 0u, 512u);      // (the body starts a 512-byte block of x)
     const int nvec = (n - head) / 8;
     const int tail0 = head + nvec * 8;
 
@@ -576,7 +579,7 @@ __global__ void __launch_bounds__(kSweepThreads, kSweepCtasPerSm) moments_bf16_s
         const int64_t n = min(len, (int64_t)(t_stop - t_first) * kTile) - off;
         const uint16_t *x = reinterpret_cast<const uint16_t *>(a.map.seg_ptr[s]) + off;
         int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
-        head = min(head, n);
+        head = aligned_head(head, n, reinterpret_cast<uintptr_t>(x), 0ull, 2u, 0u, 512u);      // (the body starts a 512-byte block of x)
         const int nv = (int)((n - head) / 8);      // (a CTA's run never exceeds device memory / grid size elements)
         const int64_t tail0 = head + (int64_t)nv * 8;
 

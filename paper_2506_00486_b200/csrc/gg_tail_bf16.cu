@@ -673,6 +673,9 @@ __device__ __forceinline__ void process_range(const uint16_t *x, TG *gout, int64
     int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 2u);
     head = min(head, n);
     if (gout != nullptr && (reinterpret_cast<uintptr_t>(gout + head) & 15u) != 0) head = n;
+    // (the body starts a block of the gradient: 1 KB of fp32 or 512 bytes of bf16 per warp step; without a gradient, of x)
+    else head = aligned_head(head, n, reinterpret_cast<uintptr_t>(x), reinterpret_cast<uintptr_t>(gout), 2u, (unsigned)sizeof(TG),
+                             gout != nullptr ? 256u * (unsigned)sizeof(TG) : 512u);
     const int64_t nvec = (n - head) / 8;
     const int64_t tail0 = head + nvec * 8;
 

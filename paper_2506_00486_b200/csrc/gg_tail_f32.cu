@@ -355,6 +355,9 @@ __device__ __forceinline__ void process_range(const float *x, TG *gout, int64_t 
     int64_t head = (int64_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 4u);
     head = min(head, n);
     if (gout != nullptr && (reinterpret_cast<uintptr_t>(gout + head) & 15u) != 0) head = n;
+    // (the body starts a block of the gradient, or of x when there is none: what a warp moves per step)
+    else head = aligned_head(head, n, reinterpret_cast<uintptr_t>(x), reinterpret_cast<uintptr_t>(gout), 4u, (unsigned)sizeof(TG),
+                             gout != nullptr ? 256u * (unsigned)sizeof(TG) : 1024u);
     const int64_t nvec = (n - head) / 8;          // units of eight elements
     const int64_t tail0 = head + nvec * 8;
 

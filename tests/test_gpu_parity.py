@@ -845,3 +845,35 @@ def test_fit_of_short_flat_topped_segments(ctx, dtype, path):
             assert_rel(float(res["beta"][which][s]), b, REL_FIT, f"beta[{s}] of call {which}")
             assert_rel(float(res["alpha"][which][s]), a, REL_FIT, f"alpha[{s}] of call {which}")
     assert large >= 150                 # (the case is what it says; most of the others clamp at 20)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_fused_segments_that_start_off_the_block_boundaries(ctx, dtype):
+    """The vector body of a run starts where the gradient (else the input) begins a 512-byte or 1 KB block, so the
+    scalar head before it is up to a few hundred elements long, depending on both addresses.  Input and gradient at
+    matching and at unrelated offsets from a 1 KB boundary, with and without a gradient; all against the oracle."""
+    from paper_2506_00486_b200 import Segments
+    rng = np.random.default_rng(83)
+    n = 3 * 16384 + 77
+    esz = 2 if dtype == torch.bfloat16 else 4
+    for xo_bytes, go_bytes in ((16, 32), (128, 256), (0, 256), (16, 0), (48, 480), (1008, 992), (0, 0)):
+        xs = [gg_synth.gg_host(rng, 0.9, 0.02, n, dtype), gg_synth.gg_host(rng, 1.7, 0.3, 300, dtype)]
+        xd, gd = [], []
+        for x in xs:
+            xb = torch.zeros(x.numel() + 1024, dtype=dtype, device="cuda:0")
+            gb = torch.full((x.numel() + 1024,), 9.0, dtype=torch.float32, device="cuda:0")
+            assert xb.data_ptr() % 512 == 0 and gb.data_ptr() % 512 == 0
+            xo = (-xb.data_ptr() % 1024 + xo_bytes) // esz
+            go = (-gb.data_ptr() % 1024 + go_bytes) // 4
+            xb[xo:xo + x.numel()].copy_(x)
+            xd.append(xb[xo:xo + x.numel()])
+            gd.append(gb[go:go + x.numel()])
+        steps = torch.full((2,), 2.0 ** -9, dtype=torch.float32, device="cuda:0")
+        out = ctx.gg_fused(Segments(xd), grad=Segments(gd), lam=1e-4, step=steps)
+        torch.cuda.synchronize()
+        check_fused(out, xs, gd, 1e-4, [0, 1], 2, steps=steps)
+        hist_only = ctx.gg_rate_hist(xd, steps)
+        fit_only = ctx.gg_fit(xd)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(hist_only["hist"].cpu().numpy(), out["hist"].cpu().numpy())
+        assert torch.equal(fit_only["beta"], out["beta"]) and torch.equal(fit_only["sum_sq"], out["sum_sq"])
