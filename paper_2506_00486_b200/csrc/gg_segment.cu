@@ -56,6 +56,37 @@ __global__ void __launch_bounds__(kSegThreads) fit_kernel(const FitArgs a)
     fit_finish(a, s, lane, s1, s2, bad, xmin, xmax);
 }
 
+// The same with one WARP per segment (eight segments per CTA), for layouts of many segments of few tiles each, where
+// a CTA per segment leaves seven of its eight warps idle and the launch takes several waves: lane l adds the tiles
+// l, l + 32, ... in order, a butterfly adds the lanes.  (Another order of additions than the kernel above: which of
+// the two serves a layout depends on the layout alone, so a layout always gets the same bits.)
+__global__ void __launch_bounds__(kSegThreads) fit_warp_kernel(const FitArgs a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int s = blockIdx.x * (kSegThreads / 32) + warp;
+    if (s >= a.map.n_seg) return;
+    const int t0 = a.map.tile_prefix[s], t1 = a.map.tile_prefix[s + 1];
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t bad = 0;
+    float xmin = INFINITY, xmax = -INFINITY;
+    for (int t = t0 + lane; t < t1; t += 32) {
+        s1 += a.part.s1[t];
+        s2 += a.part.s2[t];
+        bad += a.part.bad[t];
+        xmin = fminf(xmin, a.part.xmin[t]);
+        xmax = fmaxf(xmax, a.part.xmax[t]);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    bad = __reduce_add_sync(kFull, bad);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xmin = fminf(xmin, __shfl_xor_sync(kFull, xmin, o));
+        xmax = fmaxf(xmax, __shfl_xor_sync(kFull, xmax, o));
+    }
+    fit_finish(a, s, lane, s1, s2, bad, xmin, xmax);
+}
+
 // penalty[s] = (1/beta_s) * sum over the segment's tiles of sum |x| |g|
 //            = lambda_s * sum (|x|/alpha_s)^beta_s   since |x| |g| = lambda beta (|x|/alpha)^beta.
 __device__ __forceinline__ void penalty_finalize(const TileMap &map, const TileScratch &part, const double *beta, double *penalty, int s)
@@ -159,7 +190,10 @@ finish_kernel(const TileMap map, const TileScratch part, const double *beta, dou
 cudaError_t launch_fit(const FitArgs &a, cudaStream_t st)
 {
     if (a.map.n_seg <= 0) return cudaSuccess;
-    fit_kernel<<<a.map.n_seg, kSegThreads, 0, st>>>(a);
+    if (a.map.n_seg >= 64 && (int64_t)a.map.n_tiles <= 32 * (int64_t)a.map.n_seg)
+        fit_warp_kernel<<<(a.map.n_seg + kSegThreads / 32 - 1) / (kSegThreads / 32), kSegThreads, 0, st>>>(a);
+    else
+        fit_kernel<<<a.map.n_seg, kSegThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
